@@ -1,0 +1,198 @@
+/*
+ * sti.h - C ABI of the shard-elastic transformer execution path (STI, arXiv 2207.05022).
+ *
+ * The library executes a plan that the caller supplies: for every layer, which shard units
+ * are kept, at which bitwidth each is stored, and whether it sits in the preload buffer or is
+ * streamed while earlier layers compute.  Choosing the plan (the paper's two-stage planner,
+ * Section 5) is the caller's business; the paper's engine likewise "simply loads and executes
+ * the shards that have been selected in planning" (Section 3.2).
+ *
+ * Vocabulary (Section 4.2, Table 1).  A layer with hidden size d, M heads of width 64 and
+ * d_ff FFN neurons is cut into vertical slices.  Here the attention part and the FFN part of a
+ * slice are separate *shard units*:
+ *   attention unit h : Q_h, K_h, V_h  [64 x d]   and  O_h [d x 64]
+ *   FFN unit j       : F1_j [f x d]              and  F2_j [d x f],   f = d_ff / n_ffn_slices
+ * All matrices are out-features x in-features, row-major (y = x W^T).  The paper's shard i is
+ * the pair (attention unit i, FFN unit i) with equal keep/bits.
+ *
+ * Shard blob format (upload).  Bitwidth k in {2,3,4,5,6}: every weight is a k-bit index into
+ * the unit's table of 2^k fp32 centroids.  Index i of a matrix (row-major flat order) occupies
+ * bits [i*k, i*k+k) of a bit stream, least-significant bit first, stored as little-endian
+ * 32-bit words; the unit's matrices follow each other in the order Q,K,V,O (attention) or
+ * F1,F2 (FFN), each starting on a 16-byte boundary (automatic for the shapes accepted here).
+ * Outliers (Section 6) are (flat offset within the unit, fp32 value) pairs, offsets ascending;
+ * their slot in the index stream holds an arbitrary valid index.  Bitwidth 32 is the
+ * uncompressed version: `codes` holds the raw fp32 weights in the same order, no table.
+ *
+ * Shape limits: head_dim == 64, hidden % 128 == 0, (ffn / n_ffn_slices) % 128 == 0,
+ * max_seq <= 512.
+ *
+ * Threading/streams: a context owns one compute stream (or borrows the caller's) and one copy
+ * stream.  Forward calls are asynchronous on the compute stream; sti_sync waits for them and
+ * returns the first error a kernel reported.  A context is not thread-safe.
+ *
+ * Errors: every call returns a status and never aborts; out-parameters are left untouched on
+ * error.  Device-side waits are bounded: a kernel that gives up sets a status word that
+ * sti_sync reports as STI_ERR_TIMEOUT, and the context stays usable.
+ */
+#ifndef STI_H_
+#define STI_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+#if defined(__GNUC__)
+#pragma GCC visibility push(default)   /* the library is built with hidden visibility otherwise */
+#endif
+
+typedef struct sti_ctx sti_ctx;    /* device, streams, dense parameters, activation scratch */
+typedef struct sti_plan sti_plan;  /* which shard units, at which bits, where they live     */
+
+typedef enum {
+  STI_OK = 0,
+  STI_ERR_ARG = 1,           /* null pointer, index out of range                      */
+  STI_ERR_BITS = 2,          /* bitwidth not in {2..6, 32} or blob/plan mismatch       */
+  STI_ERR_SHAPE = 3,         /* model shape outside the limits above, batch*seq too big */
+  STI_ERR_SIZE = 4,          /* blob size does not match the unit's shape              */
+  STI_ERR_STATE = 5,         /* call not allowed in this state (e.g. upload after use) */
+  STI_ERR_SHARD_MISSING = 6, /* a kept unit was never uploaded                         */
+  STI_ERR_OOM = 7,           /* device or pinned-host allocation failed                */
+  STI_ERR_CUDA = 8,          /* CUDA runtime error                                     */
+  STI_ERR_TIMEOUT = 9        /* a bounded device-side wait ran out                     */
+} sti_status;
+
+typedef enum { STI_ATTN = 0, STI_FFN = 1 } sti_kind;
+typedef enum { STI_F32 = 0, STI_BF16 = 1 } sti_dtype;
+
+typedef struct {
+  int32_t n_layers;
+  int32_t hidden;        /* d                                         */
+  int32_t n_heads;       /* M                                         */
+  int32_t head_dim;      /* must be 64                                */
+  int32_t ffn;           /* d_ff                                      */
+  int32_t n_ffn_slices;  /* M_f                                       */
+  int32_t max_batch;
+  int32_t max_seq;       /* <= 512                                    */
+  int32_t act_dtype;     /* sti_dtype of x and y                      */
+  float ln_eps;          /* LayerNorm epsilon (BERT: 1e-12)           */
+} sti_model_desc;
+
+typedef struct {
+  uint8_t keep;      /* 0 = dropped: contributes exactly zero (Section 4.2)      */
+  uint8_t bits;      /* 2..6, or 32 = uncompressed fp32                          */
+  uint8_t resident;  /* 1 = preload buffer in device memory, 0 = streamed         */
+} sti_shard_cfg;
+
+typedef struct {
+  int32_t bits;
+  const uint32_t* codes;        /* host; index stream (or raw fp32 when bits == 32)      */
+  size_t n_code_words;          /* must equal the unit's weight count * bits / 32         */
+  const float* centroids;       /* host; 2^bits entries; NULL when bits == 32            */
+  const uint32_t* outlier_off;  /* host; flat offsets within the unit, strictly ascending */
+  const float* outlier_val;     /* host                                                   */
+  size_t n_outliers;
+} sti_shard_blob;
+
+typedef struct {
+  /* filled by sti_get_stats for the most recent sti_model_forward on the plan */
+  int32_t n_layers;
+  float compute_us[64];   /* per layer: first kernel start to last kernel end              */
+  float copy_us[64];      /* per layer: duration of its host-to-device shard copy (0 if none) */
+  float stall_us[64];     /* per layer: time compute waited for the copy beyond the previous layer's end */
+  uint64_t streamed_bytes[64];
+  uint64_t resident_bytes[64];
+  float total_us;         /* first operation of the forward to its last                    */
+} sti_stats;
+
+/* Section 3.1 (the system model: a library the app links; one model per context).
+ * Creates streams and scratch sized for max_batch*max_seq tokens on `device`.
+ * `compute_stream` is a cudaStream_t to borrow, or NULL to create one. */
+sti_status sti_ctx_create(const sti_model_desc* desc, int device, void* compute_stream, sti_ctx** out);
+
+/* Section 6 ("layer normalization and biases ... kept in memory in full fidelity").
+ * Host arrays, copied before return: bq,bk,bv [n_heads*64]; bo [d]; b1 [ffn]; b2 [d];
+ * ln1_g, ln1_b, ln2_g, ln2_b [d]. */
+sti_status sti_ctx_set_layer_params(sti_ctx* ctx, int layer,
+                                    const float* bq, const float* bk, const float* bv, const float* bo,
+                                    const float* b1, const float* b2,
+                                    const float* ln1_g, const float* ln1_b,
+                                    const float* ln2_g, const float* ln2_b);
+
+/* Section 3.2 / 5.4: a plan is the submodel with one version and one residency per shard.
+ * attn has n_layers*n_heads entries (layer-major), ffn has n_layers*n_ffn_slices.
+ * ring_slots >= 2 is the number of streamed-layer buffers in device memory. */
+sti_status sti_plan_create(sti_ctx* ctx, const sti_shard_cfg* attn, const sti_shard_cfg* ffn,
+                           int ring_slots, sti_plan** out);
+
+/* Section 4.2 "storing shards per version": hands one unit's blob to the plan.  Host pointers
+ * are only read during the call.  The blob's bits must equal the plan's.  Not allowed after
+ * the plan has been finalized. */
+sti_status sti_shard_upload(sti_plan* plan, int layer, sti_kind kind, int index, const sti_shard_blob* blob);
+
+/* Section 3.1: fills the preload buffer (resident units -> device memory) and lays every
+ * streamed layer out as one contiguous pinned-host blob ("one layer ... as a single IO job").
+ * Called implicitly by the first forward.  STI_ERR_SHARD_MISSING if a kept unit has no blob. */
+sti_status sti_plan_finalize(sti_plan* plan);
+
+/* Section 2.1 / 4.2: one layer over its kept units.  x_dev, y_dev: device, [batch, seq, hidden]
+ * contiguous in act_dtype, caller-owned; x_dev == y_dev allowed.  seq_lens_dev: device int32
+ * [batch] of valid lengths (padded keys get probability 0) or NULL.  A streamed layer is
+ * copied first (not overlapped).  Asynchronous. */
+sti_status sti_layer_forward(sti_plan* plan, int layer, const void* x_dev, void* y_dev,
+                             int batch, int seq, const int32_t* seq_lens_dev);
+
+/* Section 5.5: layers 0..n-1 in order; layer l's shard copy overlaps the compute of earlier
+ * layers, a layer starts only when its own shards have arrived, and a ring slot is reused only
+ * after its layer has finished.  Asynchronous. */
+sti_status sti_model_forward(sti_plan* plan, const void* x_dev, void* y_dev,
+                             int batch, int seq, const int32_t* seq_lens_dev);
+
+/* Same with host buffers: x_host/y_host are [batch, seq, hidden] in act_dtype (pinned memory
+ * makes the copies asynchronous), seq_lens_host int32 [batch] or NULL.  The input copy, the
+ * forward and the output copy are enqueued in order; call sti_sync before reading y_host. */
+sti_status sti_model_forward_host(sti_plan* plan, const void* x_host, void* y_host,
+                                  int batch, int seq, const int32_t* seq_lens_host);
+
+/* Waits for everything enqueued on the context; returns the first asynchronous error. */
+sti_status sti_sync(sti_ctx* ctx);
+
+/* Section 4.2 (decompression "substitut[es] dictionary indexes with floating point centroids
+ * and outliers"): decodes one matrix of an uploaded unit for inspection.  matrix: 0..3 = Q,K,V,O
+ * or 0..1 = F1,F2.  Any of the outputs may be NULL: w_dev fp32 [rows*cols] exact table values
+ * with outliers patched, codes_dev one byte per index, wbf16_dev the bf16 (round-to-nearest-
+ * even) operand values the GEMMs use.  Device pointers, caller-owned.  Asynchronous. */
+sti_status sti_shard_decode(sti_plan* plan, int layer, sti_kind kind, int index, int matrix,
+                            float* w_dev, uint8_t* codes_dev, uint16_t* wbf16_dev);
+
+/* Section 5.2 (profiling of IO and compute delays): per-layer timings of the last
+ * sti_model_forward.  Enable with sti_plan_set_profiling before that forward. */
+sti_status sti_plan_set_profiling(sti_plan* plan, int enabled);
+sti_status sti_get_stats(sti_plan* plan, sti_stats* out);
+
+/* Bytes the plan holds: preload buffer in device memory, pinned host arena, ring slots. */
+sti_status sti_plan_memory(sti_plan* plan, uint64_t* preload_bytes, uint64_t* pinned_bytes, uint64_t* ring_bytes);
+
+/* Host-only utility: re-tiles one matrix's canonical index stream (rows x cols indexes of `bits`
+ * bits) into the order the device holds it (see the upload format above; the size is unchanged).
+ * For every group of 32 rows (64 rows when cols == 64) and every 128-column chunk, the `bits`
+ * 16-byte planes of the 32 rows' 128-index runs are stored plane-major, 512 bytes per plane.
+ * Exposed so that the layout can be inspected and tested without a device. */
+sti_status sti_host_retile(const uint8_t* src, uint8_t* dst, uint32_t rows, uint32_t cols, uint32_t bits);
+
+/* Kernel launches issued by the library on this context since creation (for accounting). */
+uint64_t sti_ctx_launch_count(sti_ctx* ctx);
+
+void sti_plan_destroy(sti_plan* plan);
+void sti_ctx_destroy(sti_ctx* ctx);
+const char* sti_strerror(sti_status s);
+
+#if defined(__GNUC__)
+#pragma GCC visibility pop
+#endif
+#ifdef __cplusplus
+}
+#endif
+#endif /* STI_H_ */

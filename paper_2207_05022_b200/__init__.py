@@ -1,0 +1,15 @@
+"""B200-native shard decode + elastic transformer-layer execution (STI, arXiv 2207.05022).
+
+The package is a thin ctypes binding over the C-ABI library built from `csrc/` (sm_100a CUDA).
+Every step of the execution path runs in that library's kernels; Python only marshals arguments.
+"""
+from .binding import (  # noqa: F401
+    STI_OK, STI_ATTN, STI_FFN, STI_F32, STI_BF16,
+    StiError, StiModelDesc, StiShardCfg, StiShardBlob, StiStats,
+    load_library, library_path,
+    sti_ctx_create, sti_ctx_destroy, sti_ctx_set_layer_params, sti_plan_create, sti_plan_destroy,
+    sti_shard_upload, sti_plan_finalize, sti_layer_forward, sti_model_forward, sti_model_forward_host,
+    sti_sync, sti_shard_decode, sti_plan_set_profiling, sti_get_stats, sti_plan_memory,
+    sti_ctx_launch_count, sti_host_retile, sti_strerror,
+    Session,
+)

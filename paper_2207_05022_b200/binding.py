@@ -1,0 +1,271 @@
+"""ctypes binding of include/sti.h: same names, argument marshalling only.
+
+Device buffers are passed as integer addresses (e.g. `tensor.data_ptr()`); host arrays as
+numpy arrays.  Nothing here computes: if the shared library is missing or cannot be loaded
+the import of any entry point raises, there is no other execution path.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from typing import Optional, Sequence
+
+import numpy as np
+
+STI_OK = 0
+STI_ATTN, STI_FFN = 0, 1
+STI_F32, STI_BF16 = 0, 1
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_LIB_NAME = "libsti_b200.so"
+_lib = None
+
+
+class StiError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        msg = sti_strerror(status) if _lib is not None else str(status)
+        super().__init__(f"{where}: {msg} (status {status})")
+
+
+class StiModelDesc(C.Structure):
+    _fields_ = [("n_layers", C.c_int32), ("hidden", C.c_int32), ("n_heads", C.c_int32),
+                ("head_dim", C.c_int32), ("ffn", C.c_int32), ("n_ffn_slices", C.c_int32),
+                ("max_batch", C.c_int32), ("max_seq", C.c_int32), ("act_dtype", C.c_int32),
+                ("ln_eps", C.c_float)]
+
+
+class StiShardCfg(C.Structure):
+    _fields_ = [("keep", C.c_uint8), ("bits", C.c_uint8), ("resident", C.c_uint8)]
+
+
+class StiShardBlob(C.Structure):
+    _fields_ = [("bits", C.c_int32), ("codes", C.c_void_p), ("n_code_words", C.c_size_t),
+                ("centroids", C.c_void_p), ("outlier_off", C.c_void_p), ("outlier_val", C.c_void_p),
+                ("n_outliers", C.c_size_t)]
+
+
+class StiStats(C.Structure):
+    _fields_ = [("n_layers", C.c_int32), ("compute_us", C.c_float * 64), ("copy_us", C.c_float * 64),
+                ("stall_us", C.c_float * 64), ("streamed_bytes", C.c_uint64 * 64),
+                ("resident_bytes", C.c_uint64 * 64), ("total_us", C.c_float)]
+
+
+def library_path() -> str:
+    return os.path.join(_HERE, _LIB_NAME)
+
+
+def load_library():
+    """Loads the C-ABI library built by `python -m paper_2207_05022_b200.build`."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    path = library_path()
+    if not os.path.exists(path):
+        raise RuntimeError(f"{path} is missing: build it with `python -m paper_2207_05022_b200.build` "
+                           "(there is no fallback execution path)")
+    lib = C.CDLL(path)
+    vp, i32, u64p = C.c_void_p, C.c_int, C.POINTER(C.c_uint64)
+    sigs = {
+        "sti_ctx_create": ([C.POINTER(StiModelDesc), i32, vp, C.POINTER(vp)], i32),
+        "sti_ctx_destroy": ([vp], None),
+        "sti_ctx_set_layer_params": ([vp, i32] + [vp] * 10, i32),
+        "sti_plan_create": ([vp, C.POINTER(StiShardCfg), C.POINTER(StiShardCfg), i32, C.POINTER(vp)], i32),
+        "sti_plan_destroy": ([vp], None),
+        "sti_shard_upload": ([vp, i32, i32, i32, C.POINTER(StiShardBlob)], i32),
+        "sti_plan_finalize": ([vp], i32),
+        "sti_layer_forward": ([vp, i32, vp, vp, i32, i32, vp], i32),
+        "sti_model_forward": ([vp, vp, vp, i32, i32, vp], i32),
+        "sti_model_forward_host": ([vp, vp, vp, i32, i32, vp], i32),
+        "sti_sync": ([vp], i32),
+        "sti_shard_decode": ([vp, i32, i32, i32, i32, vp, vp, vp], i32),
+        "sti_plan_set_profiling": ([vp, i32], i32),
+        "sti_get_stats": ([vp, C.POINTER(StiStats)], i32),
+        "sti_plan_memory": ([vp, u64p, u64p, u64p], i32),
+        "sti_ctx_launch_count": ([vp], C.c_uint64),
+        "sti_host_retile": ([vp, vp, C.c_uint32, C.c_uint32, C.c_uint32], i32),
+        "sti_strerror": ([i32], C.c_char_p),
+    }
+    for name, (argtypes, restype) in sigs.items():
+        fn = getattr(lib, name)          # AttributeError if the library does not export it
+        fn.argtypes = argtypes
+        fn.restype = restype
+    _lib = lib
+    return lib
+
+
+EXPORTED = ("sti_ctx_create", "sti_ctx_destroy", "sti_ctx_set_layer_params", "sti_plan_create",
+            "sti_plan_destroy", "sti_shard_upload", "sti_plan_finalize", "sti_layer_forward",
+            "sti_model_forward", "sti_model_forward_host", "sti_sync", "sti_shard_decode",
+            "sti_plan_set_profiling", "sti_get_stats", "sti_plan_memory", "sti_ctx_launch_count",
+            "sti_host_retile", "sti_strerror")
+
+
+def _check(status: int, where: str):
+    if status != STI_OK:
+        raise StiError(status, where)
+
+
+def _host(a: Optional[np.ndarray], dtype) -> Optional[np.ndarray]:
+    if a is None:
+        return None
+    return np.ascontiguousarray(a, dtype=dtype)
+
+
+def _ptr(a: Optional[np.ndarray]):
+    return None if a is None else a.ctypes.data_as(C.c_void_p)
+
+
+def sti_strerror(status: int) -> str:
+    return load_library().sti_strerror(int(status)).decode()
+
+
+def sti_ctx_create(desc: StiModelDesc, device: int = 0, compute_stream: int = 0) -> int:
+    out = C.c_void_p()
+    _check(load_library().sti_ctx_create(C.byref(desc), device, C.c_void_p(compute_stream or None), C.byref(out)),
+           "sti_ctx_create")
+    return out.value
+
+
+def sti_ctx_destroy(ctx: int):
+    load_library().sti_ctx_destroy(C.c_void_p(ctx))
+
+
+def sti_ctx_set_layer_params(ctx: int, layer: int, bq, bk, bv, bo, b1, b2, ln1_g, ln1_b, ln2_g, ln2_b):
+    arrs = [_host(a, np.float32).reshape(-1) for a in (bq, bk, bv, bo, b1, b2, ln1_g, ln1_b, ln2_g, ln2_b)]
+    _check(load_library().sti_ctx_set_layer_params(C.c_void_p(ctx), layer, *[_ptr(a) for a in arrs]),
+           "sti_ctx_set_layer_params")
+
+
+def _cfg_array(cfgs: Sequence[Sequence[int]]):
+    arr = (StiShardCfg * len(cfgs))()
+    for i, (keep, bits, resident) in enumerate(cfgs):
+        arr[i].keep, arr[i].bits, arr[i].resident = int(bool(keep)), int(bits), int(bool(resident))
+    return arr
+
+
+def sti_plan_create(ctx: int, attn: Sequence[Sequence[int]], ffn: Sequence[Sequence[int]], ring_slots: int = 2) -> int:
+    """attn/ffn: flat, layer-major sequences of (keep, bits, resident)."""
+    out = C.c_void_p()
+    _check(load_library().sti_plan_create(C.c_void_p(ctx), _cfg_array(attn), _cfg_array(ffn), ring_slots,
+                                          C.byref(out)), "sti_plan_create")
+    return out.value
+
+
+def sti_plan_destroy(plan: int):
+    load_library().sti_plan_destroy(C.c_void_p(plan))
+
+
+def sti_shard_upload(plan: int, layer: int, kind: int, index: int, bits: int, codes: np.ndarray,
+                     centroids: Optional[np.ndarray], outlier_off: Optional[np.ndarray] = None,
+                     outlier_val: Optional[np.ndarray] = None):
+    codes = _host(codes, np.uint32)
+    cent = _host(centroids, np.float32)
+    off = _host(outlier_off, np.uint32) if outlier_off is not None and len(outlier_off) else None
+    val = _host(outlier_val, np.float32) if outlier_val is not None and len(outlier_val) else None
+    blob = StiShardBlob(bits=int(bits), codes=_ptr(codes), n_code_words=codes.size, centroids=_ptr(cent),
+                        outlier_off=_ptr(off), outlier_val=_ptr(val), n_outliers=0 if off is None else off.size)
+    _check(load_library().sti_shard_upload(C.c_void_p(plan), layer, kind, index, C.byref(blob)), "sti_shard_upload")
+
+
+def sti_plan_finalize(plan: int):
+    _check(load_library().sti_plan_finalize(C.c_void_p(plan)), "sti_plan_finalize")
+
+
+def sti_layer_forward(plan: int, layer: int, x_dev: int, y_dev: int, batch: int, seq: int, seq_lens_dev: int = 0):
+    _check(load_library().sti_layer_forward(C.c_void_p(plan), layer, C.c_void_p(x_dev), C.c_void_p(y_dev), batch, seq,
+                                            C.c_void_p(seq_lens_dev or None)), "sti_layer_forward")
+
+
+def sti_model_forward(plan: int, x_dev: int, y_dev: int, batch: int, seq: int, seq_lens_dev: int = 0):
+    _check(load_library().sti_model_forward(C.c_void_p(plan), C.c_void_p(x_dev), C.c_void_p(y_dev), batch, seq,
+                                            C.c_void_p(seq_lens_dev or None)), "sti_model_forward")
+
+
+def sti_model_forward_host(plan: int, x_host: int, y_host: int, batch: int, seq: int, seq_lens_host: int = 0):
+    """x_host / y_host: host addresses (e.g. of pinned torch tensors or numpy arrays)."""
+    _check(load_library().sti_model_forward_host(C.c_void_p(plan), C.c_void_p(x_host), C.c_void_p(y_host), batch, seq,
+                                                 C.c_void_p(seq_lens_host or None)), "sti_model_forward_host")
+
+
+def sti_sync(ctx: int):
+    _check(load_library().sti_sync(C.c_void_p(ctx)), "sti_sync")
+
+
+def sti_shard_decode(plan: int, layer: int, kind: int, index: int, matrix: int, w_dev: int = 0, codes_dev: int = 0,
+                     wbf16_dev: int = 0):
+    _check(load_library().sti_shard_decode(C.c_void_p(plan), layer, kind, index, matrix, C.c_void_p(w_dev or None),
+                                           C.c_void_p(codes_dev or None), C.c_void_p(wbf16_dev or None)),
+           "sti_shard_decode")
+
+
+def sti_plan_set_profiling(plan: int, enabled: bool):
+    _check(load_library().sti_plan_set_profiling(C.c_void_p(plan), int(enabled)), "sti_plan_set_profiling")
+
+
+def sti_get_stats(plan: int) -> StiStats:
+    st = StiStats()
+    _check(load_library().sti_get_stats(C.c_void_p(plan), C.byref(st)), "sti_get_stats")
+    return st
+
+
+def sti_plan_memory(plan: int):
+    a, b, c = C.c_uint64(), C.c_uint64(), C.c_uint64()
+    _check(load_library().sti_plan_memory(C.c_void_p(plan), C.byref(a), C.byref(b), C.byref(c)), "sti_plan_memory")
+    return {"preload_bytes": a.value, "pinned_bytes": b.value, "ring_bytes": c.value}
+
+
+def sti_ctx_launch_count(ctx: int) -> int:
+    return int(load_library().sti_ctx_launch_count(C.c_void_p(ctx)))
+
+
+def sti_host_retile(src: np.ndarray, rows: int, cols: int, bits: int) -> np.ndarray:
+    src = np.ascontiguousarray(src).view(np.uint8).reshape(-1)
+    dst = np.empty_like(src)
+    _check(load_library().sti_host_retile(_ptr(src), _ptr(dst), rows, cols, bits), "sti_host_retile")
+    return dst
+
+
+class Session:
+    """Marshals a synthetic workload (any object with the fields of `workloads.Workload`) into a
+    context and a plan: set dense parameters, create the plan, upload every kept unit."""
+
+    def __init__(self, work, device: int = 0, compute_stream: int = 0, max_batch: Optional[int] = None,
+                 max_seq: Optional[int] = None, ring_slots: Optional[int] = None, finalize: bool = True):
+        sh = work.shape
+        self.work = work
+        self.desc = StiModelDesc(n_layers=sh.n_layers, hidden=sh.hidden, n_heads=sh.n_heads, head_dim=sh.head_dim,
+                                 ffn=sh.ffn, n_ffn_slices=sh.n_ffn_slices, max_batch=max_batch or work.batch,
+                                 max_seq=max_seq or work.seq,
+                                 act_dtype=STI_BF16 if work.act_dtype == "bf16" else STI_F32, ln_eps=work.ln_eps)
+        self.ctx = sti_ctx_create(self.desc, device, compute_stream)
+        self.plan = 0
+        try:
+            for l, p in enumerate(work.dense):
+                sti_ctx_set_layer_params(self.ctx, l, p["bq"], p["bk"], p["bv"], p["bo"], p["b1"], p["b2"],
+                                         p["ln1_g"], p["ln1_b"], p["ln2_g"], p["ln2_b"])
+            attn = [(u.keep, u.bits, u.resident) for layer in work.attn_plan for u in layer]
+            ffn = [(u.keep, u.bits, u.resident) for layer in work.ffn_plan for u in layer]
+            self.plan = sti_plan_create(self.ctx, attn, ffn, ring_slots or work.ring_slots)
+            for (l, kind, idx), b in work.blobs.items():
+                sti_shard_upload(self.plan, l, kind, idx, b.bits, b.codes, b.centroids, b.outlier_off, b.outlier_val)
+            if finalize:
+                sti_plan_finalize(self.plan)
+        except Exception:
+            self.close()
+            raise
+
+    def close(self):
+        if self.plan:
+            sti_plan_destroy(self.plan)
+            self.plan = 0
+        if self.ctx:
+            sti_ctx_destroy(self.ctx)
+            self.ctx = 0
+
+    def __enter__(self):
+        return self
+
+    def __exit__(self, *exc):
+        self.close()
+        return False

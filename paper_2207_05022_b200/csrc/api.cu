@@ -1,0 +1,900 @@
+// Host runtime behind the C ABI: contexts, plans, the preload buffer, the pinned arena, the ring of
+// streamed-layer slots, tile-job tables, and the layerwise copy/compute pipeline (Sections 3.1, 5.5).
+#include <algorithm>
+#include <cstdio>
+#include <cstdlib>
+#include <cstring>
+#include <new>
+#include <string>
+#include <vector>
+
+#include <cuda_runtime.h>
+
+#include "../../include/sti.h"
+#include "retile.h"
+#include "sti_kernels.h"
+
+using namespace sti;
+
+namespace {
+
+constexpr int kMaxLayersStats = 64;
+constexpr size_t kMaxSmem = 227 * 1024;
+
+inline size_t align16(size_t v) { return (v + 15) & ~static_cast<size_t>(15); }
+inline size_t align256(size_t v) { return (v + 255) & ~static_cast<size_t>(255); }
+
+struct MatrixInfo {
+  uint32_t rows, kc;
+  uint32_t flat_base;   // first weight's flat offset in the unit
+};
+
+struct Tuning {
+  int qkv_n = 32, f1_n = 64, o_n = 64, o_group = 4, f2_n = 64, f2_group = 2;
+};
+
+struct Unit {
+  sti_shard_cfg cfg{};
+  bool uploaded = false;
+  std::vector<uint8_t> codes;          // re-tiled (or raw fp32), until finalize moves it into an arena
+  std::vector<float> table;
+  std::vector<uint32_t> out_off;
+  std::vector<float> out_val;
+  size_t off_codes = 0, off_table = 0, off_ooff = 0, off_oval = 0, bytes = 0;   // inside the layer part
+  uint8_t* dev = nullptr;              // where the unit's region starts in device memory
+};
+
+struct GemmTable {
+  Job* jobs = nullptr;
+  Seg* segs = nullptr;
+  int n_jobs = 0;
+  size_t smem = 0;
+  int n_split = 0;
+};
+
+struct Layer {
+  std::vector<Unit> attn, ffn;
+  std::vector<int> kept_heads, kept_slices;
+  size_t res_bytes = 0, str_bytes = 0;
+  uint8_t* res_dev = nullptr;          // in the preload buffer
+  uint8_t* str_host = nullptr;         // in the pinned arena
+  int slot = -1;                       // ring slot of the streamed part
+  GemmTable qkv, o, f1, f2;
+  cudaEvent_t ev_loaded = nullptr, ev_done = nullptr, ev_copy_start = nullptr, ev_comp_start = nullptr;
+};
+
+}  // namespace
+
+struct sti_ctx {
+  sti_model_desc desc{};
+  int device = 0;
+  cudaStream_t compute = nullptr, copy = nullptr;
+  bool own_compute = false;
+  float* dense = nullptr;              // [n_layers][dense_stride]
+  size_t dense_stride = 0;
+  size_t off_bq = 0, off_bk = 0, off_bv = 0, off_bo = 0, off_b1 = 0, off_b2 = 0, off_ln1g = 0, off_ln1b = 0,
+         off_ln2g = 0, off_ln2b = 0;
+  int* err_dev = nullptr;
+  uint64_t launches = 0;
+  bool simt_debug = false;
+  sti_status async_error = STI_OK;
+  MatrixInfo attn_m[4]{}, ffn_m[2]{};
+  uint32_t attn_weights = 0, ffn_weights = 0;
+};
+
+struct sti_plan {
+  sti_ctx* ctx = nullptr;
+  std::vector<Layer> layers;
+  int ring_slots = 2;
+  bool finalized = false;
+  bool attempted = false;
+  bool profiling = false;
+  Tuning tune;
+  uint8_t* preload = nullptr;  size_t preload_bytes = 0;
+  uint8_t* pinned = nullptr;   size_t pinned_bytes = 0;
+  uint8_t* ring = nullptr;     size_t slot_bytes = 0;
+  uint8_t* tables = nullptr;   size_t tables_bytes = 0;       // job/segment descriptors
+  std::vector<cudaEvent_t> slot_free;
+  cudaEvent_t ev_copy_tail = nullptr, ev_begin = nullptr, ev_end = nullptr;
+  bool copy_tail_valid = false;
+  // activation scratch
+  uint16_t* qkv = nullptr; uint16_t* attn_out = nullptr; float* partial = nullptr;
+  float* h1_f32 = nullptr; uint16_t* h1_bf16 = nullptr; uint16_t* u = nullptr;
+  void* buf[2] = {nullptr, nullptr};
+  void* x_in = nullptr; void* y_out = nullptr; int32_t* lens_dev = nullptr;
+  int max_partial = 1;
+  bool stats_valid = false;
+};
+
+namespace {
+
+#define CUDA_TRY(expr)                          \
+  do {                                          \
+    cudaError_t e__ = (expr);                   \
+    if (e__ != cudaSuccess) {                   \
+      if (e__ == cudaErrorMemoryAllocation) {   \
+        (void)cudaGetLastError();               \
+        return STI_ERR_OOM;                     \
+      }                                         \
+      return STI_ERR_CUDA;                      \
+    }                                           \
+  } while (0)
+
+size_t act_size(const sti_ctx* c) { return c->desc.act_dtype == STI_BF16 ? 2 : 4; }
+
+const MatrixInfo* unit_matrices(const sti_ctx* c, sti_kind kind, int* n) {
+  *n = kind == STI_ATTN ? 4 : 2;
+  return kind == STI_ATTN ? c->attn_m : c->ffn_m;
+}
+
+size_t matrix_code_bytes(const MatrixInfo& m, int bits) {
+  return static_cast<size_t>(m.rows) * m.kc * bits / 8;
+}
+
+void parse_tuning(Tuning* t, int tmax, const sti_model_desc& d) {
+  // more, smaller tiles when there are few tokens (spread the decode over all SMs);
+  // wider tiles when each decoded weight is reused by many token tiles
+  if (tmax > 1024) {
+    t->qkv_n = 64; t->f1_n = 64; t->o_n = 64; t->o_group = 16; t->f2_n = 64; t->f2_group = 4;
+  } else {
+    t->qkv_n = 32; t->f1_n = 64; t->o_n = 64; t->o_group = 4; t->f2_n = 64; t->f2_group = 2;
+  }
+  const char* env = getenv("STI_TUNE");     // debugging aid: "qkv_n=32,o_group=4,..."
+  if (env) {
+    std::string s(env);
+    size_t pos = 0;
+    while (pos < s.size()) {
+      size_t end = s.find(',', pos);
+      if (end == std::string::npos) end = s.size();
+      const std::string kv = s.substr(pos, end - pos);
+      const size_t eq = kv.find('=');
+      if (eq != std::string::npos) {
+        const std::string k = kv.substr(0, eq);
+        const int v = atoi(kv.c_str() + eq + 1);
+        if (k == "qkv_n") t->qkv_n = v;
+        else if (k == "f1_n") t->f1_n = v;
+        else if (k == "o_n") t->o_n = v;
+        else if (k == "o_group") t->o_group = v;
+        else if (k == "f2_n") t->f2_n = v;
+        else if (k == "f2_group") t->f2_group = v;
+      }
+      pos = end + 1;
+    }
+  }
+  auto pow2_tile = [](int v, int lo) { return (v == 32 || v == 64 || v == 128) && v >= lo ? v : lo; };
+  t->qkv_n = std::min(pow2_tile(t->qkv_n, 32), 64);
+  const int f = d.ffn / d.n_ffn_slices;
+  t->f1_n = pow2_tile(t->f1_n, 32);
+  while (f % t->f1_n) t->f1_n /= 2;
+  t->o_n = pow2_tile(t->o_n, 64);
+  t->f2_n = pow2_tile(t->f2_n, 32);
+  while (d.hidden % t->o_n) t->o_n /= 2;
+  while (d.hidden % t->f2_n) t->f2_n /= 2;
+  t->o_group = std::max(1, std::min(t->o_group, 16));
+  t->f2_group = std::max(1, std::min(t->f2_group, 16));
+  // keep every weight tile inside shared memory
+  while (t->qkv_n > 32 && gemm_smem_bytes(t->qkv_n, d.hidden, 1) > kMaxSmem) t->qkv_n /= 2;
+  while (t->f1_n > 32 && gemm_smem_bytes(t->f1_n, d.hidden, 1) > kMaxSmem) t->f1_n /= 2;
+  while (t->o_group > 1 && gemm_smem_bytes(t->o_n, t->o_group * 64, t->o_group) > kMaxSmem) --t->o_group;
+  while (t->f2_group > 1 && gemm_smem_bytes(t->f2_n, t->f2_group * f, t->f2_group) > kMaxSmem) --t->f2_group;
+}
+
+Unit* find_unit(sti_plan* p, int layer, sti_kind kind, int index) {
+  if (layer < 0 || layer >= static_cast<int>(p->layers.size())) return nullptr;
+  auto& v = kind == STI_ATTN ? p->layers[layer].attn : p->layers[layer].ffn;
+  if (index < 0 || index >= static_cast<int>(v.size())) return nullptr;
+  return &v[index];
+}
+
+// Segment for rows [row0, row0 + n_rows) of matrix `m` of `u`.
+Seg make_seg(const sti_ctx* c, const Unit& u, sti_kind kind, int m, uint32_t row0, uint32_t n_rows, uint32_t koff) {
+  int nm;
+  const MatrixInfo* mi = unit_matrices(c, kind, &nm);
+  const int bits = u.cfg.bits;
+  size_t mat_off = 0;
+  for (int i = 0; i < m; ++i) mat_off += matrix_code_bytes(mi[i], bits);
+  Seg s{};
+  s.codes = reinterpret_cast<const uint4*>(u.dev + u.off_codes + mat_off +
+                                           static_cast<size_t>(row0) * mi[m].kc * bits / 8);
+  s.table = reinterpret_cast<const float*>(u.dev + u.off_table);
+  s.flat_base = mi[m].flat_base + row0 * mi[m].kc;
+  const uint32_t flat_end = s.flat_base + n_rows * mi[m].kc;
+  const size_t lo = std::lower_bound(u.out_off.begin(), u.out_off.end(), s.flat_base) - u.out_off.begin();
+  const size_t hi = std::lower_bound(u.out_off.begin(), u.out_off.end(), flat_end) - u.out_off.begin();
+  s.out_off = reinterpret_cast<const uint32_t*>(u.dev + u.off_ooff) + lo;
+  s.out_val = reinterpret_cast<const float*>(u.dev + u.off_oval) + lo;
+  s.n_out = static_cast<uint32_t>(hi - lo);
+  s.bits = bits;
+  s.kc = mi[m].kc;
+  s.koff = koff;
+  return s;
+}
+
+struct TableBuilder {
+  std::vector<Job> jobs;
+  std::vector<Seg> segs;
+  size_t smem = 0;
+  void add(Job j, const std::vector<Seg>& ss) {
+    j.seg_begin = static_cast<uint32_t>(segs.size());
+    j.n_seg = static_cast<uint32_t>(ss.size());
+    segs.insert(segs.end(), ss.begin(), ss.end());
+    jobs.push_back(j);
+    smem = std::max(smem, gemm_smem_bytes(j.n_rows, j.k_total, j.n_seg));
+  }
+};
+
+void build_layer_tables(sti_plan* p, Layer& L, TableBuilder tb[4]) {
+  const sti_ctx* c = p->ctx;
+  const sti_model_desc& d = c->desc;
+  const Tuning& t = p->tune;
+  const uint32_t f = d.ffn / d.n_ffn_slices;
+  // QKV: one job per (kept head, matrix, row tile); full K
+  for (size_t hi = 0; hi < L.kept_heads.size(); ++hi) {
+    const int h = L.kept_heads[hi];
+    for (int which = 0; which < 3; ++which)
+      for (uint32_t r0 = 0; r0 < 64; r0 += t.qkv_n) {
+        Job j{};
+        j.n_rows = t.qkv_n; j.k_total = d.hidden; j.x_koff = 0;
+        j.out_mat = static_cast<uint32_t>(hi * 3 + which); j.out_col = r0;
+        j.bias_off = which * d.n_heads * 64 + h * 64 + static_cast<int>(r0);
+        tb[0].add(j, {make_seg(c, L.attn[h], STI_ATTN, which, r0, t.qkv_n, 0)});
+      }
+  }
+  // O projection: K is split over groups of kept heads, each group writes its own partial sum
+  const int nh = static_cast<int>(L.kept_heads.size());
+  L.o.n_split = (nh + t.o_group - 1) / t.o_group;
+  for (int sp = 0; sp < L.o.n_split; ++sp) {
+    const int first = sp * t.o_group, cnt = std::min(t.o_group, nh - first);
+    for (uint32_t n0 = 0; n0 < static_cast<uint32_t>(d.hidden); n0 += t.o_n) {
+      Job j{};
+      j.n_rows = t.o_n; j.k_total = cnt * 64; j.x_koff = first * 64;
+      j.out_mat = sp; j.out_col = n0; j.bias_off = -1;
+      std::vector<Seg> ss;
+      for (int i = 0; i < cnt; ++i)
+        ss.push_back(make_seg(c, L.attn[L.kept_heads[first + i]], STI_ATTN, 3, n0, t.o_n, i * 64));
+      tb[1].add(j, ss);
+    }
+  }
+  // FFN1: one job per (kept slice, row tile); full K
+  for (size_t ji = 0; ji < L.kept_slices.size(); ++ji) {
+    const int s = L.kept_slices[ji];
+    for (uint32_t r0 = 0; r0 < f; r0 += t.f1_n) {
+      Job j{};
+      j.n_rows = t.f1_n; j.k_total = d.hidden; j.x_koff = 0;
+      j.out_mat = 0; j.out_col = static_cast<uint32_t>(ji * f + r0);
+      j.bias_off = s * static_cast<int>(f) + static_cast<int>(r0);
+      tb[2].add(j, {make_seg(c, L.ffn[s], STI_FFN, 0, r0, t.f1_n, 0)});
+    }
+  }
+  // FFN2: K split over groups of kept slices
+  const int ns = static_cast<int>(L.kept_slices.size());
+  L.f2.n_split = (ns + t.f2_group - 1) / t.f2_group;
+  for (int sp = 0; sp < L.f2.n_split; ++sp) {
+    const int first = sp * t.f2_group, cnt = std::min(t.f2_group, ns - first);
+    for (uint32_t n0 = 0; n0 < static_cast<uint32_t>(d.hidden); n0 += t.f2_n) {
+      Job j{};
+      j.n_rows = t.f2_n; j.k_total = cnt * f; j.x_koff = first * f;
+      j.out_mat = sp; j.out_col = n0; j.bias_off = -1;
+      std::vector<Seg> ss;
+      for (int i = 0; i < cnt; ++i)
+        ss.push_back(make_seg(c, L.ffn[L.kept_slices[first + i]], STI_FFN, 1, n0, t.f2_n, i * f));
+      tb[3].add(j, ss);
+    }
+  }
+}
+
+sti_status check_async(sti_ctx* c) {
+  int flag = 0;
+  if (cudaMemcpy(&flag, c->err_dev, sizeof(int), cudaMemcpyDeviceToHost) != cudaSuccess) return STI_ERR_CUDA;
+  if (flag != ERR_NONE) {
+    int zero = 0;
+    (void)cudaMemcpy(c->err_dev, &zero, sizeof(int), cudaMemcpyHostToDevice);
+    return flag == ERR_WAIT_TIMEOUT ? STI_ERR_TIMEOUT : STI_ERR_ARG;
+  }
+  return STI_OK;
+}
+
+int m_ctas_for(int n_jobs, int T) {
+  const int n_mtiles = (T + 127) / 128;
+  int m = n_jobs > 0 ? 148 / n_jobs : 1;
+  return std::max(1, std::min(m, n_mtiles));
+}
+
+sti_status run_gemm(sti_plan* p, GemmKind kind, const GemmTable& tab, const void* x, int ldx, int T, void* out,
+                    int ldo, const float* bias) {
+  if (tab.n_jobs == 0) return STI_OK;
+  GemmLaunch g{};
+  g.jobs = tab.jobs; g.segs = tab.segs; g.n_jobs = tab.n_jobs; g.m_ctas = m_ctas_for(tab.n_jobs, T);
+  g.x = x; g.ldx = ldx; g.T = T; g.out = out; g.ldo = ldo; g.bias = bias; g.err = p->ctx->err_dev;
+  g.smem_bytes = tab.smem; g.simt_debug = p->ctx->simt_debug;
+  CUDA_TRY(launch_gemm(kind, g, p->ctx->compute));
+  p->ctx->launches++;
+  return STI_OK;
+}
+
+// The seven kernels of one layer on the compute stream.
+sti_status enqueue_layer(sti_plan* p, int li, const void* x, void* y, int batch, int seq, const int32_t* lens) {
+  sti_ctx* c = p->ctx;
+  const sti_model_desc& d = c->desc;
+  Layer& L = p->layers[li];
+  const int T = batch * seq;
+  const float* dense = c->dense + static_cast<size_t>(li) * c->dense_stride;
+  const bool bf16_act = d.act_dtype == STI_BF16;
+  const int nh = static_cast<int>(L.kept_heads.size()), ns = static_cast<int>(L.kept_slices.size());
+  const int f = d.ffn / d.n_ffn_slices;
+  sti_status st;
+  if (nh > 0) {
+    st = run_gemm(p, bf16_act ? GEMM_BF16_TO_BF16 : GEMM_F32_TO_BF16, L.qkv, x, d.hidden, T, p->qkv, 64,
+                  dense + c->off_bq);
+    if (st != STI_OK) return st;
+    CUDA_TRY(launch_attention(p->qkv, p->attn_out, nh, batch, seq, lens, c->compute));
+    c->launches++;
+    st = run_gemm(p, GEMM_BF16_TO_F32, L.o, p->attn_out, nh * 64, T, p->partial, d.hidden, nullptr);
+    if (st != STI_OK) return st;
+  }
+  LnLaunch ln{};
+  ln.partial = p->partial; ln.n_partial = nh > 0 ? L.o.n_split : 0;
+  ln.bias = dense + c->off_bo; ln.resid = x; ln.resid_bf16 = bf16_act ? 1 : 0;
+  ln.gamma = dense + c->off_ln1g; ln.beta = dense + c->off_ln1b; ln.eps = d.ln_eps; ln.T = T; ln.d = d.hidden;
+  ln.out_f32 = p->h1_f32; ln.out_bf16 = p->h1_bf16;
+  CUDA_TRY(launch_layernorm(ln, c->compute));
+  c->launches++;
+  if (ns > 0) {
+    st = run_gemm(p, GEMM_BF16_TO_BF16_GELU, L.f1, p->h1_bf16, d.hidden, T, p->u, ns * f, dense + c->off_b1);
+    if (st != STI_OK) return st;
+    st = run_gemm(p, GEMM_BF16_TO_F32, L.f2, p->u, ns * f, T, p->partial, d.hidden, nullptr);
+    if (st != STI_OK) return st;
+  }
+  LnLaunch l2{};
+  l2.partial = p->partial; l2.n_partial = ns > 0 ? L.f2.n_split : 0;
+  l2.bias = dense + c->off_b2; l2.resid = p->h1_f32; l2.resid_bf16 = 0;
+  l2.gamma = dense + c->off_ln2g; l2.beta = dense + c->off_ln2b; l2.eps = d.ln_eps; l2.T = T; l2.d = d.hidden;
+  l2.out_f32 = bf16_act ? nullptr : static_cast<float*>(y);
+  l2.out_bf16 = bf16_act ? static_cast<uint16_t*>(y) : nullptr;
+  CUDA_TRY(launch_layernorm(l2, c->compute));
+  c->launches++;
+  return STI_OK;
+}
+
+sti_status check_forward_args(sti_plan* p, const void* x, void* y, int batch, int seq) {
+  if (!p || !x || !y) return STI_ERR_ARG;
+  const sti_model_desc& d = p->ctx->desc;
+  if (batch < 1 || seq < 1 || seq > d.max_seq) return STI_ERR_SHAPE;
+  if (static_cast<long long>(batch) * seq > static_cast<long long>(d.max_batch) * d.max_seq) return STI_ERR_SHAPE;
+  return STI_OK;
+}
+
+// Copy of layer li's streamed part into its ring slot, on stream `s`.
+sti_status enqueue_layer_copy(sti_plan* p, int li, cudaStream_t s) {
+  Layer& L = p->layers[li];
+  if (L.str_bytes == 0) return STI_OK;
+  CUDA_TRY(cudaMemcpyAsync(p->ring + static_cast<size_t>(L.slot) * p->slot_bytes, L.str_host, L.str_bytes,
+                           cudaMemcpyHostToDevice, s));
+  return STI_OK;
+}
+
+sti_status model_forward_impl(sti_plan* p, const void* x, void* y, int batch, int seq, const int32_t* lens) {
+  sti_ctx* c = p->ctx;
+  const int n = static_cast<int>(p->layers.size());
+  if (p->profiling) CUDA_TRY(cudaEventRecord(p->ev_begin, c->compute));
+  // the copy stream must not run ahead of work already enqueued on the compute stream that may still
+  // read ring slots: slot_free events order that; nothing else is shared between the streams
+  const void* cur = x;
+  for (int li = 0; li < n; ++li) {
+    Layer& L = p->layers[li];
+    if (L.str_bytes > 0) {
+      // one IO job per layer (Section 3.1); the slot is reused only after its previous layer finished
+      CUDA_TRY(cudaStreamWaitEvent(c->copy, p->slot_free[L.slot], 0));
+      if (p->profiling) CUDA_TRY(cudaEventRecord(L.ev_copy_start, c->copy));
+      sti_status st = enqueue_layer_copy(p, li, c->copy);
+      if (st != STI_OK) return st;
+      CUDA_TRY(cudaEventRecord(L.ev_loaded, c->copy));
+      // a layer starts only when its own shards (and, by stream order, all earlier ones) are loaded
+      CUDA_TRY(cudaStreamWaitEvent(c->compute, L.ev_loaded, 0));
+    }
+    if (p->profiling) CUDA_TRY(cudaEventRecord(L.ev_comp_start, c->compute));
+    void* nxt = (li == n - 1) ? y : p->buf[li & 1];
+    sti_status st = enqueue_layer(p, li, cur, nxt, batch, seq, lens);
+    if (st != STI_OK) return st;
+    if (p->profiling) CUDA_TRY(cudaEventRecord(L.ev_done, c->compute));
+    if (L.str_bytes > 0) CUDA_TRY(cudaEventRecord(p->slot_free[L.slot], c->compute));
+    cur = nxt;
+  }
+  CUDA_TRY(cudaEventRecord(p->ev_copy_tail, c->copy));
+  p->copy_tail_valid = true;
+  if (p->profiling) {
+    CUDA_TRY(cudaEventRecord(p->ev_end, c->compute));
+    p->stats_valid = true;
+  }
+  return STI_OK;
+}
+
+void free_plan_device(sti_plan* p) {
+  if (!p) return;
+  cudaFree(p->preload); cudaFree(p->ring); cudaFree(p->tables);
+  if (p->pinned) cudaFreeHost(p->pinned);
+  cudaFree(p->qkv); cudaFree(p->attn_out); cudaFree(p->partial); cudaFree(p->h1_f32); cudaFree(p->h1_bf16);
+  cudaFree(p->u); cudaFree(p->buf[0]); cudaFree(p->buf[1]); cudaFree(p->x_in); cudaFree(p->y_out);
+  cudaFree(p->lens_dev);
+  for (auto& L : p->layers) {
+    if (L.ev_loaded) cudaEventDestroy(L.ev_loaded);
+    if (L.ev_done) cudaEventDestroy(L.ev_done);
+    if (L.ev_copy_start) cudaEventDestroy(L.ev_copy_start);
+    if (L.ev_comp_start) cudaEventDestroy(L.ev_comp_start);
+  }
+  for (auto e : p->slot_free) cudaEventDestroy(e);
+  if (p->ev_copy_tail) cudaEventDestroy(p->ev_copy_tail);
+  if (p->ev_begin) cudaEventDestroy(p->ev_begin);
+  if (p->ev_end) cudaEventDestroy(p->ev_end);
+}
+
+}  // namespace
+
+extern "C" {
+
+const char* sti_strerror(sti_status s) {
+  switch (s) {
+    case STI_OK: return "ok";
+    case STI_ERR_ARG: return "invalid argument";
+    case STI_ERR_BITS: return "unsupported or mismatched bitwidth";
+    case STI_ERR_SHAPE: return "unsupported shape";
+    case STI_ERR_SIZE: return "blob size does not match the unit";
+    case STI_ERR_STATE: return "call not allowed in this state";
+    case STI_ERR_SHARD_MISSING: return "a kept shard unit was never uploaded";
+    case STI_ERR_OOM: return "out of memory";
+    case STI_ERR_CUDA: return "CUDA runtime error";
+    case STI_ERR_TIMEOUT: return "a bounded device-side wait ran out";
+  }
+  return "unknown status";
+}
+
+sti_status sti_ctx_create(const sti_model_desc* desc, int device, void* compute_stream, sti_ctx** out) {
+  if (!desc || !out) return STI_ERR_ARG;
+  const sti_model_desc& d = *desc;
+  if (d.n_layers < 1 || d.n_layers > kMaxLayersStats || d.n_heads < 1 || d.n_ffn_slices < 1 || d.max_batch < 1 ||
+      d.max_seq < 1)
+    return STI_ERR_SHAPE;
+  if (d.head_dim != 64 || d.hidden < 128 || d.hidden % 128 != 0 || d.hidden > 2048 || d.ffn % d.n_ffn_slices != 0 ||
+      (d.ffn / d.n_ffn_slices) % 128 != 0 || d.max_seq > 512 || d.n_heads * 64 > 16 * 128)
+    return STI_ERR_SHAPE;
+  if (d.act_dtype != STI_F32 && d.act_dtype != STI_BF16) return STI_ERR_ARG;
+  int n_dev = 0;
+  if (cudaGetDeviceCount(&n_dev) != cudaSuccess || device < 0 || device >= n_dev) {
+    (void)cudaGetLastError();
+    return STI_ERR_CUDA;      // no usable CUDA device: there is no other execution path
+  }
+  CUDA_TRY(cudaSetDevice(device));
+  sti_ctx* c = new (std::nothrow) sti_ctx();
+  if (!c) return STI_ERR_OOM;
+  c->desc = d;
+  c->device = device;
+  const uint32_t dd = d.hidden, f = d.ffn / d.n_ffn_slices;
+  c->attn_m[0] = {64, dd, 0};
+  c->attn_m[1] = {64, dd, 64 * dd};
+  c->attn_m[2] = {64, dd, 2 * 64 * dd};
+  c->attn_m[3] = {dd, 64, 3 * 64 * dd};
+  c->attn_weights = 4 * 64 * dd;
+  c->ffn_m[0] = {f, dd, 0};
+  c->ffn_m[1] = {dd, f, f * dd};
+  c->ffn_weights = 2 * f * dd;
+  const size_t hq = static_cast<size_t>(d.n_heads) * 64;
+  size_t o = 0;
+  c->off_bq = o; o += hq;
+  c->off_bk = o; o += hq;
+  c->off_bv = o; o += hq;
+  c->off_bo = o; o += dd;
+  c->off_b1 = o; o += d.ffn;
+  c->off_b2 = o; o += dd;
+  c->off_ln1g = o; o += dd;
+  c->off_ln1b = o; o += dd;
+  c->off_ln2g = o; o += dd;
+  c->off_ln2b = o; o += dd;
+  c->dense_stride = (o + 63) / 64 * 64;
+  auto fail = [&](sti_status s) { sti_ctx_destroy(c); return s; };
+  if (compute_stream) {
+    c->compute = static_cast<cudaStream_t>(compute_stream);
+  } else {
+    if (cudaStreamCreateWithFlags(&c->compute, cudaStreamNonBlocking) != cudaSuccess) return fail(STI_ERR_CUDA);
+    c->own_compute = true;
+  }
+  if (cudaStreamCreateWithFlags(&c->copy, cudaStreamNonBlocking) != cudaSuccess) return fail(STI_ERR_CUDA);
+  if (cudaMalloc(&c->dense, c->dense_stride * d.n_layers * sizeof(float)) != cudaSuccess) return fail(STI_ERR_OOM);
+  if (cudaMemset(c->dense, 0, c->dense_stride * d.n_layers * sizeof(float)) != cudaSuccess) return fail(STI_ERR_CUDA);
+  if (cudaMalloc(&c->err_dev, sizeof(int)) != cudaSuccess) return fail(STI_ERR_OOM);
+  if (cudaMemset(c->err_dev, 0, sizeof(int)) != cudaSuccess) return fail(STI_ERR_CUDA);
+  if (gemm_configure() != cudaSuccess || attention_configure() != cudaSuccess) return fail(STI_ERR_CUDA);
+  const char* dbg = getenv("STI_DEBUG_SIMT");
+  c->simt_debug = dbg && dbg[0] == '1';
+  *out = c;
+  return STI_OK;
+}
+
+void sti_ctx_destroy(sti_ctx* c) {
+  if (!c) return;
+  cudaSetDevice(c->device);
+  if (c->compute) cudaStreamSynchronize(c->compute);
+  if (c->copy) cudaStreamSynchronize(c->copy);
+  cudaFree(c->dense);
+  cudaFree(c->err_dev);
+  if (c->own_compute && c->compute) cudaStreamDestroy(c->compute);
+  if (c->copy) cudaStreamDestroy(c->copy);
+  delete c;
+}
+
+sti_status sti_ctx_set_layer_params(sti_ctx* c, int layer, const float* bq, const float* bk, const float* bv,
+                                    const float* bo, const float* b1, const float* b2, const float* ln1_g,
+                                    const float* ln1_b, const float* ln2_g, const float* ln2_b) {
+  if (!c || !bq || !bk || !bv || !bo || !b1 || !b2 || !ln1_g || !ln1_b || !ln2_g || !ln2_b) return STI_ERR_ARG;
+  if (layer < 0 || layer >= c->desc.n_layers) return STI_ERR_ARG;
+  CUDA_TRY(cudaSetDevice(c->device));
+  std::vector<float> h(c->dense_stride, 0.f);
+  const size_t hq = static_cast<size_t>(c->desc.n_heads) * 64, d = c->desc.hidden;
+  memcpy(&h[c->off_bq], bq, hq * 4); memcpy(&h[c->off_bk], bk, hq * 4); memcpy(&h[c->off_bv], bv, hq * 4);
+  memcpy(&h[c->off_bo], bo, d * 4); memcpy(&h[c->off_b1], b1, static_cast<size_t>(c->desc.ffn) * 4);
+  memcpy(&h[c->off_b2], b2, d * 4);
+  memcpy(&h[c->off_ln1g], ln1_g, d * 4); memcpy(&h[c->off_ln1b], ln1_b, d * 4);
+  memcpy(&h[c->off_ln2g], ln2_g, d * 4); memcpy(&h[c->off_ln2b], ln2_b, d * 4);
+  CUDA_TRY(cudaStreamSynchronize(c->compute));
+  CUDA_TRY(cudaMemcpy(c->dense + static_cast<size_t>(layer) * c->dense_stride, h.data(), h.size() * 4,
+                      cudaMemcpyHostToDevice));
+  return STI_OK;
+}
+
+sti_status sti_plan_create(sti_ctx* c, const sti_shard_cfg* attn, const sti_shard_cfg* ffn, int ring_slots,
+                           sti_plan** out) {
+  if (!c || !attn || !ffn || !out) return STI_ERR_ARG;
+  if (ring_slots < 2 || ring_slots > 64) return STI_ERR_ARG;
+  const sti_model_desc& d = c->desc;
+  auto ok_bits = [](int b) { return (b >= 2 && b <= 6) || b == 32; };
+  for (int i = 0; i < d.n_layers * d.n_heads; ++i)
+    if (attn[i].keep && !ok_bits(attn[i].bits)) return STI_ERR_BITS;
+  for (int i = 0; i < d.n_layers * d.n_ffn_slices; ++i)
+    if (ffn[i].keep && !ok_bits(ffn[i].bits)) return STI_ERR_BITS;
+  sti_plan* p = new (std::nothrow) sti_plan();
+  if (!p) return STI_ERR_OOM;
+  p->ctx = c;
+  p->ring_slots = ring_slots;
+  p->layers.resize(d.n_layers);
+  for (int l = 0; l < d.n_layers; ++l) {
+    Layer& L = p->layers[l];
+    L.attn.resize(d.n_heads);
+    L.ffn.resize(d.n_ffn_slices);
+    for (int h = 0; h < d.n_heads; ++h) {
+      L.attn[h].cfg = attn[l * d.n_heads + h];
+      if (L.attn[h].cfg.keep) L.kept_heads.push_back(h);
+    }
+    for (int s = 0; s < d.n_ffn_slices; ++s) {
+      L.ffn[s].cfg = ffn[l * d.n_ffn_slices + s];
+      if (L.ffn[s].cfg.keep) L.kept_slices.push_back(s);
+    }
+  }
+  parse_tuning(&p->tune, d.max_batch * d.max_seq, d);
+  *out = p;
+  return STI_OK;
+}
+
+void sti_plan_destroy(sti_plan* p) {
+  if (!p) return;
+  cudaSetDevice(p->ctx->device);
+  cudaStreamSynchronize(p->ctx->compute);
+  cudaStreamSynchronize(p->ctx->copy);
+  free_plan_device(p);
+  delete p;
+}
+
+sti_status sti_shard_upload(sti_plan* p, int layer, sti_kind kind, int index, const sti_shard_blob* blob) {
+  if (!p || !blob || (kind != STI_ATTN && kind != STI_FFN)) return STI_ERR_ARG;
+  if (p->finalized) return STI_ERR_STATE;
+  Unit* u = find_unit(p, layer, kind, index);
+  if (!u) return STI_ERR_ARG;
+  if (!u->cfg.keep) return STI_ERR_STATE;
+  if (blob->bits != u->cfg.bits) return STI_ERR_BITS;
+  if (!blob->codes) return STI_ERR_ARG;
+  const sti_ctx* c = p->ctx;
+  int nm;
+  const MatrixInfo* mi = unit_matrices(c, kind, &nm);
+  const uint32_t n_weights = kind == STI_ATTN ? c->attn_weights : c->ffn_weights;
+  const int bits = blob->bits;
+  if (blob->n_code_words != static_cast<size_t>(n_weights) * bits / 32) return STI_ERR_SIZE;
+  if (bits != 32 && !blob->centroids) return STI_ERR_ARG;
+  if (blob->n_outliers && (!blob->outlier_off || !blob->outlier_val)) return STI_ERR_ARG;
+  if (bits == 32 && blob->n_outliers) return STI_ERR_ARG;
+  for (size_t i = 0; i < blob->n_outliers; ++i) {
+    if (blob->outlier_off[i] >= n_weights) return STI_ERR_SIZE;
+    if (i && blob->outlier_off[i] <= blob->outlier_off[i - 1]) return STI_ERR_ARG;
+  }
+  u->codes.assign(blob->n_code_words * 4, 0);
+  const uint8_t* src = reinterpret_cast<const uint8_t*>(blob->codes);
+  if (bits == 32) {
+    memcpy(u->codes.data(), src, u->codes.size());
+  } else {
+    size_t off = 0;
+    for (int m = 0; m < nm; ++m) {
+      retile_matrix(src + off, u->codes.data() + off, mi[m].rows, mi[m].kc, bits);
+      off += matrix_code_bytes(mi[m], bits);
+    }
+  }
+  u->table.clear();
+  if (bits != 32) u->table.assign(blob->centroids, blob->centroids + (1u << bits));
+  u->out_off.assign(blob->outlier_off, blob->outlier_off + blob->n_outliers);
+  u->out_val.assign(blob->outlier_val, blob->outlier_val + blob->n_outliers);
+  u->uploaded = true;
+  return STI_OK;
+}
+
+sti_status sti_plan_finalize(sti_plan* p) {
+  if (!p) return STI_ERR_ARG;
+  if (p->finalized) return STI_OK;
+  if (p->attempted) return STI_ERR_STATE;    // an earlier attempt failed half-way; the plan is unusable
+  sti_ctx* c = p->ctx;
+  const sti_model_desc& d = c->desc;
+  CUDA_TRY(cudaSetDevice(c->device));
+  // 1. every kept unit must have its blob; lay units out inside their layer's resident / streamed part
+  size_t preload_total = 0, pinned_total = 0, slot_bytes = 0;
+  int n_streamed = 0, max_heads = 0, max_slices = 0;
+  for (auto& L : p->layers) {
+    L.res_bytes = L.str_bytes = 0;
+    auto place = [&](Unit& u) -> bool {
+      if (!u.cfg.keep) return true;
+      if (!u.uploaded) return false;
+      size_t& cursor = u.cfg.resident ? L.res_bytes : L.str_bytes;
+      const size_t start = cursor;
+      u.off_codes = cursor; cursor += align16(u.codes.size());
+      u.off_table = cursor; cursor += align16(u.table.size() * 4);
+      u.off_ooff = cursor; cursor += align16(u.out_off.size() * 4);
+      u.off_oval = cursor; cursor += align16(u.out_val.size() * 4);
+      u.bytes = cursor - start;
+      return true;
+    };
+    for (auto& u : L.attn) if (!place(u)) return STI_ERR_SHARD_MISSING;
+    for (auto& u : L.ffn) if (!place(u)) return STI_ERR_SHARD_MISSING;
+    preload_total += align256(L.res_bytes);
+    pinned_total += align256(L.str_bytes);
+    slot_bytes = std::max(slot_bytes, align256(L.str_bytes));
+    if (L.str_bytes) L.slot = (n_streamed++) % p->ring_slots;
+    max_heads = std::max<int>(max_heads, L.kept_heads.size());
+    max_slices = std::max<int>(max_slices, L.kept_slices.size());
+  }
+  p->attempted = true;
+  p->preload_bytes = preload_total; p->pinned_bytes = pinned_total; p->slot_bytes = slot_bytes;
+  if (preload_total) CUDA_TRY(cudaMalloc(&p->preload, preload_total));
+  if (pinned_total) CUDA_TRY(cudaMallocHost(&p->pinned, pinned_total));
+  if (slot_bytes) CUDA_TRY(cudaMalloc(&p->ring, slot_bytes * p->ring_slots));
+  // 2. fill the preload buffer (device) and the pinned arena (host), one contiguous blob per layer
+  size_t pre_cur = 0, pin_cur = 0;
+  std::vector<uint8_t> staging;
+  for (auto& L : p->layers) {
+    L.res_dev = p->preload ? p->preload + pre_cur : nullptr;
+    L.str_host = p->pinned ? p->pinned + pin_cur : nullptr;
+    pre_cur += align256(L.res_bytes);
+    pin_cur += align256(L.str_bytes);
+    staging.assign(L.res_bytes, 0);
+    if (L.str_bytes) memset(L.str_host, 0, L.str_bytes);
+    auto emit = [&](Unit& u) {
+      if (!u.cfg.keep) return;
+      uint8_t* base = u.cfg.resident ? staging.data() : L.str_host;
+      memcpy(base + u.off_codes, u.codes.data(), u.codes.size());
+      if (!u.table.empty()) memcpy(base + u.off_table, u.table.data(), u.table.size() * 4);
+      if (!u.out_off.empty()) {
+        memcpy(base + u.off_ooff, u.out_off.data(), u.out_off.size() * 4);
+        memcpy(base + u.off_oval, u.out_val.data(), u.out_val.size() * 4);
+      }
+      u.dev = u.cfg.resident ? L.res_dev : p->ring + static_cast<size_t>(L.slot) * p->slot_bytes;
+      std::vector<uint8_t>().swap(u.codes);     // the arenas now hold the only copy
+    };
+    for (auto& u : L.attn) emit(u);
+    for (auto& u : L.ffn) emit(u);
+    if (L.res_bytes) CUDA_TRY(cudaMemcpy(L.res_dev, staging.data(), L.res_bytes, cudaMemcpyHostToDevice));
+  }
+  // 3. tile-job tables
+  std::vector<uint8_t> host_tables;
+  struct Fix { GemmTable* t; size_t jobs_off, segs_off; };
+  std::vector<Fix> fixes;
+  p->max_partial = 1;
+  for (auto& L : p->layers) {
+    TableBuilder tb[4];
+    build_layer_tables(p, L, tb);
+    GemmTable* gt[4] = {&L.qkv, &L.o, &L.f1, &L.f2};
+    for (int i = 0; i < 4; ++i) {
+      gt[i]->n_jobs = static_cast<int>(tb[i].jobs.size());
+      gt[i]->smem = tb[i].smem;
+      if (tb[i].smem > kMaxSmem) return STI_ERR_SHAPE;
+      Fix fx{gt[i], 0, 0};
+      fx.jobs_off = align16(host_tables.size());
+      host_tables.resize(fx.jobs_off + tb[i].jobs.size() * sizeof(Job));
+      if (!tb[i].jobs.empty()) memcpy(host_tables.data() + fx.jobs_off, tb[i].jobs.data(), tb[i].jobs.size() * sizeof(Job));
+      fx.segs_off = align16(host_tables.size());
+      host_tables.resize(fx.segs_off + tb[i].segs.size() * sizeof(Seg));
+      if (!tb[i].segs.empty()) memcpy(host_tables.data() + fx.segs_off, tb[i].segs.data(), tb[i].segs.size() * sizeof(Seg));
+      fixes.push_back(fx);
+    }
+    p->max_partial = std::max(p->max_partial, std::max(L.o.n_split, L.f2.n_split));
+  }
+  p->tables_bytes = std::max<size_t>(host_tables.size(), 16);
+  CUDA_TRY(cudaMalloc(&p->tables, p->tables_bytes));
+  if (!host_tables.empty())
+    CUDA_TRY(cudaMemcpy(p->tables, host_tables.data(), host_tables.size(), cudaMemcpyHostToDevice));
+  for (auto& fx : fixes) {
+    fx.t->jobs = reinterpret_cast<Job*>(p->tables + fx.jobs_off);
+    fx.t->segs = reinterpret_cast<Seg*>(p->tables + fx.segs_off);
+  }
+  // 4. activation scratch for max_batch * max_seq tokens
+  const size_t Tmax = static_cast<size_t>(d.max_batch) * d.max_seq;
+  const size_t f = d.ffn / d.n_ffn_slices;
+  CUDA_TRY(cudaMalloc(&p->qkv, std::max<size_t>(1, 3 * max_heads) * Tmax * 64 * 2));
+  CUDA_TRY(cudaMalloc(&p->attn_out, std::max<size_t>(1, max_heads) * Tmax * 64 * 2));
+  CUDA_TRY(cudaMalloc(&p->partial, static_cast<size_t>(p->max_partial) * Tmax * d.hidden * 4));
+  CUDA_TRY(cudaMalloc(&p->h1_f32, Tmax * d.hidden * 4));
+  CUDA_TRY(cudaMalloc(&p->h1_bf16, Tmax * d.hidden * 2));
+  CUDA_TRY(cudaMalloc(&p->u, std::max<size_t>(1, max_slices) * Tmax * f * 2));
+  CUDA_TRY(cudaMalloc(&p->buf[0], Tmax * d.hidden * act_size(c)));
+  CUDA_TRY(cudaMalloc(&p->buf[1], Tmax * d.hidden * act_size(c)));
+  CUDA_TRY(cudaMalloc(&p->x_in, Tmax * d.hidden * act_size(c)));
+  CUDA_TRY(cudaMalloc(&p->y_out, Tmax * d.hidden * act_size(c)));
+  CUDA_TRY(cudaMalloc(&p->lens_dev, static_cast<size_t>(d.max_batch) * 4));
+  // 5. events
+  const unsigned flags = cudaEventDefault;     // timing-capable; only recorded when profiling
+  for (auto& L : p->layers) {
+    CUDA_TRY(cudaEventCreateWithFlags(&L.ev_loaded, flags));
+    CUDA_TRY(cudaEventCreateWithFlags(&L.ev_done, flags));
+    CUDA_TRY(cudaEventCreateWithFlags(&L.ev_copy_start, flags));
+    CUDA_TRY(cudaEventCreateWithFlags(&L.ev_comp_start, flags));
+  }
+  p->slot_free.resize(p->ring_slots);
+  for (auto& e : p->slot_free) {
+    CUDA_TRY(cudaEventCreateWithFlags(&e, cudaEventDisableTiming));
+    CUDA_TRY(cudaEventRecord(e, c->compute));
+  }
+  CUDA_TRY(cudaEventCreateWithFlags(&p->ev_copy_tail, cudaEventDisableTiming));
+  CUDA_TRY(cudaEventCreateWithFlags(&p->ev_begin, flags));
+  CUDA_TRY(cudaEventCreateWithFlags(&p->ev_end, flags));
+  p->finalized = true;
+  return STI_OK;
+}
+
+sti_status sti_layer_forward(sti_plan* p, int layer, const void* x, void* y, int batch, int seq,
+                             const int32_t* lens) {
+  sti_status st = check_forward_args(p, x, y, batch, seq);
+  if (st != STI_OK) return st;
+  if (layer < 0 || layer >= static_cast<int>(p->layers.size())) return STI_ERR_ARG;
+  if ((st = sti_plan_finalize(p)) != STI_OK) return st;
+  sti_ctx* c = p->ctx;
+  CUDA_TRY(cudaSetDevice(c->device));
+  Layer& L = p->layers[layer];
+  if (L.str_bytes > 0) {
+    // not overlapped: the layer's IO job runs on the compute stream, after any copy still in flight
+    if (p->copy_tail_valid) CUDA_TRY(cudaStreamWaitEvent(c->compute, p->ev_copy_tail, 0));
+    if ((st = enqueue_layer_copy(p, layer, c->compute)) != STI_OK) return st;
+  }
+  if ((st = enqueue_layer(p, layer, x, y, batch, seq, lens)) != STI_OK) return st;
+  if (L.str_bytes > 0) CUDA_TRY(cudaEventRecord(p->slot_free[L.slot], c->compute));
+  return STI_OK;
+}
+
+sti_status sti_model_forward(sti_plan* p, const void* x, void* y, int batch, int seq, const int32_t* lens) {
+  sti_status st = check_forward_args(p, x, y, batch, seq);
+  if (st != STI_OK) return st;
+  if ((st = sti_plan_finalize(p)) != STI_OK) return st;
+  CUDA_TRY(cudaSetDevice(p->ctx->device));
+  return model_forward_impl(p, x, y, batch, seq, lens);
+}
+
+sti_status sti_model_forward_host(sti_plan* p, const void* x_host, void* y_host, int batch, int seq,
+                                  const int32_t* lens_host) {
+  sti_status st = check_forward_args(p, x_host, y_host, batch, seq);
+  if (st != STI_OK) return st;
+  if ((st = sti_plan_finalize(p)) != STI_OK) return st;
+  sti_ctx* c = p->ctx;
+  CUDA_TRY(cudaSetDevice(c->device));
+  const size_t bytes = static_cast<size_t>(batch) * seq * c->desc.hidden * act_size(c);
+  CUDA_TRY(cudaMemcpyAsync(p->x_in, x_host, bytes, cudaMemcpyHostToDevice, c->compute));
+  const int32_t* lens = nullptr;
+  if (lens_host) {
+    CUDA_TRY(cudaMemcpyAsync(p->lens_dev, lens_host, static_cast<size_t>(batch) * 4, cudaMemcpyHostToDevice, c->compute));
+    lens = p->lens_dev;
+  }
+  if ((st = model_forward_impl(p, p->x_in, p->y_out, batch, seq, lens)) != STI_OK) return st;
+  CUDA_TRY(cudaMemcpyAsync(y_host, p->y_out, bytes, cudaMemcpyDeviceToHost, c->compute));
+  return STI_OK;
+}
+
+sti_status sti_sync(sti_ctx* c) {
+  if (!c) return STI_ERR_ARG;
+  if (cudaSetDevice(c->device) != cudaSuccess) return STI_ERR_CUDA;
+  cudaError_t e1 = cudaStreamSynchronize(c->copy);
+  cudaError_t e2 = cudaStreamSynchronize(c->compute);
+  if (e1 != cudaSuccess || e2 != cudaSuccess) return STI_ERR_CUDA;
+  return check_async(c);
+}
+
+sti_status sti_shard_decode(sti_plan* p, int layer, sti_kind kind, int index, int matrix, float* w_dev,
+                            uint8_t* codes_dev, uint16_t* wbf16_dev) {
+  if (!p || (kind != STI_ATTN && kind != STI_FFN)) return STI_ERR_ARG;
+  Unit* u = find_unit(p, layer, kind, index);
+  if (!u || !u->cfg.keep) return STI_ERR_ARG;
+  sti_status st = sti_plan_finalize(p);
+  if (st != STI_OK) return st;
+  sti_ctx* c = p->ctx;
+  int nm;
+  const MatrixInfo* mi = unit_matrices(c, kind, &nm);
+  if (matrix < 0 || matrix >= nm) return STI_ERR_ARG;
+  CUDA_TRY(cudaSetDevice(c->device));
+  Layer& L = p->layers[layer];
+  if (!u->cfg.resident) {
+    if (p->copy_tail_valid) CUDA_TRY(cudaStreamWaitEvent(c->compute, p->ev_copy_tail, 0));
+    if ((st = enqueue_layer_copy(p, layer, c->compute)) != STI_OK) return st;
+  }
+  const Seg s = make_seg(c, *u, kind, matrix, 0, mi[matrix].rows, 0);
+  DecodeLaunch dl{};
+  dl.codes = s.codes; dl.table = s.table; dl.out_off = s.out_off; dl.out_val = s.out_val; dl.n_out = s.n_out;
+  dl.flat_base = s.flat_base; dl.bits = s.bits; dl.rows = mi[matrix].rows; dl.kc = mi[matrix].kc;
+  dl.w = w_dev; dl.codes_out = codes_dev; dl.wbf16 = wbf16_dev;
+  CUDA_TRY(launch_decode(dl, c->compute));
+  c->launches += (s.bits == 32 || s.n_out == 0) ? 1 : 2;
+  if (!u->cfg.resident) CUDA_TRY(cudaEventRecord(p->slot_free[L.slot], c->compute));
+  return STI_OK;
+}
+
+sti_status sti_plan_set_profiling(sti_plan* p, int enabled) {
+  if (!p) return STI_ERR_ARG;
+  p->profiling = enabled != 0;
+  p->stats_valid = false;
+  return STI_OK;
+}
+
+sti_status sti_get_stats(sti_plan* p, sti_stats* out) {
+  if (!p || !out) return STI_ERR_ARG;
+  if (!p->finalized || !p->stats_valid) return STI_ERR_STATE;
+  sti_ctx* c = p->ctx;
+  CUDA_TRY(cudaSetDevice(c->device));
+  CUDA_TRY(cudaStreamSynchronize(c->copy));
+  CUDA_TRY(cudaStreamSynchronize(c->compute));
+  sti_stats s;
+  memset(&s, 0, sizeof(s));
+  const int n = static_cast<int>(p->layers.size());
+  s.n_layers = n;
+  float prev_done = 0.f;
+  for (int l = 0; l < n; ++l) {
+    Layer& L = p->layers[l];
+    float t_start = 0.f, t_done = 0.f;
+    CUDA_TRY(cudaEventElapsedTime(&t_start, p->ev_begin, L.ev_comp_start));
+    CUDA_TRY(cudaEventElapsedTime(&t_done, p->ev_begin, L.ev_done));
+    s.compute_us[l] = (t_done - t_start) * 1e3f;
+    if (L.str_bytes) {
+      float ms = 0.f, t_loaded = 0.f;
+      CUDA_TRY(cudaEventElapsedTime(&ms, L.ev_copy_start, L.ev_loaded));
+      s.copy_us[l] = ms * 1e3f;
+      CUDA_TRY(cudaEventElapsedTime(&t_loaded, p->ev_begin, L.ev_loaded));
+      s.stall_us[l] = std::max(0.f, t_loaded - prev_done) * 1e3f;
+    }
+    s.streamed_bytes[l] = L.str_bytes;
+    s.resident_bytes[l] = L.res_bytes;
+    prev_done = t_done;
+  }
+  float tot = 0.f;
+  CUDA_TRY(cudaEventElapsedTime(&tot, p->ev_begin, p->ev_end));
+  s.total_us = tot * 1e3f;
+  *out = s;
+  return STI_OK;
+}
+
+sti_status sti_plan_memory(sti_plan* p, uint64_t* preload_bytes, uint64_t* pinned_bytes, uint64_t* ring_bytes) {
+  if (!p) return STI_ERR_ARG;
+  if (!p->finalized) return STI_ERR_STATE;
+  if (preload_bytes) *preload_bytes = p->preload_bytes;
+  if (pinned_bytes) *pinned_bytes = p->pinned_bytes;
+  if (ring_bytes) *ring_bytes = p->slot_bytes * p->ring_slots;
+  return STI_OK;
+}
+
+uint64_t sti_ctx_launch_count(sti_ctx* c) { return c ? c->launches : 0; }
+
+sti_status sti_host_retile(const uint8_t* src, uint8_t* dst, uint32_t rows, uint32_t cols, uint32_t bits) {
+  if (!src || !dst) return STI_ERR_ARG;
+  if (bits < 2 || bits > 6) return STI_ERR_BITS;
+  if (cols == 64 ? rows % 64 != 0 : (cols % 128 != 0 || rows % 32 != 0)) return STI_ERR_SHAPE;
+  retile_matrix(src, dst, rows, cols, bits);
+  return STI_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,193 @@
+// Per-head scaled-dot-product attention over the kept heads (Section 2.1: each attention head
+// independently contributes one representation; Section 4.2: any subset of heads executes).
+//
+// One CTA = (64-query tile, kept head, sequence); 4 warps x 16 query rows.  K and V of the whole
+// sequence (<= 512 keys) sit in shared memory; scores and the probability-value product run on
+// mma.sync m16n8k16 bf16 with fp32 accumulation, softmax is done in registers with warp shuffles
+// over the four lanes that share a row (online max/sum over 64-key blocks).
+// Attention is ~3 % of a layer's FLOPs at seq 128; the dense projections use tcgen05 (dqgemm.cu).
+#include <cuda_bf16.h>
+
+#include "sti_device.cuh"
+#include "sti_kernels.h"
+
+namespace sti {
+namespace {
+
+constexpr int kHeadDim = 64;
+constexpr int kQTile = 64;
+constexpr int kKStride = kHeadDim + 8;   // bf16 elements per K row in shared memory (conflict-free fragment reads)
+
+__device__ __forceinline__ void mma_bf16_16816(float (&c)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
+  asm volatile(
+      "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+      : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+      : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+
+__global__ void __launch_bounds__(128)
+attention_kernel(const uint16_t* __restrict__ qkv, uint16_t* __restrict__ out, int n_kept, int batch, int L,
+                 const int32_t* __restrict__ seq_lens) {
+  extern __shared__ __align__(16) uint8_t smem[];
+  const int qt = blockIdx.x, hi = blockIdx.y, b = blockIdx.z;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int g = lane >> 2, t4 = lane & 3;
+  const int T = batch * L;
+  const int Lpad = (L + 63) / 64 * 64;
+  const int vstride = Lpad + 8;
+  uint16_t* Ks = reinterpret_cast<uint16_t*>(smem);                       // [Lpad][72]
+  uint16_t* Vt = Ks + static_cast<size_t>(Lpad) * kKStride;               // [64][Lpad + 8]
+
+  const uint16_t* Qg = qkv + (static_cast<size_t>(hi * 3 + 0) * T + static_cast<size_t>(b) * L) * kHeadDim;
+  const uint16_t* Kg = qkv + (static_cast<size_t>(hi * 3 + 1) * T + static_cast<size_t>(b) * L) * kHeadDim;
+  const uint16_t* Vg = qkv + (static_cast<size_t>(hi * 3 + 2) * T + static_cast<size_t>(b) * L) * kHeadDim;
+
+  int valid = L;
+  if (seq_lens != nullptr) {
+    valid = seq_lens[b];
+    valid = valid < 0 ? 0 : (valid > L ? L : valid);
+  }
+
+  for (int idx = tid; idx < Lpad * 8; idx += 128) {
+    const int key = idx >> 3, piece = idx & 7;
+    uint4 v = make_uint4(0, 0, 0, 0);
+    if (key < L) v = __ldg(reinterpret_cast<const uint4*>(Kg + static_cast<size_t>(key) * kHeadDim + piece * 8));
+    *reinterpret_cast<uint4*>(Ks + static_cast<size_t>(key) * kKStride + piece * 8) = v;
+  }
+  for (int idx = tid; idx < Lpad * 8; idx += 128) {
+    const int key = idx % Lpad, piece = idx / Lpad;      // consecutive lanes -> consecutive keys
+    uint4 v = make_uint4(0, 0, 0, 0);
+    if (key < L) v = __ldg(reinterpret_cast<const uint4*>(Vg + static_cast<size_t>(key) * kHeadDim + piece * 8));
+    const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+    for (int i = 0; i < 8; ++i)
+      Vt[static_cast<size_t>(piece * 8 + i) * vstride + key] = static_cast<uint16_t>(w[i >> 1] >> ((i & 1) * 16));
+  }
+  __syncthreads();
+
+  // query fragments of this warp's 16 rows
+  const int q0 = qt * kQTile + warp * 16;
+  uint32_t qa[4][4];
+#pragma unroll
+  for (int kk = 0; kk < 4; ++kk) {
+    const int r0 = q0 + g, r1 = q0 + g + 8;
+    const int c = kk * 16 + 2 * t4;
+    qa[kk][0] = r0 < L ? __ldg(reinterpret_cast<const uint32_t*>(Qg + static_cast<size_t>(r0) * kHeadDim + c)) : 0u;
+    qa[kk][1] = r1 < L ? __ldg(reinterpret_cast<const uint32_t*>(Qg + static_cast<size_t>(r1) * kHeadDim + c)) : 0u;
+    qa[kk][2] = r0 < L ? __ldg(reinterpret_cast<const uint32_t*>(Qg + static_cast<size_t>(r0) * kHeadDim + c + 8)) : 0u;
+    qa[kk][3] = r1 < L ? __ldg(reinterpret_cast<const uint32_t*>(Qg + static_cast<size_t>(r1) * kHeadDim + c + 8)) : 0u;
+  }
+
+  const float scale_log2 = 0.125f * 1.4426950408889634f;     // 1/sqrt(64) * log2(e)
+  float o[8][4];
+#pragma unroll
+  for (int j = 0; j < 8; ++j) { o[j][0] = o[j][1] = o[j][2] = o[j][3] = 0.f; }
+  float m_run[2] = {-INFINITY, -INFINITY};
+  float l_run[2] = {0.f, 0.f};
+
+  const int n_kblocks = (valid + 63) / 64;
+  for (int kb = 0; kb < n_kblocks; ++kb) {
+    float s[8][4];
+#pragma unroll
+    for (int j = 0; j < 8; ++j) { s[j][0] = s[j][1] = s[j][2] = s[j][3] = 0.f; }
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+      const uint16_t* krow = Ks + static_cast<size_t>(kb * 64 + j * 8 + g) * kKStride + 2 * t4;
+#pragma unroll
+      for (int kk = 0; kk < 4; ++kk) {
+        const uint32_t b0 = *reinterpret_cast<const uint32_t*>(krow + kk * 16);
+        const uint32_t b1 = *reinterpret_cast<const uint32_t*>(krow + kk * 16 + 8);
+        mma_bf16_16816(s[j], qa[kk], b0, b1);
+      }
+    }
+    float mblk[2] = {-INFINITY, -INFINITY};
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+      const int key = kb * 64 + j * 8 + 2 * t4;
+#pragma unroll
+      for (int c = 0; c < 4; ++c) {
+        const float v = (key + (c & 1) < valid) ? s[j][c] * scale_log2 : -INFINITY;
+        s[j][c] = v;
+        mblk[c >> 1] = fmaxf(mblk[c >> 1], v);
+      }
+    }
+    float alpha[2], m_use[2];
+#pragma unroll
+    for (int r = 0; r < 2; ++r) {
+      mblk[r] = fmaxf(mblk[r], __shfl_xor_sync(0xffffffffu, mblk[r], 1));
+      mblk[r] = fmaxf(mblk[r], __shfl_xor_sync(0xffffffffu, mblk[r], 2));
+      const float m_new = fmaxf(m_run[r], mblk[r]);
+      m_use[r] = (m_new == -INFINITY) ? 0.f : m_new;
+      alpha[r] = exp2f(m_run[r] - m_use[r]);
+      m_run[r] = m_new;
+      l_run[r] *= alpha[r];
+    }
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+#pragma unroll
+      for (int c = 0; c < 4; ++c) {
+        const float p = exp2f(s[j][c] - m_use[c >> 1]);
+        s[j][c] = p;
+        l_run[c >> 1] += p;
+        o[j][c] *= alpha[c >> 1];
+      }
+    }
+#pragma unroll
+    for (int kk = 0; kk < 4; ++kk) {
+      uint32_t pa[4];
+      pa[0] = pack_bf16x2(s[2 * kk][0], s[2 * kk][1]);
+      pa[1] = pack_bf16x2(s[2 * kk][2], s[2 * kk][3]);
+      pa[2] = pack_bf16x2(s[2 * kk + 1][0], s[2 * kk + 1][1]);
+      pa[3] = pack_bf16x2(s[2 * kk + 1][2], s[2 * kk + 1][3]);
+#pragma unroll
+      for (int jd = 0; jd < 8; ++jd) {
+        const uint16_t* vrow = Vt + static_cast<size_t>(jd * 8 + g) * vstride + kb * 64 + kk * 16 + 2 * t4;
+        const uint32_t b0 = *reinterpret_cast<const uint32_t*>(vrow);
+        const uint32_t b1 = *reinterpret_cast<const uint32_t*>(vrow + 8);
+        mma_bf16_16816(o[jd], pa, b0, b1);
+      }
+    }
+  }
+
+  float inv[2];
+#pragma unroll
+  for (int r = 0; r < 2; ++r) {
+    float l = l_run[r];
+    l += __shfl_xor_sync(0xffffffffu, l, 1);
+    l += __shfl_xor_sync(0xffffffffu, l, 2);
+    inv[r] = l > 0.f ? 1.f / l : 0.f;
+  }
+  const int ldo = n_kept * kHeadDim;
+#pragma unroll
+  for (int r = 0; r < 2; ++r) {
+    const int row = q0 + g + 8 * r;
+    if (row < L) {
+      uint16_t* dst = out + (static_cast<size_t>(b) * L + row) * ldo + hi * kHeadDim + 2 * t4;
+#pragma unroll
+      for (int jd = 0; jd < 8; ++jd)
+        *reinterpret_cast<uint32_t*>(dst + jd * 8) = pack_bf16x2(o[jd][2 * r] * inv[r], o[jd][2 * r + 1] * inv[r]);
+    }
+  }
+}
+
+size_t attn_smem_bytes(int L) {
+  const int Lpad = (L + 63) / 64 * 64;
+  return (static_cast<size_t>(Lpad) * kKStride + static_cast<size_t>(kHeadDim) * (Lpad + 8)) * 2;
+}
+
+}  // namespace
+
+cudaError_t attention_configure() {
+  return cudaFuncSetAttribute(attention_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                              static_cast<int>(attn_smem_bytes(512)));
+}
+
+cudaError_t launch_attention(const uint16_t* qkv, uint16_t* out, int n_kept, int batch, int seq,
+                             const int32_t* seq_lens, cudaStream_t s) {
+  if (n_kept <= 0) return cudaSuccess;
+  dim3 grid((seq + kQTile - 1) / kQTile, n_kept, batch);
+  attention_kernel<<<grid, 128, attn_smem_bytes(seq), s>>>(qkv, out, n_kept, batch, seq, seq_lens);
+  return cudaGetLastError();
+}
+
+}  // namespace sti

@@ -1,0 +1,105 @@
+// Internal interface between the host runtime (api.cu) and the sm_100a kernels.
+// Nothing here is part of the public ABI.
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace sti {
+
+// One contiguous run of a unit matrix's rows feeding a weight tile.
+// Index streams are held re-tiled (see retile.h): for every group of 32 rows (64 when the
+// matrix has 64 in-features) and every 128-column chunk, the k 16-byte planes of the 32
+// per-lane quanta are stored plane-major, so that a warp reads each plane as one coalesced
+// 512-byte line and every lane ends up with 128 consecutive indexes of one row.
+struct Seg {
+  const uint4* codes;       // device; first plane of the tile's first row group (raw fp32 rows when bits == 32)
+  const float* table;       // device; 2^bits fp32 centroids (unused when bits == 32)
+  const uint32_t* out_off;  // device; outliers whose flat offset falls inside this tile
+  const float* out_val;
+  uint32_t n_out;
+  uint32_t flat_base;       // flat offset, within the unit, of the tile's first weight
+  uint32_t bits;            // 2..6 or 32
+  uint32_t kc;              // in-features (row length) of the source matrix
+  uint32_t koff;            // where this segment starts in the job's K range
+  uint32_t pad_;
+};
+
+// One weight-stationary tile: n_rows output features x k_total input features.
+struct Job {
+  uint32_t seg_begin, n_seg;
+  uint32_t n_rows;          // 32, 64 or 128 (multiple of 64 when segments have kc == 64)
+  uint32_t k_total;         // multiple of 64
+  uint32_t x_koff;          // first column of the activation operand
+  uint32_t out_mat;         // output element (t, c) goes to out[(out_mat*T + t)*ldo + out_col + c]
+  uint32_t out_col;
+  int32_t bias_off;         // index of the tile's first bias element, -1 = no bias
+};
+
+enum GemmKind : int {
+  GEMM_F32_TO_BF16 = 0,       // fp32 activations in, bf16 out (+bias)         : QKV on fp32 inputs
+  GEMM_BF16_TO_BF16 = 1,      // bf16 in, bf16 out (+bias)                     : QKV on bf16 inputs
+  GEMM_BF16_TO_BF16_GELU = 2, // bf16 in, bf16 out, +bias, erf-GELU            : FFN1
+  GEMM_BF16_TO_F32 = 3        // bf16 in, fp32 partial sums out, no bias       : O projection, FFN2
+};
+
+struct GemmLaunch {
+  const Job* jobs;
+  const Seg* segs;
+  int n_jobs;
+  int m_ctas;               // CTAs along the token dimension (each loops over its M tiles)
+  const void* x;            // [T, ldx]
+  int ldx;
+  int T;
+  void* out;
+  int ldo;
+  const float* bias;
+  int* err;                 // device status word
+  size_t smem_bytes;        // dynamic shared memory the largest job needs
+  bool simt_debug;          // compute the products on the plain ALUs instead of the tensor cores
+};
+
+size_t gemm_smem_bytes(uint32_t n_rows, uint32_t k_total, uint32_t n_seg);
+cudaError_t gemm_configure();   // opt in to large dynamic shared memory (once per device)
+cudaError_t launch_gemm(GemmKind kind, const GemmLaunch& p, cudaStream_t s);
+
+// Per-head attention over kept heads.  qkv: [(kept*3 + which)][T][64] bf16; out: [T][n_kept*64] bf16.
+cudaError_t attention_configure();
+cudaError_t launch_attention(const uint16_t* qkv, uint16_t* out, int n_kept, int batch, int seq,
+                             const int32_t* seq_lens, cudaStream_t s);
+
+// out = LayerNorm(sum_p partial[p] + bias + resid) * gamma + beta, one warp per token row.
+struct LnLaunch {
+  const float* partial;     // [n_partial][T][d]
+  int n_partial;
+  const float* bias;        // [d]
+  const void* resid;        // [T][d], fp32 or bf16
+  int resid_bf16;
+  const float* gamma;
+  const float* beta;
+  float eps;
+  int T, d;
+  float* out_f32;           // optional
+  uint16_t* out_bf16;       // optional
+};
+cudaError_t launch_layernorm(const LnLaunch& p, cudaStream_t s);
+
+// Stand-alone decode of one matrix (inspection / parity).
+struct DecodeLaunch {
+  const uint4* codes;       // re-tiled stream of the matrix (raw fp32 when bits == 32)
+  const float* table;
+  const uint32_t* out_off;  // the unit's outliers restricted to this matrix
+  const float* out_val;
+  uint32_t n_out;
+  uint32_t flat_base;       // flat offset of the matrix inside the unit
+  uint32_t bits, rows, kc;
+  float* w;                 // optional outputs
+  uint8_t* codes_out;
+  uint16_t* wbf16;
+};
+cudaError_t launch_decode(const DecodeLaunch& p, cudaStream_t s);
+
+constexpr int ERR_NONE = 0;
+constexpr int ERR_WAIT_TIMEOUT = 1;   // a bounded mbarrier wait ran out
+constexpr int ERR_BAD_JOB = 2;        // a job descriptor failed the kernel's own checks
+
+}  // namespace sti
