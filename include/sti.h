@@ -105,6 +105,12 @@ typedef struct {
   uint64_t streamed_bytes[64];
   uint64_t resident_bytes[64];
   float total_us;         /* first operation of the forward to its last                    */
+  /* kernel-level profiling only (sti_plan_set_profiling(plan, 2)); intervals between events recorded
+   * around each kernel, so each includes the launch gap before the kernel */
+  float gemm_us[64];      /* per layer: the four dequant-GEMM launches (QKV, O, FFN1, FFN2)   */
+  float attn_us[64];      /* per layer: the attention kernel                                  */
+  float ln_us[64];        /* per layer: the two residual+LayerNorm kernels                    */
+  int32_t gemm_launches;  /* dequant-GEMM launches in the forward                             */
 } sti_stats;
 
 /* Section 3.1 (the system model: a library the app links; one model per context).
@@ -168,8 +174,9 @@ sti_status sti_shard_decode(sti_plan* plan, int layer, sti_kind kind, int index,
                             float* w_dev, uint8_t* codes_dev, uint16_t* wbf16_dev);
 
 /* Section 5.2 (profiling of IO and compute delays): per-layer timings of the last
- * sti_model_forward.  Enable with sti_plan_set_profiling before that forward. */
-sti_status sti_plan_set_profiling(sti_plan* plan, int enabled);
+ * sti_model_forward.  Enable with sti_plan_set_profiling before that forward: level 0 = off,
+ * 1 = per-layer events, 2 = additionally events around every kernel (slightly slower). */
+sti_status sti_plan_set_profiling(sti_plan* plan, int level);
 sti_status sti_get_stats(sti_plan* plan, sti_stats* out);
 
 /* Bytes the plan holds: preload buffer in device memory, pinned host arena, ring slots. */

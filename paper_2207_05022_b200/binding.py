@@ -48,7 +48,9 @@ class StiShardBlob(C.Structure):
 class StiStats(C.Structure):
     _fields_ = [("n_layers", C.c_int32), ("compute_us", C.c_float * 64), ("copy_us", C.c_float * 64),
                 ("stall_us", C.c_float * 64), ("streamed_bytes", C.c_uint64 * 64),
-                ("resident_bytes", C.c_uint64 * 64), ("total_us", C.c_float)]
+                ("resident_bytes", C.c_uint64 * 64), ("total_us", C.c_float),
+                ("gemm_us", C.c_float * 64), ("attn_us", C.c_float * 64), ("ln_us", C.c_float * 64),
+                ("gemm_launches", C.c_int32)]
 
 
 def library_path() -> str:
@@ -199,8 +201,9 @@ def sti_shard_decode(plan: int, layer: int, kind: int, index: int, matrix: int, 
            "sti_shard_decode")
 
 
-def sti_plan_set_profiling(plan: int, enabled: bool):
-    _check(load_library().sti_plan_set_profiling(C.c_void_p(plan), int(enabled)), "sti_plan_set_profiling")
+def sti_plan_set_profiling(plan: int, level: int):
+    """0 = off, 1 = per-layer events, 2 = events around every kernel."""
+    _check(load_library().sti_plan_set_profiling(C.c_void_p(plan), int(level)), "sti_plan_set_profiling")
 
 
 def sti_get_stats(plan: int) -> StiStats:

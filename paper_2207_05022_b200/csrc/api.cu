@@ -61,6 +61,8 @@ struct Layer {
   int slot = -1;                       // ring slot of the streamed part
   GemmTable qkv, o, f1, f2;
   cudaEvent_t ev_loaded = nullptr, ev_done = nullptr, ev_copy_start = nullptr, ev_comp_start = nullptr;
+  cudaEvent_t ev_k[8] = {};           // boundaries of the seven kernels (kernel-level profiling)
+  bool k_ran[7] = {};
 };
 
 }  // namespace
@@ -88,7 +90,7 @@ struct sti_plan {
   int ring_slots = 2;
   bool finalized = false;
   bool attempted = false;
-  bool profiling = false;
+  int profiling = 0;                   // 0 off, 1 per layer, 2 per kernel
   Tuning tune;
   uint8_t* preload = nullptr;  size_t preload_bytes = 0;
   uint8_t* pinned = nullptr;   size_t pinned_bytes = 0;
@@ -323,15 +325,26 @@ sti_status enqueue_layer(sti_plan* p, int li, const void* x, void* y, int batch,
   const int nh = static_cast<int>(L.kept_heads.size()), ns = static_cast<int>(L.kept_slices.size());
   const int f = d.ffn / d.n_ffn_slices;
   sti_status st;
+  const bool kprof = p->profiling >= 2;
+  auto mark = [&](int i) -> cudaError_t { return kprof ? cudaEventRecord(L.ev_k[i], c->compute) : cudaSuccess; };
+  for (bool& r : L.k_ran) r = false;
+  CUDA_TRY(mark(0));
   if (nh > 0) {
     st = run_gemm(p, bf16_act ? GEMM_BF16_TO_BF16 : GEMM_F32_TO_BF16, L.qkv, x, d.hidden, T, p->qkv, 64,
                   dense + c->off_bq);
     if (st != STI_OK) return st;
+    CUDA_TRY(mark(1));
     CUDA_TRY(launch_attention(p->qkv, p->attn_out, nh, batch, seq, lens, c->compute));
     c->launches++;
+    CUDA_TRY(mark(2));
     st = run_gemm(p, GEMM_BF16_TO_F32, L.o, p->attn_out, nh * 64, T, p->partial, d.hidden, nullptr);
     if (st != STI_OK) return st;
+    L.k_ran[0] = L.k_ran[1] = L.k_ran[2] = true;
+  } else {
+    CUDA_TRY(mark(1));
+    CUDA_TRY(mark(2));
   }
+  CUDA_TRY(mark(3));
   LnLaunch ln{};
   ln.partial = p->partial; ln.n_partial = nh > 0 ? L.o.n_split : 0;
   ln.bias = dense + c->off_bo; ln.resid = x; ln.resid_bf16 = bf16_act ? 1 : 0;
@@ -339,12 +352,19 @@ sti_status enqueue_layer(sti_plan* p, int li, const void* x, void* y, int batch,
   ln.out_f32 = p->h1_f32; ln.out_bf16 = p->h1_bf16;
   CUDA_TRY(launch_layernorm(ln, c->compute));
   c->launches++;
+  L.k_ran[3] = true;
+  CUDA_TRY(mark(4));
   if (ns > 0) {
     st = run_gemm(p, GEMM_BF16_TO_BF16_GELU, L.f1, p->h1_bf16, d.hidden, T, p->u, ns * f, dense + c->off_b1);
     if (st != STI_OK) return st;
+    CUDA_TRY(mark(5));
     st = run_gemm(p, GEMM_BF16_TO_F32, L.f2, p->u, ns * f, T, p->partial, d.hidden, nullptr);
     if (st != STI_OK) return st;
+    L.k_ran[4] = L.k_ran[5] = true;
+  } else {
+    CUDA_TRY(mark(5));
   }
+  CUDA_TRY(mark(6));
   LnLaunch l2{};
   l2.partial = p->partial; l2.n_partial = ns > 0 ? L.f2.n_split : 0;
   l2.bias = dense + c->off_b2; l2.resid = p->h1_f32; l2.resid_bf16 = 0;
@@ -353,6 +373,8 @@ sti_status enqueue_layer(sti_plan* p, int li, const void* x, void* y, int batch,
   l2.out_bf16 = bf16_act ? static_cast<uint16_t*>(y) : nullptr;
   CUDA_TRY(launch_layernorm(l2, c->compute));
   c->launches++;
+  L.k_ran[6] = true;
+  CUDA_TRY(mark(7));
   return STI_OK;
 }
 
@@ -421,6 +443,7 @@ void free_plan_device(sti_plan* p) {
     if (L.ev_done) cudaEventDestroy(L.ev_done);
     if (L.ev_copy_start) cudaEventDestroy(L.ev_copy_start);
     if (L.ev_comp_start) cudaEventDestroy(L.ev_comp_start);
+    for (auto e : L.ev_k) if (e) cudaEventDestroy(e);
   }
   for (auto e : p->slot_free) cudaEventDestroy(e);
   if (p->ev_copy_tail) cudaEventDestroy(p->ev_copy_tail);
@@ -739,6 +762,7 @@ sti_status sti_plan_finalize(sti_plan* p) {
     CUDA_TRY(cudaEventCreateWithFlags(&L.ev_done, flags));
     CUDA_TRY(cudaEventCreateWithFlags(&L.ev_copy_start, flags));
     CUDA_TRY(cudaEventCreateWithFlags(&L.ev_comp_start, flags));
+    for (auto& e : L.ev_k) CUDA_TRY(cudaEventCreateWithFlags(&e, flags));
   }
   p->slot_free.resize(p->ring_slots);
   for (auto& e : p->slot_free) {
@@ -837,7 +861,7 @@ sti_status sti_shard_decode(sti_plan* p, int layer, sti_kind kind, int index, in
 
 sti_status sti_plan_set_profiling(sti_plan* p, int enabled) {
   if (!p) return STI_ERR_ARG;
-  p->profiling = enabled != 0;
+  p->profiling = enabled < 0 ? 0 : (enabled > 2 ? 2 : enabled);
   p->stats_valid = false;
   return STI_OK;
 }
@@ -866,6 +890,15 @@ sti_status sti_get_stats(sti_plan* p, sti_stats* out) {
       s.copy_us[l] = ms * 1e3f;
       CUDA_TRY(cudaEventElapsedTime(&t_loaded, p->ev_begin, L.ev_loaded));
       s.stall_us[l] = std::max(0.f, t_loaded - prev_done) * 1e3f;
+    }
+    if (p->profiling >= 2) {
+      float k[7] = {};
+      for (int i = 0; i < 7; ++i)
+        if (L.k_ran[i]) CUDA_TRY(cudaEventElapsedTime(&k[i], L.ev_k[i], L.ev_k[i + 1]));
+      s.gemm_us[l] = (k[0] + k[2] + k[4] + k[5]) * 1e3f;
+      s.attn_us[l] = k[1] * 1e3f;
+      s.ln_us[l] = (k[3] + k[6]) * 1e3f;
+      s.gemm_launches += (L.k_ran[0] ? 2 : 0) + (L.k_ran[4] ? 2 : 0);
     }
     s.streamed_bytes[l] = L.str_bytes;
     s.resident_bytes[l] = L.res_bytes;

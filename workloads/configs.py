@@ -58,7 +58,7 @@ def make_config(number: int, *, seed: int = 0, n_layers: Optional[int] = None,
                 batch: Optional[int] = None, seq: Optional[int] = None,
                 plan: str = "uniform3", resident: Optional[bool] = None,
                 resident_layers: Optional[int] = None, keep_originals: bool = False,
-                outlier_stress: float = 0.0) -> Workload:
+                outlier_stress: float = 0.0, workers: int = 1) -> Workload:
     """Workload for configuration 1..5.
 
     1  one BERT-base layer, batch 1, seq 128, every unit kept at 4 bits, fp32 activations
@@ -69,34 +69,35 @@ def make_config(number: int, *, seed: int = 0, n_layers: Optional[int] = None,
     5  BERT-large stack, batch/seq/plan given by the caller (`plan` is "uniform3" or "mixed"),
        bf16 activations, resident or streamed with a two-layer preload
 
-    `n_layers` shortens the stack (tests); `resident_layers` overrides the preload depth.
+    `n_layers` shortens the stack (tests); `resident_layers` overrides the preload depth;
+    `workers` > 1 quantizes layers in parallel processes (same result).
     """
     if number == 1:
         shape = BERT_BASE.with_layers(n_layers or 1)
         attn, ffn = _uniform_plan(shape, 4, shape.n_layers if resident_layers is None else resident_layers)
         return build_workload("cfg1_base_layer_4bit", shape, batch or 1, seq or 128, "f32", attn, ffn,
-                              seed=seed, keep_originals=keep_originals, outlier_stress=outlier_stress)
+                              seed=seed, keep_originals=keep_originals, outlier_stress=outlier_stress, workers=workers)
     if number == 2:
         shape = BERT_BASE.with_layers(n_layers or 1)
         attn, ffn = _random_plan(shape, _plan_rng(seed, 2),
                                  shape.n_layers if resident_layers is None else resident_layers,
                                  keep_heads=8, keep_slices=9)
         return build_workload("cfg2_base_layer_elastic", shape, batch or 1, seq or 128, "bf16", attn, ffn,
-                              seed=seed, keep_originals=keep_originals, outlier_stress=outlier_stress)
+                              seed=seed, keep_originals=keep_originals, outlier_stress=outlier_stress, workers=workers)
     if number == 3:
         shape = BERT_BASE.with_layers(n_layers or 12)
         attn, ffn = _random_plan(shape, _plan_rng(seed, 3), 3 if resident_layers is None else resident_layers,
                                  keep_frac_range=(0.6, 1.0))
         return build_workload("cfg3_base_model_streamed", shape, batch or 1, seq or 128, "f32", attn, ffn,
                               seed=seed, ring_slots=2, keep_originals=keep_originals,
-                              outlier_stress=outlier_stress)
+                              outlier_stress=outlier_stress, workers=workers)
     if number == 4:
         shape = BERT_LARGE.with_layers(n_layers or 24)
         attn, ffn = _random_plan(shape, _plan_rng(seed, 4), 2 if resident_layers is None else resident_layers,
                                  bit_values=_SKEW3_BITS, bit_p=_SKEW3_P)
         return build_workload("cfg4_large_model_streamed", shape, batch or 1, seq or 256, "f32", attn, ffn,
                               seed=seed, ring_slots=2, keep_originals=keep_originals,
-                              outlier_stress=outlier_stress)
+                              outlier_stress=outlier_stress, workers=workers)
     if number == 5:
         shape = BERT_LARGE.with_layers(n_layers or 24)
         res_layers = resident_layers
@@ -111,5 +112,5 @@ def make_config(number: int, *, seed: int = 0, n_layers: Optional[int] = None,
         b, s = batch or 1, seq or 128
         return build_workload(f"cfg5_large_b{b}_s{s}_{plan}_{'res' if res_layers >= shape.n_layers else 'str'}",
                               shape, b, s, "bf16", attn, ffn, seed=seed, ring_slots=2,
-                              keep_originals=keep_originals, outlier_stress=outlier_stress)
+                              keep_originals=keep_originals, outlier_stress=outlier_stress, workers=workers)
     raise ValueError("configuration number must be 1..5")
