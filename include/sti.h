@@ -189,6 +189,37 @@ sti_status sti_plan_memory(sti_plan* plan, uint64_t* preload_bytes, uint64_t* pi
  * Exposed so that the layout can be inspected and tested without a device. */
 sti_status sti_host_retile(const uint8_t* src, uint8_t* dst, uint32_t rows, uint32_t cols, uint32_t bits);
 
+/* (The paper has no counterpart to this call; it exists for callers that cannot allocate.)
+ * Decodes one matrix of a shard like sti_shard_decode, but without a context or a plan and without
+ * allocating anything, on the host or on the device.  It is meant for callers that must not call
+ * cudaMalloc: code running inside a process whose framework allocator already owns the device memory,
+ * integrity checks of shard files under an enforced memory budget, sections where the allocator's
+ * implicit device synchronisation is unwelcome.  The kernel's working copy of the shard (re-tiled
+ * index stream, centroid table, outlier lists) lives in a fixed array of STI_NOALLOC_SCRATCH_BYTES
+ * bytes inside the library image; each GPU that loads the library holds that array until exit.
+ *   device, stream : where to run; stream is a cudaStream_t or NULL for the default stream
+ *   bits           : 2..6                      rows, cols: the matrix shape, cols == 64 with rows % 64 == 0,
+ *                    or cols % 128 == 0 with rows % 32 == 0
+ *   codes          : HOST, the matrix's canonical index stream (rows*cols*bits/32 words)
+ *   centroids      : HOST, 2^bits entries
+ *   outlier_off/val: HOST, n_outliers pairs, offsets within the matrix, strictly ascending
+ *   w_dev, codes_dev, wbf16_dev : DEVICE outputs as in sti_shard_decode, caller-owned, any may be NULL
+ * Limits: rows*cols*bits/8 <= STI_NOALLOC_MAX_STREAM_BYTES and n_outliers <= STI_NOALLOC_MAX_OUTLIERS
+ * (every matrix of BERT-base and BERT-large at up to 6 bits fits); anything larger returns STI_ERR_SIZE
+ * and nothing runs.  Host inputs are consumed before the call returns; the kernel runs asynchronously
+ * on `stream`.  The first call on a device looks up the array's device address; make that first call
+ * before starting any stream capture.  All calls share the one array, which keeps the last call's
+ * contents (each call overwrites everything its kernel reads): calls on the same stream are ordered,
+ * calls whose GPU work can overlap (different streams or threads) race on it and must be serialised
+ * by the caller. */
+#define STI_NOALLOC_MAX_STREAM_BYTES 262144u
+#define STI_NOALLOC_MAX_OUTLIERS 4096u
+#define STI_NOALLOC_SCRATCH_BYTES (262144u + 256u + 2u * 4u * 4096u)
+sti_status sti_matrix_decode_noalloc(int device, void* stream, int bits, uint32_t rows, uint32_t cols,
+                                     const uint32_t* codes, const float* centroids,
+                                     const uint32_t* outlier_off, const float* outlier_val, size_t n_outliers,
+                                     float* w_dev, uint8_t* codes_dev, uint16_t* wbf16_dev);
+
 /* Kernel launches issued by the library on this context since creation (for accounting). */
 uint64_t sti_ctx_launch_count(sti_ctx* ctx);
 

@@ -87,6 +87,8 @@ def load_library():
         "sti_ctx_launch_count": ([vp], C.c_uint64),
         "sti_host_retile": ([vp, vp, C.c_uint32, C.c_uint32, C.c_uint32], i32),
         "sti_strerror": ([i32], C.c_char_p),
+        "sti_matrix_decode_noalloc": ([i32, vp, i32, C.c_uint32, C.c_uint32, vp, vp, vp, vp, C.c_size_t, vp, vp, vp],
+                                      i32),
     }
     for name, (argtypes, restype) in sigs.items():
         fn = getattr(lib, name)          # AttributeError if the library does not export it
@@ -100,7 +102,7 @@ EXPORTED = ("sti_ctx_create", "sti_ctx_destroy", "sti_ctx_set_layer_params", "st
             "sti_plan_destroy", "sti_shard_upload", "sti_plan_finalize", "sti_layer_forward",
             "sti_model_forward", "sti_model_forward_host", "sti_sync", "sti_shard_decode",
             "sti_plan_set_profiling", "sti_get_stats", "sti_plan_memory", "sti_ctx_launch_count",
-            "sti_host_retile", "sti_strerror")
+            "sti_host_retile", "sti_strerror", "sti_matrix_decode_noalloc")
 
 
 def _check(status: int, where: str):
@@ -227,6 +229,21 @@ def sti_host_retile(src: np.ndarray, rows: int, cols: int, bits: int) -> np.ndar
     dst = np.empty_like(src)
     _check(load_library().sti_host_retile(_ptr(src), _ptr(dst), rows, cols, bits), "sti_host_retile")
     return dst
+
+
+def sti_matrix_decode_noalloc(bits: int, rows: int, cols: int, codes: np.ndarray, centroids: np.ndarray,
+                              outlier_off: Optional[np.ndarray] = None, outlier_val: Optional[np.ndarray] = None,
+                              w_dev: int = 0, codes_dev: int = 0, wbf16_dev: int = 0, device: int = 0, stream: int = 0):
+    """Decode one shard matrix without a context, a plan or any allocation (see sti.h for who needs
+    that and for the size limits).  codes/centroids/outliers are host arrays, outputs device addresses."""
+    codes = _host(codes, np.uint32)
+    cent = _host(centroids, np.float32)
+    off = _host(outlier_off, np.uint32) if outlier_off is not None and len(outlier_off) else None
+    val = _host(outlier_val, np.float32) if outlier_val is not None and len(outlier_val) else None
+    _check(load_library().sti_matrix_decode_noalloc(
+        device, C.c_void_p(stream or None), int(bits), rows, cols, _ptr(codes), _ptr(cent), _ptr(off), _ptr(val),
+        0 if off is None else off.size, C.c_void_p(w_dev or None), C.c_void_p(codes_dev or None),
+        C.c_void_p(wbf16_dev or None)), "sti_matrix_decode_noalloc")
 
 
 class Session:
