@@ -49,6 +49,7 @@ struct GemmTable {
   Seg* segs = nullptr;
   int n_jobs = 0;
   size_t smem = 0;
+  uint32_t w_bytes = 0, n_stages = 0;
   int n_split = 0;
 };
 
@@ -102,6 +103,7 @@ struct sti_plan {
   // activation scratch
   uint16_t* qkv = nullptr; uint16_t* attn_out = nullptr; float* partial = nullptr;
   float* h1_f32 = nullptr; uint16_t* h1_bf16 = nullptr; uint16_t* u = nullptr;
+  uint16_t* x_bf16 = nullptr;          // bf16 copy of fp32 layer inputs (the GEMM operand)
   void* buf[2] = {nullptr, nullptr};
   void* x_in = nullptr; void* y_out = nullptr; int32_t* lens_dev = nullptr;
   int max_partial = 1;
@@ -175,10 +177,11 @@ void parse_tuning(Tuning* t, int tmax, const sti_model_desc& d) {
   t->o_group = std::max(1, std::min(t->o_group, 16));
   t->f2_group = std::max(1, std::min(t->f2_group, 16));
   // keep every weight tile inside shared memory
-  while (t->qkv_n > 32 && gemm_smem_bytes(t->qkv_n, d.hidden, 1) > kMaxSmem) t->qkv_n /= 2;
-  while (t->f1_n > 32 && gemm_smem_bytes(t->f1_n, d.hidden, 1) > kMaxSmem) t->f1_n /= 2;
-  while (t->o_group > 1 && gemm_smem_bytes(t->o_n, t->o_group * 64, t->o_group) > kMaxSmem) --t->o_group;
-  while (t->f2_group > 1 && gemm_smem_bytes(t->f2_n, t->f2_group * f, t->f2_group) > kMaxSmem) --t->f2_group;
+  auto fits = [](int n, int k) { return gemm_pick_stages(static_cast<uint32_t>(gemm_weight_bytes(n, k))) >= 4; };
+  while (t->qkv_n > 32 && !fits(t->qkv_n, d.hidden)) t->qkv_n /= 2;
+  while (t->f1_n > 32 && !fits(t->f1_n, d.hidden)) t->f1_n /= 2;
+  while (t->o_group > 1 && !fits(t->o_n, t->o_group * 64)) --t->o_group;
+  while (t->f2_group > 1 && !fits(t->f2_n, t->f2_group * f)) --t->f2_group;
 }
 
 Unit* find_unit(sti_plan* p, int layer, sti_kind kind, int index) {
@@ -215,13 +218,13 @@ Seg make_seg(const sti_ctx* c, const Unit& u, sti_kind kind, int m, uint32_t row
 struct TableBuilder {
   std::vector<Job> jobs;
   std::vector<Seg> segs;
-  size_t smem = 0;
+  uint32_t w_bytes = 0;
   void add(Job j, const std::vector<Seg>& ss) {
     j.seg_begin = static_cast<uint32_t>(segs.size());
     j.n_seg = static_cast<uint32_t>(ss.size());
     segs.insert(segs.end(), ss.begin(), ss.end());
     jobs.push_back(j);
-    smem = std::max(smem, gemm_smem_bytes(j.n_rows, j.k_total, j.n_seg));
+    w_bytes = std::max(w_bytes, static_cast<uint32_t>(gemm_weight_bytes(j.n_rows, j.k_total)));
   }
 };
 
@@ -308,14 +311,17 @@ sti_status run_gemm(sti_plan* p, GemmKind kind, const GemmTable& tab, const void
   GemmLaunch g{};
   g.jobs = tab.jobs; g.segs = tab.segs; g.n_jobs = tab.n_jobs; g.m_ctas = m_ctas_for(tab.n_jobs, T);
   g.x = x; g.ldx = ldx; g.T = T; g.out = out; g.ldo = ldo; g.bias = bias; g.err = p->ctx->err_dev;
-  g.smem_bytes = tab.smem; g.simt_debug = p->ctx->simt_debug;
+  g.smem_bytes = tab.smem; g.n_stages = tab.n_stages; g.w_bytes = tab.w_bytes; g.simt_debug = p->ctx->simt_debug;
   CUDA_TRY(launch_gemm(kind, g, p->ctx->compute));
   p->ctx->launches++;
   return STI_OK;
 }
 
 // The seven kernels of one layer on the compute stream.
-sti_status enqueue_layer(sti_plan* p, int li, const void* x, void* y, int batch, int seq, const int32_t* lens) {
+// `x_ready_bf16`: the bf16 copy of x already sits in p->x_bf16 (written by the previous layer's LayerNorm);
+// `want_next_bf16`: this layer's last kernel also writes y as bf16 into p->x_bf16 for the next layer.
+sti_status enqueue_layer(sti_plan* p, int li, const void* x, void* y, int batch, int seq, const int32_t* lens,
+                         bool x_ready_bf16, bool want_next_bf16) {
   sti_ctx* c = p->ctx;
   const sti_model_desc& d = c->desc;
   Layer& L = p->layers[li];
@@ -330,8 +336,17 @@ sti_status enqueue_layer(sti_plan* p, int li, const void* x, void* y, int batch,
   for (bool& r : L.k_ran) r = false;
   CUDA_TRY(mark(0));
   if (nh > 0) {
-    st = run_gemm(p, bf16_act ? GEMM_BF16_TO_BF16 : GEMM_F32_TO_BF16, L.qkv, x, d.hidden, T, p->qkv, 64,
-                  dense + c->off_bq);
+    const void* xq = x;
+    if (!bf16_act) {
+      // the GEMMs take bf16 operands: fp32 activations are rounded once (round-to-nearest-even)
+      if (!x_ready_bf16) {
+        CUDA_TRY(launch_cast_bf16(static_cast<const float*>(x), p->x_bf16, static_cast<size_t>(T) * d.hidden,
+                                  c->compute));
+        c->launches++;
+      }
+      xq = p->x_bf16;
+    }
+    st = run_gemm(p, GEMM_BF16_TO_BF16, L.qkv, xq, d.hidden, T, p->qkv, 64, dense + c->off_bq);
     if (st != STI_OK) return st;
     CUDA_TRY(mark(1));
     CUDA_TRY(launch_attention(p->qkv, p->attn_out, nh, batch, seq, lens, c->compute));
@@ -370,7 +385,7 @@ sti_status enqueue_layer(sti_plan* p, int li, const void* x, void* y, int batch,
   l2.bias = dense + c->off_b2; l2.resid = p->h1_f32; l2.resid_bf16 = 0;
   l2.gamma = dense + c->off_ln2g; l2.beta = dense + c->off_ln2b; l2.eps = d.ln_eps; l2.T = T; l2.d = d.hidden;
   l2.out_f32 = bf16_act ? nullptr : static_cast<float*>(y);
-  l2.out_bf16 = bf16_act ? static_cast<uint16_t*>(y) : nullptr;
+  l2.out_bf16 = bf16_act ? static_cast<uint16_t*>(y) : (want_next_bf16 ? p->x_bf16 : nullptr);
   CUDA_TRY(launch_layernorm(l2, c->compute));
   c->launches++;
   L.k_ran[6] = true;
@@ -416,7 +431,7 @@ sti_status model_forward_impl(sti_plan* p, const void* x, void* y, int batch, in
     }
     if (p->profiling) CUDA_TRY(cudaEventRecord(L.ev_comp_start, c->compute));
     void* nxt = (li == n - 1) ? y : p->buf[li & 1];
-    sti_status st = enqueue_layer(p, li, cur, nxt, batch, seq, lens);
+    sti_status st = enqueue_layer(p, li, cur, nxt, batch, seq, lens, li > 0, li + 1 < n);
     if (st != STI_OK) return st;
     if (p->profiling) CUDA_TRY(cudaEventRecord(L.ev_done, c->compute));
     if (L.str_bytes > 0) CUDA_TRY(cudaEventRecord(p->slot_free[L.slot], c->compute));
@@ -436,7 +451,7 @@ void free_plan_device(sti_plan* p) {
   cudaFree(p->preload); cudaFree(p->ring); cudaFree(p->tables);
   if (p->pinned) cudaFreeHost(p->pinned);
   cudaFree(p->qkv); cudaFree(p->attn_out); cudaFree(p->partial); cudaFree(p->h1_f32); cudaFree(p->h1_bf16);
-  cudaFree(p->u); cudaFree(p->buf[0]); cudaFree(p->buf[1]); cudaFree(p->x_in); cudaFree(p->y_out);
+  cudaFree(p->u); cudaFree(p->x_bf16); cudaFree(p->buf[0]); cudaFree(p->buf[1]); cudaFree(p->x_in); cudaFree(p->y_out);
   cudaFree(p->lens_dev);
   for (auto& L : p->layers) {
     if (L.ev_loaded) cudaEventDestroy(L.ev_loaded);
@@ -720,8 +735,11 @@ sti_status sti_plan_finalize(sti_plan* p) {
     GemmTable* gt[4] = {&L.qkv, &L.o, &L.f1, &L.f2};
     for (int i = 0; i < 4; ++i) {
       gt[i]->n_jobs = static_cast<int>(tb[i].jobs.size());
-      gt[i]->smem = tb[i].smem;
-      if (tb[i].smem > kMaxSmem) return STI_ERR_SHAPE;
+      gt[i]->w_bytes = tb[i].w_bytes;
+      gt[i]->n_stages = gemm_pick_stages(tb[i].w_bytes);
+      if (!tb[i].jobs.empty() && gt[i]->n_stages < 3) return STI_ERR_SHAPE;
+      gt[i]->smem = gemm_smem_bytes(tb[i].w_bytes, std::max(3u, gt[i]->n_stages));
+      if (gt[i]->smem > kMaxSmem && !tb[i].jobs.empty()) return STI_ERR_SHAPE;
       Fix fx{gt[i], 0, 0};
       fx.jobs_off = align16(host_tables.size());
       host_tables.resize(fx.jobs_off + tb[i].jobs.size() * sizeof(Job));
@@ -750,6 +768,7 @@ sti_status sti_plan_finalize(sti_plan* p) {
   CUDA_TRY(cudaMalloc(&p->h1_f32, Tmax * d.hidden * 4));
   CUDA_TRY(cudaMalloc(&p->h1_bf16, Tmax * d.hidden * 2));
   CUDA_TRY(cudaMalloc(&p->u, std::max<size_t>(1, max_slices) * Tmax * f * 2));
+  CUDA_TRY(cudaMalloc(&p->x_bf16, Tmax * d.hidden * 2));
   CUDA_TRY(cudaMalloc(&p->buf[0], Tmax * d.hidden * act_size(c)));
   CUDA_TRY(cudaMalloc(&p->buf[1], Tmax * d.hidden * act_size(c)));
   CUDA_TRY(cudaMalloc(&p->x_in, Tmax * d.hidden * act_size(c)));
@@ -790,7 +809,7 @@ sti_status sti_layer_forward(sti_plan* p, int layer, const void* x, void* y, int
     if (p->copy_tail_valid) CUDA_TRY(cudaStreamWaitEvent(c->compute, p->ev_copy_tail, 0));
     if ((st = enqueue_layer_copy(p, layer, c->compute)) != STI_OK) return st;
   }
-  if ((st = enqueue_layer(p, layer, x, y, batch, seq, lens)) != STI_OK) return st;
+  if ((st = enqueue_layer(p, layer, x, y, batch, seq, lens, false, false)) != STI_OK) return st;
   if (L.str_bytes > 0) CUDA_TRY(cudaEventRecord(p->slot_free[L.slot], c->compute));
   return STI_OK;
 }

@@ -2,7 +2,8 @@
 // independently contributes one representation; Section 4.2: any subset of heads executes).
 //
 // One CTA = (64-query tile, kept head, sequence); 4 warps x 16 query rows.  K and V of the whole
-// sequence (<= 512 keys) sit in shared memory; scores and the probability-value product run on
+// sequence (<= 512 keys) are brought into shared memory with cp.async (row-major, padded rows; the
+// value fragments are read with ldmatrix.trans); scores and the probability-value product run on
 // mma.sync m16n8k16 bf16 with fp32 accumulation, softmax is done in registers with warp shuffles
 // over the four lanes that share a row (online max/sum over 64-key blocks).
 // Attention is ~3 % of a layer's FLOPs at seq 128; the dense projections use tcgen05 (dqgemm.cu).
@@ -25,6 +26,16 @@ __device__ __forceinline__ void mma_bf16_16816(float (&c)[4], const uint32_t (&a
       : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
 }
 
+__device__ __forceinline__ void cp_async16(uint32_t dst, const void* src, uint32_t src_bytes) {
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "r"(src_bytes) : "memory");
+}
+
+// Two 8x8 bf16 matrices, transposed on the way in: with rows = keys this yields the B fragment
+// (k = key, n = head-dim column) of m16n8k16.  Lanes 0-7 / 8-15 give the row addresses.
+__device__ __forceinline__ void ldmatrix_x2_trans(uint32_t addr, uint32_t& r0, uint32_t& r1) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x2.trans.shared.b16 {%0, %1}, [%2];" : "=r"(r0), "=r"(r1) : "r"(addr));
+}
+
 __global__ void __launch_bounds__(128)
 attention_kernel(const uint16_t* __restrict__ qkv, uint16_t* __restrict__ out, int n_kept, int batch, int L,
                  const int32_t* __restrict__ seq_lens) {
@@ -34,9 +45,8 @@ attention_kernel(const uint16_t* __restrict__ qkv, uint16_t* __restrict__ out, i
   const int g = lane >> 2, t4 = lane & 3;
   const int T = batch * L;
   const int Lpad = (L + 63) / 64 * 64;
-  const int vstride = Lpad + 8;
   uint16_t* Ks = reinterpret_cast<uint16_t*>(smem);                       // [Lpad][72]
-  uint16_t* Vt = Ks + static_cast<size_t>(Lpad) * kKStride;               // [64][Lpad + 8]
+  uint16_t* Vs = Ks + static_cast<size_t>(Lpad) * kKStride;               // [Lpad][72]
 
   const uint16_t* Qg = qkv + (static_cast<size_t>(hi * 3 + 0) * T + static_cast<size_t>(b) * L) * kHeadDim;
   const uint16_t* Kg = qkv + (static_cast<size_t>(hi * 3 + 1) * T + static_cast<size_t>(b) * L) * kHeadDim;
@@ -48,22 +58,17 @@ attention_kernel(const uint16_t* __restrict__ qkv, uint16_t* __restrict__ out, i
     valid = valid < 0 ? 0 : (valid > L ? L : valid);
   }
 
+  // K and V rows: every 16-byte piece is its own cp.async, all in flight at once; rows past L are zero
+  const uint32_t ks_addr = smem_addr(Ks), vs_addr = smem_addr(Vs);
   for (int idx = tid; idx < Lpad * 8; idx += 128) {
     const int key = idx >> 3, piece = idx & 7;
-    uint4 v = make_uint4(0, 0, 0, 0);
-    if (key < L) v = __ldg(reinterpret_cast<const uint4*>(Kg + static_cast<size_t>(key) * kHeadDim + piece * 8));
-    *reinterpret_cast<uint4*>(Ks + static_cast<size_t>(key) * kKStride + piece * 8) = v;
+    const bool ok = key < L;
+    const size_t goff = static_cast<size_t>(ok ? key : 0) * kHeadDim + piece * 8;
+    const uint32_t soff = static_cast<uint32_t>(key * kKStride + piece * 8) * 2;
+    cp_async16(ks_addr + soff, Kg + goff, ok ? 16u : 0u);
+    cp_async16(vs_addr + soff, Vg + goff, ok ? 16u : 0u);
   }
-  for (int idx = tid; idx < Lpad * 8; idx += 128) {
-    const int key = idx % Lpad, piece = idx / Lpad;      // consecutive lanes -> consecutive keys
-    uint4 v = make_uint4(0, 0, 0, 0);
-    if (key < L) v = __ldg(reinterpret_cast<const uint4*>(Vg + static_cast<size_t>(key) * kHeadDim + piece * 8));
-    const uint32_t w[4] = {v.x, v.y, v.z, v.w};
-#pragma unroll
-    for (int i = 0; i < 8; ++i)
-      Vt[static_cast<size_t>(piece * 8 + i) * vstride + key] = static_cast<uint16_t>(w[i >> 1] >> ((i & 1) * 16));
-  }
-  __syncthreads();
+  asm volatile("cp.async.commit_group;" ::: "memory");
 
   // query fragments of this warp's 16 rows
   const int q0 = qt * kQTile + warp * 16;
@@ -77,6 +82,9 @@ attention_kernel(const uint16_t* __restrict__ qkv, uint16_t* __restrict__ out, i
     qa[kk][2] = r0 < L ? __ldg(reinterpret_cast<const uint32_t*>(Qg + static_cast<size_t>(r0) * kHeadDim + c + 8)) : 0u;
     qa[kk][3] = r1 < L ? __ldg(reinterpret_cast<const uint32_t*>(Qg + static_cast<size_t>(r1) * kHeadDim + c + 8)) : 0u;
   }
+
+  asm volatile("cp.async.wait_group 0;" ::: "memory");
+  __syncthreads();
 
   const float scale_log2 = 0.125f * 1.4426950408889634f;     // 1/sqrt(64) * log2(e)
   float o[8][4];
@@ -139,11 +147,12 @@ attention_kernel(const uint16_t* __restrict__ qkv, uint16_t* __restrict__ out, i
       pa[1] = pack_bf16x2(s[2 * kk][2], s[2 * kk][3]);
       pa[2] = pack_bf16x2(s[2 * kk + 1][0], s[2 * kk + 1][1]);
       pa[3] = pack_bf16x2(s[2 * kk + 1][2], s[2 * kk + 1][3]);
+      // lanes 0-15 address the 16 key rows of this k-step (8 rows per 8x8 matrix)
+      const uint32_t vrow = vs_addr + static_cast<uint32_t>((kb * 64 + kk * 16 + (lane & 15)) * kKStride) * 2;
 #pragma unroll
       for (int jd = 0; jd < 8; ++jd) {
-        const uint16_t* vrow = Vt + static_cast<size_t>(jd * 8 + g) * vstride + kb * 64 + kk * 16 + 2 * t4;
-        const uint32_t b0 = *reinterpret_cast<const uint32_t*>(vrow);
-        const uint32_t b1 = *reinterpret_cast<const uint32_t*>(vrow + 8);
+        uint32_t b0, b1;
+        ldmatrix_x2_trans(vrow + jd * 16, b0, b1);
         mma_bf16_16816(o[jd], pa, b0, b1);
       }
     }
@@ -172,7 +181,7 @@ attention_kernel(const uint16_t* __restrict__ qkv, uint16_t* __restrict__ out, i
 
 size_t attn_smem_bytes(int L) {
   const int Lpad = (L + 63) / 64 * 64;
-  return (static_cast<size_t>(Lpad) * kKStride + static_cast<size_t>(kHeadDim) * (Lpad + 8)) * 2;
+  return static_cast<size_t>(Lpad) * kKStride * 2 * 2;      // K and V, padded rows
 }
 
 }  // namespace

@@ -4,7 +4,8 @@
 // One CTA owns a weight tile (n_rows output features x k_total input features), decodes it ONCE
 // into shared memory as bf16 (index unpack in registers -> per-unit centroid table in shared
 // memory -> outlier patch), and then streams 128-token activation tiles past it:
-//   activation chunk [128 x 64] -> shared memory (bf16, K-major core-matrix layout)
+//   activation chunk [128 x 64] bf16 -> shared memory with cp.async, several chunks in flight
+//   (K-major core-matrix layout), issued before the decode so that their latency hides behind it
 //   tcgen05.mma (M = 128 tokens, N = n_rows, K = 16 per instruction), fp32 accumulator in TMEM
 //   epilogue: tcgen05.ld -> bias / GELU -> global.
 //
@@ -26,19 +27,19 @@ constexpr int kThreads = 256;
 constexpr int kWarps = kThreads / 32;
 constexpr int kTileM = 128;                 // tokens per MMA tile
 constexpr int kChunkK = 64;                 // activation K per pipeline stage
-constexpr int kStages = 3;
+constexpr int kMaxStages = 8;
 constexpr int kStageBytes = kTileM * kChunkK * 2;   // 16 KB
+constexpr int kHeaderBytes = 3072;          // barriers + segment tables
+constexpr int kRefillLag = 2;               // a stage is refilled two chunks after its MMAs were issued
 constexpr int kMaxSegs = 16;
 constexpr int kTableStride = 64;            // bf16 entries per segment table
 
 struct SmemHeader {
-  uint64_t mma_done[kStages];
+  uint64_t mma_done[kMaxStages];
   uint64_t acc_full;
   uint32_t tmem_base;
   uint32_t pad;
 };
-
-__host__ __device__ inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
 // ---------------------------------------------------------------------------------------
 // Weight-tile decode
@@ -93,34 +94,49 @@ __device__ __forceinline__ void decode_raw(const Seg& sg, uint8_t* wsm, uint32_t
 // ---------------------------------------------------------------------------------------
 // Activation chunk: rows [m0, m0+128) x columns [k0, k0+64) -> stage buffer
 // ---------------------------------------------------------------------------------------
-template <typename XT>
-__device__ __forceinline__ void load_x_chunk(const XT* __restrict__ x, int ldx, int T, int m0, int k0,
-                                             uint8_t* stage, uint32_t tid) {
+__device__ __forceinline__ void cp_async16_zfill(uint32_t dst, const void* src, uint32_t src_bytes) {
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "r"(src_bytes) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
+
+// Asynchronous version: 4 x 16 bytes per thread, rows past T are zero-filled.  Within a quarter warp
+// the lanes hold 8 consecutive rows of one 16-byte column piece = 128 contiguous bytes of the stage.
+__device__ __forceinline__ void load_x_chunk_async(const __nv_bfloat16* __restrict__ x, int ldx, int T, int m0, int k0,
+                                                   uint32_t stage_addr, uint32_t tid) {
   const uint32_t lane = tid & 31;
 #pragma unroll
   for (int i = 0; i < (kTileM * (kChunkK / 8)) / kThreads; ++i) {
     const uint32_t u = (i * kThreads + tid) >> 5;          // warp-level unit, 0..31
     const uint32_t row = (u & 15) * 8 + (lane & 7);
     const uint32_t piece = (u >> 4) * 4 + (lane >> 3);
+    const int t = m0 + static_cast<int>(row);
+    const bool ok = t < T;
+    const __nv_bfloat16* src = ok ? x + static_cast<size_t>(t) * ldx + k0 + piece * 8 : x;
+    cp_async16_zfill(stage_addr + piece * (kTileM * 16) + row * 16, src, ok ? 16u : 0u);
+  }
+}
+
+// Synchronous version (debug path).
+__device__ __forceinline__ void load_x_chunk(const __nv_bfloat16* __restrict__ x, int ldx, int T, int m0, int k0,
+                                             uint8_t* stage, uint32_t tid) {
+  const uint32_t lane = tid & 31;
+#pragma unroll
+  for (int i = 0; i < (kTileM * (kChunkK / 8)) / kThreads; ++i) {
+    const uint32_t u = (i * kThreads + tid) >> 5;
+    const uint32_t row = (u & 15) * 8 + (lane & 7);
+    const uint32_t piece = (u >> 4) * 4 + (lane >> 3);
     uint4 v = make_uint4(0, 0, 0, 0);
     const int t = m0 + static_cast<int>(row);
-    if (t < T) {
-      const XT* src = x + static_cast<size_t>(t) * ldx + k0 + piece * 8;
-      if constexpr (sizeof(XT) == 2) {
-        v = __ldg(reinterpret_cast<const uint4*>(src));
-      } else {
-        const float4 a = __ldg(reinterpret_cast<const float4*>(src));
-        const float4 b = __ldg(reinterpret_cast<const float4*>(src) + 1);
-        v = make_uint4(pack_bf16x2(a.x, a.y), pack_bf16x2(a.z, a.w), pack_bf16x2(b.x, b.y), pack_bf16x2(b.z, b.w));
-      }
-    }
+    if (t < T) v = __ldg(reinterpret_cast<const uint4*>(x + static_cast<size_t>(t) * ldx + k0 + piece * 8));
     *reinterpret_cast<uint4*>(stage + piece * (kTileM * 16) + row * 16) = v;
   }
 }
 
 __device__ __forceinline__ float gelu_erf(float v) { return 0.5f * v * (1.0f + erff(v * 0.70710678118654752440f)); }
 
-template <typename OutT, bool GELU>
+template <typename OutT>
 __device__ __forceinline__ void store_row16(OutT* dst, const float (&v)[16]) {
   if constexpr (sizeof(OutT) == 2) {
     uint32_t p[8];
@@ -138,38 +154,56 @@ __device__ __forceinline__ void store_row16(OutT* dst, const float (&v)[16]) {
 // ---------------------------------------------------------------------------------------
 // The kernel
 // ---------------------------------------------------------------------------------------
-template <typename XT, typename OutT, bool GELU, bool SIMT>
+template <typename OutT, bool GELU, bool SIMT>
 __global__ void __launch_bounds__(kThreads, 1)
-dqgemm_kernel(const Job* __restrict__ jobs, const Seg* __restrict__ segs, const XT* __restrict__ x, int ldx, int T,
-              OutT* __restrict__ out, int ldo, const float* __restrict__ bias, int* __restrict__ err) {
+dqgemm_kernel(const Job* __restrict__ jobs, const Seg* __restrict__ segs, const __nv_bfloat16* __restrict__ x, int ldx,
+              int T, OutT* __restrict__ out, int ldo, const float* __restrict__ bias, int* __restrict__ err,
+              uint32_t n_stages, uint32_t w_bytes) {
   extern __shared__ __align__(1024) uint8_t smem[];
   const uint32_t tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const Job job = jobs[blockIdx.x];
   const uint32_t n_rows = job.n_rows, k_total = job.k_total;
 
   SmemHeader* hdr = reinterpret_cast<SmemHeader*>(smem);
-  uint16_t* tables = reinterpret_cast<uint16_t*>(smem + 128);                       // [kMaxSegs][64]
-  uint8_t* xsm = smem + align_up(128 + kMaxSegs * kTableStride * 2, 1024);
-  uint8_t* wsm = xsm + kStages * kStageBytes;
+  uint16_t* tables = reinterpret_cast<uint16_t*>(smem + 256);                       // [kMaxSegs][64]
+  uint8_t* wsm = smem + kHeaderBytes;
+  uint8_t* xsm = wsm + w_bytes;                                                      // n_stages x 16 KB
 
   // the kernel's own checks of the descriptor: refuse rather than touch memory out of bounds
   const bool bad = job.n_seg == 0 || job.n_seg > kMaxSegs || (n_rows != 32 && n_rows != 64 && n_rows != 128) ||
-                   (k_total % kChunkK) != 0 || k_total == 0;
+                   (k_total % kChunkK) != 0 || k_total == 0 || n_rows * k_total * 2 > w_bytes ||
+                   n_stages < kRefillLag + 1 || n_stages > kMaxStages;
   if (bad) {
     if (tid == 0) atomicCAS(err, ERR_NONE, ERR_BAD_JOB);
     return;
   }
 
+  const int n_mtiles = (T + kTileM - 1) / kTileM;
+  const uint32_t n_chunks = k_total / kChunkK;
+  const uint32_t my_mtiles = blockIdx.y < static_cast<uint32_t>(n_mtiles)
+                                 ? (n_mtiles - blockIdx.y + gridDim.y - 1) / gridDim.y : 0;
+  const uint32_t total = my_mtiles * n_chunks;          // activation chunks this CTA consumes
+  const uint32_t xsm_addr = smem_addr(xsm);
+  auto issue_chunk = [&](uint32_t c) {
+    const int m0 = (blockIdx.y + (c / n_chunks) * gridDim.y) * kTileM;
+    load_x_chunk_async(x, ldx, T, m0, job.x_koff + (c % n_chunks) * kChunkK,
+                       xsm_addr + (c % n_stages) * kStageBytes, tid);
+  };
+
   uint32_t tmem_cols = 32;
   while (tmem_cols < n_rows) tmem_cols <<= 1;
   if constexpr (!SIMT) {
+    // activations first: n_stages - kRefillLag chunks in flight while the weights are decoded
+    for (uint32_t c = 0; c < n_stages - kRefillLag; ++c) {
+      if (c < total) issue_chunk(c);
+      cp_async_commit();
+    }
     if (warp == 0) {
       tmem_alloc(smem_addr(&hdr->tmem_base), tmem_cols);
       tmem_relinquish();
     }
     if (tid == 0) {
-#pragma unroll
-      for (int s = 0; s < kStages; ++s) mbar_init(smem_addr(&hdr->mma_done[s]), 1);
+      for (uint32_t s = 0; s < n_stages; ++s) mbar_init(smem_addr(&hdr->mma_done[s]), 1);
       mbar_init(smem_addr(&hdr->acc_full), 1);
       mbar_fence_init();
     }
@@ -225,25 +259,17 @@ dqgemm_kernel(const Job* __restrict__ jobs, const Seg* __restrict__ segs, const 
     __syncthreads();
   }
 
-  const int n_mtiles = (T + kTileM - 1) / kTileM;
-  const uint32_t n_chunks = k_total / kChunkK;
-  const uint32_t idesc = umma_idesc_bf16_m128(n_rows);
-  const uint32_t w_lbo = n_rows * 16;
-  uint32_t it = 0;           // activation chunks consumed so far by this CTA
-  uint32_t acc_phase = 0;
-  bool failed = false;
-
-  for (int mt = blockIdx.y; mt < n_mtiles; mt += gridDim.y) {
-    const int m0 = mt * kTileM;
-    if constexpr (SIMT) {
-      // Debug path: the same shared-memory tiles multiplied on the plain ALUs.
+  if constexpr (SIMT) {
+    // Debug path: the same shared-memory tiles multiplied on the plain ALUs.
+    for (int mt = blockIdx.y; mt < n_mtiles; mt += gridDim.y) {
+      const int m0 = mt * kTileM;
       const uint32_t row = tid & 127, chalf = tid >> 7, ncol = n_rows / 2;
       float acc[64];
 #pragma unroll
       for (int c = 0; c < 64; ++c) acc[c] = 0.f;
       for (uint32_t kc = 0; kc < n_chunks; ++kc) {
         __syncthreads();
-        load_x_chunk<XT>(x, ldx, T, m0, job.x_koff + kc * kChunkK, xsm, tid);
+        load_x_chunk(x, ldx, T, m0, job.x_koff + kc * kChunkK, xsm, tid);
         __syncthreads();
         for (uint32_t kk = 0; kk < kChunkK; ++kk) {
           const float a = __bfloat162float(
@@ -272,42 +298,60 @@ dqgemm_kernel(const Job* __restrict__ jobs, const Seg* __restrict__ segs, const 
               v[c] = GELU ? gelu_erf(a) : a;
             }
             OutT* dst = out + (static_cast<size_t>(job.out_mat) * T + t) * ldo + job.out_col + chalf * ncol + cb * 16;
-            store_row16<OutT, GELU>(dst, v);
+            store_row16<OutT>(dst, v);
           }
         }
       }
-    } else {
-      for (uint32_t kc = 0; kc < n_chunks; ++kc, ++it) {
-        const uint32_t stage = it % kStages, use = it / kStages;
-        if (use > 0 && !failed) {
-          // the MMAs that read this stage on its previous use must be done before it is overwritten
-          if (!mbar_wait_bounded(smem_addr(&hdr->mma_done[stage]), (use - 1) & 1)) failed = true;
-        }
-        if (__syncthreads_or(failed)) { failed = true; break; }
-        uint8_t* stage_ptr = xsm + stage * kStageBytes;
-        load_x_chunk<XT>(x, ldx, T, m0, job.x_koff + kc * kChunkK, stage_ptr, tid);
-        fence_proxy_async_smem();
-        __syncthreads();
-        if (tid == 0) {
-          tc_fence_after_sync();
-          const uint32_t a_base = smem_addr(stage_ptr);
-          const uint32_t b_base = smem_addr(wsm) + (kc * (kChunkK / 8)) * w_lbo;
+    }
+  } else {
+    const uint32_t idesc = umma_idesc_bf16_m128(n_rows);
+    const uint32_t w_lbo = n_rows * 16;
+    const uint32_t wsm_addr = smem_addr(wsm);
+    uint32_t acc_phase = 0;
+    uint32_t issued = 0;       // chunks whose MMAs have been issued
+    bool failed = false;
+    for (uint32_t c = 0; c < total; ++c) {
+      const uint32_t kc = c % n_chunks;
+      // refill: chunk c + S - L goes into the stage that chunk c - L used; its MMAs were issued L iterations ago
+      const uint32_t nxt = c + n_stages - kRefillLag;
+      if (nxt < total && c >= kRefillLag && !failed) {
+        const uint32_t prev = c - kRefillLag;
+        if (!mbar_wait_bounded(smem_addr(&hdr->mma_done[prev % n_stages]), (prev / n_stages) & 1)) failed = true;
+      }
+      if (nxt < total && !failed) issue_chunk(nxt);
+      cp_async_commit();
+      // chunk c is complete once at most (n_stages - kRefillLag) newer groups are pending
+      switch (n_stages - kRefillLag) {
+        case 1: cp_async_wait<1>(); break;
+        case 2: cp_async_wait<2>(); break;
+        case 3: cp_async_wait<3>(); break;
+        case 4: cp_async_wait<4>(); break;
+        case 5: cp_async_wait<5>(); break;
+        default: cp_async_wait<6>(); break;
+      }
+      fence_proxy_async_smem();
+      if (__syncthreads_or(failed)) { failed = true; break; }
+      if (tid == 0) {
+        tc_fence_after_sync();
+        const uint32_t a_base = xsm_addr + (c % n_stages) * kStageBytes;
+        const uint32_t b_base = wsm_addr + (kc * (kChunkK / 8)) * w_lbo;
 #pragma unroll
-          for (int ks = 0; ks < kChunkK / 16; ++ks) {
-            const uint64_t da = umma_smem_desc(a_base + ks * 2 * (kTileM * 16), kTileM * 16, 128);
-            const uint64_t db = umma_smem_desc(b_base + ks * 2 * w_lbo, w_lbo, 128);
-            umma_bf16_ss(tmem_base, da, db, idesc, (kc | ks) != 0 ? 1u : 0u);
-          }
-          umma_commit(smem_addr(&hdr->mma_done[stage]));
-          if (kc + 1 == n_chunks) umma_commit(smem_addr(&hdr->acc_full));
+        for (int ks = 0; ks < kChunkK / 16; ++ks) {
+          const uint64_t da = umma_smem_desc(a_base + ks * 2 * (kTileM * 16), kTileM * 16, 128);
+          const uint64_t db = umma_smem_desc(b_base + ks * 2 * w_lbo, w_lbo, 128);
+          umma_bf16_ss(tmem_base, da, db, idesc, (kc | ks) != 0 ? 1u : 0u);
         }
+        umma_commit(smem_addr(&hdr->mma_done[c % n_stages]));
+        if (kc + 1 == n_chunks) umma_commit(smem_addr(&hdr->acc_full));
       }
-      if (failed) break;
-      // ---- epilogue: accumulator -> registers -> global
+      issued = c + 1;
+      if (kc + 1 != n_chunks) continue;
+      // ---- epilogue of this token tile: accumulator -> registers -> global
       if (!mbar_wait_bounded(smem_addr(&hdr->acc_full), acc_phase)) failed = true;
       acc_phase ^= 1;
       if (__syncthreads_or(failed)) { failed = true; break; }
       tc_fence_after_sync();
+      const int m0 = (blockIdx.y + (c / n_chunks) * gridDim.y) * kTileM;
       const uint32_t q = warp & 3, chalf = warp >> 2, ncol = n_rows / 2;
       const int t = m0 + static_cast<int>(q * 32 + lane);
       for (uint32_t c0 = 0; c0 < ncol; c0 += 16) {
@@ -318,27 +362,25 @@ dqgemm_kernel(const Job* __restrict__ jobs, const Seg* __restrict__ segs, const 
         if (t < T) {
           float v[16];
 #pragma unroll
-          for (int c = 0; c < 16; ++c) {
-            float a = __uint_as_float(r[c]);
-            if (job.bias_off >= 0) a += __ldg(bias + job.bias_off + col + c);
-            v[c] = GELU ? gelu_erf(a) : a;
+          for (int i = 0; i < 16; ++i) {
+            float a = __uint_as_float(r[i]);
+            if (job.bias_off >= 0) a += __ldg(bias + job.bias_off + col + i);
+            v[i] = GELU ? gelu_erf(a) : a;
           }
           OutT* dst = out + (static_cast<size_t>(job.out_mat) * T + t) * ldo + job.out_col + col;
-          store_row16<OutT, GELU>(dst, v);
+          store_row16<OutT>(dst, v);
         }
       }
       tc_fence_before_sync();
       __syncthreads();        // all accumulator reads done before the next tile's first MMA overwrites it
     }
-  }
-
-  if constexpr (!SIMT) {
+    cp_async_wait<0>();       // no copy of this CTA may still be in flight when it exits
     if (failed && tid == 0) atomicCAS(err, ERR_NONE, ERR_WAIT_TIMEOUT);
     // Every MMA this CTA issued has completed (acc_full was waited for after the last tile) unless a
     // wait ran out; in that case give outstanding MMAs one more bounded chance before freeing TMEM.
-    if (failed && it > 0) {
-      const uint32_t last = (it - 1) % kStages, use = (it - 1) / kStages;
-      (void)mbar_wait_bounded(smem_addr(&hdr->mma_done[last]), use & 1);
+    if (failed && issued > 0) {
+      const uint32_t last = issued - 1;
+      (void)mbar_wait_bounded(smem_addr(&hdr->mma_done[last % n_stages]), (last / n_stages) & 1);
     }
     tc_fence_before_sync();
     __syncthreads();
@@ -346,15 +388,16 @@ dqgemm_kernel(const Job* __restrict__ jobs, const Seg* __restrict__ segs, const 
   }
 }
 
-template <typename XT, typename OutT, bool GELU>
+template <typename OutT, bool GELU>
 cudaError_t launch_t(const GemmLaunch& p, cudaStream_t s) {
   dim3 grid(p.n_jobs, p.m_ctas), block(kThreads);
+  const __nv_bfloat16* x = static_cast<const __nv_bfloat16*>(p.x);
   if (p.simt_debug)
-    dqgemm_kernel<XT, OutT, GELU, true><<<grid, block, p.smem_bytes, s>>>(
-        p.jobs, p.segs, static_cast<const XT*>(p.x), p.ldx, p.T, static_cast<OutT*>(p.out), p.ldo, p.bias, p.err);
+    dqgemm_kernel<OutT, GELU, true><<<grid, block, p.smem_bytes, s>>>(
+        p.jobs, p.segs, x, p.ldx, p.T, static_cast<OutT*>(p.out), p.ldo, p.bias, p.err, p.n_stages, p.w_bytes);
   else
-    dqgemm_kernel<XT, OutT, GELU, false><<<grid, block, p.smem_bytes, s>>>(
-        p.jobs, p.segs, static_cast<const XT*>(p.x), p.ldx, p.T, static_cast<OutT*>(p.out), p.ldo, p.bias, p.err);
+    dqgemm_kernel<OutT, GELU, false><<<grid, block, p.smem_bytes, s>>>(
+        p.jobs, p.segs, x, p.ldx, p.T, static_cast<OutT*>(p.out), p.ldo, p.bias, p.err, p.n_stages, p.w_bytes);
   return cudaGetLastError();
 }
 
@@ -365,30 +408,35 @@ cudaError_t set_smem(K kernel) {
 
 }  // namespace
 
-size_t gemm_smem_bytes(uint32_t n_rows, uint32_t k_total, uint32_t /*n_seg*/) {
-  return align_up(128 + kMaxSegs * kTableStride * 2, 1024) + static_cast<size_t>(kStages) * kStageBytes +
-         static_cast<size_t>(n_rows) * k_total * 2;
+size_t gemm_weight_bytes(uint32_t n_rows, uint32_t k_total) { return static_cast<size_t>(n_rows) * k_total * 2; }
+
+size_t gemm_smem_bytes(uint32_t w_bytes, uint32_t n_stages) {
+  return kHeaderBytes + static_cast<size_t>(w_bytes) + static_cast<size_t>(n_stages) * kStageBytes;
+}
+
+uint32_t gemm_pick_stages(uint32_t w_bytes) {
+  const size_t room = 227 * 1024 - kHeaderBytes - static_cast<size_t>(w_bytes);
+  const size_t s = room / kStageBytes;
+  return static_cast<uint32_t>(s > 6 ? 6 : s);       // fewer than 3 means the tile does not fit
 }
 
 cudaError_t gemm_configure() {
   cudaError_t e;
-#define STI_SET(XT, OutT, G)                                                  \
-  if ((e = set_smem(dqgemm_kernel<XT, OutT, G, false>)) != cudaSuccess) return e; \
-  if ((e = set_smem(dqgemm_kernel<XT, OutT, G, true>)) != cudaSuccess) return e;
-  STI_SET(float, __nv_bfloat16, false)
-  STI_SET(__nv_bfloat16, __nv_bfloat16, false)
-  STI_SET(__nv_bfloat16, __nv_bfloat16, true)
-  STI_SET(__nv_bfloat16, float, false)
+#define STI_SET(OutT, G)                                                  \
+  if ((e = set_smem(dqgemm_kernel<OutT, G, false>)) != cudaSuccess) return e; \
+  if ((e = set_smem(dqgemm_kernel<OutT, G, true>)) != cudaSuccess) return e;
+  STI_SET(__nv_bfloat16, false)
+  STI_SET(__nv_bfloat16, true)
+  STI_SET(float, false)
 #undef STI_SET
   return cudaSuccess;
 }
 
 cudaError_t launch_gemm(GemmKind kind, const GemmLaunch& p, cudaStream_t s) {
   switch (kind) {
-    case GEMM_F32_TO_BF16: return launch_t<float, __nv_bfloat16, false>(p, s);
-    case GEMM_BF16_TO_BF16: return launch_t<__nv_bfloat16, __nv_bfloat16, false>(p, s);
-    case GEMM_BF16_TO_BF16_GELU: return launch_t<__nv_bfloat16, __nv_bfloat16, true>(p, s);
-    case GEMM_BF16_TO_F32: return launch_t<__nv_bfloat16, float, false>(p, s);
+    case GEMM_BF16_TO_BF16: return launch_t<__nv_bfloat16, false>(p, s);
+    case GEMM_BF16_TO_BF16_GELU: return launch_t<__nv_bfloat16, true>(p, s);
+    case GEMM_BF16_TO_F32: return launch_t<float, false>(p, s);
   }
   return cudaErrorInvalidValue;
 }

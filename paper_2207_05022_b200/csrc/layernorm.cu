@@ -1,6 +1,7 @@
 // Residual + bias + LayerNorm over the split-K partial sums of the O projection and of FFN2
 // (Section 2.1; Section 6: biases and layernorm parameters stay in fp32).
-// One warp per token row; the row lives in registers, mean and variance are two-pass.
+// One CTA per token row, one float4 per thread (hidden / 4 threads): every load of a row is in
+// flight at once; mean and variance are two-pass over registers with a block reduction.
 #include <cuda_bf16.h>
 
 #include "sti_device.cuh"
@@ -9,78 +10,82 @@
 namespace sti {
 namespace {
 
-constexpr int kMaxVec = 16;   // float4 per lane: hidden <= 16 * 128 = 2048
+__device__ __forceinline__ float block_sum(float v, float* red, int tid, int n_warps) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  if ((tid & 31) == 0) red[tid >> 5] = v;
+  __syncthreads();
+  float t = 0.f;
+  for (int w = 0; w < n_warps; ++w) t += red[w];
+  __syncthreads();
+  return t;
+}
 
-__global__ void __launch_bounds__(256)
+__global__ void __launch_bounds__(512)
 layernorm_kernel(LnLaunch p) {
-  const int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
-  const int lane = threadIdx.x & 31;
-  if (warp >= p.T) return;
-  const int nvec = p.d / 128;
-  const size_t row = static_cast<size_t>(warp) * p.d;
-  float4 v[kMaxVec];
-  float sum = 0.f;
-#pragma unroll
-  for (int i = 0; i < kMaxVec; ++i) {
-    if (i < nvec) {
-      const int c = (i * 32 + lane) * 4;
-      float4 a = __ldg(reinterpret_cast<const float4*>(p.bias + c));
-      if (p.resid_bf16) {
-        const uint2 r = __ldg(reinterpret_cast<const uint2*>(static_cast<const uint16_t*>(p.resid) + row + c));
-        a.x += __uint_as_float(r.x << 16); a.y += __uint_as_float(r.x & 0xffff0000u);
-        a.z += __uint_as_float(r.y << 16); a.w += __uint_as_float(r.y & 0xffff0000u);
-      } else {
-        const float4 r = __ldg(reinterpret_cast<const float4*>(static_cast<const float*>(p.resid) + row + c));
-        a.x += r.x; a.y += r.y; a.z += r.z; a.w += r.w;
-      }
-      for (int q = 0; q < p.n_partial; ++q) {
-        const float4 s = __ldg(reinterpret_cast<const float4*>(p.partial + static_cast<size_t>(q) * p.T * p.d + row + c));
-        a.x += s.x; a.y += s.y; a.z += s.z; a.w += s.w;
-      }
-      v[i] = a;
-      sum += a.x + a.y + a.z + a.w;
-    }
+  __shared__ float red[16];
+  const int tid = threadIdx.x;
+  const int n_warps = blockDim.x >> 5;
+  const size_t row = static_cast<size_t>(blockIdx.x) * p.d;
+  const int c = tid * 4;
+  float4 a = __ldg(reinterpret_cast<const float4*>(p.bias + c));
+  if (p.resid_bf16) {
+    const uint2 r = __ldg(reinterpret_cast<const uint2*>(static_cast<const uint16_t*>(p.resid) + row + c));
+    a.x += __uint_as_float(r.x << 16); a.y += __uint_as_float(r.x & 0xffff0000u);
+    a.z += __uint_as_float(r.y << 16); a.w += __uint_as_float(r.y & 0xffff0000u);
+  } else {
+    const float4 r = __ldg(reinterpret_cast<const float4*>(static_cast<const float*>(p.resid) + row + c));
+    a.x += r.x; a.y += r.y; a.z += r.z; a.w += r.w;
   }
-#pragma unroll
-  for (int o = 16; o > 0; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
-  const float mean = sum / static_cast<float>(p.d);
-  float sq = 0.f;
-#pragma unroll
-  for (int i = 0; i < kMaxVec; ++i) {
-    if (i < nvec) {
-      const float dx = v[i].x - mean, dy = v[i].y - mean, dz = v[i].z - mean, dw = v[i].w - mean;
-      sq += dx * dx + dy * dy + dz * dz + dw * dw;
-    }
+  const size_t pstride = static_cast<size_t>(p.T) * p.d;
+  int q = 0;
+  for (; q + 4 <= p.n_partial; q += 4) {          // four independent loads at a time
+    const float4 s0 = __ldg(reinterpret_cast<const float4*>(p.partial + (q + 0) * pstride + row + c));
+    const float4 s1 = __ldg(reinterpret_cast<const float4*>(p.partial + (q + 1) * pstride + row + c));
+    const float4 s2 = __ldg(reinterpret_cast<const float4*>(p.partial + (q + 2) * pstride + row + c));
+    const float4 s3 = __ldg(reinterpret_cast<const float4*>(p.partial + (q + 3) * pstride + row + c));
+    a.x += (s0.x + s1.x) + (s2.x + s3.x); a.y += (s0.y + s1.y) + (s2.y + s3.y);
+    a.z += (s0.z + s1.z) + (s2.z + s3.z); a.w += (s0.w + s1.w) + (s2.w + s3.w);
   }
-#pragma unroll
-  for (int o = 16; o > 0; o >>= 1) sq += __shfl_xor_sync(0xffffffffu, sq, o);
-  const float rstd = rsqrtf(sq / static_cast<float>(p.d) + p.eps);
-#pragma unroll
-  for (int i = 0; i < kMaxVec; ++i) {
-    if (i < nvec) {
-      const int c = (i * 32 + lane) * 4;
-      const float4 g = __ldg(reinterpret_cast<const float4*>(p.gamma + c));
-      const float4 b = __ldg(reinterpret_cast<const float4*>(p.beta + c));
-      float4 y;
-      y.x = (v[i].x - mean) * rstd * g.x + b.x;
-      y.y = (v[i].y - mean) * rstd * g.y + b.y;
-      y.z = (v[i].z - mean) * rstd * g.z + b.z;
-      y.w = (v[i].w - mean) * rstd * g.w + b.w;
-      if (p.out_f32) *reinterpret_cast<float4*>(p.out_f32 + row + c) = y;
-      if (p.out_bf16)
-        *reinterpret_cast<uint2*>(p.out_bf16 + row + c) = make_uint2(pack_bf16x2(y.x, y.y), pack_bf16x2(y.z, y.w));
-    }
+  for (; q < p.n_partial; ++q) {
+    const float4 s = __ldg(reinterpret_cast<const float4*>(p.partial + q * pstride + row + c));
+    a.x += s.x; a.y += s.y; a.z += s.z; a.w += s.w;
   }
+  const float mean = block_sum(a.x + a.y + a.z + a.w, red, tid, n_warps) / static_cast<float>(p.d);
+  const float dx = a.x - mean, dy = a.y - mean, dz = a.z - mean, dw = a.w - mean;
+  const float var = block_sum(dx * dx + dy * dy + dz * dz + dw * dw, red, tid, n_warps) / static_cast<float>(p.d);
+  const float rstd = rsqrtf(var + p.eps);
+  const float4 g = __ldg(reinterpret_cast<const float4*>(p.gamma + c));
+  const float4 b = __ldg(reinterpret_cast<const float4*>(p.beta + c));
+  float4 y;
+  y.x = dx * rstd * g.x + b.x; y.y = dy * rstd * g.y + b.y;
+  y.z = dz * rstd * g.z + b.z; y.w = dw * rstd * g.w + b.w;
+  if (p.out_f32) *reinterpret_cast<float4*>(p.out_f32 + row + c) = y;
+  if (p.out_bf16)
+    *reinterpret_cast<uint2*>(p.out_bf16 + row + c) = make_uint2(pack_bf16x2(y.x, y.y), pack_bf16x2(y.z, y.w));
+}
+
+__global__ void cast_bf16_kernel(const float* __restrict__ in, uint16_t* __restrict__ out, size_t n4) {
+  const size_t i = static_cast<size_t>(blockIdx.x) * blockDim.x + threadIdx.x;
+  if (i >= n4) return;
+  const float4 v = __ldg(reinterpret_cast<const float4*>(in) + i);
+  reinterpret_cast<uint2*>(out)[i] = make_uint2(pack_bf16x2(v.x, v.y), pack_bf16x2(v.z, v.w));
 }
 
 }  // namespace
 
 cudaError_t launch_layernorm(const LnLaunch& p, cudaStream_t s) {
   if (p.T <= 0) return cudaSuccess;
-  if (p.d % 128 != 0 || p.d / 128 > kMaxVec) return cudaErrorInvalidValue;
-  const int warps_per_block = 8;
-  const int blocks = (p.T + warps_per_block - 1) / warps_per_block;
-  layernorm_kernel<<<blocks, warps_per_block * 32, 0, s>>>(p);
+  if (p.d % 128 != 0 || p.d > 2048) return cudaErrorInvalidValue;     // d / 4 threads, whole warps
+  layernorm_kernel<<<p.T, p.d / 4, 0, s>>>(p);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_cast_bf16(const float* in, uint16_t* out, size_t n, cudaStream_t s) {
+  if (n == 0) return cudaSuccess;
+  if (n % 4) return cudaErrorInvalidValue;
+  const size_t n4 = n / 4;
+  cast_bf16_kernel<<<static_cast<unsigned>((n4 + 255) / 256), 256, 0, s>>>(in, out, n4);
   return cudaGetLastError();
 }
 

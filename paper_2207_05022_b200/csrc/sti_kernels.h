@@ -36,8 +36,7 @@ struct Job {
 };
 
 enum GemmKind : int {
-  GEMM_F32_TO_BF16 = 0,       // fp32 activations in, bf16 out (+bias)         : QKV on fp32 inputs
-  GEMM_BF16_TO_BF16 = 1,      // bf16 in, bf16 out (+bias)                     : QKV on bf16 inputs
+  GEMM_BF16_TO_BF16 = 1,      // bf16 in, bf16 out (+bias)                     : QKV
   GEMM_BF16_TO_BF16_GELU = 2, // bf16 in, bf16 out, +bias, erf-GELU            : FFN1
   GEMM_BF16_TO_F32 = 3        // bf16 in, fp32 partial sums out, no bias       : O projection, FFN2
 };
@@ -47,18 +46,22 @@ struct GemmLaunch {
   const Seg* segs;
   int n_jobs;
   int m_ctas;               // CTAs along the token dimension (each loops over its M tiles)
-  const void* x;            // [T, ldx]
+  const void* x;            // [T, ldx] bf16
   int ldx;
   int T;
   void* out;
   int ldo;
   const float* bias;
   int* err;                 // device status word
-  size_t smem_bytes;        // dynamic shared memory the largest job needs
+  size_t smem_bytes;        // header + w_bytes + n_stages activation stages
+  uint32_t n_stages;        // activation chunks of 16 KB in the ring (3..6)
+  uint32_t w_bytes;         // shared memory reserved for the weight tile (largest job)
   bool simt_debug;          // compute the products on the plain ALUs instead of the tensor cores
 };
 
-size_t gemm_smem_bytes(uint32_t n_rows, uint32_t k_total, uint32_t n_seg);
+size_t gemm_weight_bytes(uint32_t n_rows, uint32_t k_total);
+uint32_t gemm_pick_stages(uint32_t w_bytes);        // < 3: the tile does not fit in shared memory
+size_t gemm_smem_bytes(uint32_t w_bytes, uint32_t n_stages);
 cudaError_t gemm_configure();   // opt in to large dynamic shared memory (once per device)
 cudaError_t launch_gemm(GemmKind kind, const GemmLaunch& p, cudaStream_t s);
 
@@ -82,6 +85,9 @@ struct LnLaunch {
   uint16_t* out_bf16;       // optional
 };
 cudaError_t launch_layernorm(const LnLaunch& p, cudaStream_t s);
+
+// fp32 -> bf16 (round-to-nearest-even) copy of the activations the first GEMM reads.
+cudaError_t launch_cast_bf16(const float* in, uint16_t* out, size_t n, cudaStream_t s);
 
 // Stand-alone decode of one matrix (inspection / parity).
 struct DecodeLaunch {
