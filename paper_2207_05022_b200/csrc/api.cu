@@ -299,6 +299,37 @@ sti_status check_async(sti_ctx* c) {
   return STI_OK;
 }
 
+// cuTensorMapEncodeTiled is a driver entry point; it is looked up through the runtime so that the
+// library does not link against libcuda directly.
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+EncodeTiledFn encode_tiled_fn() {
+  static EncodeTiledFn fn = [] {
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult q = cudaDriverEntryPointSymbolNotFound;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) != cudaSuccess ||
+        q != cudaDriverEntryPointSuccess)
+      p = nullptr;
+    return reinterpret_cast<EncodeTiledFn>(p);
+  }();
+  return fn;
+}
+
+// TMA view of a bf16 activation matrix [rows, ld]: boxes of 128 rows x 64 columns, 128-byte swizzle,
+// rows past `rows` read as zeros.
+bool make_xmap(CUtensorMap* map, const void* base, int ld, int rows) {
+  EncodeTiledFn fn = encode_tiled_fn();
+  if (!fn || (reinterpret_cast<uintptr_t>(base) & 15) || (ld % 8) != 0) return false;
+  const cuuint64_t dims[2] = {static_cast<cuuint64_t>(ld), static_cast<cuuint64_t>(rows)};
+  const cuuint64_t strides[1] = {static_cast<cuuint64_t>(ld) * 2};
+  const cuuint32_t box[2] = {64, 128};
+  const cuuint32_t estr[2] = {1, 1};
+  return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 int m_ctas_for(int n_jobs, int T) {
   const int n_mtiles = (T + 127) / 128;
   int m = n_jobs > 0 ? 148 / n_jobs : 1;
@@ -310,6 +341,7 @@ sti_status run_gemm(sti_plan* p, GemmKind kind, const GemmTable& tab, const void
   if (tab.n_jobs == 0) return STI_OK;
   GemmLaunch g{};
   g.jobs = tab.jobs; g.segs = tab.segs; g.n_jobs = tab.n_jobs; g.m_ctas = m_ctas_for(tab.n_jobs, T);
+  if (!make_xmap(&g.xmap, x, ldx, T)) return STI_ERR_CUDA;
   g.x = x; g.ldx = ldx; g.T = T; g.out = out; g.ldo = ldo; g.bias = bias; g.err = p->ctx->err_dev;
   g.smem_bytes = tab.smem; g.n_stages = tab.n_stages; g.w_bytes = tab.w_bytes; g.simt_debug = p->ctx->simt_debug;
   CUDA_TRY(launch_gemm(kind, g, p->ctx->compute));
@@ -738,7 +770,8 @@ sti_status sti_plan_finalize(sti_plan* p) {
       gt[i]->w_bytes = tb[i].w_bytes;
       gt[i]->n_stages = gemm_pick_stages(tb[i].w_bytes);
       if (!tb[i].jobs.empty() && gt[i]->n_stages < 3) return STI_ERR_SHAPE;
-      gt[i]->smem = gemm_smem_bytes(tb[i].w_bytes, std::max(3u, gt[i]->n_stages));
+      gt[i]->n_stages = std::max(3u, gt[i]->n_stages);
+      gt[i]->smem = gemm_smem_bytes(tb[i].w_bytes, gt[i]->n_stages);
       if (gt[i]->smem > kMaxSmem && !tb[i].jobs.empty()) return STI_ERR_SHAPE;
       Fix fx{gt[i], 0, 0};
       fx.jobs_off = align16(host_tables.size());

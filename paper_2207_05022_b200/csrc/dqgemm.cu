@@ -3,17 +3,19 @@
 // Y[T, N] = X[T, K] * W[N, K]^T where W only exists as bit-packed k-bit dictionary indexes.
 // One CTA owns a weight tile (n_rows output features x k_total input features), decodes it ONCE
 // into shared memory as bf16 (index unpack in registers -> per-unit centroid table in shared
-// memory -> outlier patch), and then streams 128-token activation tiles past it:
-//   activation chunk [128 x 64] bf16 -> shared memory with cp.async, several chunks in flight
-//   (K-major core-matrix layout), issued before the decode so that their latency hides behind it
-//   tcgen05.mma (M = 128 tokens, N = n_rows, K = 16 per instruction), fp32 accumulator in TMEM
-//   epilogue: tcgen05.ld -> bias / GELU -> global.
+// memory -> outlier patch), and then streams 128-token activation tiles past it.  After the decode
+// the CTA is warp-specialised, with no CTA-wide barrier in the main loop:
+//   warp 0  producer : TMA (cp.async.bulk.tensor, 128-byte swizzle) brings [128 x 64] bf16 activation
+//                      chunks into a ring of stages; the first stages are requested before the decode
+//   warp 1  MMA      : waits for a chunk, issues tcgen05.mma (M = 128 tokens, N = n_rows, K = 16) into
+//                      one of two TMEM accumulators, tcgen05.commit frees the stage / publishes the tile
+//   warps 4-7 epilogue: tcgen05.ld -> bias / erf-GELU -> global, while the next tile accumulates
 //
-// Shared-memory operand layout (both operands): element (row, k) lives at
-//   ((k / 8) * rows + row) * 16 + (k % 8) * 2   bytes,
-// i.e. 8x8 core matrices, 8-row groups contiguous (SBO = 128 B), K-adjacent core matrices
-// `rows * 16` bytes apart (LBO).  This is the no-swizzle K-major canonical layout; lanes that
-// hold consecutive rows write consecutive 16-byte pieces, so decode stores are conflict-free.
+// Weight tile layout in shared memory: element (row, k) at ((k / 8) * rows + row) * 16 + (k % 8) * 2,
+// the no-swizzle K-major core-matrix layout (SBO = 128 B, LBO = rows * 16 B): lanes holding consecutive
+// rows write consecutive 16-byte pieces, so decode stores are conflict-free.  Activation stages use the
+// 128-byte-swizzled K-major layout that TMA writes (SBO = 1024 B).  Every wait is bounded.
+#include <cuda.h>
 #include <cuda_bf16.h>
 
 #include "sti_device.cuh"
@@ -23,22 +25,25 @@ namespace sti {
 
 namespace {
 
-constexpr int kThreads = 256;
+constexpr int kThreads = 256;               // warp 0: TMA producer, warp 1: MMA issuer, warps 4-7: epilogue; all decode
 constexpr int kWarps = kThreads / 32;
 constexpr int kTileM = 128;                 // tokens per MMA tile
-constexpr int kChunkK = 64;                 // activation K per pipeline stage
+constexpr int kChunkK = 64;                 // activation K per pipeline stage = one 128-byte swizzle row
 constexpr int kMaxStages = 8;
 constexpr int kStageBytes = kTileM * kChunkK * 2;   // 16 KB
-constexpr int kHeaderBytes = 3072;          // barriers + segment tables
-constexpr int kRefillLag = 2;               // a stage is refilled two chunks after its MMAs were issued
+constexpr int kHeaderBytes = 4096;          // barriers + segment tables; stages start 1024-byte aligned after it
+constexpr int kAlignSlack = 1024;           // the dynamic shared-memory base is aligned up to 1024 by hand
 constexpr int kMaxSegs = 16;
 constexpr int kTableStride = 64;            // bf16 entries per segment table
+constexpr int kEpilogueWarp0 = 4;
 
 struct SmemHeader {
-  uint64_t mma_done[kMaxStages];
-  uint64_t acc_full;
+  uint64_t full[kMaxStages];     // activation chunk landed (TMA transaction bytes)
+  uint64_t empty[kMaxStages];    // the MMAs that read the chunk have completed
+  uint64_t acc_full[2];          // accumulator buffer complete
+  uint64_t acc_empty[2];         // accumulator buffer drained by the epilogue warps
   uint32_t tmem_base;
-  uint32_t pad;
+  volatile uint32_t abort;       // a bounded wait ran out somewhere in the CTA
 };
 
 // ---------------------------------------------------------------------------------------
@@ -92,46 +97,30 @@ __device__ __forceinline__ void decode_raw(const Seg& sg, uint8_t* wsm, uint32_t
 }
 
 // ---------------------------------------------------------------------------------------
-// Activation chunk: rows [m0, m0+128) x columns [k0, k0+64) -> stage buffer
+// TMA / mbarrier helpers local to this kernel
 // ---------------------------------------------------------------------------------------
-__device__ __forceinline__ void cp_async16_zfill(uint32_t dst, const void* src, uint32_t src_bytes) {
-  asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "r"(src_bytes) : "memory");
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
 }
-__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
-template <int N>
-__device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
-
-// Asynchronous version: 4 x 16 bytes per thread, rows past T are zero-filled.  Within a quarter warp
-// the lanes hold 8 consecutive rows of one 16-byte column piece = 128 contiguous bytes of the stage.
-__device__ __forceinline__ void load_x_chunk_async(const __nv_bfloat16* __restrict__ x, int ldx, int T, int m0, int k0,
-                                                   uint32_t stage_addr, uint32_t tid) {
-  const uint32_t lane = tid & 31;
-#pragma unroll
-  for (int i = 0; i < (kTileM * (kChunkK / 8)) / kThreads; ++i) {
-    const uint32_t u = (i * kThreads + tid) >> 5;          // warp-level unit, 0..31
-    const uint32_t row = (u & 15) * 8 + (lane & 7);
-    const uint32_t piece = (u >> 4) * 4 + (lane >> 3);
-    const int t = m0 + static_cast<int>(row);
-    const bool ok = t < T;
-    const __nv_bfloat16* src = ok ? x + static_cast<size_t>(t) * ldx + k0 + piece * 8 : x;
-    cp_async16_zfill(stage_addr + piece * (kTileM * 16) + row * 16, src, ok ? 16u : 0u);
-  }
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
 }
-
-// Synchronous version (debug path).
-__device__ __forceinline__ void load_x_chunk(const __nv_bfloat16* __restrict__ x, int ldx, int T, int m0, int k0,
-                                             uint8_t* stage, uint32_t tid) {
-  const uint32_t lane = tid & 31;
-#pragma unroll
-  for (int i = 0; i < (kTileM * (kChunkK / 8)) / kThreads; ++i) {
-    const uint32_t u = (i * kThreads + tid) >> 5;
-    const uint32_t row = (u & 15) * 8 + (lane & 7);
-    const uint32_t piece = (u >> 4) * 4 + (lane >> 3);
-    uint4 v = make_uint4(0, 0, 0, 0);
-    const int t = m0 + static_cast<int>(row);
-    if (t < T) v = __ldg(reinterpret_cast<const uint4*>(x + static_cast<size_t>(t) * ldx + k0 + piece * 8));
-    *reinterpret_cast<uint4*>(stage + piece * (kTileM * 16) + row * 16) = v;
-  }
+// [128 rows x 64 columns] box at (column k0, row m0); rows past the tensor's extent arrive as zeros.
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int k0, int m0, uint32_t bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+      ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(k0), "r"(m0), "r"(bar)
+      : "memory");
+}
+// K-major, 128-byte swizzle: rows of 128 bytes, 8-row groups 1024 bytes apart.
+__device__ __forceinline__ uint64_t umma_smem_desc_sw128(uint32_t saddr) {
+  uint64_t d = 0;
+  d |= static_cast<uint64_t>((saddr & 0x3FFFFu) >> 4);
+  d |= static_cast<uint64_t>(1) << 16;                 // leading byte offset: unused for this layout
+  d |= static_cast<uint64_t>(1024 >> 4) << 32;         // stride byte offset
+  d |= static_cast<uint64_t>(1) << 46;                 // descriptor version for sm_100
+  d |= static_cast<uint64_t>(2) << 61;                 // layout type: 128-byte swizzle
+  return d;
 }
 
 __device__ __forceinline__ float gelu_erf(float v) { return 0.5f * v * (1.0f + erff(v * 0.70710678118654752440f)); }
@@ -156,23 +145,24 @@ __device__ __forceinline__ void store_row16(OutT* dst, const float (&v)[16]) {
 // ---------------------------------------------------------------------------------------
 template <typename OutT, bool GELU, bool SIMT>
 __global__ void __launch_bounds__(kThreads, 1)
-dqgemm_kernel(const Job* __restrict__ jobs, const Seg* __restrict__ segs, const __nv_bfloat16* __restrict__ x, int ldx,
-              int T, OutT* __restrict__ out, int ldo, const float* __restrict__ bias, int* __restrict__ err,
-              uint32_t n_stages, uint32_t w_bytes) {
-  extern __shared__ __align__(1024) uint8_t smem[];
+dqgemm_kernel(const __grid_constant__ CUtensorMap xmap, const Job* __restrict__ jobs, const Seg* __restrict__ segs,
+              const __nv_bfloat16* __restrict__ x, int ldx, int T, OutT* __restrict__ out, int ldo,
+              const float* __restrict__ bias, int* __restrict__ err, uint32_t n_stages, uint32_t w_bytes) {
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = smem_raw + ((1024u - (smem_addr(smem_raw) & 1023u)) & 1023u);
   const uint32_t tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const Job job = jobs[blockIdx.x];
   const uint32_t n_rows = job.n_rows, k_total = job.k_total;
 
   SmemHeader* hdr = reinterpret_cast<SmemHeader*>(smem);
-  uint16_t* tables = reinterpret_cast<uint16_t*>(smem + 256);                       // [kMaxSegs][64]
-  uint8_t* wsm = smem + kHeaderBytes;
-  uint8_t* xsm = wsm + w_bytes;                                                      // n_stages x 16 KB
+  uint16_t* tables = reinterpret_cast<uint16_t*>(smem + 1024);                      // [kMaxSegs][64]
+  uint8_t* xsm = smem + kHeaderBytes;                                                // n_stages x 16 KB, 1024-aligned
+  uint8_t* wsm = xsm + n_stages * kStageBytes;
 
   // the kernel's own checks of the descriptor: refuse rather than touch memory out of bounds
   const bool bad = job.n_seg == 0 || job.n_seg > kMaxSegs || (n_rows != 32 && n_rows != 64 && n_rows != 128) ||
                    (k_total % kChunkK) != 0 || k_total == 0 || n_rows * k_total * 2 > w_bytes ||
-                   n_stages < kRefillLag + 1 || n_stages > kMaxStages;
+                   n_stages < 2 || n_stages > kMaxStages;
   if (bad) {
     if (tid == 0) atomicCAS(err, ERR_NONE, ERR_BAD_JOB);
     return;
@@ -184,28 +174,34 @@ dqgemm_kernel(const Job* __restrict__ jobs, const Seg* __restrict__ segs, const 
                                  ? (n_mtiles - blockIdx.y + gridDim.y - 1) / gridDim.y : 0;
   const uint32_t total = my_mtiles * n_chunks;          // activation chunks this CTA consumes
   const uint32_t xsm_addr = smem_addr(xsm);
-  auto issue_chunk = [&](uint32_t c) {
-    const int m0 = (blockIdx.y + (c / n_chunks) * gridDim.y) * kTileM;
-    load_x_chunk_async(x, ldx, T, m0, job.x_koff + (c % n_chunks) * kChunkK,
-                       xsm_addr + (c % n_stages) * kStageBytes, tid);
+  auto request_chunk = [&](uint32_t c) {                 // one thread
+    const uint32_t bar = smem_addr(&hdr->full[c % n_stages]);
+    mbar_expect_tx(bar, kStageBytes);
+    tma_load_2d(xsm_addr + (c % n_stages) * kStageBytes, &xmap, static_cast<int>(job.x_koff + (c % n_chunks) * kChunkK),
+                static_cast<int>((blockIdx.y + (c / n_chunks) * gridDim.y) * kTileM), bar);
   };
 
   uint32_t tmem_cols = 32;
-  while (tmem_cols < n_rows) tmem_cols <<= 1;
+  while (tmem_cols < 2 * n_rows) tmem_cols <<= 1;       // two accumulators
   if constexpr (!SIMT) {
-    // activations first: n_stages - kRefillLag chunks in flight while the weights are decoded
-    for (uint32_t c = 0; c < n_stages - kRefillLag; ++c) {
-      if (c < total) issue_chunk(c);
-      cp_async_commit();
+    if (tid == 0) {
+      for (uint32_t s = 0; s < n_stages; ++s) {
+        mbar_init(smem_addr(&hdr->full[s]), 1);
+        mbar_init(smem_addr(&hdr->empty[s]), 1);
+      }
+      for (int b = 0; b < 2; ++b) {
+        mbar_init(smem_addr(&hdr->acc_full[b]), 1);
+        mbar_init(smem_addr(&hdr->acc_empty[b]), 4);     // one arrival per epilogue warp
+      }
+      hdr->abort = 0;
+      mbar_fence_init();
+      fence_proxy_async_smem();
+      // activations first: the ring is filled while the weights are being decoded
+      for (uint32_t c = 0; c < n_stages && c < total; ++c) request_chunk(c);
     }
-    if (warp == 0) {
+    if (warp == 1) {
       tmem_alloc(smem_addr(&hdr->tmem_base), tmem_cols);
       tmem_relinquish();
-    }
-    if (tid == 0) {
-      for (uint32_t s = 0; s < n_stages; ++s) mbar_init(smem_addr(&hdr->mma_done[s]), 1);
-      mbar_init(smem_addr(&hdr->acc_full), 1);
-      mbar_fence_init();
     }
   }
   // centroid tables, rounded once to bf16 (round-to-nearest-even)
@@ -260,21 +256,16 @@ dqgemm_kernel(const Job* __restrict__ jobs, const Seg* __restrict__ segs, const 
   }
 
   if constexpr (SIMT) {
-    // Debug path: the same shared-memory tiles multiplied on the plain ALUs.
+    // Debug path: the decoded tile multiplied on the plain ALUs, activations straight from global memory.
     for (int mt = blockIdx.y; mt < n_mtiles; mt += gridDim.y) {
-      const int m0 = mt * kTileM;
       const uint32_t row = tid & 127, chalf = tid >> 7, ncol = n_rows / 2;
+      const int t = mt * kTileM + static_cast<int>(row);
       float acc[64];
 #pragma unroll
       for (int c = 0; c < 64; ++c) acc[c] = 0.f;
-      for (uint32_t kc = 0; kc < n_chunks; ++kc) {
-        __syncthreads();
-        load_x_chunk(x, ldx, T, m0, job.x_koff + kc * kChunkK, xsm, tid);
-        __syncthreads();
-        for (uint32_t kk = 0; kk < kChunkK; ++kk) {
-          const float a = __bfloat162float(
-              reinterpret_cast<const __nv_bfloat16*>(xsm)[((kk >> 3) * kTileM + row) * 8 + (kk & 7)]);
-          const uint32_t kg = kc * kChunkK + kk;
+      if (t < T) {
+        for (uint32_t kg = 0; kg < k_total; ++kg) {
+          const float a = __bfloat162float(x[static_cast<size_t>(t) * ldx + job.x_koff + kg]);
 #pragma unroll
           for (int c = 0; c < 64; ++c) {
             if (static_cast<uint32_t>(c) < ncol) {
@@ -284,9 +275,6 @@ dqgemm_kernel(const Job* __restrict__ jobs, const Seg* __restrict__ segs, const 
             }
           }
         }
-      }
-      const int t = m0 + static_cast<int>(row);
-      if (t < T) {
 #pragma unroll
         for (int cb = 0; cb < 4; ++cb) {
           if (static_cast<uint32_t>(cb * 16) < ncol) {
@@ -304,87 +292,92 @@ dqgemm_kernel(const Job* __restrict__ jobs, const Seg* __restrict__ segs, const 
       }
     }
   } else {
-    const uint32_t idesc = umma_idesc_bf16_m128(n_rows);
-    const uint32_t w_lbo = n_rows * 16;
-    const uint32_t wsm_addr = smem_addr(wsm);
-    uint32_t acc_phase = 0;
-    uint32_t issued = 0;       // chunks whose MMAs have been issued
     bool failed = false;
-    for (uint32_t c = 0; c < total; ++c) {
-      const uint32_t kc = c % n_chunks;
-      // refill: chunk c + S - L goes into the stage that chunk c - L used; its MMAs were issued L iterations ago
-      const uint32_t nxt = c + n_stages - kRefillLag;
-      if (nxt < total && c >= kRefillLag && !failed) {
-        const uint32_t prev = c - kRefillLag;
-        if (!mbar_wait_bounded(smem_addr(&hdr->mma_done[prev % n_stages]), (prev / n_stages) & 1)) failed = true;
+    if (warp == 0) {
+      // ---- producer: refill a stage as soon as the MMAs that read it have completed
+      uint32_t requested = n_stages < total ? n_stages : total;
+      for (uint32_t c = n_stages; c < total && !failed; ++c) {
+        if (hdr->abort) break;
+        if (!mbar_wait_bounded(smem_addr(&hdr->empty[c % n_stages]), ((c / n_stages) - 1) & 1)) { failed = true; break; }
+        if (lane == 0) request_chunk(c);
+        requested = c + 1;
+        __syncwarp();
       }
-      if (nxt < total && !failed) issue_chunk(nxt);
-      cp_async_commit();
-      // chunk c is complete once at most (n_stages - kRefillLag) newer groups are pending
-      switch (n_stages - kRefillLag) {
-        case 1: cp_async_wait<1>(); break;
-        case 2: cp_async_wait<2>(); break;
-        case 3: cp_async_wait<3>(); break;
-        case 4: cp_async_wait<4>(); break;
-        case 5: cp_async_wait<5>(); break;
-        default: cp_async_wait<6>(); break;
+      if (failed || hdr->abort) {
+        // give every copy this CTA requested a bounded chance to land before the CTA exits
+        const uint32_t first = requested > n_stages ? requested - n_stages : 0;
+        for (uint32_t c = first; c < requested; ++c)
+          (void)mbar_wait_bounded(smem_addr(&hdr->full[c % n_stages]), (c / n_stages) & 1);
       }
-      fence_proxy_async_smem();
-      if (__syncthreads_or(failed)) { failed = true; break; }
-      if (tid == 0) {
+    } else if (warp == 1) {
+      // ---- MMA issuer
+      const uint32_t idesc = umma_idesc_bf16_m128(n_rows);
+      const uint32_t w_lbo = n_rows * 16;
+      const uint32_t wsm_addr = smem_addr(wsm);
+      uint32_t issued = 0;
+      for (uint32_t c = 0; c < total && !failed; ++c) {
+        const uint32_t kc = c % n_chunks, ti = c / n_chunks, buf = ti & 1;
+        if (hdr->abort) break;
+        if (kc == 0 && ti >= 2) {      // the epilogue must have drained this accumulator
+          if (!mbar_wait_bounded(smem_addr(&hdr->acc_empty[buf]), ((ti >> 1) - 1) & 1)) { failed = true; break; }
+        }
+        if (!mbar_wait_bounded(smem_addr(&hdr->full[c % n_stages]), (c / n_stages) & 1)) { failed = true; break; }
         tc_fence_after_sync();
-        const uint32_t a_base = xsm_addr + (c % n_stages) * kStageBytes;
-        const uint32_t b_base = wsm_addr + (kc * (kChunkK / 8)) * w_lbo;
+        if (lane == 0) {
+          const uint32_t a_base = xsm_addr + (c % n_stages) * kStageBytes;
+          const uint32_t b_base = wsm_addr + (kc * (kChunkK / 8)) * w_lbo;
+          const uint32_t d_addr = tmem_base + buf * n_rows;
 #pragma unroll
-        for (int ks = 0; ks < kChunkK / 16; ++ks) {
-          const uint64_t da = umma_smem_desc(a_base + ks * 2 * (kTileM * 16), kTileM * 16, 128);
-          const uint64_t db = umma_smem_desc(b_base + ks * 2 * w_lbo, w_lbo, 128);
-          umma_bf16_ss(tmem_base, da, db, idesc, (kc | ks) != 0 ? 1u : 0u);
-        }
-        umma_commit(smem_addr(&hdr->mma_done[c % n_stages]));
-        if (kc + 1 == n_chunks) umma_commit(smem_addr(&hdr->acc_full));
-      }
-      issued = c + 1;
-      if (kc + 1 != n_chunks) continue;
-      // ---- epilogue of this token tile: accumulator -> registers -> global
-      if (!mbar_wait_bounded(smem_addr(&hdr->acc_full), acc_phase)) failed = true;
-      acc_phase ^= 1;
-      if (__syncthreads_or(failed)) { failed = true; break; }
-      tc_fence_after_sync();
-      const int m0 = (blockIdx.y + (c / n_chunks) * gridDim.y) * kTileM;
-      const uint32_t q = warp & 3, chalf = warp >> 2, ncol = n_rows / 2;
-      const int t = m0 + static_cast<int>(q * 32 + lane);
-      for (uint32_t c0 = 0; c0 < ncol; c0 += 16) {
-        uint32_t r[16];
-        const uint32_t col = chalf * ncol + c0;
-        tmem_ld_32x32b_x16(tmem_base + ((q * 32) << 16) + col, r);
-        tc_wait_ld();
-        if (t < T) {
-          float v[16];
-#pragma unroll
-          for (int i = 0; i < 16; ++i) {
-            float a = __uint_as_float(r[i]);
-            if (job.bias_off >= 0) a += __ldg(bias + job.bias_off + col + i);
-            v[i] = GELU ? gelu_erf(a) : a;
+          for (int ks = 0; ks < kChunkK / 16; ++ks) {
+            const uint64_t da = umma_smem_desc_sw128(a_base + ks * 32);
+            const uint64_t db = umma_smem_desc(b_base + ks * 2 * w_lbo, w_lbo, 128);
+            umma_bf16_ss(d_addr, da, db, idesc, (kc | ks) != 0 ? 1u : 0u);
           }
-          OutT* dst = out + (static_cast<size_t>(job.out_mat) * T + t) * ldo + job.out_col + col;
-          store_row16<OutT>(dst, v);
+          umma_commit(smem_addr(&hdr->empty[c % n_stages]));
+          if (kc + 1 == n_chunks) umma_commit(smem_addr(&hdr->acc_full[buf]));
         }
+        issued = c + 1;
+        __syncwarp();
       }
-      tc_fence_before_sync();
-      __syncthreads();        // all accumulator reads done before the next tile's first MMA overwrites it
+      if ((failed || hdr->abort) && issued > 0)      // outstanding MMAs: one more bounded chance before TMEM is freed
+        (void)mbar_wait_bounded(smem_addr(&hdr->empty[(issued - 1) % n_stages]), ((issued - 1) / n_stages) & 1);
+    } else if (warp >= kEpilogueWarp0) {
+      // ---- epilogue: warp w owns TMEM lanes 32*(w%4).. = token rows of the tile
+      const uint32_t q = warp & 3;
+      for (uint32_t ti = 0; ti < my_mtiles && !failed; ++ti) {
+        const uint32_t buf = ti & 1;
+        if (hdr->abort) break;
+        if (!mbar_wait_bounded(smem_addr(&hdr->acc_full[buf]), (ti >> 1) & 1)) { failed = true; break; }
+        tc_fence_after_sync();
+        const int t = static_cast<int>((blockIdx.y + ti * gridDim.y) * kTileM + q * 32 + lane);
+        for (uint32_t col = 0; col < n_rows; col += 16) {
+          uint32_t r[16];
+          tmem_ld_32x32b_x16(tmem_base + ((q * 32) << 16) + buf * n_rows + col, r);
+          tc_wait_ld();
+          if (t < T) {
+            float v[16];
+#pragma unroll
+            for (int i = 0; i < 16; ++i) {
+              float a = __uint_as_float(r[i]);
+              if (job.bias_off >= 0) a += __ldg(bias + job.bias_off + col + i);
+              v[i] = GELU ? gelu_erf(a) : a;
+            }
+            OutT* dst = out + (static_cast<size_t>(job.out_mat) * T + t) * ldo + job.out_col + col;
+            store_row16<OutT>(dst, v);
+          }
+        }
+        tc_fence_before_sync();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(smem_addr(&hdr->acc_empty[buf]));
+      }
     }
-    cp_async_wait<0>();       // no copy of this CTA may still be in flight when it exits
-    if (failed && tid == 0) atomicCAS(err, ERR_NONE, ERR_WAIT_TIMEOUT);
-    // Every MMA this CTA issued has completed (acc_full was waited for after the last tile) unless a
-    // wait ran out; in that case give outstanding MMAs one more bounded chance before freeing TMEM.
-    if (failed && issued > 0) {
-      const uint32_t last = issued - 1;
-      (void)mbar_wait_bounded(smem_addr(&hdr->mma_done[last % n_stages]), (last / n_stages) & 1);
+    if (failed) {
+      hdr->abort = 1;
+      if (lane == 0) atomicCAS(err, ERR_NONE, ERR_WAIT_TIMEOUT);
     }
     tc_fence_before_sync();
     __syncthreads();
-    if (warp == 0) tmem_dealloc(tmem_base, tmem_cols);
+    if (warp == 1) tmem_dealloc(tmem_base, tmem_cols);
   }
 }
 
@@ -394,10 +387,10 @@ cudaError_t launch_t(const GemmLaunch& p, cudaStream_t s) {
   const __nv_bfloat16* x = static_cast<const __nv_bfloat16*>(p.x);
   if (p.simt_debug)
     dqgemm_kernel<OutT, GELU, true><<<grid, block, p.smem_bytes, s>>>(
-        p.jobs, p.segs, x, p.ldx, p.T, static_cast<OutT*>(p.out), p.ldo, p.bias, p.err, p.n_stages, p.w_bytes);
+        p.xmap, p.jobs, p.segs, x, p.ldx, p.T, static_cast<OutT*>(p.out), p.ldo, p.bias, p.err, p.n_stages, p.w_bytes);
   else
     dqgemm_kernel<OutT, GELU, false><<<grid, block, p.smem_bytes, s>>>(
-        p.jobs, p.segs, x, p.ldx, p.T, static_cast<OutT*>(p.out), p.ldo, p.bias, p.err, p.n_stages, p.w_bytes);
+        p.xmap, p.jobs, p.segs, x, p.ldx, p.T, static_cast<OutT*>(p.out), p.ldo, p.bias, p.err, p.n_stages, p.w_bytes);
   return cudaGetLastError();
 }
 
@@ -411,12 +404,13 @@ cudaError_t set_smem(K kernel) {
 size_t gemm_weight_bytes(uint32_t n_rows, uint32_t k_total) { return static_cast<size_t>(n_rows) * k_total * 2; }
 
 size_t gemm_smem_bytes(uint32_t w_bytes, uint32_t n_stages) {
-  return kHeaderBytes + static_cast<size_t>(w_bytes) + static_cast<size_t>(n_stages) * kStageBytes;
+  return kAlignSlack + kHeaderBytes + static_cast<size_t>(w_bytes) + static_cast<size_t>(n_stages) * kStageBytes;
 }
 
 uint32_t gemm_pick_stages(uint32_t w_bytes) {
-  const size_t room = 227 * 1024 - kHeaderBytes - static_cast<size_t>(w_bytes);
-  const size_t s = room / kStageBytes;
+  const long room = 227L * 1024 - kAlignSlack - kHeaderBytes - static_cast<long>(w_bytes);
+  if (room < 0) return 0;
+  const long s = room / kStageBytes;
   return static_cast<uint32_t>(s > 6 ? 6 : s);       // fewer than 3 means the tile does not fit
 }
 

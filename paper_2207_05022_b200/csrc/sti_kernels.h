@@ -1,6 +1,7 @@
 // Internal interface between the host runtime (api.cu) and the sm_100a kernels.
 // Nothing here is part of the public ABI.
 #pragma once
+#include <cuda.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
 
@@ -46,6 +47,7 @@ struct GemmLaunch {
   const Seg* segs;
   int n_jobs;
   int m_ctas;               // CTAs along the token dimension (each loops over its M tiles)
+  CUtensorMap xmap;         // TMA descriptor of x: [T rows, ldx columns] bf16, box 64 x 128, 128-byte swizzle
   const void* x;            // [T, ldx] bf16
   int ldx;
   int T;
