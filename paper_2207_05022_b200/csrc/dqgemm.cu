@@ -25,7 +25,7 @@ namespace sti {
 
 namespace {
 
-constexpr int kThreads = 256;               // warp 0: TMA producer, warp 1: MMA issuer, warps 4-7: epilogue; all decode
+constexpr int kThreads = 512;               // warp 0: TMA producer, warp 1: MMA issuer, warps 4-7: epilogue; all 16 decode
 constexpr int kWarps = kThreads / 32;
 constexpr int kTileM = 128;                 // tokens per MMA tile
 constexpr int kChunkK = 64;                 // activation K per pipeline stage = one 128-byte swizzle row
@@ -35,13 +35,15 @@ constexpr int kHeaderBytes = 4096;          // barriers + segment tables; stages
 constexpr int kAlignSlack = 1024;           // the dynamic shared-memory base is aligned up to 1024 by hand
 constexpr int kMaxSegs = 16;
 constexpr int kTableStride = 64;            // bf16 entries per segment table
-constexpr int kEpilogueWarp0 = 4;
+constexpr int kEpilogueWarp0 = 4;             // epilogue warps 4..11: two per TMEM lane quadrant
+constexpr int kEpilogueWarps = 8;
 
 struct SmemHeader {
   uint64_t full[kMaxStages];     // activation chunk landed (TMA transaction bytes)
   uint64_t empty[kMaxStages];    // the MMAs that read the chunk have completed
   uint64_t acc_full[2];          // accumulator buffer complete
   uint64_t acc_empty[2];         // accumulator buffer drained by the epilogue warps
+  uint64_t drain;                // failure path only: all issued MMAs have completed
   uint32_t tmem_base;
   volatile uint32_t abort;       // a bounded wait ran out somewhere in the CTA
 };
@@ -156,6 +158,7 @@ dqgemm_kernel(const __grid_constant__ CUtensorMap xmap, const Job* __restrict__ 
 
   SmemHeader* hdr = reinterpret_cast<SmemHeader*>(smem);
   uint16_t* tables = reinterpret_cast<uint16_t*>(smem + 1024);                      // [kMaxSegs][64]
+  float* bias_sm = reinterpret_cast<float*>(smem + 1024 + kMaxSegs * kTableStride * 2);   // [n_rows] at 3072
   uint8_t* xsm = smem + kHeaderBytes;                                                // n_stages x 16 KB, 1024-aligned
   uint8_t* wsm = xsm + n_stages * kStageBytes;
 
@@ -174,11 +177,22 @@ dqgemm_kernel(const __grid_constant__ CUtensorMap xmap, const Job* __restrict__ 
                                  ? (n_mtiles - blockIdx.y + gridDim.y - 1) / gridDim.y : 0;
   const uint32_t total = my_mtiles * n_chunks;          // activation chunks this CTA consumes
   const uint32_t xsm_addr = smem_addr(xsm);
-  auto request_chunk = [&](uint32_t c) {                 // one thread
-    const uint32_t bar = smem_addr(&hdr->full[c % n_stages]);
+  // CTAs walk the K range in rotated order so that they do not all ask L2 for the same lines at once
+  const uint32_t rot = blockIdx.x % n_chunks;
+  // one thread: chunk `kcr` (rotated K index) of this CTA's token tile `ti` into ring stage `stage`
+  auto request_chunk = [&](uint32_t stage, uint32_t kcr, uint32_t ti) {
+    const uint32_t bar = smem_addr(&hdr->full[stage]);
     mbar_expect_tx(bar, kStageBytes);
-    tma_load_2d(xsm_addr + (c % n_stages) * kStageBytes, &xmap, static_cast<int>(job.x_koff + (c % n_chunks) * kChunkK),
-                static_cast<int>((blockIdx.y + (c / n_chunks) * gridDim.y) * kTileM), bar);
+    tma_load_2d(xsm_addr + stage * kStageBytes, &xmap, static_cast<int>(job.x_koff + kcr * kChunkK),
+                static_cast<int>((blockIdx.y + ti * gridDim.y) * kTileM), bar);
+  };
+  // running position of the producer: next chunk to request
+  uint32_t p_c = 0, p_stage = 0, p_kcr = rot, p_kc = 0, p_ti = 0;
+  auto producer_advance = [&]() {
+    ++p_c;
+    if (++p_stage == n_stages) p_stage = 0;
+    if (++p_kcr == n_chunks) p_kcr = 0;
+    if (++p_kc == n_chunks) { p_kc = 0; ++p_ti; }
   };
 
   uint32_t tmem_cols = 32;
@@ -191,13 +205,14 @@ dqgemm_kernel(const __grid_constant__ CUtensorMap xmap, const Job* __restrict__ 
       }
       for (int b = 0; b < 2; ++b) {
         mbar_init(smem_addr(&hdr->acc_full[b]), 1);
-        mbar_init(smem_addr(&hdr->acc_empty[b]), 4);     // one arrival per epilogue warp
+        mbar_init(smem_addr(&hdr->acc_empty[b]), kEpilogueWarps);     // one arrival per epilogue warp
       }
+      mbar_init(smem_addr(&hdr->drain), 1);
       hdr->abort = 0;
       mbar_fence_init();
       fence_proxy_async_smem();
       // activations first: the ring is filled while the weights are being decoded
-      for (uint32_t c = 0; c < n_stages && c < total; ++c) request_chunk(c);
+      while (p_c < n_stages && p_c < total) { request_chunk(p_stage, p_kcr, p_ti); producer_advance(); }
     }
     if (warp == 1) {
       tmem_alloc(smem_addr(&hdr->tmem_base), tmem_cols);
@@ -209,6 +224,15 @@ dqgemm_kernel(const __grid_constant__ CUtensorMap xmap, const Job* __restrict__ 
     const Seg& sg = segs[job.seg_begin + i / kTableStride];
     const uint32_t e = i % kTableStride;
     tables[i] = (sg.bits <= 6 && e < (1u << sg.bits)) ? bf16_bits(__ldg(sg.table + e)) : 0;
+  }
+  if (tid < n_rows) bias_sm[tid] = job.bias_off >= 0 ? __ldg(bias + job.bias_off + tid) : 0.f;
+  // outlier lists are needed right after the decode: start pulling them towards L2 now
+  for (uint32_t si = 0; si < job.n_seg; ++si) {
+    const Seg& sg = segs[job.seg_begin + si];
+    for (uint32_t o = tid * 32; o < sg.n_out; o += kThreads * 32) {
+      asm volatile("prefetch.global.L2 [%0];" ::"l"(sg.out_off + o));
+      asm volatile("prefetch.global.L2 [%0];" ::"l"(sg.out_val + o));
+    }
   }
   tc_fence_before_sync();
   __syncthreads();
@@ -258,12 +282,12 @@ dqgemm_kernel(const __grid_constant__ CUtensorMap xmap, const Job* __restrict__ 
   if constexpr (SIMT) {
     // Debug path: the decoded tile multiplied on the plain ALUs, activations straight from global memory.
     for (int mt = blockIdx.y; mt < n_mtiles; mt += gridDim.y) {
-      const uint32_t row = tid & 127, chalf = tid >> 7, ncol = n_rows / 2;
+      const uint32_t row = tid & 127, chalf = (tid >> 7) & 1, ncol = n_rows / 2;   // threads 0..255 work
       const int t = mt * kTileM + static_cast<int>(row);
       float acc[64];
 #pragma unroll
       for (int c = 0; c < 64; ++c) acc[c] = 0.f;
-      if (t < T) {
+      if (t < T && tid < 256) {
         for (uint32_t kg = 0; kg < k_total; ++kg) {
           const float a = __bfloat162float(x[static_cast<size_t>(t) * ldx + job.x_koff + kg]);
 #pragma unroll
@@ -281,8 +305,7 @@ dqgemm_kernel(const __grid_constant__ CUtensorMap xmap, const Job* __restrict__ 
             float v[16];
 #pragma unroll
             for (int c = 0; c < 16; ++c) {
-              float a = acc[cb * 16 + c];
-              if (job.bias_off >= 0) a += __ldg(bias + job.bias_off + chalf * ncol + cb * 16 + c);
+              const float a = acc[cb * 16 + c] + bias_sm[chalf * ncol + cb * 16 + c];
               v[c] = GELU ? gelu_erf(a) : a;
             }
             OutT* dst = out + (static_cast<size_t>(job.out_mat) * T + t) * ldo + job.out_col + chalf * ncol + cb * 16;
@@ -295,75 +318,109 @@ dqgemm_kernel(const __grid_constant__ CUtensorMap xmap, const Job* __restrict__ 
     bool failed = false;
     if (warp == 0) {
       // ---- producer: refill a stage as soon as the MMAs that read it have completed
-      uint32_t requested = n_stages < total ? n_stages : total;
-      for (uint32_t c = n_stages; c < total && !failed; ++c) {
-        if (hdr->abort) break;
-        if (!mbar_wait_bounded(smem_addr(&hdr->empty[c % n_stages]), ((c / n_stages) - 1) & 1)) { failed = true; break; }
-        if (lane == 0) request_chunk(c);
-        requested = c + 1;
-        __syncwarp();
+      // (thread 0 already requested the first n_stages chunks; the other lanes catch up on the counters)
+      if (lane == 0) {
+        uint32_t p_phase = 0;                 // parity of the `empty` completion being waited for
+        while (p_c < total) {
+          if (!mbar_wait_bounded_relaxed(smem_addr(&hdr->empty[p_stage]), p_phase)) { failed = true; break; }
+          request_chunk(p_stage, p_kcr, p_ti);
+          if (p_stage + 1 == n_stages) p_phase ^= 1;
+          producer_advance();
+        }
+        if (failed) {
+          // give every copy this CTA requested a bounded chance to land before the CTA exits
+          const uint32_t first = p_c > n_stages ? p_c - n_stages : 0;
+          for (uint32_t c = first; c < p_c; ++c)
+            (void)mbar_wait_bounded(smem_addr(&hdr->full[c % n_stages]), (c / n_stages) & 1);
+        }
       }
-      if (failed || hdr->abort) {
-        // give every copy this CTA requested a bounded chance to land before the CTA exits
-        const uint32_t first = requested > n_stages ? requested - n_stages : 0;
-        for (uint32_t c = first; c < requested; ++c)
-          (void)mbar_wait_bounded(smem_addr(&hdr->full[c % n_stages]), (c / n_stages) & 1);
-      }
+      __syncwarp();
     } else if (warp == 1) {
-      // ---- MMA issuer
+      // ---- MMA issuer.  Descriptors are built once; per instruction only their start address moves.
       const uint32_t idesc = umma_idesc_bf16_m128(n_rows);
       const uint32_t w_lbo = n_rows * 16;
-      const uint32_t wsm_addr = smem_addr(wsm);
-      uint32_t issued = 0;
-      for (uint32_t c = 0; c < total && !failed; ++c) {
-        const uint32_t kc = c % n_chunks, ti = c / n_chunks, buf = ti & 1;
-        if (hdr->abort) break;
-        if (kc == 0 && ti >= 2) {      // the epilogue must have drained this accumulator
-          if (!mbar_wait_bounded(smem_addr(&hdr->acc_empty[buf]), ((ti >> 1) - 1) & 1)) { failed = true; break; }
-        }
-        if (!mbar_wait_bounded(smem_addr(&hdr->full[c % n_stages]), (c / n_stages) & 1)) { failed = true; break; }
-        tc_fence_after_sync();
-        if (lane == 0) {
-          const uint32_t a_base = xsm_addr + (c % n_stages) * kStageBytes;
-          const uint32_t b_base = wsm_addr + (kc * (kChunkK / 8)) * w_lbo;
-          const uint32_t d_addr = tmem_base + buf * n_rows;
-#pragma unroll
-          for (int ks = 0; ks < kChunkK / 16; ++ks) {
-            const uint64_t da = umma_smem_desc_sw128(a_base + ks * 32);
-            const uint64_t db = umma_smem_desc(b_base + ks * 2 * w_lbo, w_lbo, 128);
-            umma_bf16_ss(d_addr, da, db, idesc, (kc | ks) != 0 ? 1u : 0u);
+      const uint64_t a_desc0 = umma_smem_desc_sw128(xsm_addr);
+      const uint64_t b_desc0 = umma_smem_desc(smem_addr(wsm), w_lbo, 128);
+      const uint32_t a_stage_step = kStageBytes >> 4;          // next ring stage
+      const uint32_t b_ks_step = (2 * w_lbo) >> 4;             // next 16 columns of the weight tile
+      const uint32_t b_chunk_step = 4 * b_ks_step;             // next 64 columns
+      if (lane == 0) {
+        uint32_t stage = 0, phase = 0, kc = 0, kcr = rot, ti = 0, issued = 0;
+        for (uint32_t c = 0; c < total; ++c) {
+          const uint32_t buf = ti & 1;
+          if (kc == 0 && ti >= 2) {      // the epilogue must have drained this accumulator
+            if (!mbar_wait_bounded(smem_addr(&hdr->acc_empty[buf]), ((ti >> 1) - 1) & 1)) { failed = true; break; }
           }
-          umma_commit(smem_addr(&hdr->empty[c % n_stages]));
+          if (!mbar_wait_bounded(smem_addr(&hdr->full[stage]), phase)) { failed = true; break; }
+          tc_fence_after_sync();
+          const uint64_t da = a_desc0 + stage * a_stage_step;
+          const uint64_t db = b_desc0 + kcr * b_chunk_step;
+          const uint32_t d_addr = tmem_base + buf * n_rows;
+          umma_bf16_ss(d_addr, da, db, idesc, kc != 0 ? 1u : 0u);
+          umma_bf16_ss(d_addr, da + 2, db + b_ks_step, idesc, 1u);          // +32 bytes inside the swizzled row
+          umma_bf16_ss(d_addr, da + 4, db + 2 * b_ks_step, idesc, 1u);
+          umma_bf16_ss(d_addr, da + 6, db + 3 * b_ks_step, idesc, 1u);
+          if (c + n_stages < total) umma_commit(smem_addr(&hdr->empty[stage]));   // only if the stage is refilled
           if (kc + 1 == n_chunks) umma_commit(smem_addr(&hdr->acc_full[buf]));
+          issued = c + 1;
+          if (++stage == n_stages) { stage = 0; phase ^= 1; }
+          if (++kcr == n_chunks) kcr = 0;
+          if (++kc == n_chunks) { kc = 0; ++ti; }
         }
-        issued = c + 1;
-        __syncwarp();
+        if (failed && issued > 0) {
+          // outstanding MMAs: a commit of its own and one more bounded chance before TMEM is freed
+          umma_commit(smem_addr(&hdr->drain));
+          (void)mbar_wait_bounded(smem_addr(&hdr->drain), 0);
+        }
       }
-      if ((failed || hdr->abort) && issued > 0)      // outstanding MMAs: one more bounded chance before TMEM is freed
-        (void)mbar_wait_bounded(smem_addr(&hdr->empty[(issued - 1) % n_stages]), ((issued - 1) / n_stages) & 1);
-    } else if (warp >= kEpilogueWarp0) {
-      // ---- epilogue: warp w owns TMEM lanes 32*(w%4).. = token rows of the tile
-      const uint32_t q = warp & 3;
-      for (uint32_t ti = 0; ti < my_mtiles && !failed; ++ti) {
+      __syncwarp();
+    } else if (warp >= kEpilogueWarp0 && warp < kEpilogueWarp0 + kEpilogueWarps) {
+      // ---- epilogue: warp w owns TMEM lanes 32*(w%4).. (token rows) and one half of the columns
+      const uint32_t q = warp & 3, half = (warp - kEpilogueWarp0) >> 2, ncol = n_rows / 2;
+      for (uint32_t ti = 0; ti < my_mtiles; ++ti) {
         const uint32_t buf = ti & 1;
-        if (hdr->abort) break;
-        if (!mbar_wait_bounded(smem_addr(&hdr->acc_full[buf]), (ti >> 1) & 1)) { failed = true; break; }
+        // one lane polls (a whole CTA's worth of pollers on one barrier word slows the MMA warp's own
+        // barrier traffic down); the warp then re-converges before it touches tensor memory
+        uint32_t ok = 1;
+        if (lane == 0) ok = mbar_wait_bounded_relaxed(smem_addr(&hdr->acc_full[buf]), (ti >> 1) & 1) ? 1u : 0u;
+        ok = __shfl_sync(0xffffffffu, ok, 0);
+        if (!ok) { failed = true; break; }
         tc_fence_after_sync();
         const int t = static_cast<int>((blockIdx.y + ti * gridDim.y) * kTileM + q * 32 + lane);
-        for (uint32_t col = 0; col < n_rows; col += 16) {
+        OutT* drow = out + (static_cast<size_t>(job.out_mat) * T + (t < T ? t : 0)) * ldo + job.out_col;
+        const uint32_t taddr = tmem_base + ((q * 32) << 16) + buf * n_rows;
+        if (ncol >= 32) {
+          // 32 columns per step: each thread then writes 128 (fp32) or 64 (bf16) contiguous bytes of its row
+          for (uint32_t col = half * ncol; col < (half + 1) * ncol; col += 32) {
+            uint32_t r[32];
+            tmem_ld_32x32b_x32(taddr + col, r);
+            tc_wait_ld();
+            if (t < T) {
+#pragma unroll
+              for (int h = 0; h < 2; ++h) {
+                float v[16];
+#pragma unroll
+                for (int i = 0; i < 16; ++i) {
+                  const float a = __uint_as_float(r[h * 16 + i]) + bias_sm[col + h * 16 + i];
+                  v[i] = GELU ? gelu_erf(a) : a;
+                }
+                store_row16<OutT>(drow + col + h * 16, v);
+              }
+            }
+          }
+        } else {
+          const uint32_t col = half * ncol;      // 16 columns
           uint32_t r[16];
-          tmem_ld_32x32b_x16(tmem_base + ((q * 32) << 16) + buf * n_rows + col, r);
+          tmem_ld_32x32b_x16(taddr + col, r);
           tc_wait_ld();
           if (t < T) {
             float v[16];
 #pragma unroll
             for (int i = 0; i < 16; ++i) {
-              float a = __uint_as_float(r[i]);
-              if (job.bias_off >= 0) a += __ldg(bias + job.bias_off + col + i);
+              const float a = __uint_as_float(r[i]) + bias_sm[col + i];
               v[i] = GELU ? gelu_erf(a) : a;
             }
-            OutT* dst = out + (static_cast<size_t>(job.out_mat) * T + t) * ldo + job.out_col + col;
-            store_row16<OutT>(dst, v);
+            store_row16<OutT>(drow + col, v);
           }
         }
         tc_fence_before_sync();
