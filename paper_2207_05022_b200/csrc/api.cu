@@ -49,7 +49,7 @@ struct GemmTable {
   Seg* segs = nullptr;
   int n_jobs = 0;
   size_t smem = 0;
-  uint32_t w_bytes = 0, n_stages = 0;
+  uint32_t w_bytes = 0, n_stages = 0, bps = 1, k_max = 0;
   int n_split = 0;
 };
 
@@ -62,6 +62,7 @@ struct Layer {
   int slot = -1;                       // ring slot of the streamed part
   GemmTable qkv, o, f1, f2;
   cudaEvent_t ev_loaded = nullptr, ev_done = nullptr, ev_copy_start = nullptr, ev_comp_start = nullptr;
+  cudaEvent_t g_ev_loaded = nullptr;   // the same role inside graph capture (captured events cannot be reused outside)
   cudaEvent_t ev_k[8] = {};           // boundaries of the seven kernels (kernel-level profiling)
   bool k_ran[7] = {};
 };
@@ -85,6 +86,17 @@ struct sti_ctx {
   uint32_t attn_weights = 0, ffn_weights = 0;
 };
 
+struct ForwardKey {
+  const void* x = nullptr; void* y = nullptr;            // device buffers (device variant)
+  const void* x_host = nullptr; void* y_host = nullptr;  // host buffers (host variant)
+  const int32_t* lens = nullptr;                         // device
+  int batch = 0, seq = 0;
+  bool operator==(const ForwardKey& o) const {
+    return x == o.x && y == o.y && x_host == o.x_host && y_host == o.y_host && lens == o.lens && batch == o.batch &&
+           seq == o.seq;
+  }
+};
+
 struct sti_plan {
   sti_ctx* ctx = nullptr;
   std::vector<Layer> layers;
@@ -97,8 +109,12 @@ struct sti_plan {
   uint8_t* pinned = nullptr;   size_t pinned_bytes = 0;
   uint8_t* ring = nullptr;     size_t slot_bytes = 0;
   uint8_t* tables = nullptr;   size_t tables_bytes = 0;       // job/segment descriptors
-  std::vector<cudaEvent_t> slot_free;
-  cudaEvent_t ev_copy_tail = nullptr, ev_begin = nullptr, ev_end = nullptr;
+  std::vector<cudaEvent_t> slot_free, g_slot_free;   // direct launches / graph capture
+  cudaEvent_t ev_copy_tail = nullptr, ev_begin = nullptr, ev_end = nullptr, ev_fork = nullptr, g_ev_join = nullptr;
+  cudaGraphExec_t gexec = nullptr;     // graph of the last forward
+  ForwardKey gkey;
+  uint64_t glaunches = 0;
+  bool graph_off = false;
   bool copy_tail_valid = false;
   // activation scratch
   uint16_t* qkv = nullptr; uint16_t* attn_out = nullptr; float* partial = nullptr;
@@ -177,7 +193,10 @@ void parse_tuning(Tuning* t, int tmax, const sti_model_desc& d) {
   t->o_group = std::max(1, std::min(t->o_group, 16));
   t->f2_group = std::max(1, std::min(t->f2_group, 16));
   // keep every weight tile inside shared memory
-  auto fits = [](int n, int k) { return gemm_pick_stages(static_cast<uint32_t>(gemm_weight_bytes(n, k))) >= 4; };
+  auto fits = [](int n, int k) {
+    uint32_t st = 0, bp = 0;
+    return gemm_pick_ring(static_cast<uint32_t>(gemm_weight_bytes(n, k)), k, &st, &bp) && st * bp >= 4;
+  };
   while (t->qkv_n > 32 && !fits(t->qkv_n, d.hidden)) t->qkv_n /= 2;
   while (t->f1_n > 32 && !fits(t->f1_n, d.hidden)) t->f1_n /= 2;
   while (t->o_group > 1 && !fits(t->o_n, t->o_group * 64)) --t->o_group;
@@ -218,13 +237,14 @@ Seg make_seg(const sti_ctx* c, const Unit& u, sti_kind kind, int m, uint32_t row
 struct TableBuilder {
   std::vector<Job> jobs;
   std::vector<Seg> segs;
-  uint32_t w_bytes = 0;
+  uint32_t w_bytes = 0, k_max = 0;
   void add(Job j, const std::vector<Seg>& ss) {
     j.seg_begin = static_cast<uint32_t>(segs.size());
     j.n_seg = static_cast<uint32_t>(ss.size());
     segs.insert(segs.end(), ss.begin(), ss.end());
     jobs.push_back(j);
     w_bytes = std::max(w_bytes, static_cast<uint32_t>(gemm_weight_bytes(j.n_rows, j.k_total)));
+    k_max = std::max(k_max, j.k_total);
   }
 };
 
@@ -343,7 +363,7 @@ sti_status run_gemm(sti_plan* p, GemmKind kind, const GemmTable& tab, const void
   g.jobs = tab.jobs; g.segs = tab.segs; g.n_jobs = tab.n_jobs; g.m_ctas = m_ctas_for(tab.n_jobs, T);
   if (!make_xmap(&g.xmap, x, ldx, T)) return STI_ERR_CUDA;
   g.x = x; g.ldx = ldx; g.T = T; g.out = out; g.ldo = ldo; g.bias = bias; g.err = p->ctx->err_dev;
-  g.smem_bytes = tab.smem; g.n_stages = tab.n_stages; g.w_bytes = tab.w_bytes; g.simt_debug = p->ctx->simt_debug;
+  g.smem_bytes = tab.smem; g.n_stages = tab.n_stages; g.bps = tab.bps; g.w_bytes = tab.w_bytes; g.simt_debug = p->ctx->simt_debug;
   CUDA_TRY(launch_gemm(kind, g, p->ctx->compute));
   p->ctx->launches++;
   return STI_OK;
@@ -442,39 +462,119 @@ sti_status enqueue_layer_copy(sti_plan* p, int li, cudaStream_t s) {
   return STI_OK;
 }
 
-sti_status model_forward_impl(sti_plan* p, const void* x, void* y, int batch, int seq, const int32_t* lens) {
+// Enqueues one whole forward: per layer the shard copy on the copy stream and the seven kernels on the
+// compute stream, ordered by events.  With `capturing` the same calls are recorded into a CUDA graph:
+// the copy stream is forked from and joined back into the compute stream, and a ring slot's "free" event
+// is only waited for when it was recorded inside this forward (stream order covers earlier forwards).
+sti_status enqueue_forward(sti_plan* p, const void* x, void* y, int batch, int seq, const int32_t* lens,
+                           bool capturing) {
   sti_ctx* c = p->ctx;
   const int n = static_cast<int>(p->layers.size());
-  if (p->profiling) CUDA_TRY(cudaEventRecord(p->ev_begin, c->compute));
-  // the copy stream must not run ahead of work already enqueued on the compute stream that may still
-  // read ring slots: slot_free events order that; nothing else is shared between the streams
+  const bool prof = p->profiling && !capturing;
+  bool any_streamed = false;
+  for (auto& L : p->layers) any_streamed |= L.str_bytes > 0;
+  std::vector<char> slot_used(p->ring_slots, 0);
+  if (prof) CUDA_TRY(cudaEventRecord(p->ev_begin, c->compute));
+  if (capturing && any_streamed) {
+    CUDA_TRY(cudaEventRecord(p->ev_fork, c->compute));
+    CUDA_TRY(cudaStreamWaitEvent(c->copy, p->ev_fork, 0));
+  }
   const void* cur = x;
   for (int li = 0; li < n; ++li) {
     Layer& L = p->layers[li];
     if (L.str_bytes > 0) {
       // one IO job per layer (Section 3.1); the slot is reused only after its previous layer finished
-      CUDA_TRY(cudaStreamWaitEvent(c->copy, p->slot_free[L.slot], 0));
-      if (p->profiling) CUDA_TRY(cudaEventRecord(L.ev_copy_start, c->copy));
+      if (!capturing) CUDA_TRY(cudaStreamWaitEvent(c->copy, p->slot_free[L.slot], 0));
+      else if (slot_used[L.slot]) CUDA_TRY(cudaStreamWaitEvent(c->copy, p->g_slot_free[L.slot], 0));
+      if (prof) CUDA_TRY(cudaEventRecord(L.ev_copy_start, c->copy));
       sti_status st = enqueue_layer_copy(p, li, c->copy);
       if (st != STI_OK) return st;
-      CUDA_TRY(cudaEventRecord(L.ev_loaded, c->copy));
+      cudaEvent_t loaded = capturing ? L.g_ev_loaded : L.ev_loaded;
+      CUDA_TRY(cudaEventRecord(loaded, c->copy));
       // a layer starts only when its own shards (and, by stream order, all earlier ones) are loaded
-      CUDA_TRY(cudaStreamWaitEvent(c->compute, L.ev_loaded, 0));
+      CUDA_TRY(cudaStreamWaitEvent(c->compute, loaded, 0));
     }
-    if (p->profiling) CUDA_TRY(cudaEventRecord(L.ev_comp_start, c->compute));
+    if (prof) CUDA_TRY(cudaEventRecord(L.ev_comp_start, c->compute));
     void* nxt = (li == n - 1) ? y : p->buf[li & 1];
     sti_status st = enqueue_layer(p, li, cur, nxt, batch, seq, lens, li > 0, li + 1 < n);
     if (st != STI_OK) return st;
-    if (p->profiling) CUDA_TRY(cudaEventRecord(L.ev_done, c->compute));
-    if (L.str_bytes > 0) CUDA_TRY(cudaEventRecord(p->slot_free[L.slot], c->compute));
+    if (prof) CUDA_TRY(cudaEventRecord(L.ev_done, c->compute));
+    if (L.str_bytes > 0) {
+      CUDA_TRY(cudaEventRecord(capturing ? p->g_slot_free[L.slot] : p->slot_free[L.slot], c->compute));
+      slot_used[L.slot] = 1;
+    }
     cur = nxt;
   }
-  CUDA_TRY(cudaEventRecord(p->ev_copy_tail, c->copy));
-  p->copy_tail_valid = true;
-  if (p->profiling) {
+  if (!capturing) {
+    CUDA_TRY(cudaEventRecord(p->ev_copy_tail, c->copy));
+    p->copy_tail_valid = true;
+  } else if (any_streamed) {
+    CUDA_TRY(cudaEventRecord(p->g_ev_join, c->copy));
+    CUDA_TRY(cudaStreamWaitEvent(c->compute, p->g_ev_join, 0));   // join the copy stream back
+  }
+  if (prof) {
     CUDA_TRY(cudaEventRecord(p->ev_end, c->compute));
     p->stats_valid = true;
   }
+  return STI_OK;
+}
+
+// Body of a forward with optional host staging of x and y (all on the compute stream around the layers).
+sti_status enqueue_forward_io(sti_plan* p, const ForwardKey& k, bool capturing) {
+  sti_ctx* c = p->ctx;
+  const size_t bytes = static_cast<size_t>(k.batch) * k.seq * c->desc.hidden * act_size(c);
+  const void* x = k.x;
+  void* y = k.y;
+  if (k.x_host) {
+    CUDA_TRY(cudaMemcpyAsync(p->x_in, k.x_host, bytes, cudaMemcpyHostToDevice, c->compute));
+    x = p->x_in;
+    y = p->y_out;
+  }
+  sti_status st = enqueue_forward(p, x, y, k.batch, k.seq, k.lens, capturing);
+  if (st != STI_OK) return st;
+  if (k.y_host) CUDA_TRY(cudaMemcpyAsync(k.y_host, p->y_out, bytes, cudaMemcpyDeviceToHost, c->compute));
+  return STI_OK;
+}
+
+// A forward with the same buffers and shape as the previous one replays its CUDA graph (one launch instead of
+// ~7 per layer, no per-kernel host work); anything else is captured anew.  Profiling runs ungraphed.
+sti_status model_forward_impl(sti_plan* p, const ForwardKey& k) {
+  sti_ctx* c = p->ctx;
+  if (p->profiling || p->graph_off) return enqueue_forward_io(p, k, false);
+  if (!(p->gexec && p->gkey == k)) {
+    if (p->gexec) { cudaGraphExecDestroy(p->gexec); p->gexec = nullptr; }
+    const uint64_t launches_before = c->launches;
+    cudaGraph_t graph = nullptr;
+    if (cudaStreamBeginCapture(c->compute, cudaStreamCaptureModeRelaxed) != cudaSuccess) {
+      (void)cudaGetLastError();
+      p->graph_off = true;
+      return enqueue_forward_io(p, k, false);
+    }
+    const sti_status st = enqueue_forward_io(p, k, true);
+    const cudaError_t ce = cudaStreamEndCapture(c->compute, &graph);
+    p->glaunches = c->launches - launches_before;
+    c->launches = launches_before;
+    if (st != STI_OK || ce != cudaSuccess || !graph) {
+      (void)cudaGetLastError();
+      if (graph) cudaGraphDestroy(graph);
+      p->graph_off = true;            // fall back to plain stream launches for this plan
+      return st != STI_OK ? st : enqueue_forward_io(p, k, false);
+    }
+    const cudaError_t ie = cudaGraphInstantiate(&p->gexec, graph, 0);
+    cudaGraphDestroy(graph);
+    if (ie != cudaSuccess) {
+      (void)cudaGetLastError();
+      p->gexec = nullptr;
+      p->graph_off = true;
+      return enqueue_forward_io(p, k, false);
+    }
+    p->gkey = k;
+  }
+  CUDA_TRY(cudaGraphLaunch(p->gexec, c->compute));
+  // later ungraphed work (profiled forwards, single layers) must not reuse a ring slot before this graph is done
+  for (auto e : p->slot_free) CUDA_TRY(cudaEventRecord(e, c->compute));
+  c->launches += p->glaunches;
+  p->copy_tail_valid = false;
   return STI_OK;
 }
 
@@ -487,13 +587,18 @@ void free_plan_device(sti_plan* p) {
   cudaFree(p->lens_dev);
   for (auto& L : p->layers) {
     if (L.ev_loaded) cudaEventDestroy(L.ev_loaded);
+    if (L.g_ev_loaded) cudaEventDestroy(L.g_ev_loaded);
     if (L.ev_done) cudaEventDestroy(L.ev_done);
     if (L.ev_copy_start) cudaEventDestroy(L.ev_copy_start);
     if (L.ev_comp_start) cudaEventDestroy(L.ev_comp_start);
     for (auto e : L.ev_k) if (e) cudaEventDestroy(e);
   }
   for (auto e : p->slot_free) cudaEventDestroy(e);
+  for (auto e : p->g_slot_free) cudaEventDestroy(e);
+  if (p->g_ev_join) cudaEventDestroy(p->g_ev_join);
   if (p->ev_copy_tail) cudaEventDestroy(p->ev_copy_tail);
+  if (p->ev_fork) cudaEventDestroy(p->ev_fork);
+  if (p->gexec) cudaGraphExecDestroy(p->gexec);
   if (p->ev_begin) cudaEventDestroy(p->ev_begin);
   if (p->ev_end) cudaEventDestroy(p->ev_end);
 }
@@ -768,10 +873,10 @@ sti_status sti_plan_finalize(sti_plan* p) {
     for (int i = 0; i < 4; ++i) {
       gt[i]->n_jobs = static_cast<int>(tb[i].jobs.size());
       gt[i]->w_bytes = tb[i].w_bytes;
-      gt[i]->n_stages = gemm_pick_stages(tb[i].w_bytes);
-      if (!tb[i].jobs.empty() && gt[i]->n_stages < 3) return STI_ERR_SHAPE;
-      gt[i]->n_stages = std::max(3u, gt[i]->n_stages);
-      gt[i]->smem = gemm_smem_bytes(tb[i].w_bytes, gt[i]->n_stages);
+      gt[i]->n_stages = 2; gt[i]->bps = 1;
+      if (!tb[i].jobs.empty() && !gemm_pick_ring(tb[i].w_bytes, tb[i].k_max, &gt[i]->n_stages, &gt[i]->bps))
+        return STI_ERR_SHAPE;
+      gt[i]->smem = gemm_smem_bytes(tb[i].w_bytes, gt[i]->n_stages, gt[i]->bps);
       if (gt[i]->smem > kMaxSmem && !tb[i].jobs.empty()) return STI_ERR_SHAPE;
       Fix fx{gt[i], 0, 0};
       fx.jobs_off = align16(host_tables.size());
@@ -811,6 +916,7 @@ sti_status sti_plan_finalize(sti_plan* p) {
   const unsigned flags = cudaEventDefault;     // timing-capable; only recorded when profiling
   for (auto& L : p->layers) {
     CUDA_TRY(cudaEventCreateWithFlags(&L.ev_loaded, flags));
+    CUDA_TRY(cudaEventCreateWithFlags(&L.g_ev_loaded, cudaEventDisableTiming));
     CUDA_TRY(cudaEventCreateWithFlags(&L.ev_done, flags));
     CUDA_TRY(cudaEventCreateWithFlags(&L.ev_copy_start, flags));
     CUDA_TRY(cudaEventCreateWithFlags(&L.ev_comp_start, flags));
@@ -822,6 +928,11 @@ sti_status sti_plan_finalize(sti_plan* p) {
     CUDA_TRY(cudaEventRecord(e, c->compute));
   }
   CUDA_TRY(cudaEventCreateWithFlags(&p->ev_copy_tail, cudaEventDisableTiming));
+  CUDA_TRY(cudaEventCreateWithFlags(&p->ev_fork, cudaEventDisableTiming));
+  CUDA_TRY(cudaEventCreateWithFlags(&p->g_ev_join, cudaEventDisableTiming));
+  p->g_slot_free.resize(p->ring_slots);
+  for (auto& e : p->g_slot_free) CUDA_TRY(cudaEventCreateWithFlags(&e, cudaEventDisableTiming));
+  { const char* ng = getenv("STI_NO_GRAPH"); p->graph_off = ng && ng[0] == '1'; }
   CUDA_TRY(cudaEventCreateWithFlags(&p->ev_begin, flags));
   CUDA_TRY(cudaEventCreateWithFlags(&p->ev_end, flags));
   p->finalized = true;
@@ -852,7 +963,9 @@ sti_status sti_model_forward(sti_plan* p, const void* x, void* y, int batch, int
   if (st != STI_OK) return st;
   if ((st = sti_plan_finalize(p)) != STI_OK) return st;
   CUDA_TRY(cudaSetDevice(p->ctx->device));
-  return model_forward_impl(p, x, y, batch, seq, lens);
+  ForwardKey k;
+  k.x = x; k.y = y; k.lens = lens; k.batch = batch; k.seq = seq;
+  return model_forward_impl(p, k);
 }
 
 sti_status sti_model_forward_host(sti_plan* p, const void* x_host, void* y_host, int batch, int seq,
@@ -862,16 +975,14 @@ sti_status sti_model_forward_host(sti_plan* p, const void* x_host, void* y_host,
   if ((st = sti_plan_finalize(p)) != STI_OK) return st;
   sti_ctx* c = p->ctx;
   CUDA_TRY(cudaSetDevice(c->device));
-  const size_t bytes = static_cast<size_t>(batch) * seq * c->desc.hidden * act_size(c);
-  CUDA_TRY(cudaMemcpyAsync(p->x_in, x_host, bytes, cudaMemcpyHostToDevice, c->compute));
-  const int32_t* lens = nullptr;
+  ForwardKey k;
+  k.x_host = x_host; k.y_host = y_host; k.batch = batch; k.seq = seq;
   if (lens_host) {
+    // sequence lengths change from call to call: staged outside the graph
     CUDA_TRY(cudaMemcpyAsync(p->lens_dev, lens_host, static_cast<size_t>(batch) * 4, cudaMemcpyHostToDevice, c->compute));
-    lens = p->lens_dev;
+    k.lens = p->lens_dev;
   }
-  if ((st = model_forward_impl(p, p->x_in, p->y_out, batch, seq, lens)) != STI_OK) return st;
-  CUDA_TRY(cudaMemcpyAsync(y_host, p->y_out, bytes, cudaMemcpyDeviceToHost, c->compute));
-  return STI_OK;
+  return model_forward_impl(p, k);
 }
 
 sti_status sti_sync(sti_ctx* c) {

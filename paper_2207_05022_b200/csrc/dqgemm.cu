@@ -28,9 +28,9 @@ namespace {
 constexpr int kThreads = 512;               // warp 0: TMA producer, warp 1: MMA issuer, warps 4-7: epilogue; all 16 decode
 constexpr int kWarps = kThreads / 32;
 constexpr int kTileM = 128;                 // tokens per MMA tile
-constexpr int kChunkK = 64;                 // activation K per pipeline stage = one 128-byte swizzle row
+constexpr int kChunkK = 64;                 // one TMA box = 64 columns = one 128-byte swizzle row; a stage holds 1, 2 or 4 boxes
 constexpr int kMaxStages = 8;
-constexpr int kStageBytes = kTileM * kChunkK * 2;   // 16 KB
+constexpr int kBoxBytes = kTileM * kChunkK * 2;     // 16 KB
 constexpr int kHeaderBytes = 4096;          // barriers + segment tables; stages start 1024-byte aligned after it
 constexpr int kAlignSlack = 1024;           // the dynamic shared-memory base is aligned up to 1024 by hand
 constexpr int kMaxSegs = 16;
@@ -149,7 +149,8 @@ template <typename OutT, bool GELU, bool SIMT>
 __global__ void __launch_bounds__(kThreads, 1)
 dqgemm_kernel(const __grid_constant__ CUtensorMap xmap, const Job* __restrict__ jobs, const Seg* __restrict__ segs,
               const __nv_bfloat16* __restrict__ x, int ldx, int T, OutT* __restrict__ out, int ldo,
-              const float* __restrict__ bias, int* __restrict__ err, uint32_t n_stages, uint32_t w_bytes) {
+              const float* __restrict__ bias, int* __restrict__ err, uint32_t n_stages, uint32_t bps,
+              uint32_t w_bytes) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = smem_raw + ((1024u - (smem_addr(smem_raw) & 1023u)) & 1023u);
   const uint32_t tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -160,19 +161,21 @@ dqgemm_kernel(const __grid_constant__ CUtensorMap xmap, const Job* __restrict__ 
   uint16_t* tables = reinterpret_cast<uint16_t*>(smem + 1024);                      // [kMaxSegs][64]
   float* bias_sm = reinterpret_cast<float*>(smem + 1024 + kMaxSegs * kTableStride * 2);   // [n_rows] at 3072
   uint8_t* xsm = smem + kHeaderBytes;                                                // n_stages x 16 KB, 1024-aligned
-  uint8_t* wsm = xsm + n_stages * kStageBytes;
+  const uint32_t stage_bytes = bps * kBoxBytes;          // bps boxes of 64 columns per stage
+  uint8_t* wsm = xsm + n_stages * stage_bytes;
 
   // the kernel's own checks of the descriptor: refuse rather than touch memory out of bounds
   const bool bad = job.n_seg == 0 || job.n_seg > kMaxSegs || (n_rows != 32 && n_rows != 64 && n_rows != 128) ||
                    (k_total % kChunkK) != 0 || k_total == 0 || n_rows * k_total * 2 > w_bytes ||
-                   n_stages < 2 || n_stages > kMaxStages;
+                   n_stages < 2 || n_stages > kMaxStages || (bps != 1 && bps != 2 && bps != 4);
   if (bad) {
     if (tid == 0) atomicCAS(err, ERR_NONE, ERR_BAD_JOB);
     return;
   }
 
   const int n_mtiles = (T + kTileM - 1) / kTileM;
-  const uint32_t n_chunks = k_total / kChunkK;
+  const uint32_t n_boxes = k_total / kChunkK;
+  const uint32_t n_chunks = (n_boxes + bps - 1) / bps;  // pipeline steps per token tile
   const uint32_t my_mtiles = blockIdx.y < static_cast<uint32_t>(n_mtiles)
                                  ? (n_mtiles - blockIdx.y + gridDim.y - 1) / gridDim.y : 0;
   const uint32_t total = my_mtiles * n_chunks;          // activation chunks this CTA consumes
@@ -182,9 +185,13 @@ dqgemm_kernel(const __grid_constant__ CUtensorMap xmap, const Job* __restrict__ 
   // one thread: chunk `kcr` (rotated K index) of this CTA's token tile `ti` into ring stage `stage`
   auto request_chunk = [&](uint32_t stage, uint32_t kcr, uint32_t ti) {
     const uint32_t bar = smem_addr(&hdr->full[stage]);
-    mbar_expect_tx(bar, kStageBytes);
-    tma_load_2d(xsm_addr + stage * kStageBytes, &xmap, static_cast<int>(job.x_koff + kcr * kChunkK),
-                static_cast<int>((blockIdx.y + ti * gridDim.y) * kTileM), bar);
+    const uint32_t box0 = kcr * bps;
+    const uint32_t nb = n_boxes - box0 < bps ? n_boxes - box0 : bps;
+    mbar_expect_tx(bar, nb * kBoxBytes);
+    for (uint32_t b = 0; b < nb; ++b)
+      tma_load_2d(xsm_addr + stage * stage_bytes + b * kBoxBytes, &xmap,
+                  static_cast<int>(job.x_koff + (box0 + b) * kChunkK),
+                  static_cast<int>((blockIdx.y + ti * gridDim.y) * kTileM), bar);
   };
   // running position of the producer: next chunk to request
   uint32_t p_c = 0, p_stage = 0, p_kcr = rot, p_kc = 0, p_ti = 0;
@@ -341,7 +348,8 @@ dqgemm_kernel(const __grid_constant__ CUtensorMap xmap, const Job* __restrict__ 
       const uint32_t w_lbo = n_rows * 16;
       const uint64_t a_desc0 = umma_smem_desc_sw128(xsm_addr);
       const uint64_t b_desc0 = umma_smem_desc(smem_addr(wsm), w_lbo, 128);
-      const uint32_t a_stage_step = kStageBytes >> 4;          // next ring stage
+      const uint32_t a_stage_step = stage_bytes >> 4;          // next ring stage
+      const uint32_t a_box_step = kBoxBytes >> 4;              // next 64-column box inside a stage
       const uint32_t b_ks_step = (2 * w_lbo) >> 4;             // next 16 columns of the weight tile
       const uint32_t b_chunk_step = 4 * b_ks_step;             // next 64 columns
       if (lane == 0) {
@@ -353,13 +361,17 @@ dqgemm_kernel(const __grid_constant__ CUtensorMap xmap, const Job* __restrict__ 
           }
           if (!mbar_wait_bounded(smem_addr(&hdr->full[stage]), phase)) { failed = true; break; }
           tc_fence_after_sync();
-          const uint64_t da = a_desc0 + stage * a_stage_step;
-          const uint64_t db = b_desc0 + kcr * b_chunk_step;
+          const uint32_t box0 = kcr * bps;
+          const uint32_t nb = n_boxes - box0 < bps ? n_boxes - box0 : bps;
+          uint64_t da = a_desc0 + stage * a_stage_step;
+          uint64_t db = b_desc0 + box0 * b_chunk_step;
           const uint32_t d_addr = tmem_base + buf * n_rows;
-          umma_bf16_ss(d_addr, da, db, idesc, kc != 0 ? 1u : 0u);
-          umma_bf16_ss(d_addr, da + 2, db + b_ks_step, idesc, 1u);          // +32 bytes inside the swizzled row
-          umma_bf16_ss(d_addr, da + 4, db + 2 * b_ks_step, idesc, 1u);
-          umma_bf16_ss(d_addr, da + 6, db + 3 * b_ks_step, idesc, 1u);
+          for (uint32_t b = 0; b < nb; ++b, da += a_box_step, db += b_chunk_step) {
+            umma_bf16_ss(d_addr, da, db, idesc, (kc | b) != 0 ? 1u : 0u);
+            umma_bf16_ss(d_addr, da + 2, db + b_ks_step, idesc, 1u);          // +32 bytes inside the swizzled row
+            umma_bf16_ss(d_addr, da + 4, db + 2 * b_ks_step, idesc, 1u);
+            umma_bf16_ss(d_addr, da + 6, db + 3 * b_ks_step, idesc, 1u);
+          }
           if (c + n_stages < total) umma_commit(smem_addr(&hdr->empty[stage]));   // only if the stage is refilled
           if (kc + 1 == n_chunks) umma_commit(smem_addr(&hdr->acc_full[buf]));
           issued = c + 1;
@@ -444,10 +456,10 @@ cudaError_t launch_t(const GemmLaunch& p, cudaStream_t s) {
   const __nv_bfloat16* x = static_cast<const __nv_bfloat16*>(p.x);
   if (p.simt_debug)
     dqgemm_kernel<OutT, GELU, true><<<grid, block, p.smem_bytes, s>>>(
-        p.xmap, p.jobs, p.segs, x, p.ldx, p.T, static_cast<OutT*>(p.out), p.ldo, p.bias, p.err, p.n_stages, p.w_bytes);
+        p.xmap, p.jobs, p.segs, x, p.ldx, p.T, static_cast<OutT*>(p.out), p.ldo, p.bias, p.err, p.n_stages, p.bps, p.w_bytes);
   else
     dqgemm_kernel<OutT, GELU, false><<<grid, block, p.smem_bytes, s>>>(
-        p.xmap, p.jobs, p.segs, x, p.ldx, p.T, static_cast<OutT*>(p.out), p.ldo, p.bias, p.err, p.n_stages, p.w_bytes);
+        p.xmap, p.jobs, p.segs, x, p.ldx, p.T, static_cast<OutT*>(p.out), p.ldo, p.bias, p.err, p.n_stages, p.bps, p.w_bytes);
   return cudaGetLastError();
 }
 
@@ -460,15 +472,21 @@ cudaError_t set_smem(K kernel) {
 
 size_t gemm_weight_bytes(uint32_t n_rows, uint32_t k_total) { return static_cast<size_t>(n_rows) * k_total * 2; }
 
-size_t gemm_smem_bytes(uint32_t w_bytes, uint32_t n_stages) {
-  return kAlignSlack + kHeaderBytes + static_cast<size_t>(w_bytes) + static_cast<size_t>(n_stages) * kStageBytes;
+size_t gemm_smem_bytes(uint32_t w_bytes, uint32_t n_stages, uint32_t bps) {
+  return kAlignSlack + kHeaderBytes + static_cast<size_t>(w_bytes) + static_cast<size_t>(n_stages) * bps * kBoxBytes;
 }
 
-uint32_t gemm_pick_stages(uint32_t w_bytes) {
+// Ring shape for a weight tile of `w_bytes` and a K range of `k_total`: boxes per stage and stages.
+// Fewer, larger stages mean fewer waits for the single MMA-issuing thread; at least ~64 KB stay in flight.
+bool gemm_pick_ring(uint32_t w_bytes, uint32_t k_total, uint32_t* n_stages, uint32_t* bps) {
   const long room = 227L * 1024 - kAlignSlack - kHeaderBytes - static_cast<long>(w_bytes);
-  if (room < 0) return 0;
-  const long s = room / kStageBytes;
-  return static_cast<uint32_t>(s > 6 ? 6 : s);       // fewer than 3 means the tile does not fit
+  if (room < 3L * kBoxBytes) return false;           // the tile does not fit
+  const uint32_t n_boxes = k_total / kChunkK;
+  if (n_boxes <= 8 && room >= 2L * 4 * kBoxBytes) { *bps = 4; *n_stages = 2; return true; }   // a tile's K in <= 2 stages
+  if (room >= 3L * 2 * kBoxBytes) { *bps = 2; *n_stages = static_cast<uint32_t>(room / (2 * kBoxBytes) > 4 ? 4 : room / (2 * kBoxBytes)); return true; }
+  *bps = 1;
+  *n_stages = static_cast<uint32_t>(room / kBoxBytes > 6 ? 6 : room / kBoxBytes);
+  return true;
 }
 
 cudaError_t gemm_configure() {

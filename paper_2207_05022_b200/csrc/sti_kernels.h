@@ -56,14 +56,15 @@ struct GemmLaunch {
   const float* bias;
   int* err;                 // device status word
   size_t smem_bytes;        // header + w_bytes + n_stages activation stages
-  uint32_t n_stages;        // activation chunks of 16 KB in the ring (3..6)
+  uint32_t n_stages;        // stages in the activation ring
+  uint32_t bps;             // 16 KB boxes (64 columns) per stage: 1, 2 or 4
   uint32_t w_bytes;         // shared memory reserved for the weight tile (largest job)
   bool simt_debug;          // compute the products on the plain ALUs instead of the tensor cores
 };
 
 size_t gemm_weight_bytes(uint32_t n_rows, uint32_t k_total);
-uint32_t gemm_pick_stages(uint32_t w_bytes);        // < 3: the tile does not fit in shared memory
-size_t gemm_smem_bytes(uint32_t w_bytes, uint32_t n_stages);
+bool gemm_pick_ring(uint32_t w_bytes, uint32_t k_total, uint32_t* n_stages, uint32_t* bps);   // false: tile does not fit
+size_t gemm_smem_bytes(uint32_t w_bytes, uint32_t n_stages, uint32_t bps);
 cudaError_t gemm_configure();   // opt in to large dynamic shared memory (once per device)
 cudaError_t launch_gemm(GemmKind kind, const GemmLaunch& p, cudaStream_t s);
 
