@@ -352,20 +352,23 @@ dqgemm_kernel(const __grid_constant__ CUtensorMap xmap, const Job* __restrict__ 
       const uint32_t a_box_step = kBoxBytes >> 4;              // next 64-column box inside a stage
       const uint32_t b_ks_step = (2 * w_lbo) >> 4;             // next 16 columns of the weight tile
       const uint32_t b_chunk_step = 4 * b_ks_step;             // next 64 columns
-      if (lane == 0) {
-        uint32_t stage = 0, phase = 0, kc = 0, kcr = rot, ti = 0, issued = 0;
-        for (uint32_t c = 0; c < total; ++c) {
-          const uint32_t buf = ti & 1;
-          if (kc == 0 && ti >= 2) {      // the epilogue must have drained this accumulator
-            if (!mbar_wait_bounded(smem_addr(&hdr->acc_empty[buf]), ((ti >> 1) - 1) & 1)) { failed = true; break; }
-          }
-          if (!mbar_wait_bounded(smem_addr(&hdr->full[stage]), phase)) { failed = true; break; }
-          tc_fence_after_sync();
-          const uint32_t box0 = kcr * bps;
-          const uint32_t nb = n_boxes - box0 < bps ? n_boxes - box0 : bps;
-          uint64_t da = a_desc0 + stage * a_stage_step;
-          uint64_t db = b_desc0 + box0 * b_chunk_step;
-          const uint32_t d_addr = tmem_base + buf * n_rows;
+      // The whole warp runs the loop converged; one elected lane issues.
+      uint32_t stage = 0, phase = 0, kc = 0, kcr = rot, ti = 0, issued = 0;
+      for (uint32_t c = 0; c < total; ++c) {
+        const uint32_t buf = ti & 1;
+        bool ok = true;
+        if (kc == 0 && ti >= 2)        // the epilogue must have drained this accumulator
+          ok = __all_sync(0xffffffffu, mbar_wait_bounded(smem_addr(&hdr->acc_empty[buf]), ((ti >> 1) - 1) & 1));
+        if (ok) ok = __all_sync(0xffffffffu, mbar_wait_bounded(smem_addr(&hdr->full[stage]), phase));
+        if (!ok) { failed = true; break; }
+        tc_fence_after_sync();
+        const uint32_t box0 = kcr * bps;
+        const uint32_t nb = n_boxes - box0 < bps ? n_boxes - box0 : bps;
+        const uint64_t da0 = a_desc0 + stage * a_stage_step;
+        const uint64_t db0 = b_desc0 + box0 * b_chunk_step;
+        const uint32_t d_addr = tmem_base + buf * n_rows;
+        if (elect_one()) {
+          uint64_t da = da0, db = db0;
           for (uint32_t b = 0; b < nb; ++b, da += a_box_step, db += b_chunk_step) {
             umma_bf16_ss(d_addr, da, db, idesc, (kc | b) != 0 ? 1u : 0u);
             umma_bf16_ss(d_addr, da + 2, db + b_ks_step, idesc, 1u);          // +32 bytes inside the swizzled row
@@ -374,18 +377,19 @@ dqgemm_kernel(const __grid_constant__ CUtensorMap xmap, const Job* __restrict__ 
           }
           if (c + n_stages < total) umma_commit(smem_addr(&hdr->empty[stage]));   // only if the stage is refilled
           if (kc + 1 == n_chunks) umma_commit(smem_addr(&hdr->acc_full[buf]));
-          issued = c + 1;
-          if (++stage == n_stages) { stage = 0; phase ^= 1; }
-          if (++kcr == n_chunks) kcr = 0;
-          if (++kc == n_chunks) { kc = 0; ++ti; }
         }
-        if (failed && issued > 0) {
-          // outstanding MMAs: a commit of its own and one more bounded chance before TMEM is freed
-          umma_commit(smem_addr(&hdr->drain));
-          (void)mbar_wait_bounded(smem_addr(&hdr->drain), 0);
-        }
+        __syncwarp();
+        issued = c + 1;
+        if (++stage == n_stages) { stage = 0; phase ^= 1; }
+        if (++kcr == n_chunks) kcr = 0;
+        if (++kc == n_chunks) { kc = 0; ++ti; }
       }
-      __syncwarp();
+      if (failed && issued > 0) {
+        // outstanding MMAs: a commit of its own and one more bounded chance before TMEM is freed
+        if (elect_one()) umma_commit(smem_addr(&hdr->drain));
+        __syncwarp();
+        (void)mbar_wait_bounded(smem_addr(&hdr->drain), 0);
+      }
     } else if (warp >= kEpilogueWarp0 && warp < kEpilogueWarp0 + kEpilogueWarps) {
       // ---- epilogue: warp w owns TMEM lanes 32*(w%4).. (token rows) and one half of the columns
       const uint32_t q = warp & 3, half = (warp - kEpilogueWarp0) >> 2, ncol = n_rows / 2;
