@@ -81,6 +81,7 @@ struct sti_ctx {
   int* err_dev = nullptr;
   uint64_t launches = 0;
   bool simt_debug = false;
+  bool pdl = true;                     // programmatic dependent launch between the kernels of a layer
   sti_status async_error = STI_OK;
   MatrixInfo attn_m[4]{}, ffn_m[2]{};
   uint32_t attn_weights = 0, ffn_weights = 0;
@@ -363,7 +364,7 @@ sti_status run_gemm(sti_plan* p, GemmKind kind, const GemmTable& tab, const void
   g.jobs = tab.jobs; g.segs = tab.segs; g.n_jobs = tab.n_jobs; g.m_ctas = m_ctas_for(tab.n_jobs, T);
   if (!make_xmap(&g.xmap, x, ldx, T)) return STI_ERR_CUDA;
   g.x = x; g.ldx = ldx; g.T = T; g.out = out; g.ldo = ldo; g.bias = bias; g.err = p->ctx->err_dev;
-  g.smem_bytes = tab.smem; g.n_stages = tab.n_stages; g.bps = tab.bps; g.w_bytes = tab.w_bytes; g.simt_debug = p->ctx->simt_debug;
+  g.smem_bytes = tab.smem; g.n_stages = tab.n_stages; g.bps = tab.bps; g.w_bytes = tab.w_bytes; g.simt_debug = p->ctx->simt_debug; g.pdl = p->ctx->pdl;
   CUDA_TRY(launch_gemm(kind, g, p->ctx->compute));
   p->ctx->launches++;
   return STI_OK;
@@ -393,7 +394,7 @@ sti_status enqueue_layer(sti_plan* p, int li, const void* x, void* y, int batch,
       // the GEMMs take bf16 operands: fp32 activations are rounded once (round-to-nearest-even)
       if (!x_ready_bf16) {
         CUDA_TRY(launch_cast_bf16(static_cast<const float*>(x), p->x_bf16, static_cast<size_t>(T) * d.hidden,
-                                  c->compute));
+                                  c->compute, c->pdl));
         c->launches++;
       }
       xq = p->x_bf16;
@@ -401,7 +402,7 @@ sti_status enqueue_layer(sti_plan* p, int li, const void* x, void* y, int batch,
     st = run_gemm(p, GEMM_BF16_TO_BF16, L.qkv, xq, d.hidden, T, p->qkv, 64, dense + c->off_bq);
     if (st != STI_OK) return st;
     CUDA_TRY(mark(1));
-    CUDA_TRY(launch_attention(p->qkv, p->attn_out, nh, batch, seq, lens, c->compute));
+    CUDA_TRY(launch_attention(p->qkv, p->attn_out, nh, batch, seq, lens, c->compute, c->pdl));
     c->launches++;
     CUDA_TRY(mark(2));
     st = run_gemm(p, GEMM_BF16_TO_F32, L.o, p->attn_out, nh * 64, T, p->partial, d.hidden, nullptr);
@@ -417,7 +418,7 @@ sti_status enqueue_layer(sti_plan* p, int li, const void* x, void* y, int batch,
   ln.bias = dense + c->off_bo; ln.resid = x; ln.resid_bf16 = bf16_act ? 1 : 0;
   ln.gamma = dense + c->off_ln1g; ln.beta = dense + c->off_ln1b; ln.eps = d.ln_eps; ln.T = T; ln.d = d.hidden;
   ln.out_f32 = p->h1_f32; ln.out_bf16 = p->h1_bf16;
-  CUDA_TRY(launch_layernorm(ln, c->compute));
+  CUDA_TRY(launch_layernorm(ln, c->compute, c->pdl));
   c->launches++;
   L.k_ran[3] = true;
   CUDA_TRY(mark(4));
@@ -438,7 +439,7 @@ sti_status enqueue_layer(sti_plan* p, int li, const void* x, void* y, int batch,
   l2.gamma = dense + c->off_ln2g; l2.beta = dense + c->off_ln2b; l2.eps = d.ln_eps; l2.T = T; l2.d = d.hidden;
   l2.out_f32 = bf16_act ? nullptr : static_cast<float*>(y);
   l2.out_bf16 = bf16_act ? static_cast<uint16_t*>(y) : (want_next_bf16 ? p->x_bf16 : nullptr);
-  CUDA_TRY(launch_layernorm(l2, c->compute));
+  CUDA_TRY(launch_layernorm(l2, c->compute, c->pdl));
   c->launches++;
   L.k_ran[6] = true;
   CUDA_TRY(mark(7));
@@ -680,6 +681,8 @@ sti_status sti_ctx_create(const sti_model_desc* desc, int device, void* compute_
   if (gemm_configure() != cudaSuccess || attention_configure() != cudaSuccess) return fail(STI_ERR_CUDA);
   const char* dbg = getenv("STI_DEBUG_SIMT");
   c->simt_debug = dbg && dbg[0] == '1';
+  const char* nopdl = getenv("STI_NO_PDL");
+  c->pdl = !(nopdl && nopdl[0] == '1');
   *out = c;
   return STI_OK;
 }

@@ -52,6 +52,8 @@ attention_kernel(const uint16_t* __restrict__ qkv, uint16_t* __restrict__ out, i
   const uint16_t* Kg = qkv + (static_cast<size_t>(hi * 3 + 1) * T + static_cast<size_t>(b) * L) * kHeadDim;
   const uint16_t* Vg = qkv + (static_cast<size_t>(hi * 3 + 2) * T + static_cast<size_t>(b) * L) * kHeadDim;
 
+  pdl_launch_dependents();
+  pdl_wait();          // q, k, v (and possibly seq_lens) come from the preceding kernels
   int valid = L;
   if (seq_lens != nullptr) {
     valid = seq_lens[b];
@@ -192,11 +194,11 @@ cudaError_t attention_configure() {
 }
 
 cudaError_t launch_attention(const uint16_t* qkv, uint16_t* out, int n_kept, int batch, int seq,
-                             const int32_t* seq_lens, cudaStream_t s) {
+                             const int32_t* seq_lens, cudaStream_t s, bool pdl) {
   if (n_kept <= 0) return cudaSuccess;
   dim3 grid((seq + kQTile - 1) / kQTile, n_kept, batch);
-  attention_kernel<<<grid, 128, attn_smem_bytes(seq), s>>>(qkv, out, n_kept, batch, seq, seq_lens);
-  return cudaGetLastError();
+  return launch_kernel(attention_kernel, grid, dim3(128), attn_smem_bytes(seq), s, pdl, qkv, out, n_kept, batch, seq,
+                       seq_lens);
 }
 
 }  // namespace sti

@@ -202,6 +202,7 @@ dqgemm_kernel(const __grid_constant__ CUtensorMap xmap, const Job* __restrict__ 
     if (++p_kc == n_chunks) { p_kc = 0; ++p_ti; }
   };
 
+  pdl_launch_dependents();     // the next kernel may start its own weight decode while this one runs
   uint32_t tmem_cols = 32;
   while (tmem_cols < 2 * n_rows) tmem_cols <<= 1;       // two accumulators
   if constexpr (!SIMT) {
@@ -218,8 +219,6 @@ dqgemm_kernel(const __grid_constant__ CUtensorMap xmap, const Job* __restrict__ 
       hdr->abort = 0;
       mbar_fence_init();
       fence_proxy_async_smem();
-      // activations first: the ring is filled while the weights are being decoded
-      while (p_c < n_stages && p_c < total) { request_chunk(p_stage, p_kcr, p_ti); producer_advance(); }
     }
     if (warp == 1) {
       tmem_alloc(smem_addr(&hdr->tmem_base), tmem_cols);
@@ -285,6 +284,9 @@ dqgemm_kernel(const __grid_constant__ CUtensorMap xmap, const Job* __restrict__ 
     fence_proxy_async_smem();
     __syncthreads();
   }
+  // Everything above read only weights, descriptors and parameters.  The activations are the previous
+  // kernel's output: from here on this kernel depends on it.
+  pdl_wait();
 
   if constexpr (SIMT) {
     // Debug path: the decoded tile multiplied on the plain ALUs, activations straight from global memory.
@@ -324,9 +326,9 @@ dqgemm_kernel(const __grid_constant__ CUtensorMap xmap, const Job* __restrict__ 
   } else {
     bool failed = false;
     if (warp == 0) {
-      // ---- producer: refill a stage as soon as the MMAs that read it have completed
-      // (thread 0 already requested the first n_stages chunks; the other lanes catch up on the counters)
+      // ---- producer: fill the ring, then refill a stage as soon as the MMAs that read it have completed
       if (lane == 0) {
+        while (p_c < n_stages && p_c < total) { request_chunk(p_stage, p_kcr, p_ti); producer_advance(); }
         uint32_t p_phase = 0;                 // parity of the `empty` completion being waited for
         while (p_c < total) {
           if (!mbar_wait_bounded_relaxed(smem_addr(&hdr->empty[p_stage]), p_phase)) { failed = true; break; }
@@ -459,11 +461,9 @@ cudaError_t launch_t(const GemmLaunch& p, cudaStream_t s) {
   dim3 grid(p.n_jobs, p.m_ctas), block(kThreads);
   const __nv_bfloat16* x = static_cast<const __nv_bfloat16*>(p.x);
   if (p.simt_debug)
-    dqgemm_kernel<OutT, GELU, true><<<grid, block, p.smem_bytes, s>>>(
-        p.xmap, p.jobs, p.segs, x, p.ldx, p.T, static_cast<OutT*>(p.out), p.ldo, p.bias, p.err, p.n_stages, p.bps, p.w_bytes);
+    return launch_kernel(dqgemm_kernel<OutT, GELU, true>, grid, block, p.smem_bytes, s, p.pdl, p.xmap, p.jobs, p.segs, x, p.ldx, p.T, static_cast<OutT*>(p.out), p.ldo, p.bias, p.err, p.n_stages, p.bps, p.w_bytes);
   else
-    dqgemm_kernel<OutT, GELU, false><<<grid, block, p.smem_bytes, s>>>(
-        p.xmap, p.jobs, p.segs, x, p.ldx, p.T, static_cast<OutT*>(p.out), p.ldo, p.bias, p.err, p.n_stages, p.bps, p.w_bytes);
+    return launch_kernel(dqgemm_kernel<OutT, GELU, false>, grid, block, p.smem_bytes, s, p.pdl, p.xmap, p.jobs, p.segs, x, p.ldx, p.T, static_cast<OutT*>(p.out), p.ldo, p.bias, p.err, p.n_stages, p.bps, p.w_bytes);
   return cudaGetLastError();
 }
 

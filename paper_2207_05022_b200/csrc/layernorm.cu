@@ -28,7 +28,11 @@ layernorm_kernel(LnLaunch p) {
   const int n_warps = blockDim.x >> 5;
   const size_t row = static_cast<size_t>(blockIdx.x) * p.d;
   const int c = tid * 4;
-  float4 a = __ldg(reinterpret_cast<const float4*>(p.bias + c));
+  pdl_launch_dependents();
+  float4 a = __ldg(reinterpret_cast<const float4*>(p.bias + c));      // parameters: not written by any kernel
+  const float4 g = __ldg(reinterpret_cast<const float4*>(p.gamma + c));
+  const float4 b = __ldg(reinterpret_cast<const float4*>(p.beta + c));
+  pdl_wait();                                                          // residual and partial sums are
   if (p.resid_bf16) {
     const uint2 r = __ldg(reinterpret_cast<const uint2*>(static_cast<const uint16_t*>(p.resid) + row + c));
     a.x += __uint_as_float(r.x << 16); a.y += __uint_as_float(r.x & 0xffff0000u);
@@ -55,8 +59,6 @@ layernorm_kernel(LnLaunch p) {
   const float dx = a.x - mean, dy = a.y - mean, dz = a.z - mean, dw = a.w - mean;
   const float var = block_sum(dx * dx + dy * dy + dz * dz + dw * dw, red, tid, n_warps) / static_cast<float>(p.d);
   const float rstd = rsqrtf(var + p.eps);
-  const float4 g = __ldg(reinterpret_cast<const float4*>(p.gamma + c));
-  const float4 b = __ldg(reinterpret_cast<const float4*>(p.beta + c));
   float4 y;
   y.x = dx * rstd * g.x + b.x; y.y = dy * rstd * g.y + b.y;
   y.z = dz * rstd * g.z + b.z; y.w = dw * rstd * g.w + b.w;
@@ -67,6 +69,8 @@ layernorm_kernel(LnLaunch p) {
 
 __global__ void cast_bf16_kernel(const float* __restrict__ in, uint16_t* __restrict__ out, size_t n4) {
   const size_t i = static_cast<size_t>(blockIdx.x) * blockDim.x + threadIdx.x;
+  pdl_launch_dependents();
+  pdl_wait();
   if (i >= n4) return;
   const float4 v = __ldg(reinterpret_cast<const float4*>(in) + i);
   reinterpret_cast<uint2*>(out)[i] = make_uint2(pack_bf16x2(v.x, v.y), pack_bf16x2(v.z, v.w));
@@ -74,19 +78,17 @@ __global__ void cast_bf16_kernel(const float* __restrict__ in, uint16_t* __restr
 
 }  // namespace
 
-cudaError_t launch_layernorm(const LnLaunch& p, cudaStream_t s) {
+cudaError_t launch_layernorm(const LnLaunch& p, cudaStream_t s, bool pdl) {
   if (p.T <= 0) return cudaSuccess;
   if (p.d % 128 != 0 || p.d > 2048) return cudaErrorInvalidValue;     // d / 4 threads, whole warps
-  layernorm_kernel<<<p.T, p.d / 4, 0, s>>>(p);
-  return cudaGetLastError();
+  return launch_kernel(layernorm_kernel, dim3(p.T), dim3(p.d / 4), 0, s, pdl, p);
 }
 
-cudaError_t launch_cast_bf16(const float* in, uint16_t* out, size_t n, cudaStream_t s) {
+cudaError_t launch_cast_bf16(const float* in, uint16_t* out, size_t n, cudaStream_t s, bool pdl) {
   if (n == 0) return cudaSuccess;
   if (n % 4) return cudaErrorInvalidValue;
   const size_t n4 = n / 4;
-  cast_bf16_kernel<<<static_cast<unsigned>((n4 + 255) / 256), 256, 0, s>>>(in, out, n4);
-  return cudaGetLastError();
+  return launch_kernel(cast_bf16_kernel, dim3(static_cast<unsigned>((n4 + 255) / 256)), dim3(256), 0, s, pdl, in, out, n4);
 }
 
 }  // namespace sti

@@ -91,6 +91,13 @@ __device__ __forceinline__ bool mbar_wait_bounded_relaxed(uint32_t bar, uint32_t
   }
 }
 
+// Programmatic dependent launch: a kernel launched with the attribute may start while its predecessor
+// on the stream still runs.  `pdl_wait` blocks until the predecessor has completed and its writes are
+// visible - everything before it may only touch data no kernel writes (weights, descriptors, parameters);
+// `pdl_launch_dependents` lets the successor start launching.  Both are no-ops for ordinary launches.
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
 // Make generic-proxy shared-memory writes visible to the async proxy (tensor core reads).
 __device__ __forceinline__ void fence_proxy_async_smem() {
   asm volatile("fence.proxy.async.shared::cta;" ::: "memory");

@@ -60,6 +60,7 @@ struct GemmLaunch {
   uint32_t bps;             // 16 KB boxes (64 columns) per stage: 1, 2 or 4
   uint32_t w_bytes;         // shared memory reserved for the weight tile (largest job)
   bool simt_debug;          // compute the products on the plain ALUs instead of the tensor cores
+  bool pdl;                 // launch with programmatic dependent launch
 };
 
 size_t gemm_weight_bytes(uint32_t n_rows, uint32_t k_total);
@@ -71,7 +72,7 @@ cudaError_t launch_gemm(GemmKind kind, const GemmLaunch& p, cudaStream_t s);
 // Per-head attention over kept heads.  qkv: [(kept*3 + which)][T][64] bf16; out: [T][n_kept*64] bf16.
 cudaError_t attention_configure();
 cudaError_t launch_attention(const uint16_t* qkv, uint16_t* out, int n_kept, int batch, int seq,
-                             const int32_t* seq_lens, cudaStream_t s);
+                             const int32_t* seq_lens, cudaStream_t s, bool pdl);
 
 // out = LayerNorm(sum_p partial[p] + bias + resid) * gamma + beta, one warp per token row.
 struct LnLaunch {
@@ -87,10 +88,10 @@ struct LnLaunch {
   float* out_f32;           // optional
   uint16_t* out_bf16;       // optional
 };
-cudaError_t launch_layernorm(const LnLaunch& p, cudaStream_t s);
+cudaError_t launch_layernorm(const LnLaunch& p, cudaStream_t s, bool pdl);
 
 // fp32 -> bf16 (round-to-nearest-even) copy of the activations the first GEMM reads.
-cudaError_t launch_cast_bf16(const float* in, uint16_t* out, size_t n, cudaStream_t s);
+cudaError_t launch_cast_bf16(const float* in, uint16_t* out, size_t n, cudaStream_t s, bool pdl);
 
 // Stand-alone decode of one matrix (inspection / parity).
 struct DecodeLaunch {
@@ -106,6 +107,24 @@ struct DecodeLaunch {
   uint16_t* wbf16;
 };
 cudaError_t launch_decode(const DecodeLaunch& p, cudaStream_t s);
+
+// Launch with or without the programmatic-dependent-launch attribute (every kernel of the layer calls
+// pdl_wait before it reads what its predecessor wrote, so consecutive kernels may overlap their prologues).
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_kernel(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t s, bool pdl,
+                                 Args... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = s;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = pdl ? 1 : 0;
+  return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
 
 constexpr int ERR_NONE = 0;
 constexpr int ERR_WAIT_TIMEOUT = 1;   // a bounded mbarrier wait ran out
