@@ -196,6 +196,82 @@ def time_layer_config(sti, torch, number, peaks, iters=60):
             "l2": "flushed before every call"}
 
 
+def run_sweep(args):
+    """Configuration 5: BERT-large stack, batch {1,8,32,64} x seq {128,512}, uniform 3-bit and mixed 2-6-bit
+    plans, shards resident vs streamed (2-layer preload).  Prints one JSON object with a row per point."""
+    import workloads as W
+    from workloads.shards import round_to_bf16
+    n_layers = args.layers or 24
+    works = {plan: W.make_config(5, n_layers=n_layers, plan=plan, resident=False, batch=1, seq=128,
+                                 workers=min(8, os.cpu_count() or 1)) for plan in ("uniform3", "mixed")}
+    import torch
+    import paper_2207_05022_b200 as sti
+    from paper_2207_05022_b200 import build
+    build.build_library()
+    peaks, peak_src = load_peaks()
+    for k, v in FALLBACK_PEAKS.items():
+        peaks.setdefault(k, v)
+    stream = torch.cuda.Stream()
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
+    batches = [int(b) for b in args.sweep_batches.split(",")]
+    seqs = [int(q) for q in args.sweep_seqs.split(",")]
+    rows = []
+    rng = np.random.default_rng(0)
+    for plan, work in works.items():
+        sessions = {"resident": sti.Session(with_residency(work, n_layers), compute_stream=stream.cuda_stream,
+                                            max_batch=max(batches), max_seq=max(seqs)),
+                    "streamed": sti.Session(work, compute_stream=stream.cuda_stream, max_batch=max(batches),
+                                            max_seq=max(seqs))}
+        packed = work.packed_bytes()
+        for B in batches:
+            for L in seqs:
+                bits16, _ = round_to_bf16(rng.standard_normal((B, L, work.shape.hidden), dtype=np.float32))
+                x = torch.from_numpy(bits16.view(np.int16)).cuda().view(torch.bfloat16)
+                y = torch.empty_like(x)
+                shaped = dataclasses.replace(work, batch=B, seq=L)
+                flops_g, flops_a = gemm_flops(shaped), attn_flops(shaped)
+                row = {"plan": plan, "batch": B, "seq": L, "tokens": B * L, "packed_bytes": packed}
+                for name, sess in sessions.items():
+                    ms = []
+                    with torch.cuda.stream(stream):
+                        for i in range(args.warmup + args.steps):
+                            flush.zero_()
+                            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                            e0.record(stream)
+                            sti.sti_model_forward(sess.plan, x.data_ptr(), y.data_ptr(), B, L)
+                            e1.record(stream)
+                            stream.synchronize()
+                            if i >= args.warmup:
+                                ms.append(e0.elapsed_time(e1))
+                    sti.sti_sync(sess.ctx)
+                    row[f"ms_{name}"] = float(np.median(ms))
+                sess = sessions["resident"]
+                sti.sti_plan_set_profiling(sess.plan, 2)
+                gemm_us = []
+                with torch.cuda.stream(stream):
+                    for i in range(3):
+                        flush.zero_()
+                        sti.sti_model_forward(sess.plan, x.data_ptr(), y.data_ptr(), B, L)
+                        st = sti.sti_get_stats(sess.plan)
+                        gemm_us.append(sum(st.gemm_us[:st.n_layers]))
+                sti.sti_plan_set_profiling(sess.plan, 0)
+                g_s = float(np.median(gemm_us)) * 1e-6
+                t_res = row["ms_resident"] * 1e-3
+                row.update({
+                    "gemm_ms": g_s * 1e3, "gemm_TFLOPs": flops_g / g_s / 1e12,
+                    "gemm_frac_of_tensor_peak": flops_g / g_s / 1e12 / peaks["bf16_tflops_sustained"],
+                    "gemm_packed_GBps": packed / g_s / 1e9,
+                    "e2e_TFLOPs_resident": (flops_g + flops_a) / t_res / 1e12,
+                    "packed_GBps_resident": packed / t_res / 1e9,
+                    "packed_GBps_streamed": packed / (row["ms_streamed"] * 1e-3) / 1e9,
+                    "streamed_over_resident": row["ms_streamed"] / row["ms_resident"]})
+                rows.append(row)
+        for sess in sessions.values():
+            sess.close()
+    print(json.dumps({"sweep": "configs[4]: BERT-large stack, bf16 activations", "n_layers": n_layers,
+                      "peak_source": peak_src, "rows": rows}))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -204,9 +280,16 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--layers", type=int, default=0, help="shorten the stack (profiler captures only)")
     ap.add_argument("--no-extras", action="store_true", help="skip the cpu baseline and single-layer extras")
+    ap.add_argument("--sweep", action="store_true", help="configuration 5 sweep instead of the headline workload")
+    ap.add_argument("--sweep-batches", default="1,8,32,64")
+    ap.add_argument("--sweep-seqs", default="128,512")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)
+        return
+    if args.sweep:
+        args.steps = min(args.steps, 10)
+        run_sweep(args)
         return
     args.warmup = max(args.warmup, 3)
 

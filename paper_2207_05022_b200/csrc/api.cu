@@ -158,7 +158,7 @@ void parse_tuning(Tuning* t, int tmax, const sti_model_desc& d) {
   if (tmax > 1024) {
     t->qkv_n = 64; t->f1_n = 64; t->o_n = 64; t->o_group = 16; t->f2_n = 64; t->f2_group = 4;
   } else {
-    t->qkv_n = 32; t->f1_n = 64; t->o_n = 64; t->o_group = 4; t->f2_n = 64; t->f2_group = 2;
+    t->qkv_n = 64; t->f1_n = 64; t->o_n = 64; t->o_group = 8; t->f2_n = 64; t->f2_group = 2;
   }
   const char* env = getenv("STI_TUNE");     // debugging aid: "qkv_n=32,o_group=4,..."
   if (env) {
