@@ -49,7 +49,7 @@ struct GemmTable {
   Seg* segs = nullptr;
   int n_jobs = 0;
   size_t smem = 0;
-  uint32_t w_bytes = 0, n_stages = 0, bps = 1, k_max = 0;
+  uint32_t w_bytes = 0, n_stages = 0, bps = 1, k_max = 0, hdr_bytes = 0;
   int n_split = 0;
 };
 
@@ -196,7 +196,7 @@ void parse_tuning(Tuning* t, int tmax, const sti_model_desc& d) {
   // keep every weight tile inside shared memory
   auto fits = [](int n, int k) {
     uint32_t st = 0, bp = 0;
-    return gemm_pick_ring(static_cast<uint32_t>(gemm_weight_bytes(n, k)), k, &st, &bp) && st * bp >= 4;
+    return gemm_pick_ring(static_cast<uint32_t>(gemm_weight_bytes(n, k)), k, gemm_header_bytes(16), &st, &bp) && st * bp >= 4;
   };
   while (t->qkv_n > 32 && !fits(t->qkv_n, d.hidden)) t->qkv_n /= 2;
   while (t->f1_n > 32 && !fits(t->f1_n, d.hidden)) t->f1_n /= 2;
@@ -238,7 +238,7 @@ Seg make_seg(const sti_ctx* c, const Unit& u, sti_kind kind, int m, uint32_t row
 struct TableBuilder {
   std::vector<Job> jobs;
   std::vector<Seg> segs;
-  uint32_t w_bytes = 0, k_max = 0;
+  uint32_t w_bytes = 0, k_max = 0, seg_max = 0;
   void add(Job j, const std::vector<Seg>& ss) {
     j.seg_begin = static_cast<uint32_t>(segs.size());
     j.n_seg = static_cast<uint32_t>(ss.size());
@@ -246,6 +246,7 @@ struct TableBuilder {
     jobs.push_back(j);
     w_bytes = std::max(w_bytes, static_cast<uint32_t>(gemm_weight_bytes(j.n_rows, j.k_total)));
     k_max = std::max(k_max, j.k_total);
+    seg_max = std::max(seg_max, j.n_seg);
   }
 };
 
@@ -364,7 +365,7 @@ sti_status run_gemm(sti_plan* p, GemmKind kind, const GemmTable& tab, const void
   g.jobs = tab.jobs; g.segs = tab.segs; g.n_jobs = tab.n_jobs; g.m_ctas = m_ctas_for(tab.n_jobs, T);
   if (!make_xmap(&g.xmap, x, ldx, T)) return STI_ERR_CUDA;
   g.x = x; g.ldx = ldx; g.T = T; g.out = out; g.ldo = ldo; g.bias = bias; g.err = p->ctx->err_dev;
-  g.smem_bytes = tab.smem; g.n_stages = tab.n_stages; g.bps = tab.bps; g.w_bytes = tab.w_bytes; g.simt_debug = p->ctx->simt_debug; g.pdl = p->ctx->pdl;
+  g.smem_bytes = tab.smem; g.n_stages = tab.n_stages; g.bps = tab.bps; g.w_bytes = tab.w_bytes; g.hdr_bytes = tab.hdr_bytes; g.simt_debug = p->ctx->simt_debug; g.pdl = p->ctx->pdl;
   CUDA_TRY(launch_gemm(kind, g, p->ctx->compute));
   p->ctx->launches++;
   return STI_OK;
@@ -877,9 +878,11 @@ sti_status sti_plan_finalize(sti_plan* p) {
       gt[i]->n_jobs = static_cast<int>(tb[i].jobs.size());
       gt[i]->w_bytes = tb[i].w_bytes;
       gt[i]->n_stages = 2; gt[i]->bps = 1;
-      if (!tb[i].jobs.empty() && !gemm_pick_ring(tb[i].w_bytes, tb[i].k_max, &gt[i]->n_stages, &gt[i]->bps))
+      gt[i]->hdr_bytes = gemm_header_bytes(tb[i].seg_max);
+      if (!tb[i].jobs.empty() &&
+          !gemm_pick_ring(tb[i].w_bytes, tb[i].k_max, gt[i]->hdr_bytes, &gt[i]->n_stages, &gt[i]->bps))
         return STI_ERR_SHAPE;
-      gt[i]->smem = gemm_smem_bytes(tb[i].w_bytes, gt[i]->n_stages, gt[i]->bps);
+      gt[i]->smem = gemm_smem_bytes(tb[i].w_bytes, gt[i]->n_stages, gt[i]->bps, gt[i]->hdr_bytes);
       if (gt[i]->smem > kMaxSmem && !tb[i].jobs.empty()) return STI_ERR_SHAPE;
       Fix fx{gt[i], 0, 0};
       fx.jobs_off = align16(host_tables.size());

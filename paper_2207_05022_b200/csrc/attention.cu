@@ -16,7 +16,6 @@ namespace sti {
 namespace {
 
 constexpr int kHeadDim = 64;
-constexpr int kQTile = 64;
 constexpr int kKStride = kHeadDim + 8;   // bf16 elements per K row in shared memory (conflict-free fragment reads)
 
 __device__ __forceinline__ void mma_bf16_16816(float (&c)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
@@ -36,7 +35,8 @@ __device__ __forceinline__ void ldmatrix_x2_trans(uint32_t addr, uint32_t& r0, u
   asm volatile("ldmatrix.sync.aligned.m8n8.x2.trans.shared.b16 {%0, %1}, [%2];" : "=r"(r0), "=r"(r1) : "r"(addr));
 }
 
-__global__ void __launch_bounds__(128)
+template <int WARPS>      // 16 query rows per warp; K and V of the sequence are shared by the CTA's warps
+__global__ void __launch_bounds__(32 * WARPS)
 attention_kernel(const uint16_t* __restrict__ qkv, uint16_t* __restrict__ out, int n_kept, int batch, int L,
                  const int32_t* __restrict__ seq_lens) {
   extern __shared__ __align__(16) uint8_t smem[];
@@ -62,7 +62,7 @@ attention_kernel(const uint16_t* __restrict__ qkv, uint16_t* __restrict__ out, i
 
   // K and V rows: every 16-byte piece is its own cp.async, all in flight at once; rows past L are zero
   const uint32_t ks_addr = smem_addr(Ks), vs_addr = smem_addr(Vs);
-  for (int idx = tid; idx < Lpad * 8; idx += 128) {
+  for (int idx = tid; idx < Lpad * 8; idx += 32 * WARPS) {
     const int key = idx >> 3, piece = idx & 7;
     const bool ok = key < L;
     const size_t goff = static_cast<size_t>(ok ? key : 0) * kHeadDim + piece * 8;
@@ -73,7 +73,7 @@ attention_kernel(const uint16_t* __restrict__ qkv, uint16_t* __restrict__ out, i
   asm volatile("cp.async.commit_group;" ::: "memory");
 
   // query fragments of this warp's 16 rows
-  const int q0 = qt * kQTile + warp * 16;
+  const int q0 = qt * (16 * WARPS) + warp * 16;
   uint32_t qa[4][4];
 #pragma unroll
   for (int kk = 0; kk < 4; ++kk) {
@@ -189,15 +189,25 @@ size_t attn_smem_bytes(int L) {
 }  // namespace
 
 cudaError_t attention_configure() {
-  return cudaFuncSetAttribute(attention_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+  cudaError_t e = cudaFuncSetAttribute(attention_kernel<4>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                       static_cast<int>(attn_smem_bytes(512)));
+  if (e != cudaSuccess) return e;
+  return cudaFuncSetAttribute(attention_kernel<8>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                               static_cast<int>(attn_smem_bytes(512)));
 }
 
 cudaError_t launch_attention(const uint16_t* qkv, uint16_t* out, int n_kept, int batch, int seq,
                              const int32_t* seq_lens, cudaStream_t s, bool pdl) {
   if (n_kept <= 0) return cudaSuccess;
-  dim3 grid((seq + kQTile - 1) / kQTile, n_kept, batch);
-  return launch_kernel(attention_kernel, grid, dim3(128), attn_smem_bytes(seq), s, pdl, qkv, out, n_kept, batch, seq,
+  // 128-query CTAs when there are enough of them to fill the GPU (fewer K/V re-reads per head), 64 otherwise
+  const long ctas128 = static_cast<long>((seq + 127) / 128) * n_kept * batch;
+  if (seq >= 128 && ctas128 >= 148) {
+    dim3 grid((seq + 127) / 128, n_kept, batch);
+    return launch_kernel(attention_kernel<8>, grid, dim3(256), attn_smem_bytes(seq), s, pdl, qkv, out, n_kept, batch,
+                         seq, seq_lens);
+  }
+  dim3 grid((seq + 63) / 64, n_kept, batch);
+  return launch_kernel(attention_kernel<4>, grid, dim3(128), attn_smem_bytes(seq), s, pdl, qkv, out, n_kept, batch, seq,
                        seq_lens);
 }
 

@@ -31,7 +31,9 @@ constexpr int kTileM = 128;                 // tokens per MMA tile
 constexpr int kChunkK = 64;                 // one TMA box = 64 columns = one 128-byte swizzle row; a stage holds 1, 2 or 4 boxes
 constexpr int kMaxStages = 8;
 constexpr int kBoxBytes = kTileM * kChunkK * 2;     // 16 KB
-constexpr int kHeaderBytes = 4096;          // barriers + segment tables; stages start 1024-byte aligned after it
+// header = barriers (256 B) + bias (512 B) + one 128-byte table per segment; stages start 1024-aligned after it
+constexpr int kHeaderSmall = 1024;          // single-segment tiles (QKV, FFN1)
+constexpr int kHeaderLarge = 3072;          // up to 16 segments (O projection, FFN2)
 constexpr int kAlignSlack = 1024;           // the dynamic shared-memory base is aligned up to 1024 by hand
 constexpr int kMaxSegs = 16;
 constexpr int kTableStride = 64;            // bf16 entries per segment table
@@ -162,7 +164,7 @@ __global__ void __launch_bounds__(kThreads, 1)
 dqgemm_kernel(const __grid_constant__ CUtensorMap xmap, const Job* __restrict__ jobs, const Seg* __restrict__ segs,
               const __nv_bfloat16* __restrict__ x, int ldx, int T, OutT* __restrict__ out, int ldo,
               const float* __restrict__ bias, int* __restrict__ err, uint32_t n_stages, uint32_t bps,
-              uint32_t w_bytes) {
+              uint32_t w_bytes, uint32_t hdr_bytes) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = smem_raw + ((1024u - (smem_addr(smem_raw) & 1023u)) & 1023u);
   const uint32_t tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -170,16 +172,17 @@ dqgemm_kernel(const __grid_constant__ CUtensorMap xmap, const Job* __restrict__ 
   const uint32_t n_rows = job.n_rows, k_total = job.k_total;
 
   SmemHeader* hdr = reinterpret_cast<SmemHeader*>(smem);
-  uint16_t* tables = reinterpret_cast<uint16_t*>(smem + 1024);                      // [kMaxSegs][64]
-  float* bias_sm = reinterpret_cast<float*>(smem + 1024 + kMaxSegs * kTableStride * 2);   // [n_rows] at 3072
-  uint8_t* xsm = smem + kHeaderBytes;                                                // n_stages x 16 KB, 1024-aligned
+  float* bias_sm = reinterpret_cast<float*>(smem + 256);                            // [n_rows <= 128]
+  uint16_t* tables = reinterpret_cast<uint16_t*>(smem + 768);                       // [n_seg][64]
+  uint8_t* xsm = smem + hdr_bytes;                                                   // stages, 1024-aligned
   const uint32_t stage_bytes = bps * kBoxBytes;          // bps boxes of 64 columns per stage
   uint8_t* wsm = xsm + n_stages * stage_bytes;
 
   // the kernel's own checks of the descriptor: refuse rather than touch memory out of bounds
   const bool bad = job.n_seg == 0 || job.n_seg > kMaxSegs || (n_rows != 32 && n_rows != 64 && n_rows != 128) ||
                    (k_total % kChunkK) != 0 || k_total == 0 || n_rows * k_total * 2 > w_bytes ||
-                   n_stages < 2 || n_stages > kMaxStages || (bps != 1 && bps != 2 && bps != 4);
+                   n_stages < 2 || n_stages > kMaxStages || (bps != 1 && bps != 2 && bps != 4) ||
+                   768 + job.n_seg * kTableStride * 2 > hdr_bytes || (hdr_bytes & 1023) != 0;
   if (bad) {
     if (tid == 0) atomicCAS(err, ERR_NONE, ERR_BAD_JOB);
     return;
@@ -473,9 +476,9 @@ cudaError_t launch_t(const GemmLaunch& p, cudaStream_t s) {
   dim3 grid(p.n_jobs, p.m_ctas), block(kThreads);
   const __nv_bfloat16* x = static_cast<const __nv_bfloat16*>(p.x);
   if (p.simt_debug)
-    return launch_kernel(dqgemm_kernel<OutT, GELU, true>, grid, block, p.smem_bytes, s, p.pdl, p.xmap, p.jobs, p.segs, x, p.ldx, p.T, static_cast<OutT*>(p.out), p.ldo, p.bias, p.err, p.n_stages, p.bps, p.w_bytes);
+    return launch_kernel(dqgemm_kernel<OutT, GELU, true>, grid, block, p.smem_bytes, s, p.pdl, p.xmap, p.jobs, p.segs, x, p.ldx, p.T, static_cast<OutT*>(p.out), p.ldo, p.bias, p.err, p.n_stages, p.bps, p.w_bytes, p.hdr_bytes);
   else
-    return launch_kernel(dqgemm_kernel<OutT, GELU, false>, grid, block, p.smem_bytes, s, p.pdl, p.xmap, p.jobs, p.segs, x, p.ldx, p.T, static_cast<OutT*>(p.out), p.ldo, p.bias, p.err, p.n_stages, p.bps, p.w_bytes);
+    return launch_kernel(dqgemm_kernel<OutT, GELU, false>, grid, block, p.smem_bytes, s, p.pdl, p.xmap, p.jobs, p.segs, x, p.ldx, p.T, static_cast<OutT*>(p.out), p.ldo, p.bias, p.err, p.n_stages, p.bps, p.w_bytes, p.hdr_bytes);
   return cudaGetLastError();
 }
 
@@ -488,14 +491,16 @@ cudaError_t set_smem(K kernel) {
 
 size_t gemm_weight_bytes(uint32_t n_rows, uint32_t k_total) { return static_cast<size_t>(n_rows) * k_total * 2; }
 
-size_t gemm_smem_bytes(uint32_t w_bytes, uint32_t n_stages, uint32_t bps) {
-  return kAlignSlack + kHeaderBytes + static_cast<size_t>(w_bytes) + static_cast<size_t>(n_stages) * bps * kBoxBytes;
+uint32_t gemm_header_bytes(uint32_t max_segs) { return max_segs <= 1 ? kHeaderSmall : kHeaderLarge; }
+
+size_t gemm_smem_bytes(uint32_t w_bytes, uint32_t n_stages, uint32_t bps, uint32_t hdr_bytes) {
+  return kAlignSlack + hdr_bytes + static_cast<size_t>(w_bytes) + static_cast<size_t>(n_stages) * bps * kBoxBytes;
 }
 
 // Ring shape for a weight tile of `w_bytes` and a K range of `k_total`: boxes per stage and stages.
-// Fewer, larger stages mean fewer waits for the single MMA-issuing thread; at least ~64 KB stay in flight.
-bool gemm_pick_ring(uint32_t w_bytes, uint32_t k_total, uint32_t* n_stages, uint32_t* bps) {
-  const long room = 227L * 1024 - kAlignSlack - kHeaderBytes - static_cast<long>(w_bytes);
+// Fewer, larger stages mean fewer waits for the MMA-issuing warp; at least ~64 KB stay in flight.
+bool gemm_pick_ring(uint32_t w_bytes, uint32_t k_total, uint32_t hdr_bytes, uint32_t* n_stages, uint32_t* bps) {
+  const long room = 227L * 1024 - kAlignSlack - static_cast<long>(hdr_bytes) - static_cast<long>(w_bytes);
   if (room < 3L * kBoxBytes) return false;           // the tile does not fit
   const uint32_t n_boxes = k_total / kChunkK;
   if (n_boxes <= 8 && room >= 2L * 4 * kBoxBytes) { *bps = 4; *n_stages = 2; return true; }   // a tile's K in <= 2 stages

@@ -59,13 +59,15 @@ struct GemmLaunch {
   uint32_t n_stages;        // stages in the activation ring
   uint32_t bps;             // 16 KB boxes (64 columns) per stage: 1, 2 or 4
   uint32_t w_bytes;         // shared memory reserved for the weight tile (largest job)
+  uint32_t hdr_bytes;       // barriers + bias + per-segment tables: 1024 (one segment per tile) or 3072
   bool simt_debug;          // compute the products on the plain ALUs instead of the tensor cores
   bool pdl;                 // launch with programmatic dependent launch
 };
 
 size_t gemm_weight_bytes(uint32_t n_rows, uint32_t k_total);
-bool gemm_pick_ring(uint32_t w_bytes, uint32_t k_total, uint32_t* n_stages, uint32_t* bps);   // false: tile does not fit
-size_t gemm_smem_bytes(uint32_t w_bytes, uint32_t n_stages, uint32_t bps);
+uint32_t gemm_header_bytes(uint32_t max_segs);
+bool gemm_pick_ring(uint32_t w_bytes, uint32_t k_total, uint32_t hdr_bytes, uint32_t* n_stages, uint32_t* bps);   // false: does not fit
+size_t gemm_smem_bytes(uint32_t w_bytes, uint32_t n_stages, uint32_t bps, uint32_t hdr_bytes);
 cudaError_t gemm_configure();   // opt in to large dynamic shared memory (once per device)
 cudaError_t launch_gemm(GemmKind kind, const GemmLaunch& p, cudaStream_t s);
 
