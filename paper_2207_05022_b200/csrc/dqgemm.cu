@@ -386,11 +386,12 @@ dqgemm_kernel(const __grid_constant__ CUtensorMap xmap, const Job* __restrict__ 
         const uint32_t d_addr = tmem_base + buf * n_rows;
         if (elect_one()) {
           uint64_t da = da0, db = db0;
-          for (uint32_t b = 0; b < nb; ++b, da += a_box_step, db += b_chunk_step) {
-            umma_bf16_ss(d_addr, da, db, idesc, (kc | b) != 0 ? 1u : 0u);
-            umma_bf16_ss(d_addr, da + 2, db + b_ks_step, idesc, 1u);          // +32 bytes inside the swizzled row
-            umma_bf16_ss(d_addr, da + 4, db + 2 * b_ks_step, idesc, 1u);
-            umma_bf16_ss(d_addr, da + 6, db + 3 * b_ks_step, idesc, 1u);
+          // per box: four K = 16 steps, +32 bytes inside the swizzled activation row, +2 core-matrix columns of W
+          umma_bf16_ss_x4(d_addr, da, db, 2, b_ks_step, idesc, kc != 0 ? 1u : 0u);
+          for (uint32_t b = 1; b < nb; ++b) {
+            da += a_box_step;
+            db += b_chunk_step;
+            umma_bf16_ss_x4(d_addr, da, db, 2, b_ks_step, idesc, 1u);
           }
           if (c + n_stages < total) umma_commit(smem_addr(&hdr->empty[stage]));   // only if the stage is refilled
           if (kc + 1 == n_chunks) umma_commit(smem_addr(&hdr->acc_full[buf]));

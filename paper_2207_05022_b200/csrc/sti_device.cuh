@@ -165,6 +165,27 @@ __device__ __forceinline__ void umma_bf16_ss(uint32_t tmem_d, uint64_t desc_a, u
       ::"r"(tmem_d), "l"(desc_a), "l"(desc_b), "r"(idesc), "r"(accumulate)
       : "memory");
 }
+// Four consecutive K = 16 steps of one 64-column box in a single instruction group: the A descriptor
+// advances by `a_step`, the B descriptor by `b_step` (both in 16-byte units) per step; only the first
+// step may overwrite the accumulator.  One predicate set-up for the four instructions.
+__device__ __forceinline__ void umma_bf16_ss_x4(uint32_t tmem_d, uint64_t desc_a, uint64_t desc_b, uint32_t a_step,
+                                                uint32_t b_step, uint32_t idesc, uint32_t accumulate_first) {
+  asm volatile(
+      "{\n\t.reg .pred p0, p1;\n\t.reg .b64 a1, a2, a3, b1, b2, b3, as, bs;\n\t"
+      "setp.ne.b32 p0, %6, 0;\n\t"
+      "setp.eq.b32 p1, 0, 0;\n\t"
+      "cvt.u64.u32 as, %3;\n\t"
+      "cvt.u64.u32 bs, %4;\n\t"
+      "add.u64 a1, %1, as;\n\tadd.u64 a2, a1, as;\n\tadd.u64 a3, a2, as;\n\t"
+      "add.u64 b1, %2, bs;\n\tadd.u64 b2, b1, bs;\n\tadd.u64 b3, b2, bs;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %5, p0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], a1, b1, %5, p1;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], a2, b2, %5, p1;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], a3, b3, %5, p1;\n\t}"
+      ::"r"(tmem_d), "l"(desc_a), "l"(desc_b), "r"(a_step), "r"(b_step), "r"(idesc), "r"(accumulate_first)
+      : "memory");
+}
+
 // Arrive on an mbarrier once all MMAs issued so far by this thread have completed.
 __device__ __forceinline__ void umma_commit(uint32_t bar) {
   asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
