@@ -163,10 +163,11 @@ def device_act(torch, work):
     return torch.from_numpy(work.x_dev).cuda()
 
 
-def time_layer_config(sti, torch, number, peaks, iters=60):
-    """Cold-L2 latency of one sti_layer_forward on configuration 1 or 2 (microseconds)."""
+def time_layer_config(sti, torch, number, peaks, iters=60, seq=None):
+    """Cold-L2 latency of one sti_layer_forward on configuration 1 or 2 (microseconds); `seq` shortens the
+    sequence for the weight-streaming probe shapes (few tokens: the GEMMs are HBM-bound by the roofline)."""
     import workloads as W
-    work = W.make_config(number)
+    work = W.make_config(number, seq=seq)
     stream = torch.cuda.Stream()
     flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
     times = []
@@ -190,7 +191,10 @@ def time_layer_config(sti, torch, number, peaks, iters=60):
     act = 2 * work.x_dev.nbytes
     floor_us = max((packed + act) / (peaks["hbm_gbs"] * 1e9), flops / (peaks["bf16_tflops_sustained"] * 1e12)) * 1e6
     med = float(np.median(times))
-    return {"layer_us_median": med, "layer_us_p10": float(np.percentile(times, 10)),
+    t_hbm = (packed + act) / (peaks["hbm_gbs"] * 1e9) * 1e6
+    return {"tokens": work.batch * work.seq, "bound": "hbm" if t_hbm >= floor_us * 0.999 else "tensor",
+            "packed_frac_of_hbm_peak": packed / med / 1e3 / peaks["hbm_gbs"],
+            "layer_us_median": med, "layer_us_p10": float(np.percentile(times, 10)),
             "layer_us_p90": float(np.percentile(times, 90)), "packed_bytes": packed, "flops": flops,
             "packed_GBps": packed / med / 1e3, "roofline_floor_us": floor_us, "x_of_floor": med / floor_us,
             "l2": "flushed before every call"}
@@ -408,6 +412,8 @@ def main():
     if rank == 0 and world == 1 and not args.no_extras:
         for num in (1, 2):
             extras[f"config{num}_layer"] = time_layer_config(sti, torch, num, peaks)
+        for probe_seq in (8, 32):
+            extras[f"config1_layer_probe_seq{probe_seq}"] = time_layer_config(sti, torch, 1, peaks, seq=probe_seq)
     s_res.close()
     s_str.close()
 

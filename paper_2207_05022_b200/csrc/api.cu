@@ -92,8 +92,9 @@ struct ForwardKey {
   const void* x_host = nullptr; void* y_host = nullptr;  // host buffers (host variant)
   const int32_t* lens = nullptr;                         // device
   int batch = 0, seq = 0;
+  int layer = -1;                                        // >= 0: a single layer (sti_layer_forward)
   bool operator==(const ForwardKey& o) const {
-    return x == o.x && y == o.y && x_host == o.x_host && y_host == o.y_host && lens == o.lens && batch == o.batch &&
+    return layer == o.layer && x == o.x && y == o.y && x_host == o.x_host && y_host == o.y_host && lens == o.lens && batch == o.batch &&
            seq == o.seq;
   }
 };
@@ -112,9 +113,9 @@ struct sti_plan {
   uint8_t* tables = nullptr;   size_t tables_bytes = 0;       // job/segment descriptors
   std::vector<cudaEvent_t> slot_free, g_slot_free;   // direct launches / graph capture
   cudaEvent_t ev_copy_tail = nullptr, ev_begin = nullptr, ev_end = nullptr, ev_fork = nullptr, g_ev_join = nullptr;
-  cudaGraphExec_t gexec = nullptr;     // graph of the last forward
-  ForwardKey gkey;
-  uint64_t glaunches = 0;
+  struct CachedGraph { ForwardKey key; cudaGraphExec_t exec = nullptr; uint64_t launches = 0; uint64_t last_use = 0; };
+  std::vector<CachedGraph> graphs;     // captured forwards, a few most recently used (buffers + shape + layer)
+  uint64_t graph_clock = 0;
   bool graph_off = false;
   bool copy_tail_valid = false;
   // activation scratch
@@ -532,7 +533,19 @@ sti_status enqueue_forward_io(sti_plan* p, const ForwardKey& k, bool capturing) 
     x = p->x_in;
     y = p->y_out;
   }
-  sti_status st = enqueue_forward(p, x, y, k.batch, k.seq, k.lens, capturing);
+  sti_status st;
+  if (k.layer >= 0) {
+    // a single layer: its IO job (if it has streamed units) runs on the compute stream, not overlapped
+    Layer& L = p->layers[k.layer];
+    if (L.str_bytes > 0) {
+      if (!capturing && p->copy_tail_valid) CUDA_TRY(cudaStreamWaitEvent(c->compute, p->ev_copy_tail, 0));
+      if ((st = enqueue_layer_copy(p, k.layer, c->compute)) != STI_OK) return st;
+    }
+    st = enqueue_layer(p, k.layer, x, y, k.batch, k.seq, k.lens, false, false);
+    if (st == STI_OK && L.str_bytes > 0 && !capturing) CUDA_TRY(cudaEventRecord(p->slot_free[L.slot], c->compute));
+  } else {
+    st = enqueue_forward(p, x, y, k.batch, k.seq, k.lens, capturing);
+  }
   if (st != STI_OK) return st;
   if (k.y_host) CUDA_TRY(cudaMemcpyAsync(k.y_host, p->y_out, bytes, cudaMemcpyDeviceToHost, c->compute));
   return STI_OK;
@@ -543,8 +556,9 @@ sti_status enqueue_forward_io(sti_plan* p, const ForwardKey& k, bool capturing) 
 sti_status model_forward_impl(sti_plan* p, const ForwardKey& k) {
   sti_ctx* c = p->ctx;
   if (p->profiling || p->graph_off) return enqueue_forward_io(p, k, false);
-  if (!(p->gexec && p->gkey == k)) {
-    if (p->gexec) { cudaGraphExecDestroy(p->gexec); p->gexec = nullptr; }
+  sti_plan::CachedGraph* hit = nullptr;
+  for (auto& g : p->graphs) if (g.exec && g.key == k) hit = &g;
+  if (!hit) {
     const uint64_t launches_before = c->launches;
     cudaGraph_t graph = nullptr;
     if (cudaStreamBeginCapture(c->compute, cudaStreamCaptureModeRelaxed) != cudaSuccess) {
@@ -554,7 +568,7 @@ sti_status model_forward_impl(sti_plan* p, const ForwardKey& k) {
     }
     const sti_status st = enqueue_forward_io(p, k, true);
     const cudaError_t ce = cudaStreamEndCapture(c->compute, &graph);
-    p->glaunches = c->launches - launches_before;
+    const uint64_t n_launches = c->launches - launches_before;
     c->launches = launches_before;
     if (st != STI_OK || ce != cudaSuccess || !graph) {
       (void)cudaGetLastError();
@@ -562,20 +576,31 @@ sti_status model_forward_impl(sti_plan* p, const ForwardKey& k) {
       p->graph_off = true;            // fall back to plain stream launches for this plan
       return st != STI_OK ? st : enqueue_forward_io(p, k, false);
     }
-    const cudaError_t ie = cudaGraphInstantiate(&p->gexec, graph, 0);
+    cudaGraphExec_t exec = nullptr;
+    const cudaError_t ie = cudaGraphInstantiate(&exec, graph, 0);
     cudaGraphDestroy(graph);
-    if (ie != cudaSuccess) {
+    if (ie != cudaSuccess || !exec) {
       (void)cudaGetLastError();
-      p->gexec = nullptr;
       p->graph_off = true;
       return enqueue_forward_io(p, k, false);
     }
-    p->gkey = k;
+    constexpr size_t kMaxGraphs = 8;
+    if (p->graphs.size() < kMaxGraphs) {
+      p->graphs.emplace_back();
+      hit = &p->graphs.back();
+    } else {                          // replace the least recently used one
+      hit = &p->graphs[0];
+      for (auto& g : p->graphs) if (g.last_use < hit->last_use) hit = &g;
+      (void)cudaStreamSynchronize(c->compute);      // it may still be running
+      cudaGraphExecDestroy(hit->exec);
+    }
+    hit->key = k; hit->exec = exec; hit->launches = n_launches;
   }
-  CUDA_TRY(cudaGraphLaunch(p->gexec, c->compute));
+  hit->last_use = ++p->graph_clock;
+  CUDA_TRY(cudaGraphLaunch(hit->exec, c->compute));
   // later ungraphed work (profiled forwards, single layers) must not reuse a ring slot before this graph is done
   for (auto e : p->slot_free) CUDA_TRY(cudaEventRecord(e, c->compute));
-  c->launches += p->glaunches;
+  c->launches += hit->launches;
   p->copy_tail_valid = false;
   return STI_OK;
 }
@@ -600,7 +625,7 @@ void free_plan_device(sti_plan* p) {
   if (p->g_ev_join) cudaEventDestroy(p->g_ev_join);
   if (p->ev_copy_tail) cudaEventDestroy(p->ev_copy_tail);
   if (p->ev_fork) cudaEventDestroy(p->ev_fork);
-  if (p->gexec) cudaGraphExecDestroy(p->gexec);
+  for (auto& g : p->graphs) if (g.exec) cudaGraphExecDestroy(g.exec);
   if (p->ev_begin) cudaEventDestroy(p->ev_begin);
   if (p->ev_end) cudaEventDestroy(p->ev_end);
 }
@@ -953,15 +978,13 @@ sti_status sti_layer_forward(sti_plan* p, int layer, const void* x, void* y, int
   if ((st = sti_plan_finalize(p)) != STI_OK) return st;
   sti_ctx* c = p->ctx;
   CUDA_TRY(cudaSetDevice(c->device));
-  Layer& L = p->layers[layer];
-  if (L.str_bytes > 0) {
-    // not overlapped: the layer's IO job runs on the compute stream, after any copy still in flight
-    if (p->copy_tail_valid) CUDA_TRY(cudaStreamWaitEvent(c->compute, p->ev_copy_tail, 0));
-    if ((st = enqueue_layer_copy(p, layer, c->compute)) != STI_OK) return st;
+  if (p->copy_tail_valid) {       // an ungraphed forward may still have copies in flight on the copy stream
+    CUDA_TRY(cudaStreamWaitEvent(c->compute, p->ev_copy_tail, 0));
+    p->copy_tail_valid = false;
   }
-  if ((st = enqueue_layer(p, layer, x, y, batch, seq, lens, false, false)) != STI_OK) return st;
-  if (L.str_bytes > 0) CUDA_TRY(cudaEventRecord(p->slot_free[L.slot], c->compute));
-  return STI_OK;
+  ForwardKey k;
+  k.x = x; k.y = y; k.lens = lens; k.batch = batch; k.seq = seq; k.layer = layer;
+  return model_forward_impl(p, k);
 }
 
 sti_status sti_model_forward(sti_plan* p, const void* x, void* y, int batch, int seq, const int32_t* lens) {
