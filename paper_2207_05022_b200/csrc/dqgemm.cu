@@ -217,7 +217,6 @@ dqgemm_kernel(const __grid_constant__ CUtensorMap xmap, const Job* __restrict__ 
     if (++p_kc == n_chunks) { p_kc = 0; ++p_ti; }
   };
 
-  pdl_launch_dependents();     // the next kernel may start its own weight decode while this one runs
   uint32_t tmem_cols = 32;
   while (tmem_cols < 2 * n_rows) tmem_cols <<= 1;       // two accumulators
   if constexpr (!SIMT) {
@@ -259,6 +258,10 @@ dqgemm_kernel(const __grid_constant__ CUtensorMap xmap, const Job* __restrict__ 
   __syncthreads();
   tc_fence_after_sync();
   const uint32_t tmem_base = SIMT ? 0u : hdr->tmem_base;
+  // Only now may the next kernel's CTAs start (and decode their weights while this kernel runs): this CTA
+  // already owns its tensor memory, so a successor that allocates and then waits for this kernel to finish
+  // can never starve it of columns.
+  pdl_launch_dependents();
 
   // ---- decode the weight tile once
   {
