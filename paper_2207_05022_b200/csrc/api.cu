@@ -31,6 +31,7 @@ struct MatrixInfo {
 
 struct Tuning {
   int qkv_n = 32, f1_n = 64, o_n = 64, o_group = 4, f2_n = 64, f2_group = 2;
+  int pair_min_tiles = 8;              // two-CTA GEMM from this many 128-token tiles on (0 = never)
 };
 
 struct Unit {
@@ -50,6 +51,7 @@ struct GemmTable {
   int n_jobs = 0;
   size_t smem = 0;
   uint32_t w_bytes = 0, n_stages = 0, bps = 1, k_max = 0, hdr_bytes = 0;
+  bool pair_ok = false;                // consecutive jobs can share two-CTA MMAs (64-row tiles, same K range)
   int n_split = 0;
 };
 
@@ -179,6 +181,7 @@ void parse_tuning(Tuning* t, int tmax, const sti_model_desc& d) {
         else if (k == "o_group") t->o_group = v;
         else if (k == "f2_n") t->f2_n = v;
         else if (k == "f2_group") t->f2_group = v;
+        else if (k == "pair_min_tiles") t->pair_min_tiles = v;
       }
       pos = end + 1;
     }
@@ -364,6 +367,12 @@ sti_status run_gemm(sti_plan* p, GemmKind kind, const GemmTable& tab, const void
   if (tab.n_jobs == 0) return STI_OK;
   GemmLaunch g{};
   g.jobs = tab.jobs; g.segs = tab.segs; g.n_jobs = tab.n_jobs; g.m_ctas = m_ctas_for(tab.n_jobs, T);
+  const int n_mtiles = (T + 127) / 128;
+  g.pair = tab.pair_ok && p->tune.pair_min_tiles > 0 && n_mtiles >= p->tune.pair_min_tiles;
+  if (g.pair) {      // a pair of CTAs takes two token tiles at a time
+    const int n_mpairs = (n_mtiles + 1) / 2;
+    g.m_ctas = std::max(1, std::min(n_mpairs, 148 / tab.n_jobs));
+  }
   if (!make_xmap(&g.xmap, x, ldx, T)) return STI_ERR_CUDA;
   g.x = x; g.ldx = ldx; g.T = T; g.out = out; g.ldo = ldo; g.bias = bias; g.err = p->ctx->err_dev;
   g.smem_bytes = tab.smem; g.n_stages = tab.n_stages; g.bps = tab.bps; g.w_bytes = tab.w_bytes; g.hdr_bytes = tab.hdr_bytes; g.simt_debug = p->ctx->simt_debug; g.pdl = p->ctx->pdl;
@@ -904,6 +913,11 @@ sti_status sti_plan_finalize(sti_plan* p) {
       gt[i]->w_bytes = tb[i].w_bytes;
       gt[i]->n_stages = 2; gt[i]->bps = 1;
       gt[i]->hdr_bytes = gemm_header_bytes(tb[i].seg_max);
+      gt[i]->pair_ok = !tb[i].jobs.empty() && tb[i].jobs.size() % 2 == 0;
+      for (size_t j = 0; gt[i]->pair_ok && j < tb[i].jobs.size(); j += 2) {
+        const Job &a = tb[i].jobs[j], &b = tb[i].jobs[j + 1];
+        gt[i]->pair_ok = a.n_rows == 64 && b.n_rows == 64 && a.k_total == b.k_total && a.x_koff == b.x_koff;
+      }
       if (!tb[i].jobs.empty() &&
           !gemm_pick_ring(tb[i].w_bytes, tb[i].k_max, gt[i]->hdr_bytes, &gt[i]->n_stages, &gt[i]->bps))
         return STI_ERR_SHAPE;

@@ -157,6 +157,70 @@ __device__ __forceinline__ void store_row16(OutT* dst, const float (&v)[16]) {
 }
 
 // ---------------------------------------------------------------------------------------
+// Pieces shared by the one-CTA and the two-CTA kernel
+// ---------------------------------------------------------------------------------------
+// Centroid tables of the job's segments, rounded once to bf16 (round-to-nearest-even), and a head start
+// for the outlier lists, which are needed right after the decode.
+__device__ __forceinline__ void load_tables(const Job& job, const Seg* __restrict__ segs, uint16_t* tables, uint32_t tid) {
+  for (uint32_t i = tid; i < job.n_seg * kTableStride; i += kThreads) {
+    const Seg& sg = segs[job.seg_begin + i / kTableStride];
+    const uint32_t e = i % kTableStride;
+    tables[i] = (sg.bits <= 6 && e < (1u << sg.bits)) ? bf16_bits(__ldg(sg.table + e)) : 0;
+  }
+  for (uint32_t si = 0; si < job.n_seg; ++si) {
+    const Seg& sg = segs[job.seg_begin + si];
+    for (uint32_t o = tid * 32; o < sg.n_out; o += kThreads * 32) {
+      asm volatile("prefetch.global.L2 [%0];" ::"l"(sg.out_off + o));
+      asm volatile("prefetch.global.L2 [%0];" ::"l"(sg.out_val + o));
+    }
+  }
+}
+
+// Decode of the job's weight tile into `wsm` (all threads of the CTA; ends with the tile visible to the
+// tensor core: proxy fence + CTA barrier).  Needs the tables in place (a CTA barrier after load_tables).
+__device__ __forceinline__ void decode_weight_tile(const Job& job, const Seg* __restrict__ segs, const uint16_t* tables,
+                                                   uint8_t* wsm, uint32_t tid) {
+  const uint32_t lane = tid & 31, warp = tid >> 5;
+  const uint32_t n_rows = job.n_rows, k_total = job.k_total;
+  const Seg& s0 = segs[job.seg_begin];
+  const uint32_t rows_per_group = s0.kc >= 128 ? 32 : 64;
+  const uint32_t chunks = s0.kc >= 128 ? s0.kc / 128 : 1;
+  const uint32_t tasks_per_seg = (n_rows / rows_per_group) * chunks;
+  const uint32_t n_tasks = tasks_per_seg * job.n_seg;
+  for (uint32_t t = warp; t < n_tasks; t += kWarps) {
+    const uint32_t si = t / tasks_per_seg, task = t % tasks_per_seg;
+    const Seg& sg = segs[job.seg_begin + si];
+    const uint16_t* tab = tables + si * kTableStride;
+    switch (sg.bits) {
+      case 2: decode_task<2>(sg, tab, wsm, n_rows, task, lane); break;
+      case 3: decode_task<3>(sg, tab, wsm, n_rows, task, lane); break;
+      case 4: decode_task<4>(sg, tab, wsm, n_rows, task, lane); break;
+      case 5: decode_task<5>(sg, tab, wsm, n_rows, task, lane); break;
+      case 6: decode_task<6>(sg, tab, wsm, n_rows, task, lane); break;
+      default: break;
+    }
+  }
+  for (uint32_t si = 0; si < job.n_seg; ++si) {
+    const Seg& sg = segs[job.seg_begin + si];
+    if (sg.bits == 32) decode_raw(sg, wsm, n_rows, tid);
+  }
+  __syncthreads();
+  // outliers keep their original value (Section 6): overwrite their slot
+  for (uint32_t si = 0; si < job.n_seg; ++si) {
+    const Seg& sg = segs[job.seg_begin + si];
+    for (uint32_t o = tid; o < sg.n_out; o += kThreads) {
+      const uint32_t local = __ldg(sg.out_off + o) - sg.flat_base;
+      const uint32_t row = local / sg.kc, kk = sg.koff + local % sg.kc;
+      if (row < n_rows && kk < k_total)
+        reinterpret_cast<uint16_t*>(wsm)[(static_cast<size_t>(kk >> 3) * n_rows + row) * 8 + (kk & 7)] =
+            bf16_bits(__ldg(sg.out_val + o));
+    }
+  }
+  fence_proxy_async_smem();
+  __syncthreads();
+}
+
+// ---------------------------------------------------------------------------------------
 // The kernel
 // ---------------------------------------------------------------------------------------
 template <typename OutT, bool GELU, bool SIMT>
@@ -239,21 +303,8 @@ dqgemm_kernel(const __grid_constant__ CUtensorMap xmap, const Job* __restrict__ 
       tmem_relinquish();
     }
   }
-  // centroid tables, rounded once to bf16 (round-to-nearest-even)
-  for (uint32_t i = tid; i < job.n_seg * kTableStride; i += kThreads) {
-    const Seg& sg = segs[job.seg_begin + i / kTableStride];
-    const uint32_t e = i % kTableStride;
-    tables[i] = (sg.bits <= 6 && e < (1u << sg.bits)) ? bf16_bits(__ldg(sg.table + e)) : 0;
-  }
+  load_tables(job, segs, tables, tid);
   if (tid < n_rows) bias_sm[tid] = job.bias_off >= 0 ? __ldg(bias + job.bias_off + tid) : 0.f;
-  // outlier lists are needed right after the decode: start pulling them towards L2 now
-  for (uint32_t si = 0; si < job.n_seg; ++si) {
-    const Seg& sg = segs[job.seg_begin + si];
-    for (uint32_t o = tid * 32; o < sg.n_out; o += kThreads * 32) {
-      asm volatile("prefetch.global.L2 [%0];" ::"l"(sg.out_off + o));
-      asm volatile("prefetch.global.L2 [%0];" ::"l"(sg.out_val + o));
-    }
-  }
   tc_fence_before_sync();
   __syncthreads();
   tc_fence_after_sync();
@@ -263,45 +314,7 @@ dqgemm_kernel(const __grid_constant__ CUtensorMap xmap, const Job* __restrict__ 
   // can never starve it of columns.
   pdl_launch_dependents();
 
-  // ---- decode the weight tile once
-  {
-    const Seg& s0 = segs[job.seg_begin];
-    const uint32_t rows_per_group = s0.kc >= 128 ? 32 : 64;
-    const uint32_t chunks = s0.kc >= 128 ? s0.kc / 128 : 1;
-    const uint32_t tasks_per_seg = (n_rows / rows_per_group) * chunks;
-    const uint32_t n_tasks = tasks_per_seg * job.n_seg;
-    for (uint32_t t = warp; t < n_tasks; t += kWarps) {
-      const uint32_t si = t / tasks_per_seg, task = t % tasks_per_seg;
-      const Seg& sg = segs[job.seg_begin + si];
-      const uint16_t* tab = tables + si * kTableStride;
-      switch (sg.bits) {
-        case 2: decode_task<2>(sg, tab, wsm, n_rows, task, lane); break;
-        case 3: decode_task<3>(sg, tab, wsm, n_rows, task, lane); break;
-        case 4: decode_task<4>(sg, tab, wsm, n_rows, task, lane); break;
-        case 5: decode_task<5>(sg, tab, wsm, n_rows, task, lane); break;
-        case 6: decode_task<6>(sg, tab, wsm, n_rows, task, lane); break;
-        default: break;
-      }
-    }
-    for (uint32_t si = 0; si < job.n_seg; ++si) {
-      const Seg& sg = segs[job.seg_begin + si];
-      if (sg.bits == 32) decode_raw(sg, wsm, n_rows, tid);
-    }
-    __syncthreads();
-    // outliers keep their original value (Section 6): overwrite their slot
-    for (uint32_t si = 0; si < job.n_seg; ++si) {
-      const Seg& sg = segs[job.seg_begin + si];
-      for (uint32_t o = tid; o < sg.n_out; o += kThreads) {
-        const uint32_t local = __ldg(sg.out_off + o) - sg.flat_base;
-        const uint32_t row = local / sg.kc, kk = sg.koff + local % sg.kc;
-        if (row < n_rows && kk < k_total)
-          reinterpret_cast<uint16_t*>(wsm)[(static_cast<size_t>(kk >> 3) * n_rows + row) * 8 + (kk & 7)] =
-              bf16_bits(__ldg(sg.out_val + o));
-      }
-    }
-    fence_proxy_async_smem();
-    __syncthreads();
-  }
+  decode_weight_tile(job, segs, tables, wsm, tid);
   // Everything above read only weights, descriptors and parameters.  The activations are the previous
   // kernel's output: from here on this kernel depends on it.
   pdl_wait();
@@ -475,15 +488,290 @@ dqgemm_kernel(const __grid_constant__ CUtensorMap xmap, const Job* __restrict__ 
   }
 }
 
+// ---------------------------------------------------------------------------------------
+// Two-CTA variant (cta_group::2) for many tokens.
+//
+// A cluster of two CTAs shares one MMA: M = 256 (each CTA contributes its own 128-token activation tile),
+// N = 128 (each CTA contributes the 64 decoded weight rows of its own job).  Per instruction the pair does
+// twice the work of the one-CTA kernel per SM for the same issue cost, and every activation byte brought in
+// from L2 is used against 128 instead of 64 output features - the one-CTA kernel is bound by exactly these
+// two things once there are thousands of tokens.  CTA 0 issues; tcgen05.commit multicasts completions to both
+// CTAs; both CTAs' TMA loads report to CTA 0's `full` barriers; each CTA drains its own accumulator rows
+// (its 128 tokens x all 128 features) and reports to CTA 0's `acc_empty`.
+// ---------------------------------------------------------------------------------------
+__device__ __forceinline__ uint32_t cluster_ctarank() {
+  uint32_t r;
+  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+  return r;
+}
+__device__ __forceinline__ void cluster_sync_all() {     // every thread of both CTAs
+  asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+__device__ __forceinline__ uint32_t map_to_cta(uint32_t saddr, uint32_t rank) {   // same offset in CTA `rank`
+  uint32_t r;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(saddr), "r"(rank));
+  return r;
+}
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr) {
+  asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+}
+__device__ __forceinline__ void tmem_alloc_pair(uint32_t smem_dst, uint32_t n_cols) {     // one warp in each CTA
+  asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_dst), "r"(n_cols)
+               : "memory");
+}
+__device__ __forceinline__ void tmem_relinquish_pair() {
+  asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc_pair(uint32_t taddr, uint32_t n_cols) {
+  asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(n_cols) : "memory");
+}
+// Own tile into own shared memory, completion bytes credited to the barrier at `bar_cluster_addr` (CTA 0's).
+__device__ __forceinline__ void tma_load_2d_pair(uint32_t dst, const CUtensorMap* map, int k0, int m0,
+                                                 uint32_t bar_cluster_addr) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+      ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(k0), "r"(m0), "r"(bar_cluster_addr)
+      : "memory");
+}
+__device__ __forceinline__ void umma_bf16_ss_x4_pair(uint32_t tmem_d, uint64_t desc_a, uint64_t desc_b, uint32_t a_step,
+                                                     uint32_t b_step, uint32_t idesc, uint32_t accumulate_first) {
+  asm volatile(
+      "{\n\t.reg .pred p0, p1;\n\t.reg .b64 a1, a2, a3, b1, b2, b3, as, bs;\n\t"
+      "setp.ne.b32 p0, %6, 0;\n\t"
+      "setp.eq.b32 p1, 0, 0;\n\t"
+      "cvt.u64.u32 as, %3;\n\t"
+      "cvt.u64.u32 bs, %4;\n\t"
+      "add.u64 a1, %1, as;\n\tadd.u64 a2, a1, as;\n\tadd.u64 a3, a2, as;\n\t"
+      "add.u64 b1, %2, bs;\n\tadd.u64 b2, b1, bs;\n\tadd.u64 b3, b2, bs;\n\t"
+      "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %5, p0;\n\t"
+      "tcgen05.mma.cta_group::2.kind::f16 [%0], a1, b1, %5, p1;\n\t"
+      "tcgen05.mma.cta_group::2.kind::f16 [%0], a2, b2, %5, p1;\n\t"
+      "tcgen05.mma.cta_group::2.kind::f16 [%0], a3, b3, %5, p1;\n\t}"
+      ::"r"(tmem_d), "l"(desc_a), "l"(desc_b), "r"(a_step), "r"(b_step), "r"(idesc), "r"(accumulate_first)
+      : "memory");
+}
+// Completion of all MMAs issued so far -> the barrier at this offset in both CTAs.
+__device__ __forceinline__ void umma_commit_pair(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+               ::"r"(bar), "h"(static_cast<uint16_t>(3)) : "memory");
+}
+
+template <typename OutT, bool GELU>
+__global__ void __launch_bounds__(kThreads, 1)
+dqgemm_pair_kernel(const __grid_constant__ CUtensorMap xmap, const Job* __restrict__ jobs, const Seg* __restrict__ segs,
+                   int T, OutT* __restrict__ out, int ldo, const float* __restrict__ bias, int* __restrict__ err,
+                   uint32_t n_stages, uint32_t bps, uint32_t w_bytes, uint32_t hdr_bytes) {
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = smem_raw + ((1024u - (smem_addr(smem_raw) & 1023u)) & 1023u);
+  const uint32_t tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const uint32_t rank = cluster_ctarank();                 // 0 issues the MMAs
+  const uint32_t pair_base = blockIdx.x & ~1u;
+  const Job job = jobs[blockIdx.x];                        // the 64 weight rows this CTA decodes
+  const Job job0 = jobs[pair_base], job1 = jobs[pair_base + 1];   // columns 0-63 / 64-127 of the accumulator
+  const uint32_t k_total = job.k_total;
+
+  SmemHeader* hdr = reinterpret_cast<SmemHeader*>(smem);
+  float* bias_sm = reinterpret_cast<float*>(smem + 256);            // [128]
+  uint16_t* tables = reinterpret_cast<uint16_t*>(smem + 768);       // [n_seg][64]
+  uint8_t* xsm = smem + hdr_bytes;
+  const uint32_t stage_bytes = bps * kBoxBytes;
+  uint8_t* wsm = xsm + n_stages * stage_bytes;
+
+  // both CTAs evaluate the same conditions, so a refused pair leaves together
+  const bool bad = job0.n_rows != 64 || job1.n_rows != 64 || job0.k_total != job1.k_total || job0.x_koff != job1.x_koff ||
+                   job0.n_seg == 0 || job0.n_seg > kMaxSegs || job1.n_seg == 0 || job1.n_seg > kMaxSegs ||
+                   (k_total % kChunkK) != 0 || k_total == 0 || 64 * k_total * 2 > w_bytes || n_stages < 2 ||
+                   n_stages > kMaxStages || (bps != 1 && bps != 2 && bps != 4) ||
+                   768 + (job0.n_seg > job1.n_seg ? job0.n_seg : job1.n_seg) * kTableStride * 2 > hdr_bytes ||
+                   (hdr_bytes & 1023) != 0 || (gridDim.x & 1) != 0;
+  if (bad) {
+    if (tid == 0) atomicCAS(err, ERR_NONE, ERR_BAD_JOB);
+    return;
+  }
+
+  const int n_mtiles = (T + kTileM - 1) / kTileM;
+  const uint32_t n_mpairs = (n_mtiles + 1) / 2;           // the pair takes token tiles 2p (CTA 0) and 2p + 1 (CTA 1)
+  const uint32_t n_boxes = k_total / kChunkK;
+  const uint32_t n_chunks = (n_boxes + bps - 1) / bps;
+  const uint32_t my_pairs = blockIdx.y < n_mpairs ? (n_mpairs - blockIdx.y + gridDim.y - 1) / gridDim.y : 0;
+  const uint32_t total = my_pairs * n_chunks;
+  const uint32_t xsm_addr = smem_addr(xsm);
+  const uint32_t rot = (blockIdx.x >> 1) % n_chunks;      // both CTAs of a pair walk K in the same order
+  auto tile_row0 = [&](uint32_t ti) { return static_cast<int>((2 * (blockIdx.y + ti * gridDim.y) + rank) * kTileM); };
+
+  constexpr uint32_t kAccCols = 128, kTmemCols = 256;      // two accumulators of 128 columns
+  if (tid == 0) {
+    for (uint32_t s = 0; s < n_stages; ++s) {
+      mbar_init(smem_addr(&hdr->full[s]), 1);              // used in CTA 0 only
+      mbar_init(smem_addr(&hdr->empty[s]), 1);
+    }
+    for (int b = 0; b < 2; ++b) {
+      mbar_init(smem_addr(&hdr->acc_full[b]), 1);
+      mbar_init(smem_addr(&hdr->acc_empty[b]), 2 * kEpilogueWarps);   // CTA 0 only: both CTAs' epilogue warps
+    }
+    mbar_init(smem_addr(&hdr->drain), 1);
+    hdr->abort = 0;
+    mbar_fence_init();
+    fence_proxy_async_smem();
+  }
+  if (warp == 1) {
+    tmem_alloc_pair(smem_addr(&hdr->tmem_base), kTmemCols);
+    tmem_relinquish_pair();
+  }
+  load_tables(job, segs, tables, tid);
+  if (tid < 128) {
+    const Job& jb = tid < 64 ? job0 : job1;
+    bias_sm[tid] = jb.bias_off >= 0 ? __ldg(bias + jb.bias_off + (tid & 63)) : 0.f;
+  }
+  tc_fence_before_sync();
+  __syncthreads();
+  tc_fence_after_sync();
+  const uint32_t tmem_base = hdr->tmem_base;
+  pdl_launch_dependents();          // this CTA owns its tensor memory now (see the one-CTA kernel)
+
+  decode_weight_tile(job, segs, tables, wsm, tid);
+  cluster_sync_all();               // both halves of the weight tile are in place, all barriers initialised
+  pdl_wait();                       // from here on: the previous kernel's output
+
+  bool failed = false;
+  if (warp == 0) {
+    // ---- producer (one in each CTA): own token tile into own ring, completion reported to CTA 0
+    if (lane == 0) {
+      uint32_t c = 0, stage = 0, phase = 0, kcr = rot, kc = 0, ti = 0;
+      for (; c < total; ++c) {
+        if (c >= n_stages) {
+          if (!mbar_wait_bounded_relaxed(smem_addr(&hdr->empty[stage]), phase)) { failed = true; break; }
+        }
+        const uint32_t box0 = kcr * bps;
+        const uint32_t nb = n_boxes - box0 < bps ? n_boxes - box0 : bps;
+        if (rank == 0) mbar_expect_tx(smem_addr(&hdr->full[stage]), 2 * nb * kBoxBytes);    // both CTAs' bytes
+        const uint32_t bar = map_to_cta(smem_addr(&hdr->full[stage]), 0);
+        for (uint32_t b = 0; b < nb; ++b)
+          tma_load_2d_pair(xsm_addr + stage * stage_bytes + b * kBoxBytes, &xmap,
+                           static_cast<int>(job.x_koff + (box0 + b) * kChunkK), tile_row0(ti), bar);
+        if (++stage == n_stages) { stage = 0; if (c >= n_stages) phase ^= 1; }
+        if (++kcr == n_chunks) kcr = 0;
+        if (++kc == n_chunks) { kc = 0; ++ti; }
+      }
+    }
+    __syncwarp();
+  } else if (warp == 1) {
+    if (rank == 0) {
+      // ---- MMA issuer of the pair
+      const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((128u >> 3) << 17) | ((256u >> 4) << 24);
+      const uint32_t w_lbo = 64 * 16;
+      const uint64_t a_desc0 = umma_smem_desc_sw128(xsm_addr);
+      const uint64_t b_desc0 = umma_smem_desc(smem_addr(wsm), w_lbo, 128);
+      const uint32_t a_stage_step = stage_bytes >> 4, a_box_step = kBoxBytes >> 4;
+      const uint32_t b_ks_step = (2 * w_lbo) >> 4, b_chunk_step = 4 * b_ks_step;
+      uint32_t stage = 0, phase = 0, kc = 0, kcr = rot, ti = 0, issued = 0;
+      for (uint32_t c = 0; c < total; ++c) {
+        const uint32_t buf = ti & 1;
+        bool ok = true;
+        if (kc == 0 && ti >= 2)
+          ok = __all_sync(0xffffffffu, mbar_wait_bounded(smem_addr(&hdr->acc_empty[buf]), ((ti >> 1) - 1) & 1));
+        if (ok) ok = __all_sync(0xffffffffu, mbar_wait_bounded(smem_addr(&hdr->full[stage]), phase));
+        if (!ok) { failed = true; break; }
+        tc_fence_after_sync();
+        const uint32_t box0 = kcr * bps;
+        const uint32_t nb = n_boxes - box0 < bps ? n_boxes - box0 : bps;
+        const uint64_t da0 = a_desc0 + stage * a_stage_step;
+        const uint64_t db0 = b_desc0 + box0 * b_chunk_step;
+        const uint32_t d_addr = tmem_base + buf * kAccCols;
+        if (elect_one()) {
+          uint64_t da = da0, db = db0;
+          umma_bf16_ss_x4_pair(d_addr, da, db, 2, b_ks_step, idesc, kc != 0 ? 1u : 0u);
+          for (uint32_t b = 1; b < nb; ++b) {
+            da += a_box_step;
+            db += b_chunk_step;
+            umma_bf16_ss_x4_pair(d_addr, da, db, 2, b_ks_step, idesc, 1u);
+          }
+          if (c + n_stages < total) umma_commit_pair(smem_addr(&hdr->empty[stage]));
+          if (kc + 1 == n_chunks) umma_commit_pair(smem_addr(&hdr->acc_full[buf]));
+        }
+        __syncwarp();
+        issued = c + 1;
+        if (++stage == n_stages) { stage = 0; phase ^= 1; }
+        if (++kcr == n_chunks) kcr = 0;
+        if (++kc == n_chunks) { kc = 0; ++ti; }
+      }
+      if (failed && issued > 0) {
+        if (elect_one()) umma_commit_pair(smem_addr(&hdr->drain));
+        __syncwarp();
+        (void)mbar_wait_bounded(smem_addr(&hdr->drain), 0);
+      }
+    }
+  } else if (warp >= kEpilogueWarp0 && warp < kEpilogueWarp0 + kEpilogueWarps) {
+    // ---- epilogue: this CTA's 128 token rows; warp = (lane quadrant, which job's 64 columns)
+    const uint32_t q = warp & 3, half = (warp - kEpilogueWarp0) >> 2;
+    const Job& jb = half ? job1 : job0;
+    for (uint32_t ti = 0; ti < my_pairs; ++ti) {
+      const uint32_t buf = ti & 1;
+      uint32_t ok = 1;
+      if (lane == 0) ok = mbar_wait_bounded_relaxed(smem_addr(&hdr->acc_full[buf]), (ti >> 1) & 1) ? 1u : 0u;
+      ok = __shfl_sync(0xffffffffu, ok, 0);
+      if (!ok) { failed = true; break; }
+      tc_fence_after_sync();
+      const int t = tile_row0(ti) + static_cast<int>(q * 32 + lane);
+      OutT* drow = out + (static_cast<size_t>(jb.out_mat) * T + (t < T ? t : 0)) * ldo + jb.out_col;
+      const uint32_t taddr = tmem_base + ((q * 32) << 16) + buf * kAccCols + half * 64;
+#pragma unroll
+      for (uint32_t col = 0; col < 64; col += 32) {
+        uint32_t r[32];
+        tmem_ld_32x32b_x32(taddr + col, r);
+        tc_wait_ld();
+        if (t < T) {
+#pragma unroll
+          for (int h = 0; h < 2; ++h) {
+            float v[16];
+#pragma unroll
+            for (int i = 0; i < 16; ++i) {
+              const float a = __uint_as_float(r[h * 16 + i]) + bias_sm[half * 64 + col + h * 16 + i];
+              v[i] = GELU ? gelu_erf(a) : a;
+            }
+            store_row16<OutT>(drow + col + h * 16, v);
+          }
+        }
+      }
+      tc_fence_before_sync();
+      __syncwarp();
+      if (lane == 0) mbar_arrive_cluster(map_to_cta(smem_addr(&hdr->acc_empty[buf]), 0));
+    }
+  }
+  if (failed) {
+    hdr->abort = 1;
+    if (lane == 0) atomicCAS(err, ERR_NONE, ERR_WAIT_TIMEOUT);
+  }
+  tc_fence_before_sync();
+  __syncthreads();
+  cluster_sync_all();      // neither CTA frees tensor memory or exits while the pair's MMAs may still use it
+  if (warp == 1) tmem_dealloc_pair(tmem_base, kTmemCols);
+}
+
 template <typename OutT, bool GELU>
 cudaError_t launch_t(const GemmLaunch& p, cudaStream_t s) {
-  dim3 grid(p.n_jobs, p.m_ctas), block(kThreads);
   const __nv_bfloat16* x = static_cast<const __nv_bfloat16*>(p.x);
+  if (p.pair && !p.simt_debug) {
+    // clusters of two CTAs along x (consecutive jobs = the two halves of a 128-feature tile)
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(p.n_jobs, p.m_ctas);
+    cfg.blockDim = dim3(kThreads);
+    cfg.dynamicSmemBytes = p.smem_bytes;
+    cfg.stream = s;
+    cudaLaunchAttribute attr[2];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[1].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = p.pdl ? 2 : 1;
+    return cudaLaunchKernelEx(&cfg, dqgemm_pair_kernel<OutT, GELU>, p.xmap, p.jobs, p.segs, p.T, static_cast<OutT*>(p.out),
+                              p.ldo, p.bias, p.err, p.n_stages, p.bps, p.w_bytes, p.hdr_bytes);
+  }
+  dim3 grid(p.n_jobs, p.m_ctas), block(kThreads);
   if (p.simt_debug)
     return launch_kernel(dqgemm_kernel<OutT, GELU, true>, grid, block, p.smem_bytes, s, p.pdl, p.xmap, p.jobs, p.segs, x, p.ldx, p.T, static_cast<OutT*>(p.out), p.ldo, p.bias, p.err, p.n_stages, p.bps, p.w_bytes, p.hdr_bytes);
-  else
-    return launch_kernel(dqgemm_kernel<OutT, GELU, false>, grid, block, p.smem_bytes, s, p.pdl, p.xmap, p.jobs, p.segs, x, p.ldx, p.T, static_cast<OutT*>(p.out), p.ldo, p.bias, p.err, p.n_stages, p.bps, p.w_bytes, p.hdr_bytes);
-  return cudaGetLastError();
+  return launch_kernel(dqgemm_kernel<OutT, GELU, false>, grid, block, p.smem_bytes, s, p.pdl, p.xmap, p.jobs, p.segs, x, p.ldx, p.T, static_cast<OutT*>(p.out), p.ldo, p.bias, p.err, p.n_stages, p.bps, p.w_bytes, p.hdr_bytes);
 }
 
 template <typename K>
@@ -518,7 +806,8 @@ cudaError_t gemm_configure() {
   cudaError_t e;
 #define STI_SET(OutT, G)                                                  \
   if ((e = set_smem(dqgemm_kernel<OutT, G, false>)) != cudaSuccess) return e; \
-  if ((e = set_smem(dqgemm_kernel<OutT, G, true>)) != cudaSuccess) return e;
+  if ((e = set_smem(dqgemm_kernel<OutT, G, true>)) != cudaSuccess) return e;  \
+  if ((e = set_smem(dqgemm_pair_kernel<OutT, G>)) != cudaSuccess) return e;
   STI_SET(__nv_bfloat16, false)
   STI_SET(__nv_bfloat16, true)
   STI_SET(float, false)

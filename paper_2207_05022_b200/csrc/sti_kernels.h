@@ -62,6 +62,7 @@ struct GemmLaunch {
   uint32_t hdr_bytes;       // barriers + bias + per-segment tables: 1024 (one segment per tile) or 3072
   bool simt_debug;          // compute the products on the plain ALUs instead of the tensor cores
   bool pdl;                 // launch with programmatic dependent launch
+  bool pair;                // two-CTA clusters (cta_group::2): jobs 2i and 2i+1 share one M=256 x N=128 MMA
 };
 
 size_t gemm_weight_bytes(uint32_t n_rows, uint32_t k_total);
