@@ -117,6 +117,22 @@ class ClockSampler:
                 "power_w_max": max(power) if power else None, "samples": len(sm), "reasons": sorted(reasons)}
 
 
+def max_over_ranks(local_ms: float, world: int, device: str = "cuda") -> float:
+    """Timing rule for N > 1: every rank times its own replica on its device, the job's time is the slowest rank's."""
+    if world <= 1:
+        return float(local_ms)
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor([local_ms], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def aggregate_throughput(units_per_rank: float, world: int, ms_per_step: float) -> float:
+    """Whole-job throughput of `world` independent replicas (weak scaling): all ranks' units over the slowest time."""
+    return units_per_rank * world / (ms_per_step * 1e-3)
+
+
 def oracle_forward_timed(work, layers):
     from oracle import sti_oracle as O
     t0 = time.perf_counter()
@@ -361,11 +377,7 @@ def main():
                 fn()
                 e1.record(stream)
             barrier()
-        ms = sum(e0.elapsed_time(e1) for e0, e1 in ev)
-        t = torch.tensor([ms], dtype=torch.float64, device="cuda")
-        if world > 1:
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        return float(t.item())
+        return max_over_ranks(sum(e0.elapsed_time(e1) for e0, e1 in ev), world)
 
     sampler.start()
     launches0 = sti.sti_ctx_launch_count(s_res.ctx)
@@ -433,7 +445,7 @@ def main():
     t_floor_ms = max((packed + 2 * x_bytes) / (peak_hbm * 1e9),
                      (flops_gemm + attn_flops(work_str)) / (peak_tf * 1e12)) * 1e3
     line = {
-        "metric": METRIC, "value": packed * world / (t_res * 1e-3) / 1e9, "unit": UNIT, "n_gpus": world,
+        "metric": METRIC, "value": aggregate_throughput(packed, world, t_res) / 1e9, "unit": UNIT, "n_gpus": world,
         "steps": K, "warmup": Wm, "ms_per_step": t_res, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
         "config": {"workload": WORKLOAD, "n_layers": work_str.shape.n_layers, "batch": B, "seq": L,
@@ -441,7 +453,7 @@ def main():
                    "l2": "256 MiB memset before every step; packed weights (136 MB) also exceed the 126 MB L2",
                    "value_arm": "all shards resident in device memory",
                    "e2e_arm": "2-layer preload, layers 2.. streamed from pinned host memory"},
-        "e2e": {"value": packed * world / (ms_e2e / K * 1e-3) / 1e9, "unit": UNIT, "ms_per_step": ms_e2e / K,
+        "e2e": {"value": aggregate_throughput(packed, world, ms_e2e / K) / 1e9, "unit": UNIT, "ms_per_step": ms_e2e / K,
                 "h2d_bytes_per_step": int(streamed_bytes + x_bytes), "d2h_bytes_per_step": int(x_bytes)},
         "gpu_launches": int(launches),
         "clocks": clocks,

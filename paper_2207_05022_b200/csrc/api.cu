@@ -31,6 +31,7 @@ struct MatrixInfo {
 
 struct Tuning {
   int qkv_n = 32, f1_n = 64, o_n = 64, o_group = 4, f2_n = 64, f2_group = 2;
+  int cta_budget = 148;                // CTAs a GEMM launch may use when it splits the token tiles over CTAs
   int pair_min_tiles = 8;              // two-CTA GEMM from this many 128-token tiles on (0 = never)
 };
 
@@ -182,6 +183,7 @@ void parse_tuning(Tuning* t, int tmax, const sti_model_desc& d) {
         else if (k == "f2_n") t->f2_n = v;
         else if (k == "f2_group") t->f2_group = v;
         else if (k == "pair_min_tiles") t->pair_min_tiles = v;
+        else if (k == "cta_budget") t->cta_budget = std::max(1, v);
       }
       pos = end + 1;
     }
@@ -356,9 +358,9 @@ bool make_xmap(CUtensorMap* map, const void* base, int ld, int rows) {
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-int m_ctas_for(int n_jobs, int T) {
+int m_ctas_for(int n_jobs, int T, int cta_budget) {
   const int n_mtiles = (T + 127) / 128;
-  int m = n_jobs > 0 ? 148 / n_jobs : 1;
+  int m = n_jobs > 0 ? cta_budget / n_jobs : 1;
   return std::max(1, std::min(m, n_mtiles));
 }
 
@@ -366,12 +368,12 @@ sti_status run_gemm(sti_plan* p, GemmKind kind, const GemmTable& tab, const void
                     int ldo, const float* bias) {
   if (tab.n_jobs == 0) return STI_OK;
   GemmLaunch g{};
-  g.jobs = tab.jobs; g.segs = tab.segs; g.n_jobs = tab.n_jobs; g.m_ctas = m_ctas_for(tab.n_jobs, T);
+  g.jobs = tab.jobs; g.segs = tab.segs; g.n_jobs = tab.n_jobs; g.m_ctas = m_ctas_for(tab.n_jobs, T, p->tune.cta_budget);
   const int n_mtiles = (T + 127) / 128;
   g.pair = tab.pair_ok && p->tune.pair_min_tiles > 0 && n_mtiles >= p->tune.pair_min_tiles;
   if (g.pair) {      // a pair of CTAs takes two token tiles at a time
     const int n_mpairs = (n_mtiles + 1) / 2;
-    g.m_ctas = std::max(1, std::min(n_mpairs, 148 / tab.n_jobs));
+    g.m_ctas = std::max(1, std::min(n_mpairs, p->tune.cta_budget / tab.n_jobs));
   }
   if (!make_xmap(&g.xmap, x, ldx, T)) return STI_ERR_CUDA;
   g.x = x; g.ldx = ldx; g.T = T; g.out = out; g.ldo = ldo; g.bias = bias; g.err = p->ctx->err_dev;
