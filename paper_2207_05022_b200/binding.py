@@ -102,7 +102,7 @@ EXPORTED = ("sti_ctx_create", "sti_ctx_destroy", "sti_ctx_set_layer_params", "st
             "sti_plan_destroy", "sti_shard_upload", "sti_plan_finalize", "sti_layer_forward",
             "sti_model_forward", "sti_model_forward_host", "sti_sync", "sti_shard_decode",
             "sti_plan_set_profiling", "sti_get_stats", "sti_plan_memory", "sti_ctx_launch_count",
-            "sti_host_retile", "sti_strerror", "sti_matrix_decode_noalloc")
+            "sti_host_retile", "sti_strerror", "sti_matrix_decode_noalloc", "sti_plan_auto")
 
 
 def _check(status: int, where: str):
@@ -244,6 +244,57 @@ def sti_matrix_decode_noalloc(bits: int, rows: int, cols: int, codes: np.ndarray
         device, C.c_void_p(stream or None), int(bits), rows, cols, _ptr(codes), _ptr(cent), _ptr(off), _ptr(val),
         0 if off is None else off.size, C.c_void_p(w_dev or None), C.c_void_p(codes_dev or None),
         C.c_void_p(wbf16_dev or None)), "sti_matrix_decode_noalloc")
+
+class StiPlannerProfile(C.Structure):
+    _fields_ = [("n_layers", C.c_int32), ("n_slices", C.c_int32), ("t_comp_us", C.POINTER(C.c_double)),
+                ("t_io_us", C.c_double * 6), ("shard_bytes", C.c_uint64 * 6),
+                ("importance", C.POINTER(C.c_float))]
+
+
+class StiPlannerRequest(C.Structure):
+    _fields_ = [("target_us", C.c_double), ("preload_bytes", C.c_uint64),
+                ("preloaded_bits", C.POINTER(C.c_uint8))]
+
+
+class StiPlannerResult(C.Structure):
+    _fields_ = [("n", C.c_int32), ("m", C.c_int32), ("pass1_bits", C.c_int32), ("valid", C.c_int32),
+                ("keep", C.POINTER(C.c_uint8)), ("bits", C.POINTER(C.c_uint8)),
+                ("preload", C.POINTER(C.c_uint8)), ("aib_us", C.POINTER(C.c_double))]
+
+
+def sti_plan_auto(target_us: float, n_layers: int, n_slices: int, t_comp_us, t_io_us, shard_bytes,
+                  importance, preload_bytes: int, preloaded_bits=None) -> dict:
+    """Two-stage planner (Section 5.3 and 5.4); marshals arrays, returns the result fields as numpy arrays."""
+    lib = load_library()
+    tc = _host(t_comp_us, np.float64)
+    imp = _host(importance, np.float32).reshape(-1)
+    if tc.size != n_slices + 1 or imp.size != n_layers * n_slices or len(t_io_us) != 6 or len(shard_bytes) != 6:
+        raise ValueError("planner table sizes do not match n_layers / n_slices")
+    pf = StiPlannerProfile(n_layers, n_slices, tc.ctypes.data_as(C.POINTER(C.c_double)),
+                           (C.c_double * 6)(*[float(v) for v in t_io_us]),
+                           (C.c_uint64 * 6)(*[int(v) for v in shard_bytes]),
+                           imp.ctypes.data_as(C.POINTER(C.c_float)))
+    pre = None if preloaded_bits is None else _host(preloaded_bits, np.uint8).reshape(-1)
+    if pre is not None and pre.size != n_layers * n_slices:
+        raise ValueError("preloaded_bits must have n_layers * n_slices entries")
+    rq = StiPlannerRequest(float(target_us), int(preload_bytes),
+                           None if pre is None else pre.ctypes.data_as(C.POINTER(C.c_uint8)))
+    keep = np.zeros(n_layers * n_slices, np.uint8)
+    bits = np.zeros_like(keep)
+    preload = np.zeros_like(keep)
+    aib = np.zeros(n_layers, np.float64)
+    res = StiPlannerResult(0, 0, 0, 0, keep.ctypes.data_as(C.POINTER(C.c_uint8)),
+                           bits.ctypes.data_as(C.POINTER(C.c_uint8)),
+                           preload.ctypes.data_as(C.POINTER(C.c_uint8)),
+                           aib.ctypes.data_as(C.POINTER(C.c_double)))
+    lib.sti_plan_auto.restype = C.c_int
+    lib.sti_plan_auto.argtypes = [C.POINTER(StiPlannerProfile), C.POINTER(StiPlannerRequest),
+                                  C.POINTER(StiPlannerResult)]
+    _check(lib.sti_plan_auto(C.byref(pf), C.byref(rq), C.byref(res)), "sti_plan_auto")
+    shape = (n_layers, n_slices)
+    return {"n": res.n, "m": res.m, "pass1_bits": res.pass1_bits, "valid": bool(res.valid),
+            "keep": keep.reshape(shape), "bits": bits.reshape(shape), "preload": preload.reshape(shape),
+            "aib_us": aib}
 
 
 class Session:
