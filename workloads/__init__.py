@@ -13,4 +13,4 @@ from .shards import (  # noqa: F401
     quantize_unit, pack_codes, make_unit_weights, make_dense_params, make_activations,
     build_workload,
 )
-from .configs import make_config  # noqa: F401
+from .configs import make_config, make_planned  # noqa: F401

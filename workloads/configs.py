@@ -114,3 +114,21 @@ def make_config(number: int, *, seed: int = 0, n_layers: Optional[int] = None,
                               shape, b, s, "bf16", attn, ffn, seed=seed, ring_slots=2,
                               keep_originals=keep_originals, outlier_stress=outlier_stress, workers=workers)
     raise ValueError("configuration number must be 1..5")
+
+
+def make_planned(keep, bits, preload, *, batch: int = 1, seq: int = 256, seed: int = 0,
+                 act_dtype: str = "bf16", workers: int = 1, ring_slots: int = 4) -> Workload:
+    """BERT-large workload for a planner result: `keep`, `bits`, `preload` are [n_layers][16] grids over
+    the paper's shards; shard i of a layer is attention head i plus FFN slice i, which share the entry.
+    Layers with no kept shard (beyond the submodel's depth) are left out.  `ring_slots` streamed-layer
+    buffers let the copy engine run that many layers ahead of the computation."""
+    keep = np.asarray(keep)
+    depth = int(max(l + 1 for l in range(keep.shape[0]) if keep[l].any()))
+    shape = BERT_LARGE.with_layers(depth)
+    if keep.shape[1] != shape.n_heads or shape.n_ffn_slices != shape.n_heads:
+        raise ValueError("planner grid must have one column per head / FFN slice")
+    def grid():
+        return [[UnitPlan(bool(keep[l][i]), int(bits[l][i]) if keep[l][i] else 2, bool(preload[l][i]))
+                 for i in range(shape.n_heads)] for l in range(depth)]
+    return build_workload(f"planned_large_b{batch}_s{seq}", shape, batch, seq, act_dtype, grid(), grid(),
+                          seed=seed, ring_slots=ring_slots, workers=workers)
