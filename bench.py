@@ -38,6 +38,12 @@ WORKLOAD = ("configs[3]: 24-layer BERT-large (hidden 1024, 16 heads x 64, FFN 40
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
 
+# dram__bytes_read.sum + dram__bytes_write.sum per dequant-GEMM launch (mean over one layer's QKV, O, FFN1, FFN2
+# launches; BERT-large layer, batch 1, seq 256) from the ncu capture summarised in
+# profiles/dqgemm_bertlarge_seq256_ncu_full.md.  Set to None whenever dqgemm.cu changes after that capture.
+NCU_DRAM_BYTES_PER_GEMM_LAUNCH = 2534464
+
+
 def load_peaks():
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(path):
@@ -591,7 +597,11 @@ def main():
         "clocks": clocks,
         "roofline": {"kernel": "dqgemm_kernel (fused dequant-GEMM, 4 launches per layer)", "bound": "tensor",
                      "achieved": ach_tflops, "peak": peak_tf, "unit": "TFLOP/s",
-                     "frac": ach_tflops / peak_tf if peak_tf else None, "traffic": None,
+                     "frac": ach_tflops / peak_tf if peak_tf else None,
+                     "traffic": NCU_DRAM_BYTES_PER_GEMM_LAUNCH if work_str.shape.hidden == 1024 and work_str.seq == 256
+                     and work_str.batch == 1 else None,
+                     "traffic_note": "dram read+write bytes per launch, mean of a layer's four launches, one ncu "
+                                     "capture of this kernel build (cold caches); algorithmic: packed shards + bf16 operands",
                      "peak_source": f"bf16_tflops_sustained, {peak_src}",
                      "flops_per_launch": flops_gemm * K / gemm_launches if gemm_launches else None,
                      "avg_launch_us": gemm_us / gemm_launches if gemm_launches else None,
