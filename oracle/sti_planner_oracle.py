@@ -141,3 +141,23 @@ def plan(T: float, N: int, M: int, t_comp: Sequence[float], t_io_list: Sequence[
         bgrid[s[0]][s[1]] = bits[s]
         pgrid[s[0]][s[1]] = 1 if s in S else 0
     return PlannerResult(n, m, k1, bool(valid and fits), keep, bgrid, pgrid, list(aib))
+
+
+def retain_after_run(keep: Sequence[Sequence[int]], bits: Sequence[Sequence[int]], shard_bytes_list: Sequence[int],
+                     buffer_bytes: int) -> Tuple[List[List[int]], int]:
+    """Section 3.2 (caching between back-to-back executions) with Section 5.5's eviction order: loaded
+    shards are dropped from the top layer down until what remains fits the buffer.  Returns the grid of
+    retained versions (0 = not cached) and the bytes used."""
+    nbytes = dict(zip(VERSIONS, shard_bytes_list))
+    N, M = len(keep), len(keep[0])
+    loaded = [(l, i) for l in range(N) for i in range(M) if keep[l][i]]
+    total = sum(nbytes[bits[l][i]] for l, i in loaded)
+    while loaded and total > buffer_bytes:          # evict the topmost remaining shard
+        l, i = loaded.pop()
+        total -= nbytes[bits[l][i]]
+    # the walk from the bottom stops at the first shard that does not fit: a shard above an evicted one
+    # is evicted too, which the pop-from-the-top loop guarantees
+    grid = [[0] * M for _ in range(N)]
+    for l, i in loaded:
+        grid[l][i] = bits[l][i]
+    return grid, total

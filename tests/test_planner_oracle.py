@@ -199,3 +199,45 @@ def test_more_time_never_shrinks_the_submodel():
         r = run_oracle(inst)
         sizes.append(r.n * r.m)
     assert sizes == sorted(sizes)
+
+
+# ------------------------------------------------------------------ caching between back-to-back runs
+def test_retained_shards_are_the_longest_bottom_up_prefix_that_fits():
+    """Section 5.5: eviction goes from the top layer down until the buffer is filled, so what stays is a
+    prefix of the loaded shards in layer order; checked against brute force over all prefixes."""
+    rng = np.random.default_rng(21)
+    for _ in range(60):
+        inst = random_instance(rng)
+        r = run_oracle(inst)
+        order = [(l, i) for l in range(inst["N"]) for i in range(inst["M"]) if r.keep[l][i]]
+        sizes = [inst["nbytes"][VERS.index(r.bits[l][i])] for l, i in order]
+        budget = int(rng.integers(0, sum(sizes) + 2000))
+        grid, used = po.retain_after_run(r.keep, r.bits, inst["nbytes"], budget)
+        best = max(k for k in range(len(order) + 1) if sum(sizes[:k]) <= budget)
+        kept = [(l, i) for l, i in order if grid[l][i]]
+        assert kept == order[:best] and used == sum(sizes[:best])
+        assert all(grid[l][i] == r.bits[l][i] for l, i in kept)
+    assert po.retain_after_run([[1, 1]], [[2, 3]], [10, 20, 30, 40, 50, 60], 0) == ([[0, 0]], 0)
+    assert po.retain_after_run([[1, 1]], [[2, 3]], [10, 20, 30, 40, 50, 60], 29) == ([[2, 0]], 10)
+    assert po.retain_after_run([[1, 1]], [[2, 3]], [10, 20, 30, 40, 50, 60], 30) == ([[2, 3]], 30)
+
+
+def test_replanning_with_cached_shards_spends_the_freed_io_time():
+    """Section 3.2: with more shards cached the next plan stays stall-free (pipeline simulation) and no
+    streamed shard gets a lower uniform version than before."""
+    rng = np.random.default_rng(22)
+    for _ in range(40):
+        inst = random_instance(rng, N=int(rng.integers(2, 7)), M=int(rng.integers(2, 6)))
+        first = run_oracle(inst)
+        if not first.valid:
+            continue
+        t_io = dict(zip(VERS, inst["t_io"]))
+        grown = inst["S"] + int(rng.integers(1, 6)) * 4000
+        cached, _ = po.retain_after_run(first.keep, first.bits, inst["nbytes"], grown)
+        second = run_oracle(inst, cached)
+        assert (second.n, second.m) == (first.n, first.m) and second.valid
+        assert second.preload == [[1 if c else 0 for c in row] for row in cached]
+        assert all(second.bits[l][i] == cached[l][i] for l in range(inst["N"]) for i in range(inst["M"]) if cached[l][i])
+        assert simulate_pipeline(second.n, inst["t_comp"][second.m], t_io, second.bits, second.preload)[1] <= 1e-7
+        if any(k and not c for kr, cr in zip(second.keep, cached) for k, c in zip(kr, cr)):
+            assert VERS.index(second.pass1_bits) >= VERS.index(first.pass1_bits)
