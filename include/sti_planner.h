@@ -68,6 +68,20 @@ typedef struct {                       /* arrays are caller-allocated, [n_layers
 sti_status sti_plan_auto(const sti_planner_profile* profile, const sti_planner_request* request,
                          sti_planner_result* result);
 
+/* Back-to-back executions (Section 3.2) with the eviction rule of Section 5.5: after a run the loaded
+ * shards may stay cached in an enlarged preload buffer.  Shards are evicted from the top layer downwards
+ * until the rest fits, i.e. walking the executed submodel in layer order (layer 0 first, slices in index
+ * order) shards are retained, at the version they ran with, while they fit in buffer_bytes; the walk
+ * stops at the first shard that does not fit.  keep / bits are the executed plan's grids
+ * ([n_layers * n_slices], layer-major); out_preloaded_bits (same shape, caller-allocated) receives 0 or the
+ * retained version and is what sti_plan_auto takes as `preloaded_bits` for the next execution, whose
+ * planner then spends the IO time no longer needed on higher versions of the other shards.
+ * out_used_bytes (optional) receives the bytes retained.  STI_ERR_ARG on null pointers, empty grids or a
+ * kept shard whose version is not one of 2,3,4,5,6,32.  Host only. */
+sti_status sti_preload_after_run(int32_t n_layers, int32_t n_slices, const uint8_t* keep, const uint8_t* bits,
+                                 const uint64_t shard_bytes[STI_N_VERSIONS], uint64_t buffer_bytes,
+                                 uint8_t* out_preloaded_bits, uint64_t* out_used_bytes);
+
 #if defined(__GNUC__)
 #pragma GCC visibility pop
 #endif

@@ -102,7 +102,8 @@ EXPORTED = ("sti_ctx_create", "sti_ctx_destroy", "sti_ctx_set_layer_params", "st
             "sti_plan_destroy", "sti_shard_upload", "sti_plan_finalize", "sti_layer_forward",
             "sti_model_forward", "sti_model_forward_host", "sti_sync", "sti_shard_decode",
             "sti_plan_set_profiling", "sti_get_stats", "sti_plan_memory", "sti_ctx_launch_count",
-            "sti_host_retile", "sti_strerror", "sti_matrix_decode_noalloc", "sti_plan_auto")
+            "sti_host_retile", "sti_strerror", "sti_matrix_decode_noalloc", "sti_plan_auto",
+            "sti_preload_after_run")
 
 
 def _check(status: int, where: str):
@@ -295,6 +296,25 @@ def sti_plan_auto(target_us: float, n_layers: int, n_slices: int, t_comp_us, t_i
     return {"n": res.n, "m": res.m, "pass1_bits": res.pass1_bits, "valid": bool(res.valid),
             "keep": keep.reshape(shape), "bits": bits.reshape(shape), "preload": preload.reshape(shape),
             "aib_us": aib}
+
+
+def sti_preload_after_run(keep, bits, shard_bytes, buffer_bytes: int):
+    """Section 3.2 / 5.5: which loaded shards stay cached in a buffer of `buffer_bytes` after a run.
+    Returns (preloaded_bits grid for the next sti_plan_auto call, bytes used)."""
+    k = _host(keep, np.uint8)
+    b = _host(bits, np.uint8)
+    if k.ndim != 2 or k.shape != b.shape or len(shard_bytes) != 6:
+        raise ValueError("keep and bits must be [n_layers, n_slices] grids; shard_bytes has 6 entries")
+    out = np.zeros(k.shape, np.uint8)
+    used = C.c_uint64()
+    lib = load_library()
+    lib.sti_preload_after_run.restype = C.c_int
+    lib.sti_preload_after_run.argtypes = [C.c_int32, C.c_int32, C.c_void_p, C.c_void_p, C.POINTER(C.c_uint64),
+                                          C.c_uint64, C.c_void_p, C.POINTER(C.c_uint64)]
+    _check(lib.sti_preload_after_run(k.shape[0], k.shape[1], _ptr(k), _ptr(b),
+                                     (C.c_uint64 * 6)(*[int(v) for v in shard_bytes]), int(buffer_bytes),
+                                     _ptr(out), C.byref(used)), "sti_preload_after_run")
+    return out, int(used.value)
 
 
 class Session:

@@ -164,3 +164,24 @@ extern "C" sti_status sti_plan_auto(const sti_planner_profile* pf, const sti_pla
   out->valid = (valid && fits) ? 1 : 0;
   return STI_OK;
 }
+
+extern "C" sti_status sti_preload_after_run(int32_t n_layers, int32_t n_slices, const uint8_t* keep,
+                                            const uint8_t* bits, const uint64_t shard_bytes[STI_N_VERSIONS],
+                                            uint64_t buffer_bytes, uint8_t* out_preloaded_bits,
+                                            uint64_t* out_used_bytes) {
+  if (!keep || !bits || !shard_bytes || !out_preloaded_bits || n_layers < 1 || n_slices < 1) return STI_ERR_ARG;
+  const int total = n_layers * n_slices;
+  for (int i = 0; i < total; ++i)
+    if (keep[i] && version_of(bits[i]) < 0) return STI_ERR_ARG;
+  std::fill(out_preloaded_bits, out_preloaded_bits + total, 0);
+  uint64_t used = 0;
+  for (int i = 0; i < total; ++i) {        // layer-major order is the bottom-up walk
+    if (!keep[i]) continue;
+    const uint64_t b = shard_bytes[version_of(bits[i])];
+    if (used + b > buffer_bytes) break;     // this shard and everything above it is evicted
+    used += b;
+    out_preloaded_bits[i] = bits[i];
+  }
+  if (out_used_bytes) *out_used_bytes = used;
+  return STI_OK;
+}

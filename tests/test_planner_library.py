@@ -48,3 +48,17 @@ def test_library_planner_rejects_bad_arguments(sti):
     with pytest.raises(ValueError):
         sti.sti_plan_auto(5.0, 2, 2, [0, 1], [1, 2, 3, 4, 5, 6], [1] * 6, np.ones((2, 2)), 0)
     del C
+
+
+def test_library_retention_equals_oracle(sti):
+    rng = np.random.default_rng(31)
+    for _ in range(100):
+        inst = random_instance(rng)
+        r = run_oracle(inst)
+        total = sum(inst["nbytes"][VERS.index(b)] for row in r.bits for b in row if b)
+        budget = int(rng.integers(0, total + 3000))
+        want, want_used = po.retain_after_run(r.keep, r.bits, inst["nbytes"], budget)
+        got, used = sti.sti_preload_after_run(np.array(r.keep), np.array(r.bits), inst["nbytes"], budget)
+        assert got.tolist() == want and used == want_used
+    with pytest.raises(sti.StiError):                                      # a kept shard with an unknown version
+        sti.sti_preload_after_run(np.ones((1, 2)), np.array([[2, 7]]), [1] * 6, 10)
