@@ -10,8 +10,8 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB_NAME = "libsti_b200.so"
 LIB_PATH = os.path.join(HERE, LIB_NAME)
-SOURCES = ["api.cu", "dqgemm.cu", "attention.cu", "layernorm.cu", "decode.cu", "noalloc.cu", "planner.cu"]
-HEADERS = ["sti_kernels.h", "sti_device.cuh", "retile.h", os.path.join("..", "..", "include", "sti.h"),
+SOURCES = ["api.cu", "dqgemm.cu", "attention.cu", "layernorm.cu", "layerfused.cu", "decode.cu", "noalloc.cu", "planner.cu"]
+HEADERS = ["sti_kernels.h", "sti_device.cuh", "gemm_device.cuh", "retile.h", os.path.join("..", "..", "include", "sti.h"),
            os.path.join("..", "..", "include", "sti_planner.h")]
 NVCC_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",

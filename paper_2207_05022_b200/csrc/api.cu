@@ -33,6 +33,7 @@ struct Tuning {
   int qkv_n = 32, f1_n = 64, o_n = 64, o_group = 4, f2_n = 64, f2_group = 2;
   int cta_budget = 148;                // CTAs a GEMM launch may use when it splits the token tiles over CTAs
   int pair_min_tiles = 8;              // two-CTA GEMM from this many 128-token tiles on (0 = never)
+  int fused_max_tokens = 0;            // whole-layer kernel up to this many tokens (0 = never; STI_TUNE turns it on)
 };
 
 struct Unit {
@@ -54,6 +55,7 @@ struct GemmTable {
   uint32_t w_bytes = 0, n_stages = 0, bps = 1, k_max = 0, hdr_bytes = 0;
   bool pair_ok = false;                // consecutive jobs can share two-CTA MMAs (64-row tiles, same K range)
   int n_split = 0;
+  uint32_t f_stages = 0, f_bps = 0;    // activation ring inside the whole-layer kernel (0: the tile does not fit there)
 };
 
 struct Layer {
@@ -128,6 +130,8 @@ struct sti_plan {
   void* buf[2] = {nullptr, nullptr};
   void* x_in = nullptr; void* y_out = nullptr; int32_t* lens_dev = nullptr;
   int max_partial = 1;
+  unsigned int* fused_ctr = nullptr;   // one grid-barrier counter per layer, zeroed at the start of every forward
+  bool fused_off = false;
   bool stats_valid = false;
 };
 
@@ -184,6 +188,7 @@ void parse_tuning(Tuning* t, int tmax, const sti_model_desc& d) {
         else if (k == "f2_group") t->f2_group = v;
         else if (k == "pair_min_tiles") t->pair_min_tiles = v;
         else if (k == "cta_budget") t->cta_budget = std::max(1, v);
+        else if (k == "fused_max_tokens") t->fused_max_tokens = std::max(0, v);
       }
       pos = end + 1;
     }
@@ -322,7 +327,8 @@ sti_status check_async(sti_ctx* c) {
   if (flag != ERR_NONE) {
     int zero = 0;
     (void)cudaMemcpy(c->err_dev, &zero, sizeof(int), cudaMemcpyHostToDevice);
-    return flag == ERR_WAIT_TIMEOUT ? STI_ERR_TIMEOUT : STI_ERR_ARG;
+    if (getenv("STI_VERBOSE")) fprintf(stderr, "sti: device status word 0x%08x\n", static_cast<unsigned>(flag));
+    return (flag & 0xff) == ERR_WAIT_TIMEOUT ? STI_ERR_TIMEOUT : STI_ERR_ARG;
   }
   return STI_OK;
 }
@@ -383,6 +389,65 @@ sti_status run_gemm(sti_plan* p, GemmKind kind, const GemmTable& tab, const void
   return STI_OK;
 }
 
+// One launch for the whole layer (few tokens): returns STI_OK and sets *done when the layer was enqueued
+// through the whole-layer kernel, leaves *done false when the shapes call for the seven-kernel path.
+sti_status enqueue_layer_fused(sti_plan* p, int li, const void* xq, const void* x, void* y, int batch, int seq,
+                               const int32_t* lens, bool want_next_bf16, bool* done) {
+  *done = false;
+  sti_ctx* c = p->ctx;
+  const sti_model_desc& d = c->desc;
+  Layer& L = p->layers[li];
+  const int T = batch * seq;
+  const int nh = static_cast<int>(L.kept_heads.size()), ns = static_cast<int>(L.kept_slices.size());
+  if (p->fused_off || c->simt_debug || p->profiling >= 2 || nh == 0 || ns == 0 || T > p->tune.fused_max_tokens) return STI_OK;
+  const GemmTable* gt[4] = {&L.qkv, &L.o, &L.f1, &L.f2};
+  int grid = 1;
+  for (const GemmTable* t : gt) {
+    if (t->f_stages == 0 || t->n_jobs < 1 || t->n_jobs > kFusedMaxCtas) return STI_OK;
+    grid = std::max(grid, t->n_jobs * m_ctas_for(t->n_jobs, T, kFusedMaxCtas));
+  }
+  const size_t top = fused_smem_total() - 1024, attn_end = fused_low_offset() + fused_attention_bytes(seq);
+  if (attn_end > top) return STI_OK;
+  const float* dense = c->dense + static_cast<size_t>(li) * c->dense_stride;
+  const bool bf16_act = d.act_dtype == STI_BF16;
+  const int f = d.ffn / d.n_ffn_slices;
+  FusedLayerParams fp{};
+  const void* xs[4] = {xq, p->attn_out, p->h1_bf16, p->u};
+  const int ldx[4] = {d.hidden, nh * 64, d.hidden, ns * f};
+  void* outs[4] = {p->qkv, p->partial, p->u, p->partial};
+  const int ldo[4] = {64, d.hidden, ns * f, d.hidden};
+  const float* bias[4] = {dense + c->off_bq, nullptr, dense + c->off_b1, nullptr};
+  const int kinds[4] = {GEMM_BF16_TO_BF16, GEMM_BF16_TO_F32, GEMM_BF16_TO_BF16_GELU, GEMM_BF16_TO_F32};
+  for (int i = 0; i < 4; ++i) {
+    FusedGemm& g = fp.g[i];
+    if (!make_xmap(&g.xmap, xs[i], ldx[i], T)) return STI_ERR_CUDA;
+    g.jobs = gt[i]->jobs; g.segs = gt[i]->segs; g.out = outs[i]; g.bias = bias[i];
+    g.n_jobs = gt[i]->n_jobs; g.m_ctas = m_ctas_for(gt[i]->n_jobs, T, kFusedMaxCtas);
+    g.ldo = ldo[i]; g.kind = kinds[i];
+    g.n_stages = gt[i]->f_stages; g.bps = gt[i]->f_bps; g.w_bytes = gt[i]->w_bytes;
+    g.ahead = 1;
+  }
+  fp.g[0].ahead = 0;
+  fp.g[1].ahead = attn_end + L.o.w_bytes <= top ? 1 : 0;    // the O tile must fit above the attention buffers
+  LnLaunch& l1 = fp.ln[0];
+  l1.partial = p->partial; l1.n_partial = L.o.n_split; l1.bias = dense + c->off_bo; l1.resid = x;
+  l1.resid_bf16 = bf16_act ? 1 : 0; l1.gamma = dense + c->off_ln1g; l1.beta = dense + c->off_ln1b; l1.eps = d.ln_eps;
+  l1.T = T; l1.d = d.hidden; l1.out_f32 = p->h1_f32; l1.out_bf16 = p->h1_bf16;
+  LnLaunch& l2 = fp.ln[1];
+  l2.partial = p->partial; l2.n_partial = L.f2.n_split; l2.bias = dense + c->off_b2; l2.resid = p->h1_f32;
+  l2.resid_bf16 = 0; l2.gamma = dense + c->off_ln2g; l2.beta = dense + c->off_ln2b; l2.eps = d.ln_eps;
+  l2.T = T; l2.d = d.hidden;
+  l2.out_f32 = bf16_act ? nullptr : static_cast<float*>(y);
+  l2.out_bf16 = bf16_act ? static_cast<uint16_t*>(y) : (want_next_bf16 ? p->x_bf16 : nullptr);
+  fp.qkv = p->qkv; fp.attn_out = p->attn_out; fp.seq_lens = lens;
+  fp.n_kept_heads = nh; fp.batch = batch; fp.seq = seq; fp.T = T;
+  fp.barrier = p->fused_ctr + li; fp.err = c->err_dev;
+  CUDA_TRY(launch_fused_layer(fp, grid, c->compute, c->pdl));
+  c->launches++;
+  *done = true;
+  return STI_OK;
+}
+
 // The seven kernels of one layer on the compute stream.
 // `x_ready_bf16`: the bf16 copy of x already sits in p->x_bf16 (written by the previous layer's LayerNorm);
 // `want_next_bf16`: this layer's last kernel also writes y as bf16 into p->x_bf16 for the next layer.
@@ -411,6 +476,13 @@ sti_status enqueue_layer(sti_plan* p, int li, const void* x, void* y, int batch,
         c->launches++;
       }
       xq = p->x_bf16;
+    }
+    bool fused = false;
+    st = enqueue_layer_fused(p, li, xq, x, y, batch, seq, lens, want_next_bf16, &fused);
+    if (st != STI_OK) return st;
+    if (fused) {
+      for (int i = 1; i <= 7; ++i) CUDA_TRY(mark(i));
+      return STI_OK;
     }
     st = run_gemm(p, GEMM_BF16_TO_BF16, L.qkv, xq, d.hidden, T, p->qkv, 64, dense + c->off_bq);
     if (st != STI_OK) return st;
@@ -544,6 +616,8 @@ sti_status enqueue_forward_io(sti_plan* p, const ForwardKey& k, bool capturing) 
     x = p->x_in;
     y = p->y_out;
   }
+  // grid-barrier counters of the whole-layer kernels start every forward at zero
+  CUDA_TRY(cudaMemsetAsync(p->fused_ctr, 0, p->layers.size() * sizeof(unsigned int), c->compute));
   sti_status st;
   if (k.layer >= 0) {
     // a single layer: its IO job (if it has streamed units) runs on the compute stream, not overlapped
@@ -623,6 +697,7 @@ void free_plan_device(sti_plan* p) {
   cudaFree(p->qkv); cudaFree(p->attn_out); cudaFree(p->partial); cudaFree(p->h1_f32); cudaFree(p->h1_bf16);
   cudaFree(p->u); cudaFree(p->x_bf16); cudaFree(p->buf[0]); cudaFree(p->buf[1]); cudaFree(p->x_in); cudaFree(p->y_out);
   cudaFree(p->lens_dev);
+  cudaFree(p->fused_ctr);
   for (auto& L : p->layers) {
     if (L.ev_loaded) cudaEventDestroy(L.ev_loaded);
     if (L.g_ev_loaded) cudaEventDestroy(L.g_ev_loaded);
@@ -715,7 +790,8 @@ sti_status sti_ctx_create(const sti_model_desc* desc, int device, void* compute_
   if (cudaMemset(c->dense, 0, c->dense_stride * d.n_layers * sizeof(float)) != cudaSuccess) return fail(STI_ERR_CUDA);
   if (cudaMalloc(&c->err_dev, sizeof(int)) != cudaSuccess) return fail(STI_ERR_OOM);
   if (cudaMemset(c->err_dev, 0, sizeof(int)) != cudaSuccess) return fail(STI_ERR_CUDA);
-  if (gemm_configure() != cudaSuccess || attention_configure() != cudaSuccess) return fail(STI_ERR_CUDA);
+  if (gemm_configure() != cudaSuccess || attention_configure() != cudaSuccess || fused_configure() != cudaSuccess)
+    return fail(STI_ERR_CUDA);
   const char* dbg = getenv("STI_DEBUG_SIMT");
   c->simt_debug = dbg && dbg[0] == '1';
   const char* nopdl = getenv("STI_NO_PDL");
@@ -924,6 +1000,10 @@ sti_status sti_plan_finalize(sti_plan* p) {
           !gemm_pick_ring(tb[i].w_bytes, tb[i].k_max, gt[i]->hdr_bytes, &gt[i]->n_stages, &gt[i]->bps))
         return STI_ERR_SHAPE;
       gt[i]->smem = gemm_smem_bytes(tb[i].w_bytes, gt[i]->n_stages, gt[i]->bps, gt[i]->hdr_bytes);
+      // the whole-layer kernel keeps both header slots resident: its activation ring starts further up
+      if (tb[i].jobs.empty() || tb[i].seg_max > 16 ||
+          !gemm_pick_ring(tb[i].w_bytes, tb[i].k_max, static_cast<uint32_t>(fused_low_offset()), &gt[i]->f_stages, &gt[i]->f_bps))
+        gt[i]->f_stages = gt[i]->f_bps = 0;
       if (gt[i]->smem > kMaxSmem && !tb[i].jobs.empty()) return STI_ERR_SHAPE;
       Fix fx{gt[i], 0, 0};
       fx.jobs_off = align16(host_tables.size());
@@ -959,6 +1039,8 @@ sti_status sti_plan_finalize(sti_plan* p) {
   CUDA_TRY(cudaMalloc(&p->x_in, Tmax * d.hidden * act_size(c)));
   CUDA_TRY(cudaMalloc(&p->y_out, Tmax * d.hidden * act_size(c)));
   CUDA_TRY(cudaMalloc(&p->lens_dev, static_cast<size_t>(d.max_batch) * 4));
+  CUDA_TRY(cudaMalloc(&p->fused_ctr, static_cast<size_t>(d.n_layers) * sizeof(unsigned int)));
+  CUDA_TRY(cudaMemset(p->fused_ctr, 0, static_cast<size_t>(d.n_layers) * sizeof(unsigned int)));
   // 5. events
   const unsigned flags = cudaEventDefault;     // timing-capable; only recorded when profiling
   for (auto& L : p->layers) {
@@ -980,6 +1062,7 @@ sti_status sti_plan_finalize(sti_plan* p) {
   p->g_slot_free.resize(p->ring_slots);
   for (auto& e : p->g_slot_free) CUDA_TRY(cudaEventCreateWithFlags(&e, cudaEventDisableTiming));
   { const char* ng = getenv("STI_NO_GRAPH"); p->graph_off = ng && ng[0] == '1'; }
+  { const char* nf = getenv("STI_NO_FUSED"); p->fused_off = nf && nf[0] == '1'; }
   CUDA_TRY(cudaEventCreateWithFlags(&p->ev_begin, flags));
   CUDA_TRY(cudaEventCreateWithFlags(&p->ev_end, flags));
   p->finalized = true;

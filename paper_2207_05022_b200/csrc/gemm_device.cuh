@@ -1,0 +1,210 @@
+// Device-side pieces of the fused dequant-GEMM that more than one kernel uses: tile constants, the
+// shared-memory header with the mbarriers, the weight-tile decode (Section 4.2 decompression: index
+// unpack -> per-unit centroid table -> outlier patch), TMA / descriptor helpers and the epilogue maths.
+#pragma once
+#include <cuda.h>
+#include <cuda_bf16.h>
+
+#include "sti_device.cuh"
+#include "sti_kernels.h"
+
+namespace sti {
+namespace {
+
+constexpr int kThreads = 512;               // warp 0: TMA producer, warp 1: MMA issuer, warps 4-7: epilogue; all 16 decode
+constexpr int kWarps = kThreads / 32;
+constexpr int kTileM = 128;                 // tokens per MMA tile
+constexpr int kChunkK = 64;                 // one TMA box = 64 columns = one 128-byte swizzle row; a stage holds 1, 2 or 4 boxes
+constexpr int kMaxStages = 8;
+constexpr int kBoxBytes = kTileM * kChunkK * 2;     // 16 KB
+// header = barriers (256 B) + bias (512 B) + one 128-byte table per segment; stages start 1024-aligned after it
+constexpr int kHeaderSmall = 1024;          // single-segment tiles (QKV, FFN1)
+constexpr int kHeaderLarge = 3072;          // up to 16 segments (O projection, FFN2)
+constexpr int kAlignSlack = 1024;           // the dynamic shared-memory base is aligned up to 1024 by hand
+constexpr int kMaxSegs = 16;
+constexpr int kTableStride = 64;            // bf16 entries per segment table
+constexpr int kEpilogueWarp0 = 4;             // epilogue warps 4..11: two per TMEM lane quadrant
+constexpr int kEpilogueWarps = 8;
+
+struct SmemHeader {
+  uint64_t full[kMaxStages];     // activation chunk landed (TMA transaction bytes)
+  uint64_t empty[kMaxStages];    // the MMAs that read the chunk have completed
+  uint64_t acc_full[2];          // accumulator buffer complete
+  uint64_t acc_empty[2];         // accumulator buffer drained by the epilogue warps
+  uint64_t drain;                // failure path only: all issued MMAs have completed
+  uint32_t tmem_base;
+  volatile uint32_t abort;       // a bounded wait ran out somewhere in the CTA
+};
+
+// ---------------------------------------------------------------------------------------
+// Weight-tile decode
+// ---------------------------------------------------------------------------------------
+template <int BITS>
+__device__ __forceinline__ void decode_task(const Seg& sg, const uint16_t* __restrict__ tab, uint8_t* wsm,
+                                            uint32_t n_rows, uint32_t task, uint32_t lane) {
+  // task = (row group, 128-column chunk); the k planes of the group are contiguous.
+  const uint32_t chunks = sg.kc >= 128 ? sg.kc / 128 : 1;
+  const uint32_t g = task / chunks, j = task % chunks;
+  const uint4* src = sg.codes + (static_cast<size_t>(g) * chunks + j) * (BITS * 32) + lane;
+  uint32_t w[4 * BITS];
+#pragma unroll
+  for (int p = 0; p < BITS; ++p) {
+    const uint4 v = __ldg(src + p * 32);
+    w[4 * p + 0] = v.x; w[4 * p + 1] = v.y; w[4 * p + 2] = v.z; w[4 * p + 3] = v.w;
+  }
+  const bool narrow = sg.kc < 128;     // 64 in-features: the quantum is rows (l, l + 32) of a 64-row group
+  const uint32_t row0 = narrow ? g * 64 + lane : g * 32 + lane;
+  const uint32_t kcore0 = (sg.koff + (narrow ? 0 : j * 128)) >> 3;
+#pragma unroll
+  for (int s = 0; s < 16; ++s) {
+    uint32_t pk[4];
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+      const uint32_t c0 = extract_index<BITS>(w, 8 * s + 2 * e);
+      const uint32_t c1 = extract_index<BITS>(w, 8 * s + 2 * e + 1);
+      pk[e] = static_cast<uint32_t>(tab[c0]) | (static_cast<uint32_t>(tab[c1]) << 16);
+    }
+    const uint32_t row = narrow ? row0 + 32 * (s >> 3) : row0;
+    const uint32_t kcore = narrow ? kcore0 + (s & 7) : kcore0 + s;
+    *reinterpret_cast<uint4*>(wsm + (static_cast<size_t>(kcore) * n_rows + row) * 16) =
+        make_uint4(pk[0], pk[1], pk[2], pk[3]);
+  }
+}
+
+// Uncompressed (32-bit) version of a unit: rows are plain fp32, converted to bf16 on the way in.
+__device__ __forceinline__ void decode_raw(const Seg& sg, uint8_t* wsm, uint32_t n_rows, uint32_t tid) {
+  const float* src = reinterpret_cast<const float*>(sg.codes);
+  const uint32_t pieces_per_row = sg.kc / 8;
+  const uint32_t total = n_rows * pieces_per_row;
+  for (uint32_t idx = tid; idx < total; idx += kThreads) {
+    const uint32_t row = idx % n_rows, piece = idx / n_rows;
+    const float4 a = __ldg(reinterpret_cast<const float4*>(src + static_cast<size_t>(row) * sg.kc + piece * 8));
+    const float4 b = __ldg(reinterpret_cast<const float4*>(src + static_cast<size_t>(row) * sg.kc + piece * 8 + 4));
+    const uint32_t kcore = (sg.koff >> 3) + piece;
+    *reinterpret_cast<uint4*>(wsm + (static_cast<size_t>(kcore) * n_rows + row) * 16) =
+        make_uint4(pack_bf16x2(a.x, a.y), pack_bf16x2(a.z, a.w), pack_bf16x2(b.x, b.y), pack_bf16x2(b.z, b.w));
+  }
+}
+
+// ---------------------------------------------------------------------------------------
+// TMA / mbarrier helpers local to this kernel
+// ---------------------------------------------------------------------------------------
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+// [128 rows x 64 columns] box at (column k0, row m0); rows past the tensor's extent arrive as zeros.
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int k0, int m0, uint32_t bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+      ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(k0), "r"(m0), "r"(bar)
+      : "memory");
+}
+// K-major, 128-byte swizzle: rows of 128 bytes, 8-row groups 1024 bytes apart.
+__device__ __forceinline__ uint64_t umma_smem_desc_sw128(uint32_t saddr) {
+  uint64_t d = 0;
+  d |= static_cast<uint64_t>((saddr & 0x3FFFFu) >> 4);
+  d |= static_cast<uint64_t>(1) << 16;                 // leading byte offset: unused for this layout
+  d |= static_cast<uint64_t>(1024 >> 4) << 32;         // stride byte offset
+  d |= static_cast<uint64_t>(1) << 46;                 // descriptor version for sm_100
+  d |= static_cast<uint64_t>(2) << 61;                 // layout type: 128-byte swizzle
+  return d;
+}
+
+// erf-GELU.  erf through the rational approximation 7.1.26 of Abramowitz & Stegun (absolute error
+// below 1.5e-7, three orders of magnitude under the bf16 rounding of the result) with the hardware
+// exponential; the epilogue runs it for every element of the FFN1 output.
+__device__ __forceinline__ float gelu_erf(float v) {
+  const float x = fabsf(v) * 0.70710678118654752440f;
+  const float t = __fdividef(1.0f, fmaf(0.3275911f, x, 1.0f));
+  float poly = fmaf(1.061405429f, t, -1.453152027f);
+  poly = fmaf(poly, t, 1.421413741f);
+  poly = fmaf(poly, t, -0.284496736f);
+  poly = fmaf(poly, t, 0.254829592f);
+  const float erf_abs = 1.0f - poly * t * __expf(-x * x);
+  return 0.5f * v * (1.0f + copysignf(erf_abs, v));
+}
+
+template <typename OutT>
+__device__ __forceinline__ void store_row16(OutT* dst, const float (&v)[16]) {
+  if constexpr (sizeof(OutT) == 2) {
+    uint32_t p[8];
+#pragma unroll
+    for (int i = 0; i < 8; ++i) p[i] = pack_bf16x2(v[2 * i], v[2 * i + 1]);
+    reinterpret_cast<uint4*>(dst)[0] = make_uint4(p[0], p[1], p[2], p[3]);
+    reinterpret_cast<uint4*>(dst)[1] = make_uint4(p[4], p[5], p[6], p[7]);
+  } else {
+#pragma unroll
+    for (int i = 0; i < 4; ++i)
+      reinterpret_cast<float4*>(dst)[i] = make_float4(v[4 * i], v[4 * i + 1], v[4 * i + 2], v[4 * i + 3]);
+  }
+}
+
+// ---------------------------------------------------------------------------------------
+// Pieces shared by the one-CTA and the two-CTA kernel
+// ---------------------------------------------------------------------------------------
+// Centroid tables of the job's segments, rounded once to bf16 (round-to-nearest-even), and a head start
+// for the outlier lists, which are needed right after the decode.
+__device__ __forceinline__ void load_tables(const Job& job, const Seg* __restrict__ segs, uint16_t* tables, uint32_t tid) {
+  for (uint32_t i = tid; i < job.n_seg * kTableStride; i += kThreads) {
+    const Seg& sg = segs[job.seg_begin + i / kTableStride];
+    const uint32_t e = i % kTableStride;
+    tables[i] = (sg.bits <= 6 && e < (1u << sg.bits)) ? bf16_bits(__ldg(sg.table + e)) : 0;
+  }
+  for (uint32_t si = 0; si < job.n_seg; ++si) {
+    const Seg& sg = segs[job.seg_begin + si];
+    for (uint32_t o = tid * 32; o < sg.n_out; o += kThreads * 32) {
+      asm volatile("prefetch.global.L2 [%0];" ::"l"(sg.out_off + o));
+      asm volatile("prefetch.global.L2 [%0];" ::"l"(sg.out_val + o));
+    }
+  }
+}
+
+// Decode of the job's weight tile into `wsm` (all threads of the CTA; ends with the tile visible to the
+// tensor core: proxy fence + CTA barrier).  Needs the tables in place (a CTA barrier after load_tables).
+__device__ __forceinline__ void decode_weight_tile(const Job& job, const Seg* __restrict__ segs, const uint16_t* tables,
+                                                   uint8_t* wsm, uint32_t tid) {
+  const uint32_t lane = tid & 31, warp = tid >> 5;
+  const uint32_t n_rows = job.n_rows, k_total = job.k_total;
+  const Seg& s0 = segs[job.seg_begin];
+  const uint32_t rows_per_group = s0.kc >= 128 ? 32 : 64;
+  const uint32_t chunks = s0.kc >= 128 ? s0.kc / 128 : 1;
+  const uint32_t tasks_per_seg = (n_rows / rows_per_group) * chunks;
+  const uint32_t n_tasks = tasks_per_seg * job.n_seg;
+  for (uint32_t t = warp; t < n_tasks; t += kWarps) {
+    const uint32_t si = t / tasks_per_seg, task = t % tasks_per_seg;
+    const Seg& sg = segs[job.seg_begin + si];
+    const uint16_t* tab = tables + si * kTableStride;
+    switch (sg.bits) {
+      case 2: decode_task<2>(sg, tab, wsm, n_rows, task, lane); break;
+      case 3: decode_task<3>(sg, tab, wsm, n_rows, task, lane); break;
+      case 4: decode_task<4>(sg, tab, wsm, n_rows, task, lane); break;
+      case 5: decode_task<5>(sg, tab, wsm, n_rows, task, lane); break;
+      case 6: decode_task<6>(sg, tab, wsm, n_rows, task, lane); break;
+      default: break;
+    }
+  }
+  for (uint32_t si = 0; si < job.n_seg; ++si) {
+    const Seg& sg = segs[job.seg_begin + si];
+    if (sg.bits == 32) decode_raw(sg, wsm, n_rows, tid);
+  }
+  __syncthreads();
+  // outliers keep their original value (Section 6): overwrite their slot
+  for (uint32_t si = 0; si < job.n_seg; ++si) {
+    const Seg& sg = segs[job.seg_begin + si];
+    for (uint32_t o = tid; o < sg.n_out; o += kThreads) {
+      const uint32_t local = __ldg(sg.out_off + o) - sg.flat_base;
+      const uint32_t row = local / sg.kc, kk = sg.koff + local % sg.kc;
+      if (row < n_rows && kk < k_total)
+        reinterpret_cast<uint16_t*>(wsm)[(static_cast<size_t>(kk >> 3) * n_rows + row) * 8 + (kk & 7)] =
+            bf16_bits(__ldg(sg.out_val + o));
+    }
+  }
+  fence_proxy_async_smem();
+  __syncthreads();
+}
+
+}  // namespace
+}  // namespace sti

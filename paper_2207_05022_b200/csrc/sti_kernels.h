@@ -111,6 +111,49 @@ struct DecodeLaunch {
 };
 cudaError_t launch_decode(const DecodeLaunch& p, cudaStream_t s);
 
+// ---------------------------------------------------------------------------------------
+// Whole-layer kernel for few tokens (one launch per layer instead of seven).
+// A grid of at most one CTA per SM runs the layer's seven steps one after the other - QKV GEMM,
+// attention, O projection, residual + LayerNorm, FFN1 + GELU, FFN2, residual + LayerNorm - with a
+// grid-wide barrier between steps.  Between arriving at a barrier and waiting on it a CTA decodes the
+// weight tile of its next GEMM step (weights depend on no activation), so shard decode never sits on
+// the critical path, and the barriers replace the kernel boundaries.
+// ---------------------------------------------------------------------------------------
+struct FusedGemm {
+  CUtensorMap xmap;         // activation operand of this step: [T, ld] bf16, box 64 x 128, 128-byte swizzle
+  const Job* jobs;
+  const Seg* segs;
+  void* out;
+  const float* bias;
+  int n_jobs;
+  int m_ctas;               // CTAs per job along the token dimension; n_jobs * m_ctas <= grid
+  int ldo;
+  int kind;                 // GemmKind
+  uint32_t n_stages, bps;   // activation ring: stages, 16 KB boxes per stage
+  uint32_t w_bytes;         // shared memory of the largest weight tile of this step
+  uint32_t ahead;           // 1: the tile is decoded before the preceding barrier wait (its shared memory is free then)
+};
+
+struct FusedLayerParams {
+  FusedGemm g[4];           // QKV, O projection, FFN1, FFN2
+  LnLaunch ln[2];           // after the O projection, after FFN2
+  const uint16_t* qkv;      // attention operands / result, as in launch_attention
+  uint16_t* attn_out;
+  const int32_t* seq_lens;
+  int n_kept_heads, batch, seq, T;
+  unsigned int* barrier;    // one counter per launch, zero when the kernel starts
+  int* err;
+};
+
+constexpr int kFusedMaxCtas = 148;
+cudaError_t fused_configure();
+// Shared memory the attention step needs for sequences of `seq` tokens, counted from the start of the
+// activation area; the O-projection tile may be decoded ahead only if it fits above that.
+size_t fused_attention_bytes(int seq);
+size_t fused_smem_total();      // dynamic shared memory of the kernel
+size_t fused_low_offset();      // where the activation stages / attention buffers start
+cudaError_t launch_fused_layer(const FusedLayerParams& p, int grid, cudaStream_t s, bool pdl);
+
 // Launch with or without the programmatic-dependent-launch attribute (every kernel of the layer calls
 // pdl_wait before it reads what its predecessor wrote, so consecutive kernels may overlap their prologues).
 template <typename... KArgs, typename... Args>
