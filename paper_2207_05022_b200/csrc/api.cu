@@ -52,7 +52,7 @@ struct GemmTable {
   Seg* segs = nullptr;
   int n_jobs = 0;
   size_t smem = 0;
-  uint32_t w_bytes = 0, n_stages = 0, bps = 1, k_max = 0, hdr_bytes = 0;
+  uint32_t w_bytes = 0, n_stages = 0, bps = 1, k_max = 0, hdr_bytes = 0, seg_stride = 0;
   bool pair_ok = false;                // consecutive jobs can share two-CTA MMAs (64-row tiles, same K range)
   int n_split = 0;
   uint32_t f_stages = 0, f_bps = 0;    // activation ring inside the whole-layer kernel (0: the tile does not fit there)
@@ -65,6 +65,7 @@ struct Layer {
   uint8_t* res_dev = nullptr;          // in the preload buffer
   uint8_t* str_host = nullptr;         // in the pinned arena
   int slot = -1;                       // ring slot of the streamed part
+  size_t tables_off = 0, tables_bytes = 0;   // this layer's tile-job descriptors inside the plan's table buffer
   GemmTable qkv, o, f1, f2;
   cudaEvent_t ev_loaded = nullptr, ev_done = nullptr, ev_copy_start = nullptr, ev_comp_start = nullptr;
   cudaEvent_t g_ev_loaded = nullptr;   // the same role inside graph capture (captured events cannot be reused outside)
@@ -207,7 +208,7 @@ void parse_tuning(Tuning* t, int tmax, const sti_model_desc& d) {
   // keep every weight tile inside shared memory
   auto fits = [](int n, int k) {
     uint32_t st = 0, bp = 0;
-    return gemm_pick_ring(static_cast<uint32_t>(gemm_weight_bytes(n, k)), k, gemm_header_bytes(16), &st, &bp) && st * bp >= 4;
+    return gemm_pick_ring(static_cast<uint32_t>(gemm_weight_bytes(n, k)), k, gemm_header_bytes(), &st, &bp) && st * bp >= 4;
   };
   while (t->qkv_n > 32 && !fits(t->qkv_n, d.hidden)) t->qkv_n /= 2;
   while (t->f1_n > 32 && !fits(t->f1_n, d.hidden)) t->f1_n /= 2;
@@ -248,16 +249,24 @@ Seg make_seg(const sti_ctx* c, const Unit& u, sti_kind kind, int m, uint32_t row
 
 struct TableBuilder {
   std::vector<Job> jobs;
-  std::vector<Seg> segs;
-  uint32_t w_bytes = 0, k_max = 0, seg_max = 0;
+  std::vector<std::vector<Seg>> job_segs;
+  std::vector<Seg> segs;               // filled by finish(): job j's segments start at j * seg_stride
+  uint32_t w_bytes = 0, k_max = 0, seg_stride = 0;
   void add(Job j, const std::vector<Seg>& ss) {
-    j.seg_begin = static_cast<uint32_t>(segs.size());
     j.n_seg = static_cast<uint32_t>(ss.size());
-    segs.insert(segs.end(), ss.begin(), ss.end());
     jobs.push_back(j);
+    job_segs.push_back(ss);
     w_bytes = std::max(w_bytes, static_cast<uint32_t>(gemm_weight_bytes(j.n_rows, j.k_total)));
     k_max = std::max(k_max, j.k_total);
-    seg_max = std::max(seg_max, j.n_seg);
+    seg_stride = std::max(seg_stride, j.n_seg);
+  }
+  // A fixed stride lets a CTA fetch its job and its segments in the same memory round trip.
+  void finish() {
+    segs.assign(jobs.size() * seg_stride, Seg{});
+    for (size_t j = 0; j < jobs.size(); ++j) {
+      jobs[j].seg_begin = static_cast<uint32_t>(j * seg_stride);
+      std::copy(job_segs[j].begin(), job_segs[j].end(), segs.begin() + j * seg_stride);
+    }
   }
 };
 
@@ -370,8 +379,20 @@ int m_ctas_for(int n_jobs, int T, int cta_budget) {
   return std::max(1, std::min(m, n_mtiles));
 }
 
+// The packed shards of layer `li` as (address, bytes) ranges: its part of the preload buffer and its ring slot.
+void layer_ranges(const sti_plan* p, int li, const uint8_t* ptr[4], uint32_t bytes[4]) {
+  for (int r = 0; r < 4; ++r) { ptr[r] = nullptr; bytes[r] = 0; }
+  if (li < 0 || li >= static_cast<int>(p->layers.size())) return;
+  const Layer& L = p->layers[li];
+  if (L.res_bytes) { ptr[0] = L.res_dev; bytes[0] = static_cast<uint32_t>(L.res_bytes); }
+  if (L.str_bytes) { ptr[1] = p->ring + static_cast<size_t>(L.slot) * p->slot_bytes; bytes[1] = static_cast<uint32_t>(L.str_bytes); }
+  ptr[2] = p->tables + L.tables_off; bytes[2] = static_cast<uint32_t>(L.tables_bytes);
+  ptr[3] = reinterpret_cast<const uint8_t*>(p->ctx->dense + static_cast<size_t>(li) * p->ctx->dense_stride);
+  bytes[3] = static_cast<uint32_t>(p->ctx->dense_stride * sizeof(float));
+}
+
 sti_status run_gemm(sti_plan* p, GemmKind kind, const GemmTable& tab, const void* x, int ldx, int T, void* out,
-                    int ldo, const float* bias) {
+                    int ldo, const float* bias, int prefetch_layer = -1) {
   if (tab.n_jobs == 0) return STI_OK;
   GemmLaunch g{};
   g.jobs = tab.jobs; g.segs = tab.segs; g.n_jobs = tab.n_jobs; g.m_ctas = m_ctas_for(tab.n_jobs, T, p->tune.cta_budget);
@@ -382,8 +403,9 @@ sti_status run_gemm(sti_plan* p, GemmKind kind, const GemmTable& tab, const void
     g.m_ctas = std::max(1, std::min(n_mpairs, p->tune.cta_budget / tab.n_jobs));
   }
   if (!make_xmap(&g.xmap, x, ldx, T)) return STI_ERR_CUDA;
+  layer_ranges(p, prefetch_layer, g.pf_ptr, g.pf_bytes);
   g.x = x; g.ldx = ldx; g.T = T; g.out = out; g.ldo = ldo; g.bias = bias; g.err = p->ctx->err_dev;
-  g.smem_bytes = tab.smem; g.n_stages = tab.n_stages; g.bps = tab.bps; g.w_bytes = tab.w_bytes; g.hdr_bytes = tab.hdr_bytes; g.simt_debug = p->ctx->simt_debug; g.pdl = p->ctx->pdl;
+  g.smem_bytes = tab.smem; g.n_stages = tab.n_stages; g.bps = tab.bps; g.w_bytes = tab.w_bytes; g.hdr_bytes = tab.hdr_bytes; g.seg_stride = tab.seg_stride; g.simt_debug = p->ctx->simt_debug; g.pdl = p->ctx->pdl;
   CUDA_TRY(launch_gemm(kind, g, p->ctx->compute));
   p->ctx->launches++;
   return STI_OK;
@@ -392,7 +414,7 @@ sti_status run_gemm(sti_plan* p, GemmKind kind, const GemmTable& tab, const void
 // One launch for the whole layer (few tokens): returns STI_OK and sets *done when the layer was enqueued
 // through the whole-layer kernel, leaves *done false when the shapes call for the seven-kernel path.
 sti_status enqueue_layer_fused(sti_plan* p, int li, const void* xq, const void* x, void* y, int batch, int seq,
-                               const int32_t* lens, bool want_next_bf16, bool* done) {
+                               const int32_t* lens, bool want_next_bf16, int next_layer, bool* done) {
   *done = false;
   sti_ctx* c = p->ctx;
   const sti_model_desc& d = c->desc;
@@ -406,7 +428,7 @@ sti_status enqueue_layer_fused(sti_plan* p, int li, const void* xq, const void* 
     if (t->f_stages == 0 || t->n_jobs < 1 || t->n_jobs > kFusedMaxCtas) return STI_OK;
     grid = std::max(grid, t->n_jobs * m_ctas_for(t->n_jobs, T, kFusedMaxCtas));
   }
-  const size_t top = fused_smem_total() - 1024, attn_end = fused_low_offset() + fused_attention_bytes(seq);
+  const size_t top = fused_smem_total(), attn_end = fused_low_offset() + fused_attention_bytes(seq);
   if (attn_end > top) return STI_OK;
   const float* dense = c->dense + static_cast<size_t>(li) * c->dense_stride;
   const bool bf16_act = d.act_dtype == STI_BF16;
@@ -424,7 +446,7 @@ sti_status enqueue_layer_fused(sti_plan* p, int li, const void* xq, const void* 
     g.jobs = gt[i]->jobs; g.segs = gt[i]->segs; g.out = outs[i]; g.bias = bias[i];
     g.n_jobs = gt[i]->n_jobs; g.m_ctas = m_ctas_for(gt[i]->n_jobs, T, kFusedMaxCtas);
     g.ldo = ldo[i]; g.kind = kinds[i];
-    g.n_stages = gt[i]->f_stages; g.bps = gt[i]->f_bps; g.w_bytes = gt[i]->w_bytes;
+    g.n_stages = gt[i]->f_stages; g.bps = gt[i]->f_bps; g.w_bytes = gt[i]->w_bytes; g.seg_stride = gt[i]->seg_stride;
     g.ahead = 1;
   }
   fp.g[0].ahead = 0;
@@ -442,6 +464,7 @@ sti_status enqueue_layer_fused(sti_plan* p, int li, const void* xq, const void* 
   fp.qkv = p->qkv; fp.attn_out = p->attn_out; fp.seq_lens = lens;
   fp.n_kept_heads = nh; fp.batch = batch; fp.seq = seq; fp.T = T;
   fp.barrier = p->fused_ctr + li; fp.err = c->err_dev;
+  layer_ranges(p, next_layer, fp.pf_ptr, fp.pf_bytes);
   CUDA_TRY(launch_fused_layer(fp, grid, c->compute, c->pdl));
   c->launches++;
   *done = true;
@@ -452,7 +475,7 @@ sti_status enqueue_layer_fused(sti_plan* p, int li, const void* xq, const void* 
 // `x_ready_bf16`: the bf16 copy of x already sits in p->x_bf16 (written by the previous layer's LayerNorm);
 // `want_next_bf16`: this layer's last kernel also writes y as bf16 into p->x_bf16 for the next layer.
 sti_status enqueue_layer(sti_plan* p, int li, const void* x, void* y, int batch, int seq, const int32_t* lens,
-                         bool x_ready_bf16, bool want_next_bf16) {
+                         bool x_ready_bf16, bool want_next_bf16, int next_layer = -1) {
   sti_ctx* c = p->ctx;
   const sti_model_desc& d = c->desc;
   Layer& L = p->layers[li];
@@ -478,13 +501,13 @@ sti_status enqueue_layer(sti_plan* p, int li, const void* x, void* y, int batch,
       xq = p->x_bf16;
     }
     bool fused = false;
-    st = enqueue_layer_fused(p, li, xq, x, y, batch, seq, lens, want_next_bf16, &fused);
+    st = enqueue_layer_fused(p, li, xq, x, y, batch, seq, lens, want_next_bf16, next_layer, &fused);
     if (st != STI_OK) return st;
     if (fused) {
       for (int i = 1; i <= 7; ++i) CUDA_TRY(mark(i));
       return STI_OK;
     }
-    st = run_gemm(p, GEMM_BF16_TO_BF16, L.qkv, xq, d.hidden, T, p->qkv, 64, dense + c->off_bq);
+    st = run_gemm(p, GEMM_BF16_TO_BF16, L.qkv, xq, d.hidden, T, p->qkv, 64, dense + c->off_bq, next_layer);
     if (st != STI_OK) return st;
     CUDA_TRY(mark(1));
     CUDA_TRY(launch_attention(p->qkv, p->attn_out, nh, batch, seq, lens, c->compute, c->pdl));
@@ -582,7 +605,8 @@ sti_status enqueue_forward(sti_plan* p, const void* x, void* y, int batch, int s
     }
     if (prof) CUDA_TRY(cudaEventRecord(L.ev_comp_start, c->compute));
     void* nxt = (li == n - 1) ? y : p->buf[li & 1];
-    sti_status st = enqueue_layer(p, li, cur, nxt, batch, seq, lens, li > 0, li + 1 < n);
+    // the layer's first GEMM also pulls the next layer's packed shards into L2 (if they are on the device yet)
+    sti_status st = enqueue_layer(p, li, cur, nxt, batch, seq, lens, li > 0, li + 1 < n, li + 1 < n ? li + 1 : -1);
     if (st != STI_OK) return st;
     if (prof) CUDA_TRY(cudaEventRecord(L.ev_done, c->compute));
     if (L.str_bytes > 0) {
@@ -984,13 +1008,16 @@ sti_status sti_plan_finalize(sti_plan* p) {
   p->max_partial = 1;
   for (auto& L : p->layers) {
     TableBuilder tb[4];
+    L.tables_off = align16(host_tables.size());
     build_layer_tables(p, L, tb);
     GemmTable* gt[4] = {&L.qkv, &L.o, &L.f1, &L.f2};
     for (int i = 0; i < 4; ++i) {
+      tb[i].finish();
+      gt[i]->seg_stride = tb[i].seg_stride;
       gt[i]->n_jobs = static_cast<int>(tb[i].jobs.size());
       gt[i]->w_bytes = tb[i].w_bytes;
       gt[i]->n_stages = 2; gt[i]->bps = 1;
-      gt[i]->hdr_bytes = gemm_header_bytes(tb[i].seg_max);
+      gt[i]->hdr_bytes = gemm_header_bytes();
       gt[i]->pair_ok = !tb[i].jobs.empty() && tb[i].jobs.size() % 2 == 0;
       for (size_t j = 0; gt[i]->pair_ok && j < tb[i].jobs.size(); j += 2) {
         const Job &a = tb[i].jobs[j], &b = tb[i].jobs[j + 1];
@@ -1001,7 +1028,7 @@ sti_status sti_plan_finalize(sti_plan* p) {
         return STI_ERR_SHAPE;
       gt[i]->smem = gemm_smem_bytes(tb[i].w_bytes, gt[i]->n_stages, gt[i]->bps, gt[i]->hdr_bytes);
       // the whole-layer kernel keeps both header slots resident: its activation ring starts further up
-      if (tb[i].jobs.empty() || tb[i].seg_max > 16 ||
+      if (tb[i].jobs.empty() || tb[i].seg_stride > 16 ||
           !gemm_pick_ring(tb[i].w_bytes, tb[i].k_max, static_cast<uint32_t>(fused_low_offset()), &gt[i]->f_stages, &gt[i]->f_bps))
         gt[i]->f_stages = gt[i]->f_bps = 0;
       if (gt[i]->smem > kMaxSmem && !tb[i].jobs.empty()) return STI_ERR_SHAPE;
@@ -1014,6 +1041,7 @@ sti_status sti_plan_finalize(sti_plan* p) {
       if (!tb[i].segs.empty()) memcpy(host_tables.data() + fx.segs_off, tb[i].segs.data(), tb[i].segs.size() * sizeof(Seg));
       fixes.push_back(fx);
     }
+    L.tables_bytes = host_tables.size() - L.tables_off;
     p->max_partial = std::max(p->max_partial, std::max(L.o.n_split, L.f2.n_split));
   }
   p->tables_bytes = std::max<size_t>(host_tables.size(), 16);

@@ -9,31 +9,14 @@
 // Attention is ~3 % of a layer's FLOPs at seq 128; the dense projections use tcgen05 (dqgemm.cu).
 #include <cuda_bf16.h>
 
-#include "sti_device.cuh"
+#include "attention_device.cuh"
 #include "sti_kernels.h"
 
 namespace sti {
 namespace {
 
 constexpr int kHeadDim = 64;
-constexpr int kKStride = kHeadDim + 8;   // bf16 elements per K row in shared memory (conflict-free fragment reads)
-
-__device__ __forceinline__ void mma_bf16_16816(float (&c)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
-  asm volatile(
-      "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
-      : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
-      : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
-}
-
-__device__ __forceinline__ void cp_async16(uint32_t dst, const void* src, uint32_t src_bytes) {
-  asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "r"(src_bytes) : "memory");
-}
-
-// Two 8x8 bf16 matrices, transposed on the way in: with rows = keys this yields the B fragment
-// (k = key, n = head-dim column) of m16n8k16.  Lanes 0-7 / 8-15 give the row addresses.
-__device__ __forceinline__ void ldmatrix_x2_trans(uint32_t addr, uint32_t& r0, uint32_t& r1) {
-  asm volatile("ldmatrix.sync.aligned.m8n8.x2.trans.shared.b16 {%0, %1}, [%2];" : "=r"(r0), "=r"(r1) : "r"(addr));
-}
+constexpr int kKStride = kAttnKStride;
 
 template <int WARPS>      // 16 query rows per warp; K and V of the sequence are shared by the CTA's warps
 __global__ void __launch_bounds__(32 * WARPS)
@@ -181,6 +164,21 @@ attention_kernel(const uint16_t* __restrict__ qkv, uint16_t* __restrict__ out, i
   }
 }
 
+// Few tokens: one CTA of 16 warps per (64-query tile, kept head, sequence), keys split four ways inside the
+// CTA - a quarter of the serial key loop of the kernel above, at the price of one merge through shared memory.
+__global__ void __launch_bounds__(kAttnThreads)
+attention_split_kernel(AttnArgs p) {
+  extern __shared__ __align__(16) uint8_t smem[];
+  pdl_launch_dependents();
+  pdl_wait();          // q, k, v (and possibly seq_lens) come from the preceding kernels
+  attention_step(p, blockIdx.x, gridDim.x, smem, threadIdx.x);
+}
+
+size_t attn_split_smem_bytes(int L) {
+  const int Lpad = (L + 63) / 64 * 64;
+  return static_cast<size_t>(Lpad) * kAttnKStride * 2 * 2 + kAttnMergeBytes;
+}
+
 size_t attn_smem_bytes(int L) {
   const int Lpad = (L + 63) / 64 * 64;
   return static_cast<size_t>(Lpad) * kKStride * 2 * 2;      // K and V, padded rows
@@ -192,8 +190,11 @@ cudaError_t attention_configure() {
   cudaError_t e = cudaFuncSetAttribute(attention_kernel<4>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                        static_cast<int>(attn_smem_bytes(512)));
   if (e != cudaSuccess) return e;
-  return cudaFuncSetAttribute(attention_kernel<8>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                              static_cast<int>(attn_smem_bytes(512)));
+  e = cudaFuncSetAttribute(attention_kernel<8>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                           static_cast<int>(attn_smem_bytes(512)));
+  if (e != cudaSuccess) return e;
+  return cudaFuncSetAttribute(attention_split_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                              static_cast<int>(attn_split_smem_bytes(512)));
 }
 
 cudaError_t launch_attention(const uint16_t* qkv, uint16_t* out, int n_kept, int batch, int seq,
@@ -205,6 +206,12 @@ cudaError_t launch_attention(const uint16_t* qkv, uint16_t* out, int n_kept, int
     dim3 grid((seq + 127) / 128, n_kept, batch);
     return launch_kernel(attention_kernel<8>, grid, dim3(256), attn_smem_bytes(seq), s, pdl, qkv, out, n_kept, batch,
                          seq, seq_lens);
+  }
+  const long items = static_cast<long>((seq + 63) / 64) * n_kept * batch;
+  if (items <= 2 * 148 && seq > 64) {          // too few CTAs to fill the GPU: shorten each CTA's key loop instead
+    AttnArgs a{qkv, out, seq_lens, n_kept, batch, seq, batch * seq};
+    return launch_kernel(attention_split_kernel, dim3(static_cast<unsigned>(items)), dim3(kAttnThreads),
+                         attn_split_smem_bytes(seq), s, pdl, a);
   }
   dim3 grid((seq + 63) / 64, n_kept, batch);
   return launch_kernel(attention_kernel<4>, grid, dim3(128), attn_smem_bytes(seq), s, pdl, qkv, out, n_kept, batch, seq,

@@ -32,16 +32,17 @@ __global__ void __launch_bounds__(kThreads, 1)
 dqgemm_kernel(const __grid_constant__ CUtensorMap xmap, const Job* __restrict__ jobs, const Seg* __restrict__ segs,
               const __nv_bfloat16* __restrict__ x, int ldx, int T, OutT* __restrict__ out, int ldo,
               const float* __restrict__ bias, int* __restrict__ err, uint32_t n_stages, uint32_t bps,
-              uint32_t w_bytes, uint32_t hdr_bytes) {
-  extern __shared__ uint8_t smem_raw[];
-  uint8_t* smem = smem_raw + ((1024u - (smem_addr(smem_raw) & 1023u)) & 1023u);
+              uint32_t w_bytes, uint32_t hdr_bytes, uint32_t seg_stride, PrefetchRanges pf) {
+  extern __shared__ __align__(1024) uint8_t smem_raw[];
+  uint8_t* smem = smem_raw;
   const uint32_t tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const Job job = jobs[blockIdx.x];
+  const Seg* my_segs = segs + static_cast<size_t>(blockIdx.x) * seg_stride;     // independent of the job load
   const uint32_t n_rows = job.n_rows, k_total = job.k_total;
 
   SmemHeader* hdr = reinterpret_cast<SmemHeader*>(smem);
   float* bias_sm = reinterpret_cast<float*>(smem + 256);                            // [n_rows <= 128]
-  uint16_t* tables = reinterpret_cast<uint16_t*>(smem + 768);                       // [n_seg][64]
+  uint16_t* tables = reinterpret_cast<uint16_t*>(smem + 768);                       // [warp][64]
   uint8_t* xsm = smem + hdr_bytes;                                                   // stages, 1024-aligned
   const uint32_t stage_bytes = bps * kBoxBytes;          // bps boxes of 64 columns per stage
   uint8_t* wsm = xsm + n_stages * stage_bytes;
@@ -50,7 +51,8 @@ dqgemm_kernel(const __grid_constant__ CUtensorMap xmap, const Job* __restrict__ 
   const bool bad = job.n_seg == 0 || job.n_seg > kMaxSegs || (n_rows != 32 && n_rows != 64 && n_rows != 128) ||
                    (k_total % kChunkK) != 0 || k_total == 0 || n_rows * k_total * 2 > w_bytes ||
                    n_stages < 2 || n_stages > kMaxStages || (bps != 1 && bps != 2 && bps != 4) ||
-                   768 + job.n_seg * kTableStride * 2 > hdr_bytes || (hdr_bytes & 1023) != 0;
+                   768 + kWarps * kTableStride * 2 > hdr_bytes || (hdr_bytes & 1023) != 0 ||
+                   (smem_addr(smem_raw) & 1023u) != 0 || job.seg_begin != blockIdx.x * seg_stride || job.n_seg > seg_stride;
   if (bad) {
     if (tid == 0) atomicCAS(err, ERR_NONE, ERR_BAD_JOB);
     return;
@@ -107,7 +109,6 @@ dqgemm_kernel(const __grid_constant__ CUtensorMap xmap, const Job* __restrict__ 
       tmem_relinquish();
     }
   }
-  load_tables(job, segs, tables, tid);
   if (tid < n_rows) bias_sm[tid] = job.bias_off >= 0 ? __ldg(bias + job.bias_off + tid) : 0.f;
   tc_fence_before_sync();
   __syncthreads();
@@ -118,7 +119,7 @@ dqgemm_kernel(const __grid_constant__ CUtensorMap xmap, const Job* __restrict__ 
   // can never starve it of columns.
   pdl_launch_dependents();
 
-  decode_weight_tile(job, segs, tables, wsm, tid);
+  decode_weight_tile(job, my_segs, tables, wsm, tid);
   // Everything above read only weights, descriptors and parameters.  The activations are the previous
   // kernel's output: from here on this kernel depends on it.
   pdl_wait();
@@ -228,6 +229,10 @@ dqgemm_kernel(const __grid_constant__ CUtensorMap xmap, const Job* __restrict__ 
         __syncwarp();
         (void)mbar_wait_bounded(smem_addr(&hdr->drain), 0);
       }
+    } else if (warp == 2 || warp == 3) {
+      // ---- otherwise idle: pull the packed shards of a later launch into L2
+      const uint32_t n_cta = gridDim.x * gridDim.y, me = (blockIdx.y * gridDim.x + blockIdx.x) * 64 + (tid - 64);
+      for (int r = 0; r < 4; ++r) prefetch_range_l2(pf.ptr[r], pf.bytes[r], me, n_cta * 64);
     } else if (warp >= kEpilogueWarp0 && warp < kEpilogueWarp0 + kEpilogueWarps) {
       // ---- epilogue: warp w owns TMEM lanes 32*(w%4).. (token rows) and one half of the columns
       const uint32_t q = warp & 3, half = (warp - kEpilogueWarp0) >> 2, ncol = n_rows / 2;
@@ -364,9 +369,9 @@ template <typename OutT, bool GELU>
 __global__ void __launch_bounds__(kThreads, 1)
 dqgemm_pair_kernel(const __grid_constant__ CUtensorMap xmap, const Job* __restrict__ jobs, const Seg* __restrict__ segs,
                    int T, OutT* __restrict__ out, int ldo, const float* __restrict__ bias, int* __restrict__ err,
-                   uint32_t n_stages, uint32_t bps, uint32_t w_bytes, uint32_t hdr_bytes) {
-  extern __shared__ uint8_t smem_raw[];
-  uint8_t* smem = smem_raw + ((1024u - (smem_addr(smem_raw) & 1023u)) & 1023u);
+                   uint32_t n_stages, uint32_t bps, uint32_t w_bytes, uint32_t hdr_bytes, uint32_t seg_stride) {
+  extern __shared__ __align__(1024) uint8_t smem_raw[];
+  uint8_t* smem = smem_raw;
   const uint32_t tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const uint32_t rank = cluster_ctarank();                 // 0 issues the MMAs
   const uint32_t pair_base = blockIdx.x & ~1u;
@@ -376,7 +381,8 @@ dqgemm_pair_kernel(const __grid_constant__ CUtensorMap xmap, const Job* __restri
 
   SmemHeader* hdr = reinterpret_cast<SmemHeader*>(smem);
   float* bias_sm = reinterpret_cast<float*>(smem + 256);            // [128]
-  uint16_t* tables = reinterpret_cast<uint16_t*>(smem + 768);       // [n_seg][64]
+  uint16_t* tables = reinterpret_cast<uint16_t*>(smem + 768);       // [warp][64]
+  const Seg* my_segs = segs + static_cast<size_t>(blockIdx.x) * seg_stride;
   uint8_t* xsm = smem + hdr_bytes;
   const uint32_t stage_bytes = bps * kBoxBytes;
   uint8_t* wsm = xsm + n_stages * stage_bytes;
@@ -386,8 +392,9 @@ dqgemm_pair_kernel(const __grid_constant__ CUtensorMap xmap, const Job* __restri
                    job0.n_seg == 0 || job0.n_seg > kMaxSegs || job1.n_seg == 0 || job1.n_seg > kMaxSegs ||
                    (k_total % kChunkK) != 0 || k_total == 0 || 64 * k_total * 2 > w_bytes || n_stages < 2 ||
                    n_stages > kMaxStages || (bps != 1 && bps != 2 && bps != 4) ||
-                   768 + (job0.n_seg > job1.n_seg ? job0.n_seg : job1.n_seg) * kTableStride * 2 > hdr_bytes ||
-                   (hdr_bytes & 1023) != 0 || (gridDim.x & 1) != 0;
+                   768 + kWarps * kTableStride * 2 > hdr_bytes || (hdr_bytes & 1023) != 0 || (gridDim.x & 1) != 0 ||
+                   (smem_addr(smem_raw) & 1023u) != 0 || job0.n_seg > seg_stride || job1.n_seg > seg_stride ||
+                   job0.seg_begin != pair_base * seg_stride || job1.seg_begin != (pair_base + 1) * seg_stride;
   if (bad) {
     if (tid == 0) atomicCAS(err, ERR_NONE, ERR_BAD_JOB);
     return;
@@ -422,7 +429,6 @@ dqgemm_pair_kernel(const __grid_constant__ CUtensorMap xmap, const Job* __restri
     tmem_alloc_pair(smem_addr(&hdr->tmem_base), kTmemCols);
     tmem_relinquish_pair();
   }
-  load_tables(job, segs, tables, tid);
   if (tid < 128) {
     const Job& jb = tid < 64 ? job0 : job1;
     bias_sm[tid] = jb.bias_off >= 0 ? __ldg(bias + jb.bias_off + (tid & 63)) : 0.f;
@@ -433,7 +439,7 @@ dqgemm_pair_kernel(const __grid_constant__ CUtensorMap xmap, const Job* __restri
   const uint32_t tmem_base = hdr->tmem_base;
   pdl_launch_dependents();          // this CTA owns its tensor memory now (see the one-CTA kernel)
 
-  decode_weight_tile(job, segs, tables, wsm, tid);
+  decode_weight_tile(job, my_segs, tables, wsm, tid);
   cluster_sync_all();               // both halves of the weight tile are in place, all barriers initialised
   pdl_wait();                       // from here on: the previous kernel's output
 
@@ -570,12 +576,14 @@ cudaError_t launch_t(const GemmLaunch& p, cudaStream_t s) {
     cfg.attrs = attr;
     cfg.numAttrs = p.pdl ? 2 : 1;
     return cudaLaunchKernelEx(&cfg, dqgemm_pair_kernel<OutT, GELU>, p.xmap, p.jobs, p.segs, p.T, static_cast<OutT*>(p.out),
-                              p.ldo, p.bias, p.err, p.n_stages, p.bps, p.w_bytes, p.hdr_bytes);
+                              p.ldo, p.bias, p.err, p.n_stages, p.bps, p.w_bytes, p.hdr_bytes, p.seg_stride);
   }
   dim3 grid(p.n_jobs, p.m_ctas), block(kThreads);
+  PrefetchRanges pf;
+  for (int r = 0; r < 4; ++r) { pf.ptr[r] = p.pf_ptr[r]; pf.bytes[r] = p.pf_bytes[r]; }
   if (p.simt_debug)
-    return launch_kernel(dqgemm_kernel<OutT, GELU, true>, grid, block, p.smem_bytes, s, p.pdl, p.xmap, p.jobs, p.segs, x, p.ldx, p.T, static_cast<OutT*>(p.out), p.ldo, p.bias, p.err, p.n_stages, p.bps, p.w_bytes, p.hdr_bytes);
-  return launch_kernel(dqgemm_kernel<OutT, GELU, false>, grid, block, p.smem_bytes, s, p.pdl, p.xmap, p.jobs, p.segs, x, p.ldx, p.T, static_cast<OutT*>(p.out), p.ldo, p.bias, p.err, p.n_stages, p.bps, p.w_bytes, p.hdr_bytes);
+    return launch_kernel(dqgemm_kernel<OutT, GELU, true>, grid, block, p.smem_bytes, s, p.pdl, p.xmap, p.jobs, p.segs, x, p.ldx, p.T, static_cast<OutT*>(p.out), p.ldo, p.bias, p.err, p.n_stages, p.bps, p.w_bytes, p.hdr_bytes, p.seg_stride, pf);
+  return launch_kernel(dqgemm_kernel<OutT, GELU, false>, grid, block, p.smem_bytes, s, p.pdl, p.xmap, p.jobs, p.segs, x, p.ldx, p.T, static_cast<OutT*>(p.out), p.ldo, p.bias, p.err, p.n_stages, p.bps, p.w_bytes, p.hdr_bytes, p.seg_stride, pf);
 }
 
 template <typename K>
@@ -587,16 +595,16 @@ cudaError_t set_smem(K kernel) {
 
 size_t gemm_weight_bytes(uint32_t n_rows, uint32_t k_total) { return static_cast<size_t>(n_rows) * k_total * 2; }
 
-uint32_t gemm_header_bytes(uint32_t max_segs) { return max_segs <= 1 ? kHeaderSmall : kHeaderLarge; }
+uint32_t gemm_header_bytes() { return kHeaderBytes; }
 
 size_t gemm_smem_bytes(uint32_t w_bytes, uint32_t n_stages, uint32_t bps, uint32_t hdr_bytes) {
-  return kAlignSlack + hdr_bytes + static_cast<size_t>(w_bytes) + static_cast<size_t>(n_stages) * bps * kBoxBytes;
+  return hdr_bytes + static_cast<size_t>(w_bytes) + static_cast<size_t>(n_stages) * bps * kBoxBytes;
 }
 
 // Ring shape for a weight tile of `w_bytes` and a K range of `k_total`: boxes per stage and stages.
 // Fewer, larger stages mean fewer waits for the MMA-issuing warp; at least ~64 KB stay in flight.
 bool gemm_pick_ring(uint32_t w_bytes, uint32_t k_total, uint32_t hdr_bytes, uint32_t* n_stages, uint32_t* bps) {
-  const long room = 227L * 1024 - kAlignSlack - static_cast<long>(hdr_bytes) - static_cast<long>(w_bytes);
+  const long room = 227L * 1024 - static_cast<long>(hdr_bytes) - static_cast<long>(w_bytes);
   if (room < 3L * kBoxBytes) return false;           // the tile does not fit
   const uint32_t n_boxes = k_total / kChunkK;
   if (n_boxes <= 8 && room >= 2L * 4 * kBoxBytes) { *bps = 4; *n_stages = 2; return true; }   // a tile's K in <= 2 stages

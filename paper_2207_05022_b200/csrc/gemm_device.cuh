@@ -17,10 +17,8 @@ constexpr int kTileM = 128;                 // tokens per MMA tile
 constexpr int kChunkK = 64;                 // one TMA box = 64 columns = one 128-byte swizzle row; a stage holds 1, 2 or 4 boxes
 constexpr int kMaxStages = 8;
 constexpr int kBoxBytes = kTileM * kChunkK * 2;     // 16 KB
-// header = barriers (256 B) + bias (512 B) + one 128-byte table per segment; stages start 1024-aligned after it
-constexpr int kHeaderSmall = 1024;          // single-segment tiles (QKV, FFN1)
-constexpr int kHeaderLarge = 3072;          // up to 16 segments (O projection, FFN2)
-constexpr int kAlignSlack = 1024;           // the dynamic shared-memory base is aligned up to 1024 by hand
+// header = barriers (256 B) + bias (512 B) + one 128-byte centroid table per warp; stages start 1024-aligned after it
+constexpr int kHeaderBytes = 3072;
 constexpr int kMaxSegs = 16;
 constexpr int kTableStride = 64;            // bf16 entries per segment table
 constexpr int kEpilogueWarp0 = 4;             // epilogue warps 4..11: two per TMEM lane quadrant
@@ -39,19 +37,33 @@ struct SmemHeader {
 // ---------------------------------------------------------------------------------------
 // Weight-tile decode
 // ---------------------------------------------------------------------------------------
-template <int BITS>
-__device__ __forceinline__ void decode_task(const Seg& sg, const uint16_t* __restrict__ tab, uint8_t* wsm,
-                                            uint32_t n_rows, uint32_t task, uint32_t lane) {
-  // task = (row group, 128-column chunk); the k planes of the group are contiguous.
+// The k index planes of one task = (row group, 128-column chunk), one coalesced 128-bit load per plane.
+// `bits` is only known at run time here, so that the loads can be issued before anything else of the
+// task is ready; planes beyond `bits` are not touched.
+__device__ __forceinline__ void load_planes(const Seg& sg, uint32_t task, uint32_t lane, uint32_t (&w)[24]) {
+  const uint32_t bits = sg.bits;
   const uint32_t chunks = sg.kc >= 128 ? sg.kc / 128 : 1;
   const uint32_t g = task / chunks, j = task % chunks;
-  const uint4* src = sg.codes + (static_cast<size_t>(g) * chunks + j) * (BITS * 32) + lane;
+  const uint4* src = sg.codes + (static_cast<size_t>(g) * chunks + j) * (bits * 32) + lane;
+#pragma unroll
+  for (int p = 0; p < 6; ++p) {
+    if (static_cast<uint32_t>(p) < bits) {
+      const uint4 v = __ldg(src + p * 32);
+      w[4 * p + 0] = v.x; w[4 * p + 1] = v.y; w[4 * p + 2] = v.z; w[4 * p + 3] = v.w;
+    }
+  }
+}
+
+// Index unpack in registers -> bf16 table lookup in shared memory -> 16-byte stores into the K-major
+// core-matrix layout.  Each lane holds 128 consecutive indexes of its own row.
+template <int BITS>
+__device__ __forceinline__ void unpack_task(const uint32_t (&planes)[24], const Seg& sg, const uint16_t* __restrict__ tab,
+                                            uint8_t* wsm, uint32_t n_rows, uint32_t task, uint32_t lane) {
   uint32_t w[4 * BITS];
 #pragma unroll
-  for (int p = 0; p < BITS; ++p) {
-    const uint4 v = __ldg(src + p * 32);
-    w[4 * p + 0] = v.x; w[4 * p + 1] = v.y; w[4 * p + 2] = v.z; w[4 * p + 3] = v.w;
-  }
+  for (int i = 0; i < 4 * BITS; ++i) w[i] = planes[i];
+  const uint32_t chunks = sg.kc >= 128 ? sg.kc / 128 : 1;
+  const uint32_t g = task / chunks, j = task % chunks;
   const bool narrow = sg.kc < 128;     // 64 in-features: the quantum is rows (l, l + 32) of a 64-row group
   const uint32_t row0 = narrow ? g * 64 + lane : g * 32 + lane;
   const uint32_t kcore0 = (sg.koff + (narrow ? 0 : j * 128)) >> 3;
@@ -142,64 +154,100 @@ __device__ __forceinline__ void store_row16(OutT* dst, const float (&v)[16]) {
   }
 }
 
-// ---------------------------------------------------------------------------------------
-// Pieces shared by the one-CTA and the two-CTA kernel
-// ---------------------------------------------------------------------------------------
-// Centroid tables of the job's segments, rounded once to bf16 (round-to-nearest-even), and a head start
-// for the outlier lists, which are needed right after the decode.
-__device__ __forceinline__ void load_tables(const Job& job, const Seg* __restrict__ segs, uint16_t* tables, uint32_t tid) {
-  for (uint32_t i = tid; i < job.n_seg * kTableStride; i += kThreads) {
-    const Seg& sg = segs[job.seg_begin + i / kTableStride];
-    const uint32_t e = i % kTableStride;
-    tables[i] = (sg.bits <= 6 && e < (1u << sg.bits)) ? bf16_bits(__ldg(sg.table + e)) : 0;
+struct PrefetchRanges {
+  const uint8_t* ptr[4];
+  uint32_t bytes[4];
+};
+
+// Pulls [ptr, ptr + bytes) into L2, one 128-byte line per instruction, the range shared out over
+// `n_threads` threads of which this is number `t`.  Packed shards are read once per forward, so without
+// this every decode starts with address translation and DRAM latency on its critical path.
+__device__ __forceinline__ void prefetch_range_l2(const uint8_t* ptr, uint32_t bytes, uint32_t t, uint32_t n_threads) {
+  // plain loads whose values are dropped: unlike a prefetch hint they also bring the translation in
+  uint32_t sink = 0;
+  for (uint32_t off = t * 128u; off < bytes; off += n_threads * 128u) {
+    uint32_t v;
+    asm volatile("ld.global.cg.b32 %0, [%1];" : "=r"(v) : "l"(ptr + off) : "memory");
+    sink |= v;
   }
-  for (uint32_t si = 0; si < job.n_seg; ++si) {
-    const Seg& sg = segs[job.seg_begin + si];
-    for (uint32_t o = tid * 32; o < sg.n_out; o += kThreads * 32) {
-      asm volatile("prefetch.global.L2 [%0];" ::"l"(sg.out_off + o));
-      asm volatile("prefetch.global.L2 [%0];" ::"l"(sg.out_val + o));
-    }
-  }
+  asm volatile("" ::"r"(sink));
 }
 
-// Decode of the job's weight tile into `wsm` (all threads of the CTA; ends with the tile visible to the
-// tensor core: proxy fence + CTA barrier).  Needs the tables in place (a CTA barrier after load_tables).
-__device__ __forceinline__ void decode_weight_tile(const Job& job, const Seg* __restrict__ segs, const uint16_t* tables,
+// ---------------------------------------------------------------------------------------
+// Decode of one job's weight tile (shared by every GEMM kernel)
+// ---------------------------------------------------------------------------------------
+// One outlier (Section 6: outliers keep their original value) into its slot of the decoded tile.
+__device__ __forceinline__ void patch_outlier(const Seg& sg, uint32_t off, float val, uint8_t* wsm, uint32_t n_rows,
+                                              uint32_t k_total) {
+  const uint32_t local = off - sg.flat_base;
+  const uint32_t row = local / sg.kc, kk = sg.koff + local % sg.kc;
+  if (row < n_rows && kk < k_total)
+    reinterpret_cast<uint16_t*>(wsm)[(static_cast<size_t>(kk >> 3) * n_rows + row) * 8 + (kk & 7)] = bf16_bits(val);
+}
+
+// Decodes the job's weight tile into `wsm` (all threads of the CTA; ends with the tile visible to the tensor
+// core: proxy fence + CTA barrier).  `segs` are the job's own segments.  The whole prologue is two memory
+// round trips: the segment descriptors, then - issued together - the index planes, the centroid table and
+// the outliers.  A warp keeps the table of the segment it works on (rounded once to bf16, round-to-nearest-
+// even) in its own 128 bytes of `warp_tables`, so no CTA-wide barrier sits between the loads and the unpack.
+__device__ __forceinline__ void decode_weight_tile(const Job& job, const Seg* __restrict__ segs, uint16_t* warp_tables,
                                                    uint8_t* wsm, uint32_t tid) {
   const uint32_t lane = tid & 31, warp = tid >> 5;
   const uint32_t n_rows = job.n_rows, k_total = job.k_total;
-  const Seg& s0 = segs[job.seg_begin];
+  const Seg& s0 = segs[0];
   const uint32_t rows_per_group = s0.kc >= 128 ? 32 : 64;
   const uint32_t chunks = s0.kc >= 128 ? s0.kc / 128 : 1;
   const uint32_t tasks_per_seg = (n_rows / rows_per_group) * chunks;
   const uint32_t n_tasks = tasks_per_seg * job.n_seg;
+  // outlier number `tid` of the tile (segments in order): fetched now, applied once the tile is written
+  uint32_t o_seg = 0xffffffffu, o_off = 0, n_out_total = 0;
+  float o_val = 0.f;
+  for (uint32_t si = 0; si < job.n_seg; ++si) {
+    const uint32_t n = segs[si].n_out;
+    if (o_seg == 0xffffffffu && tid >= n_out_total && tid - n_out_total < n) {
+      o_seg = si;
+      o_off = __ldg(segs[si].out_off + (tid - n_out_total));
+      o_val = __ldg(segs[si].out_val + (tid - n_out_total));
+    }
+    n_out_total += n;
+  }
+  uint16_t* tab = warp_tables + warp * kTableStride;
   for (uint32_t t = warp; t < n_tasks; t += kWarps) {
     const uint32_t si = t / tasks_per_seg, task = t % tasks_per_seg;
-    const Seg& sg = segs[job.seg_begin + si];
-    const uint16_t* tab = tables + si * kTableStride;
-    switch (sg.bits) {
-      case 2: decode_task<2>(sg, tab, wsm, n_rows, task, lane); break;
-      case 3: decode_task<3>(sg, tab, wsm, n_rows, task, lane); break;
-      case 4: decode_task<4>(sg, tab, wsm, n_rows, task, lane); break;
-      case 5: decode_task<5>(sg, tab, wsm, n_rows, task, lane); break;
-      case 6: decode_task<6>(sg, tab, wsm, n_rows, task, lane); break;
+    const Seg& sg = segs[si];
+    const uint32_t bits = sg.bits;
+    if (bits > 6) continue;            // raw fp32 segments are handled below
+    const uint32_t n_entries = 1u << bits;
+    const float c0 = lane < n_entries ? __ldg(sg.table + lane) : 0.f;
+    const float c1 = lane + 32 < n_entries ? __ldg(sg.table + lane + 32) : 0.f;
+    uint32_t planes[24];
+    load_planes(sg, task, lane, planes);
+    tab[lane] = bf16_bits(c0);
+    tab[lane + 32] = bf16_bits(c1);
+    __syncwarp();
+    switch (bits) {
+      case 2: unpack_task<2>(planes, sg, tab, wsm, n_rows, task, lane); break;
+      case 3: unpack_task<3>(planes, sg, tab, wsm, n_rows, task, lane); break;
+      case 4: unpack_task<4>(planes, sg, tab, wsm, n_rows, task, lane); break;
+      case 5: unpack_task<5>(planes, sg, tab, wsm, n_rows, task, lane); break;
+      case 6: unpack_task<6>(planes, sg, tab, wsm, n_rows, task, lane); break;
       default: break;
     }
+    __syncwarp();                      // the table is overwritten by the warp's next task
   }
   for (uint32_t si = 0; si < job.n_seg; ++si) {
-    const Seg& sg = segs[job.seg_begin + si];
+    const Seg& sg = segs[si];
     if (sg.bits == 32) decode_raw(sg, wsm, n_rows, tid);
   }
   __syncthreads();
-  // outliers keep their original value (Section 6): overwrite their slot
-  for (uint32_t si = 0; si < job.n_seg; ++si) {
-    const Seg& sg = segs[job.seg_begin + si];
-    for (uint32_t o = tid; o < sg.n_out; o += kThreads) {
-      const uint32_t local = __ldg(sg.out_off + o) - sg.flat_base;
-      const uint32_t row = local / sg.kc, kk = sg.koff + local % sg.kc;
-      if (row < n_rows && kk < k_total)
-        reinterpret_cast<uint16_t*>(wsm)[(static_cast<size_t>(kk >> 3) * n_rows + row) * 8 + (kk & 7)] =
-            bf16_bits(__ldg(sg.out_val + o));
+  if (o_seg != 0xffffffffu) patch_outlier(segs[o_seg], o_off, o_val, wsm, n_rows, k_total);
+  if (n_out_total > kThreads) {        // more outliers than threads: the rest, one pass per 512
+    uint32_t base = 0;
+    for (uint32_t si = 0; si < job.n_seg; ++si) {
+      const Seg& sg = segs[si];
+      for (uint32_t o = tid; o < sg.n_out; o += kThreads)
+        if (base + o >= kThreads) patch_outlier(sg, __ldg(sg.out_off + o), __ldg(sg.out_val + o), wsm, n_rows, k_total);
+      base += sg.n_out;
     }
   }
   fence_proxy_async_smem();

@@ -13,7 +13,7 @@
 //
 // Shared memory map (offsets from the 1024-aligned base):
 //   [0, 256)      mbarriers, TMEM base, abort flag          [256, 512)  LayerNorm reduction scratch
-//   [512, 3072)   header slot 0: bias (512 B) + 16 segment tables (128 B each)
+//   [512, 3072)   header slot 0: bias (512 B) + one 128-byte centroid table per warp
 //   [3072, 5632)  header slot 1 (consecutive GEMM steps alternate, so a tile can be decoded ahead)
 //   [6144, ...)   activation ring of the running GEMM step / K, V and merge buffers of attention
 //   [..., top)    weight tile of the running or the next GEMM step, placed at the top end
@@ -22,6 +22,7 @@
 #include <cuda.h>
 #include <cuda_bf16.h>
 
+#include "attention_device.cuh"
 #include "gemm_device.cuh"
 
 namespace sti {
@@ -29,10 +30,8 @@ namespace {
 
 constexpr uint32_t kSlotOff0 = 512, kSlotBytes = 2560, kSlotOff1 = kSlotOff0 + kSlotBytes;
 constexpr uint32_t kLowOff = 6144;                       // 1024-aligned start of the activation area
-constexpr uint32_t kFusedTotal = 226 * 1024;             // usable bytes after the alignment slack
+constexpr uint32_t kFusedTotal = 227 * 1024;             // dynamic shared memory of the kernel
 constexpr uint32_t kFusedTmemCols = 256;                 // two accumulators of up to 128 columns
-constexpr int kAttnKStride = 64 + 8;                     // bf16 per K / V row in shared memory
-constexpr uint32_t kAttnMergeBytes = 3 * 4 * 32 * 36 * 4;   // three key-split partners x four query groups
 
 struct FusedScratch {                // lives at offset 256
   float red[2][16];                  // LayerNorm: per row group, one partial per warp
@@ -82,9 +81,11 @@ __device__ __forceinline__ void gemm_prologue(const FusedGemm& g, int gi, uint32
   FusedScratch* sc = reinterpret_cast<FusedScratch*>(smem + 256);
   const uint32_t n_items = static_cast<uint32_t>(g.n_jobs) * static_cast<uint32_t>(g.m_ctas);
   if (cta >= n_items) return;                            // uniform over the CTA
-  const Job job = g.jobs[cta % static_cast<uint32_t>(g.n_jobs)];
+  const uint32_t job_i = cta % static_cast<uint32_t>(g.n_jobs);
+  const Job job = g.jobs[job_i];
+  const Seg* my_segs = g.segs + static_cast<size_t>(job_i) * g.seg_stride;      // independent of the job load
   const uint32_t n_rows = job.n_rows, k_total = job.k_total;
-  const bool bad = job.n_seg == 0 || job.n_seg > kMaxSegs || (n_rows != 32 && n_rows != 64 && n_rows != 128) ||
+  const bool bad = job.seg_begin != job_i * g.seg_stride || job.n_seg > g.seg_stride || job.n_seg == 0 || job.n_seg > kMaxSegs || (n_rows != 32 && n_rows != 64 && n_rows != 128) ||
                    (k_total % kChunkK) != 0 || k_total == 0 || n_rows * k_total * 2 > g.w_bytes ||
                    g.n_stages < 2 || g.n_stages > kMaxStages || (g.bps != 1 && g.bps != 2 && g.bps != 4) ||
                    kLowOff + g.n_stages * g.bps * kBoxBytes + g.w_bytes > kFusedTotal;
@@ -95,10 +96,8 @@ __device__ __forceinline__ void gemm_prologue(const FusedGemm& g, int gi, uint32
   }
   float* bias_sm = reinterpret_cast<float*>(smem + slot_off);
   uint16_t* tables = reinterpret_cast<uint16_t*>(smem + slot_off + 512);
-  load_tables(job, g.segs, tables, tid);
   if (tid < n_rows) bias_sm[tid] = job.bias_off >= 0 ? __ldg(g.bias + job.bias_off + tid) : 0.f;
-  __syncthreads();
-  decode_weight_tile(job, g.segs, tables, smem + kFusedTotal - g.w_bytes, tid);
+  decode_weight_tile(job, my_segs, tables, smem + kFusedTotal - g.w_bytes, tid);
 }
 
 // ---------------------------------------------------------------------------------------
@@ -125,7 +124,7 @@ __device__ __forceinline__ void drain_tile(uint32_t taddr, uint32_t col0, uint32
 
 // Returns false when a bounded wait ran out.
 __device__ __forceinline__ bool gemm_main(const FusedGemm& g, int gi, uint32_t cta, int T, uint8_t* smem, uint32_t slot_off,
-                                          uint32_t tmem_base, uint32_t tid) {
+                                          uint32_t tmem_base, uint32_t tid, const FusedLayerParams* pf = nullptr) {
   SmemHeader* hdr = reinterpret_cast<SmemHeader*>(smem);
   FusedScratch* sc = reinterpret_cast<FusedScratch*>(smem + 256);
   const uint32_t lane = tid & 31, warp = tid >> 5;
@@ -245,6 +244,9 @@ __device__ __forceinline__ bool gemm_main(const FusedGemm& g, int gi, uint32_t c
       __syncwarp();
       (void)mbar_wait_bounded(smem_addr(&hdr->drain), 0);
     }
+  } else if ((warp == 2 || warp == 3) && pf != nullptr) {
+    // ---- otherwise idle: pull the next layer's packed shards into L2
+    for (int r = 0; r < 4; ++r) prefetch_range_l2(pf->pf_ptr[r], pf->pf_bytes[r], cta * 64 + (tid - 64), n_items * 64);
   } else if (warp >= kEpilogueWarp0 && warp < kEpilogueWarp0 + kEpilogueWarps) {
     // ---- epilogue: warp w owns TMEM lanes 32*(w%4).. (token rows) and one half of the columns
     const uint32_t q = warp & 3, half = (warp - kEpilogueWarp0) >> 2, ncol = n_rows / 2;
@@ -291,196 +293,6 @@ __device__ __forceinline__ bool gemm_main(const FusedGemm& g, int gi, uint32_t c
     mbar_inval(smem_addr(&hdr->drain));
   }
   return hdr->abort == 0;
-}
-
-// ---------------------------------------------------------------------------------------
-// Attention step (Section 2.1; kept heads only).  Work item = (64-query tile, kept head, sequence).
-// The CTA's 16 warps form 4 query groups (16 rows each) x 4 key splits: warp (qg, ks) walks the 64-key
-// blocks kb = ks, ks + 4, ... with mma.sync m16n8k16 and an online softmax in registers; the four
-// partial (max, sum, output) triples of a query group are merged through shared memory.
-// ---------------------------------------------------------------------------------------
-__device__ __forceinline__ void mma_bf16_16816(float (&c)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
-  asm volatile(
-      "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
-      : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
-      : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
-}
-__device__ __forceinline__ void cp_async16(uint32_t dst, const void* src, uint32_t src_bytes) {
-  asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "r"(src_bytes) : "memory");
-}
-__device__ __forceinline__ void ldmatrix_x2_trans(uint32_t addr, uint32_t& r0, uint32_t& r1) {
-  asm volatile("ldmatrix.sync.aligned.m8n8.x2.trans.shared.b16 {%0, %1}, [%2];" : "=r"(r0), "=r"(r1) : "r"(addr));
-}
-
-__device__ __forceinline__ void attention_step(const FusedLayerParams& p, uint32_t cta, uint32_t n_ctas, uint8_t* smem,
-                                               uint32_t tid) {
-  const int L = p.seq, T = p.T, n_kept = p.n_kept_heads;
-  const int lane = tid & 31, warp = tid >> 5;
-  const int g = lane >> 2, t4 = lane & 3;
-  const int qg = warp & 3, ks = warp >> 2;
-  const int Lpad = (L + 63) / 64 * 64;
-  const int q_tiles = (L + 63) / 64;
-  const int n_items = q_tiles * n_kept * p.batch;
-  uint16_t* Ks = reinterpret_cast<uint16_t*>(smem + kLowOff);
-  uint16_t* Vs = Ks + static_cast<size_t>(Lpad) * kAttnKStride;
-  float* merge = reinterpret_cast<float*>(Vs + static_cast<size_t>(Lpad) * kAttnKStride);   // [3][4][36][32]
-  const uint32_t ks_addr = smem_addr(Ks), vs_addr = smem_addr(Vs);
-  const float scale_log2 = 0.125f * 1.4426950408889634f;     // 1/sqrt(64) * log2(e)
-
-  for (int item = cta; item < n_items; item += n_ctas) {
-    const int qt = item % q_tiles, hi = (item / q_tiles) % n_kept, b = item / (q_tiles * n_kept);
-    const uint16_t* Qg = p.qkv + (static_cast<size_t>(hi * 3 + 0) * T + static_cast<size_t>(b) * L) * 64;
-    const uint16_t* Kg = p.qkv + (static_cast<size_t>(hi * 3 + 1) * T + static_cast<size_t>(b) * L) * 64;
-    const uint16_t* Vg = p.qkv + (static_cast<size_t>(hi * 3 + 2) * T + static_cast<size_t>(b) * L) * 64;
-    int valid = L;
-    if (p.seq_lens != nullptr) {
-      valid = p.seq_lens[b];
-      valid = valid < 0 ? 0 : (valid > L ? L : valid);
-    }
-    for (int idx = tid; idx < Lpad * 8; idx += kThreads) {
-      const int key = idx >> 3, piece = idx & 7;
-      const bool ok = key < L;
-      const size_t goff = static_cast<size_t>(ok ? key : 0) * 64 + piece * 8;
-      const uint32_t soff = static_cast<uint32_t>(key * kAttnKStride + piece * 8) * 2;
-      cp_async16(ks_addr + soff, Kg + goff, ok ? 16u : 0u);
-      cp_async16(vs_addr + soff, Vg + goff, ok ? 16u : 0u);
-    }
-    asm volatile("cp.async.commit_group;" ::: "memory");
-
-    const int q0 = qt * 64 + qg * 16;
-    uint32_t qa[4][4];
-#pragma unroll
-    for (int kk = 0; kk < 4; ++kk) {
-      const int r0 = q0 + g, r1 = q0 + g + 8;
-      const int c = kk * 16 + 2 * t4;
-      qa[kk][0] = r0 < L ? *reinterpret_cast<const uint32_t*>(Qg + static_cast<size_t>(r0) * 64 + c) : 0u;
-      qa[kk][1] = r1 < L ? *reinterpret_cast<const uint32_t*>(Qg + static_cast<size_t>(r1) * 64 + c) : 0u;
-      qa[kk][2] = r0 < L ? *reinterpret_cast<const uint32_t*>(Qg + static_cast<size_t>(r0) * 64 + c + 8) : 0u;
-      qa[kk][3] = r1 < L ? *reinterpret_cast<const uint32_t*>(Qg + static_cast<size_t>(r1) * 64 + c + 8) : 0u;
-    }
-    asm volatile("cp.async.wait_group 0;" ::: "memory");
-    __syncthreads();
-
-    float o[8][4];
-#pragma unroll
-    for (int j = 0; j < 8; ++j) { o[j][0] = o[j][1] = o[j][2] = o[j][3] = 0.f; }
-    float m_run[2] = {-INFINITY, -INFINITY};
-    float l_run[2] = {0.f, 0.f};
-    const int n_kblocks = (valid + 63) / 64;
-    for (int kb = ks; kb < n_kblocks; kb += 4) {
-      float s[8][4];
-#pragma unroll
-      for (int j = 0; j < 8; ++j) { s[j][0] = s[j][1] = s[j][2] = s[j][3] = 0.f; }
-#pragma unroll
-      for (int j = 0; j < 8; ++j) {
-        const uint16_t* krow = Ks + static_cast<size_t>(kb * 64 + j * 8 + g) * kAttnKStride + 2 * t4;
-#pragma unroll
-        for (int kk = 0; kk < 4; ++kk) {
-          const uint32_t b0 = *reinterpret_cast<const uint32_t*>(krow + kk * 16);
-          const uint32_t b1 = *reinterpret_cast<const uint32_t*>(krow + kk * 16 + 8);
-          mma_bf16_16816(s[j], qa[kk], b0, b1);
-        }
-      }
-      float mblk[2] = {-INFINITY, -INFINITY};
-#pragma unroll
-      for (int j = 0; j < 8; ++j) {
-        const int key = kb * 64 + j * 8 + 2 * t4;
-#pragma unroll
-        for (int c = 0; c < 4; ++c) {
-          const float v = (key + (c & 1) < valid) ? s[j][c] * scale_log2 : -INFINITY;
-          s[j][c] = v;
-          mblk[c >> 1] = fmaxf(mblk[c >> 1], v);
-        }
-      }
-      float alpha[2], m_use[2];
-#pragma unroll
-      for (int r = 0; r < 2; ++r) {
-        mblk[r] = fmaxf(mblk[r], __shfl_xor_sync(0xffffffffu, mblk[r], 1));
-        mblk[r] = fmaxf(mblk[r], __shfl_xor_sync(0xffffffffu, mblk[r], 2));
-        const float m_new = fmaxf(m_run[r], mblk[r]);
-        m_use[r] = (m_new == -INFINITY) ? 0.f : m_new;
-        alpha[r] = exp2f(m_run[r] - m_use[r]);
-        m_run[r] = m_new;
-        l_run[r] *= alpha[r];
-      }
-#pragma unroll
-      for (int j = 0; j < 8; ++j) {
-#pragma unroll
-        for (int c = 0; c < 4; ++c) {
-          const float pr = exp2f(s[j][c] - m_use[c >> 1]);
-          s[j][c] = pr;
-          l_run[c >> 1] += pr;
-          o[j][c] *= alpha[c >> 1];
-        }
-      }
-#pragma unroll
-      for (int kk = 0; kk < 4; ++kk) {
-        uint32_t pa[4];
-        pa[0] = pack_bf16x2(s[2 * kk][0], s[2 * kk][1]);
-        pa[1] = pack_bf16x2(s[2 * kk][2], s[2 * kk][3]);
-        pa[2] = pack_bf16x2(s[2 * kk + 1][0], s[2 * kk + 1][1]);
-        pa[3] = pack_bf16x2(s[2 * kk + 1][2], s[2 * kk + 1][3]);
-        const uint32_t vrow = vs_addr + static_cast<uint32_t>((kb * 64 + kk * 16 + (lane & 15)) * kAttnKStride) * 2;
-#pragma unroll
-        for (int jd = 0; jd < 8; ++jd) {
-          uint32_t b0, b1;
-          ldmatrix_x2_trans(vrow + jd * 16, b0, b1);
-          mma_bf16_16816(o[jd], pa, b0, b1);
-        }
-      }
-    }
-    // the four lanes of a row hold disjoint keys: complete the row sums before merging
-#pragma unroll
-    for (int r = 0; r < 2; ++r) {
-      l_run[r] += __shfl_xor_sync(0xffffffffu, l_run[r], 1);
-      l_run[r] += __shfl_xor_sync(0xffffffffu, l_run[r], 2);
-    }
-    // key splits 1..3 hand their partial result to split 0 of the same query group
-    if (ks > 0) {
-      float* dst = merge + (static_cast<size_t>(ks - 1) * 4 + qg) * 36 * 32 + lane;
-      dst[0 * 32] = m_run[0]; dst[1 * 32] = m_run[1]; dst[2 * 32] = l_run[0]; dst[3 * 32] = l_run[1];
-#pragma unroll
-      for (int j = 0; j < 8; ++j)
-#pragma unroll
-        for (int c = 0; c < 4; ++c) dst[(4 + j * 4 + c) * 32] = o[j][c];
-    }
-    __syncthreads();
-    if (ks == 0) {
-#pragma unroll 1
-      for (int part = 0; part < 3; ++part) {
-        const float* src = merge + (static_cast<size_t>(part) * 4 + qg) * 36 * 32 + lane;
-        float f_old[2], f_new[2];
-#pragma unroll
-        for (int r = 0; r < 2; ++r) {
-          const float m_o = src[r * 32], l_o = src[(2 + r) * 32];
-          const float m_new = fmaxf(m_run[r], m_o);
-          const float m_use = (m_new == -INFINITY) ? 0.f : m_new;
-          f_old[r] = exp2f(m_run[r] - m_use);
-          f_new[r] = exp2f(m_o - m_use);
-          l_run[r] = l_run[r] * f_old[r] + l_o * f_new[r];
-          m_run[r] = m_new;
-        }
-#pragma unroll
-        for (int j = 0; j < 8; ++j)
-#pragma unroll
-          for (int c = 0; c < 4; ++c)
-            o[j][c] = o[j][c] * f_old[c >> 1] + src[(4 + j * 4 + c) * 32] * f_new[c >> 1];
-      }
-      const int ldo = n_kept * 64;
-#pragma unroll
-      for (int r = 0; r < 2; ++r) {
-        const float inv = l_run[r] > 0.f ? 1.f / l_run[r] : 0.f;
-        const int row = q0 + g + 8 * r;
-        if (row < L) {
-          uint16_t* dst = p.attn_out + (static_cast<size_t>(b) * L + row) * ldo + hi * 64 + 2 * t4;
-#pragma unroll
-          for (int jd = 0; jd < 8; ++jd)
-            *reinterpret_cast<uint32_t*>(dst + jd * 8) = pack_bf16x2(o[jd][2 * r] * inv, o[jd][2 * r + 1] * inv);
-        }
-      }
-    }
-    __syncthreads();        // K, V and the merge buffer are reused by the CTA's next item
-  }
 }
 
 // ---------------------------------------------------------------------------------------
@@ -556,10 +368,14 @@ __device__ __forceinline__ void layernorm_step(const LnLaunch& p, uint32_t cta, 
 // ---------------------------------------------------------------------------------------
 __global__ void __launch_bounds__(kThreads, 1)
 fused_layer_kernel(const __grid_constant__ FusedLayerParams p) {
-  extern __shared__ uint8_t smem_raw[];
-  uint8_t* smem = smem_raw + ((1024u - (smem_addr(smem_raw) & 1023u)) & 1023u);
+  extern __shared__ __align__(1024) uint8_t smem_raw[];
+  uint8_t* smem = smem_raw;
   const uint32_t tid = threadIdx.x, warp = tid >> 5;
   const uint32_t cta = blockIdx.x, G = gridDim.x;
+  if ((smem_addr(smem_raw) & 1023u) != 0) {            // the swizzled TMA stages need this alignment
+    if (tid == 0) atomicCAS(p.err, ERR_NONE, ERR_BAD_JOB);
+    return;
+  }
   SmemHeader* hdr = reinterpret_cast<SmemHeader*>(smem);
   FusedScratch* sc = reinterpret_cast<FusedScratch*>(smem + 256);
   if (tid == 0) { hdr->abort = 0; sc->where = 0; }
@@ -586,9 +402,12 @@ fused_layer_kernel(const __grid_constant__ FusedLayerParams p) {
 
   gemm_prologue(p.g[0], 0, cta, smem, kSlotOff0, p.err, tid);
   pdl_wait();                       // from here on: the previous kernel's output (the layer input)
-  alive = gemm_main(p.g[0], 0, cta, p.T, smem, kSlotOff0, tmem_base, tid);
+  alive = gemm_main(p.g[0], 0, cta, p.T, smem, kSlotOff0, tmem_base, tid, &p);
   barrier(1, kSlotOff1);
-  if (alive) attention_step(p, cta, G, smem, tid);
+  if (alive) {
+    AttnArgs aa{p.qkv, p.attn_out, p.seq_lens, p.n_kept_heads, p.batch, p.seq, p.T};
+    attention_step(aa, cta, G, smem + kLowOff, tid);
+  }
   barrier(-1, 0);
   if (alive) {
     if (!p.g[1].ahead) gemm_prologue(p.g[1], 1, cta, smem, kSlotOff1, p.err, tid);
@@ -622,7 +441,7 @@ size_t fused_attention_bytes(int seq) {
   const int Lpad = (seq + 63) / 64 * 64;
   return static_cast<size_t>(Lpad) * kAttnKStride * 2 * 2 + kAttnMergeBytes;
 }
-size_t fused_smem_total() { return kFusedTotal + kAlignSlack; }
+size_t fused_smem_total() { return kFusedTotal; }
 size_t fused_low_offset() { return kLowOff; }
 
 cudaError_t fused_configure() {

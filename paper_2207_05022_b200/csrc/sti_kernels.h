@@ -59,14 +59,17 @@ struct GemmLaunch {
   uint32_t n_stages;        // stages in the activation ring
   uint32_t bps;             // 16 KB boxes (64 columns) per stage: 1, 2 or 4
   uint32_t w_bytes;         // shared memory reserved for the weight tile (largest job)
-  uint32_t hdr_bytes;       // barriers + bias + per-segment tables: 1024 (one segment per tile) or 3072
+  uint32_t hdr_bytes;       // barriers + bias + per-warp centroid tables
+  uint32_t seg_stride;      // the segments of job j start at segs[j * seg_stride]
+  const uint8_t* pf_ptr[4]; // what the next layer reads first (packed shards, tile descriptors, dense parameters):
+  uint32_t pf_bytes[4];     // pulled into L2 by this launch's idle warps
   bool simt_debug;          // compute the products on the plain ALUs instead of the tensor cores
   bool pdl;                 // launch with programmatic dependent launch
   bool pair;                // two-CTA clusters (cta_group::2): jobs 2i and 2i+1 share one M=256 x N=128 MMA
 };
 
 size_t gemm_weight_bytes(uint32_t n_rows, uint32_t k_total);
-uint32_t gemm_header_bytes(uint32_t max_segs);
+uint32_t gemm_header_bytes();
 bool gemm_pick_ring(uint32_t w_bytes, uint32_t k_total, uint32_t hdr_bytes, uint32_t* n_stages, uint32_t* bps);   // false: does not fit
 size_t gemm_smem_bytes(uint32_t w_bytes, uint32_t n_stages, uint32_t bps, uint32_t hdr_bytes);
 cudaError_t gemm_configure();   // opt in to large dynamic shared memory (once per device)
@@ -122,7 +125,7 @@ cudaError_t launch_decode(const DecodeLaunch& p, cudaStream_t s);
 struct FusedGemm {
   CUtensorMap xmap;         // activation operand of this step: [T, ld] bf16, box 64 x 128, 128-byte swizzle
   const Job* jobs;
-  const Seg* segs;
+  const Seg* segs;          // the segments of job j start at segs[j * seg_stride]
   void* out;
   const float* bias;
   int n_jobs;
@@ -131,6 +134,7 @@ struct FusedGemm {
   int kind;                 // GemmKind
   uint32_t n_stages, bps;   // activation ring: stages, 16 KB boxes per stage
   uint32_t w_bytes;         // shared memory of the largest weight tile of this step
+  uint32_t seg_stride;
   uint32_t ahead;           // 1: the tile is decoded before the preceding barrier wait (its shared memory is free then)
 };
 
@@ -142,6 +146,8 @@ struct FusedLayerParams {
   const int32_t* seq_lens;
   int n_kept_heads, batch, seq, T;
   unsigned int* barrier;    // one counter per launch, zero when the kernel starts
+  const uint8_t* pf_ptr[4]; // the next layer's packed shards, tile descriptors and dense parameters,
+  uint32_t pf_bytes[4];     // pulled into L2 while this layer computes
   int* err;
 };
 

@@ -1,0 +1,95 @@
+"""The whole-layer kernel (one launch per layer, grid barriers between the steps) and the key-split attention
+kernel against the CPU oracle: same inputs, same 2e-2 relative max-abs bound as the seven-kernel path."""
+import os
+
+import dataclasses
+
+import numpy as np
+import pytest
+
+import workloads as W
+from oracle import sti_oracle as O
+
+pytestmark = pytest.mark.gpu
+
+sti = pytest.importorskip("paper_2207_05022_b200")
+
+
+@pytest.fixture(scope="module", autouse=True)
+def _built():
+    from paper_2207_05022_b200 import build
+    build.build_library()
+    sti.load_library()
+
+
+def _with_env(env, fn):
+    old = {k: os.environ.get(k) for k in env}
+    os.environ.update(env)
+    try:
+        return fn()
+    finally:
+        for k, v in old.items():
+            if v is None:
+                os.environ.pop(k, None)
+            else:
+                os.environ[k] = v
+
+
+def _mixed_workload(act, batch, seq, seed):
+    shape = W.ModelShape(n_layers=3, hidden=256, n_heads=4, head_dim=64, ffn=1024, n_ffn_slices=4)
+    bits = [2, 3, 4, 5, 6, 32]
+    attn = [[W.UnitPlan((l + i) % 4 != 1, bits[(l + i) % 6], l < 1) for i in range(4)] for l in range(3)]
+    ffn = [[W.UnitPlan((l + 2 * i) % 5 != 0, bits[(l + 3 * i) % 6], l < 1) for i in range(4)] for l in range(3)]
+    return W.build_workload("fused", shape, batch, seq, act, attn, ffn, seed=seed, ring_slots=2)
+
+
+@pytest.mark.parametrize("act,batch,seq", [("f32", 1, 100), ("bf16", 2, 150), ("f32", 1, 320)])
+def test_whole_layer_kernel_matches_oracle(act, batch, seq):
+    from gpu_util import run_model, rel_err, REL_TOL
+    work = _mixed_workload(act, batch, seq, seed=41)
+    ref = O.run_workload(work)
+
+    def run():
+        with sti.Session(work) as s:
+            first = run_model(s, work)
+            second = run_model(s, work)              # graph replay: the barrier counters start again at zero
+            return first, second, sti.sti_ctx_launch_count(s.ctx)
+
+    y, y2, launches = _with_env({"STI_TUNE": "fused_max_tokens=512"}, run)
+    assert rel_err(y, ref) <= REL_TOL
+    assert np.array_equal(y, y2)
+    casts = 1 if act == "f32" else 0
+    assert launches == 2 * (3 + casts)               # one launch per layer (+ the fp32 -> bf16 cast of the input)
+    y_seven, _, launches_seven = _with_env({"STI_TUNE": "fused_max_tokens=0"}, run)
+    assert launches_seven == 2 * (3 * 7 + casts)
+    assert rel_err(y, y_seven) <= 5e-3               # same operands, different attention summation order
+
+
+def test_whole_layer_kernel_with_padding_mask_and_single_layer_call():
+    from gpu_util import run_model, run_layer, rel_err, REL_TOL
+    work = _mixed_workload("f32", 2, 130, seed=43)
+    lens = [130, 57]
+    ref = O.run_workload(dataclasses.replace(work, seq_lens=np.asarray(lens, np.int32)))
+    ref_l1 = O.run_workload(work, layers=[1])
+
+    def run():
+        with sti.Session(work) as s:
+            return run_model(s, work, lens=lens), run_layer(s, work, 1)
+
+    y, y_l1 = _with_env({"STI_TUNE": "fused_max_tokens=512"}, run)
+    assert rel_err(y, ref) <= REL_TOL
+    assert rel_err(y_l1, ref_l1) <= REL_TOL
+
+
+def test_key_split_attention_long_sequence_and_mask():
+    """seq 512 (eight key blocks, two per key split) with a ragged mask through the stand-alone kernels."""
+    from gpu_util import run_model, rel_err, REL_TOL
+    shape = W.ModelShape(n_layers=1, hidden=256, n_heads=4, head_dim=64, ffn=1024, n_ffn_slices=4)
+    attn = [[W.UnitPlan(True, 4, True) for _ in range(4)]]
+    ffn = [[W.UnitPlan(True, 3, True) for _ in range(4)]]
+    work = W.build_workload("attn512", shape, 2, 512, "bf16", attn, ffn, seed=47, ring_slots=2)
+    lens = [512, 301]
+    ref = O.run_workload(dataclasses.replace(work, seq_lens=np.asarray(lens, np.int32)))
+    with sti.Session(work) as s:
+        y = run_model(s, work, lens=lens)
+    assert rel_err(y, ref) <= REL_TOL
