@@ -298,11 +298,9 @@ def run_sweep(args):
                       "peak_source": peak_src, "rows": rows}))
 
 
-def run_planner(args):
-    """Section 5 end to end: profile the device (T_io per version, T_comp per width m), let the library's
-    two-stage planner pick (n, m), bitwidths and the preload prefix for each target latency, execute the
-    plan streamed from pinned host memory and report how much of the copy time the pipeline hid.
-    Shard importance is a seeded uniform table (the paper profiles it on a dev set)."""
+def planner_profile(args):
+    """Section 5.2's two offline profiles on the device in use: T_io per stored version and T_comp per submodel
+    width m (see run_planner).  Returns everything the plan-and-execute modes need."""
     import workloads as W
     B, L = args.planner_batch, args.planner_seq
     workers = min(8, os.cpu_count() or 1)
@@ -379,7 +377,21 @@ def run_planner(args):
     pipe_us = max(0.0, (stack_ms(narrowed(4, streamed_from=1)) * 1e3 - measured[3] * depth) / (depth - 1))
     t_comp_us = [0.0] + [float(np.interp(m, widths, measured)) + pipe_us for m in range(1, M + 1)]
     t_comp_us = list(np.maximum.accumulate(t_comp_us))
+    return dict(W=W, sti=sti, torch=torch, stream=stream, flush=flush, forward_ms=forward_ms, B=B, L=L, N=N, M=M,
+                workers=workers, versions=versions, shard_bytes=shard_bytes, ring=ring, h2d_gbps=h2d_gbps,
+                t_io_us=t_io_us, t_comp_us=t_comp_us, pipe_us=pipe_us, measured=measured, t_comp16_6bit=t_comp16_6bit)
 
+
+def run_planner(args):
+    """Section 5 end to end: profile the device (T_io per version, T_comp per width m), let the library's
+    two-stage planner pick (n, m), bitwidths and the preload prefix for each target latency, execute the
+    plan streamed from pinned host memory and report how much of the copy time the pipeline hid.
+    Shard importance is a seeded uniform table (the paper profiles it on a dev set)."""
+    pf = planner_profile(args)
+    W, sti, torch, stream, flush, forward_ms = pf["W"], pf["sti"], pf["torch"], pf["stream"], pf["flush"], pf["forward_ms"]
+    B, L, N, M, workers, ring = pf["B"], pf["L"], pf["N"], pf["M"], pf["workers"], pf["ring"]
+    shard_bytes, h2d_gbps, t_io_us, t_comp_us, pipe_us = pf["shard_bytes"], pf["h2d_gbps"], pf["t_io_us"], pf["t_comp_us"], pf["pipe_us"]
+    measured, t_comp16_6bit = pf["measured"], pf["t_comp16_6bit"]
     importance = np.random.default_rng(np.random.SeedSequence([0, 77])).uniform(0, 1, (N, M)).astype(np.float32)
     preload_bytes = int(args.planner_preload_mb * (1 << 20))
     def execute(plan, target_ms):
@@ -446,6 +458,91 @@ def run_planner(args):
                       "ring_slots": ring, "rows": rows, "back_to_back": series}))
 
 
+def run_baselines(args):
+    """Section 7.1's comparison systems as plans of this library, next to the two-stage planner, for the same
+    target latencies on the same profiled device tables (latency only; accuracy needs trained weights):
+      Load&Exec       32-bit shards, everything loaded before layer 0 starts (IO + compute add up)
+      StdPL-X         uniform X bits, layerwise pipeline, nothing preloaded
+      PreloadModel-X  uniform X bits, the whole submodel resident (no IO at run time)
+      STI             sti_plan_auto: per-shard bitwidths, preload prefix, layerwise pipeline
+    Each baseline picks the submodel with Section 5.3's rule (most shards, then deepest) under its own
+    delay model, the plan is executed, and measured latency, fidelity (bits) and memory are reported."""
+    pf = planner_profile(args)
+    W, sti, torch, stream, flush, forward_ms = pf["W"], pf["sti"], pf["torch"], pf["stream"], pf["flush"], pf["forward_ms"]
+    B, L, N, M, workers = pf["B"], pf["L"], pf["N"], pf["M"], pf["workers"]
+    versions, shard_bytes, t_io_us, t_comp_us = pf["versions"], pf["shard_bytes"], pf["t_io_us"], pf["t_comp_us"]
+    importance = np.random.default_rng(np.random.SeedSequence([0, 77])).uniform(0, 1, (N, M)).astype(np.float32)
+    preload_bytes = int(args.planner_preload_mb * (1 << 20))
+    X = args.baseline_bits
+    vi = {k: i for i, k in enumerate(versions)}
+
+    def pick(delay_us, target_us):
+        best = None
+        for n in range(1, N + 1):
+            for m in range(1, M + 1):
+                if delay_us(n, m) <= target_us and (best is None or n * m > best[0] * best[1] or
+                                                    (n * m == best[0] * best[1] and n > best[0])):
+                    best = (n, m)
+        return best
+
+    def pipeline_us(n, m, bits):
+        """Layerwise pipeline with nothing preloaded: layer k starts when its shards and layer k-1 are done."""
+        io_done = comp_done = 0.0
+        for _ in range(n):
+            io_done += m * t_io_us[vi[bits]]
+            comp_done = max(comp_done, io_done) + t_comp_us[m]
+        return comp_done
+
+    def grids(n, m, bits, preload):
+        keep = np.zeros((N, M), np.uint8)
+        rank = np.argsort(-importance, axis=1, kind="stable")
+        for l in range(n):
+            keep[l, rank[l, :m]] = 1                     # the m most important shards of the layer
+        return keep, keep * bits, keep * (1 if preload else 0)
+
+    def execute(name, keep, bits, preload, target_ms, predicted_us, overlap=True):
+        streamed_layers = int(((keep > 0) & (preload == 0)).any(axis=1).sum())
+        work = W.make_planned(keep, bits, preload, batch=B, seq=L, workers=workers, ring_slots=max(2, streamed_layers))
+        kept_bits = bits[keep > 0]
+        with sti.Session(work, compute_stream=stream.cuda_stream) as sess:
+            if not overlap:
+                sti.sti_plan_set_overlap(sess.plan, False)
+            x = device_act(torch, work)
+            y = torch.empty_like(x)
+            ms = forward_ms(sess, work, x, y, args.steps)
+            mem = sti.sti_plan_memory(sess.plan)
+        return {"system": name, "target_ms": target_ms, "n": int(keep.any(axis=1).sum()), "m": int(keep[0].sum()),
+                "mean_bits": float(kept_bits.astype(np.float64).mean()),
+                "bits_hist": {int(b): int((kept_bits == b).sum()) for b in np.unique(kept_bits)},
+                "predicted_ms": predicted_us * 1e-3, "measured_ms": ms, "meets_target": bool(ms <= target_ms * 1.02),
+                "device_bytes_resident": mem["preload_bytes"], "device_bytes_ring": mem["ring_bytes"],
+                "streamed_bytes": work.packed_bytes() - mem["preload_bytes"]}
+
+    rows = []
+    for target_ms in [float(t) for t in args.planner_targets_ms.split(",")]:
+        T = target_ms * 1e3
+        # Load&Exec: IO of all 32-bit shards, then compute
+        load_exec = lambda n, m: n * m * t_io_us[vi[32]] + n * t_comp_us[m]
+        nm = pick(load_exec, T)
+        if nm:
+            rows.append(execute("Load&Exec", *grids(nm[0], nm[1], 32, False), target_ms, load_exec(*nm), overlap=False))
+        else:
+            rows.append({"system": "Load&Exec", "target_ms": target_ms, "n": 0, "m": 0, "note": "no submodel fits"})
+        nm = pick(lambda n, m: pipeline_us(n, m, X), T)
+        if nm:
+            rows.append(execute(f"StdPL-{X}", *grids(nm[0], nm[1], X, False), target_ms, pipeline_us(nm[0], nm[1], X)))
+        else:
+            rows.append({"system": f"StdPL-{X}", "target_ms": target_ms, "n": 0, "m": 0, "note": "no submodel fits"})
+        nm = pick(lambda n, m: n * t_comp_us[m], T)
+        rows.append(execute(f"PreloadModel-{X}", *grids(nm[0], nm[1], X, True), target_ms, nm[0] * t_comp_us[nm[1]]))
+        plan = sti.sti_plan_auto(T, N, M, t_comp_us, t_io_us, shard_bytes, importance, preload_bytes)
+        rows.append(execute("STI", plan["keep"], plan["bits"], plan["preload"], target_ms,
+                            plan["n"] * t_comp_us[plan["m"]]))
+    print(json.dumps({"baselines": "Section 7.1 systems as plans, BERT-large 24x16 store", "batch": B, "seq": L,
+                      "X": X, "preload_budget_bytes": preload_bytes, "h2d_GBps": pf["h2d_gbps"],
+                      "t_io_us": t_io_us, "t_comp_us": t_comp_us[1:], "rows": rows}))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -464,6 +561,9 @@ def main():
     ap.add_argument("--planner-preload-mb", type=float, default=8.0)
     ap.add_argument("--planner-series-mb", default="8,32,64",
                     help="preload buffer sizes of consecutive back-to-back executions at the last target")
+    ap.add_argument("--baselines", action="store_true",
+                    help="Load&Exec / StdPL-X / PreloadModel-X / planner comparison on the profiled device")
+    ap.add_argument("--baseline-bits", type=int, default=6, choices=[2, 3, 4, 5, 6])
     ap.add_argument("--planner-ring", type=int, default=24,
                     help="most streamed-layer buffers on the device (the IO budgets assume loading runs ahead freely)")
     args = ap.parse_args()
@@ -477,6 +577,10 @@ def main():
     if args.planner:
         args.steps = min(args.steps, 20)
         run_planner(args)
+        return
+    if args.baselines:
+        args.steps = min(args.steps, 20)
+        run_baselines(args)
         return
     args.warmup = max(args.warmup, 3)
 

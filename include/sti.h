@@ -179,6 +179,13 @@ sti_status sti_shard_decode(sti_plan* plan, int layer, sti_kind kind, int index,
 sti_status sti_plan_set_profiling(sti_plan* plan, int level);
 sti_status sti_get_stats(sti_plan* plan, sti_stats* out);
 
+/* Section 7.1 (the Load&Exec baseline "loads model as a whole and executes it"): with overlap = 0 a model
+ * forward first copies every streamed layer into its ring slot and only then starts layer 0, so IO and
+ * compute delays add up; overlap = 1 (the default) is the layerwise pipeline of Section 3.1.  Results are
+ * identical.  overlap = 0 needs one ring slot per streamed layer (STI_ERR_STATE otherwise: a slot could
+ * only be reused after a layer that has not started).  Takes effect at the next forward. */
+sti_status sti_plan_set_overlap(sti_plan* plan, int overlap);
+
 /* Bytes the plan holds: preload buffer in device memory, pinned host arena, ring slots. */
 sti_status sti_plan_memory(sti_plan* plan, uint64_t* preload_bytes, uint64_t* pinned_bytes, uint64_t* ring_bytes);
 

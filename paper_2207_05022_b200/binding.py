@@ -82,6 +82,7 @@ def load_library():
         "sti_sync": ([vp], i32),
         "sti_shard_decode": ([vp, i32, i32, i32, i32, vp, vp, vp], i32),
         "sti_plan_set_profiling": ([vp, i32], i32),
+        "sti_plan_set_overlap": ([vp, i32], i32),
         "sti_get_stats": ([vp, C.POINTER(StiStats)], i32),
         "sti_plan_memory": ([vp, u64p, u64p, u64p], i32),
         "sti_ctx_launch_count": ([vp], C.c_uint64),
@@ -101,7 +102,7 @@ def load_library():
 EXPORTED = ("sti_ctx_create", "sti_ctx_destroy", "sti_ctx_set_layer_params", "sti_plan_create",
             "sti_plan_destroy", "sti_shard_upload", "sti_plan_finalize", "sti_layer_forward",
             "sti_model_forward", "sti_model_forward_host", "sti_sync", "sti_shard_decode",
-            "sti_plan_set_profiling", "sti_get_stats", "sti_plan_memory", "sti_ctx_launch_count",
+            "sti_plan_set_profiling", "sti_plan_set_overlap", "sti_get_stats", "sti_plan_memory", "sti_ctx_launch_count",
             "sti_host_retile", "sti_strerror", "sti_matrix_decode_noalloc", "sti_plan_auto",
             "sti_preload_after_run")
 
@@ -207,6 +208,11 @@ def sti_shard_decode(plan: int, layer: int, kind: int, index: int, matrix: int, 
 def sti_plan_set_profiling(plan: int, level: int):
     """0 = off, 1 = per-layer events, 2 = events around every kernel."""
     _check(load_library().sti_plan_set_profiling(C.c_void_p(plan), int(level)), "sti_plan_set_profiling")
+
+
+def sti_plan_set_overlap(plan: int, overlap: bool):
+    """False: load every streamed layer, then execute (the Load&Exec order); True: the layerwise pipeline."""
+    _check(load_library().sti_plan_set_overlap(C.c_void_p(plan), int(bool(overlap))), "sti_plan_set_overlap")
 
 
 def sti_get_stats(plan: int) -> StiStats:

@@ -133,6 +133,8 @@ struct sti_plan {
   int max_partial = 1;
   unsigned int* fused_ctr = nullptr;   // one grid-barrier counter per layer, zeroed at the start of every forward
   bool fused_off = false;
+  bool overlap = true;                 // false: load every streamed layer, then execute (Load&Exec)
+  int n_streamed_layers = 0;
   bool stats_valid = false;
 };
 
@@ -588,10 +590,25 @@ sti_status enqueue_forward(sti_plan* p, const void* x, void* y, int batch, int s
     CUDA_TRY(cudaEventRecord(p->ev_fork, c->compute));
     CUDA_TRY(cudaStreamWaitEvent(c->copy, p->ev_fork, 0));
   }
+  if (!p->overlap && any_streamed) {
+    // load-then-execute: every IO job first (each layer has its own slot), compute waits for the last one
+    cudaEvent_t last = nullptr;
+    for (int li = 0; li < n; ++li) {
+      Layer& L = p->layers[li];
+      if (L.str_bytes == 0) continue;
+      if (!capturing) CUDA_TRY(cudaStreamWaitEvent(c->copy, p->slot_free[L.slot], 0));
+      if (prof) CUDA_TRY(cudaEventRecord(L.ev_copy_start, c->copy));
+      sti_status st = enqueue_layer_copy(p, li, c->copy);
+      if (st != STI_OK) return st;
+      last = capturing ? L.g_ev_loaded : L.ev_loaded;
+      CUDA_TRY(cudaEventRecord(last, c->copy));
+    }
+    CUDA_TRY(cudaStreamWaitEvent(c->compute, last, 0));
+  }
   const void* cur = x;
   for (int li = 0; li < n; ++li) {
     Layer& L = p->layers[li];
-    if (L.str_bytes > 0) {
+    if (L.str_bytes > 0 && p->overlap) {
       // one IO job per layer (Section 3.1); the slot is reused only after its previous layer finished
       if (!capturing) CUDA_TRY(cudaStreamWaitEvent(c->copy, p->slot_free[L.slot], 0));
       else if (slot_used[L.slot]) CUDA_TRY(cudaStreamWaitEvent(c->copy, p->g_slot_free[L.slot], 0));
@@ -967,6 +984,7 @@ sti_status sti_plan_finalize(sti_plan* p) {
     pinned_total += align256(L.str_bytes);
     slot_bytes = std::max(slot_bytes, align256(L.str_bytes));
     if (L.str_bytes) L.slot = (n_streamed++) % p->ring_slots;
+    p->n_streamed_layers = n_streamed;
     max_heads = std::max<int>(max_heads, L.kept_heads.size());
     max_slices = std::max<int>(max_slices, L.kept_slices.size());
   }
@@ -1236,6 +1254,25 @@ sti_status sti_plan_memory(sti_plan* p, uint64_t* preload_bytes, uint64_t* pinne
   if (preload_bytes) *preload_bytes = p->preload_bytes;
   if (pinned_bytes) *pinned_bytes = p->pinned_bytes;
   if (ring_bytes) *ring_bytes = p->slot_bytes * p->ring_slots;
+  return STI_OK;
+}
+
+sti_status sti_plan_set_overlap(sti_plan* p, int overlap) {
+  if (!p) return STI_ERR_ARG;
+  if (!overlap) {
+    sti_status st = sti_plan_finalize(p);
+    if (st != STI_OK) return st;
+    if (p->n_streamed_layers > p->ring_slots) return STI_ERR_STATE;
+  }
+  const bool want = overlap != 0;
+  if (want != p->overlap) {
+    // captured forwards encode the old order
+    cudaSetDevice(p->ctx->device);
+    cudaStreamSynchronize(p->ctx->compute);
+    for (auto& g : p->graphs) if (g.exec) { cudaGraphExecDestroy(g.exec); g.exec = nullptr; }
+    p->graphs.clear();
+    p->overlap = want;
+  }
   return STI_OK;
 }
 

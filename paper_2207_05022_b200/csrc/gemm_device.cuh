@@ -67,19 +67,32 @@ __device__ __forceinline__ void unpack_task(const uint32_t (&planes)[24], const 
   const bool narrow = sg.kc < 128;     // 64 in-features: the quantum is rows (l, l + 32) of a 64-row group
   const uint32_t row0 = narrow ? g * 64 + lane : g * 32 + lane;
   const uint32_t kcore0 = (sg.koff + (narrow ? 0 : j * 128)) >> 3;
+  // 32 indexes = exactly BITS words, whatever BITS is: the loop below is rolled over the four such groups
+  // of the quantum and always reads w[0 .. BITS), the words moving down by BITS after each group.  A
+  // quarter of the instructions of the fully unrolled form: the decode runs once per CTA, so its code is
+  // fetched cold and its size is what it costs.
+#pragma unroll 1
+  for (int grp = 0; grp < 4; ++grp) {
+    uint32_t lo[BITS];
 #pragma unroll
-  for (int s = 0; s < 16; ++s) {
-    uint32_t pk[4];
+    for (int i = 0; i < BITS; ++i) lo[i] = w[i];
 #pragma unroll
-    for (int e = 0; e < 4; ++e) {
-      const uint32_t c0 = extract_index<BITS>(w, 8 * s + 2 * e);
-      const uint32_t c1 = extract_index<BITS>(w, 8 * s + 2 * e + 1);
-      pk[e] = static_cast<uint32_t>(tab[c0]) | (static_cast<uint32_t>(tab[c1]) << 16);
+    for (int ss = 0; ss < 4; ++ss) {
+      uint32_t pk[4];
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        const uint32_t c0 = extract_index_words<BITS>(lo, 8 * ss + 2 * e);
+        const uint32_t c1 = extract_index_words<BITS>(lo, 8 * ss + 2 * e + 1);
+        pk[e] = static_cast<uint32_t>(tab[c0]) | (static_cast<uint32_t>(tab[c1]) << 16);
+      }
+      const uint32_t sidx = 4 * grp + ss;
+      const uint32_t row = narrow ? row0 + 32 * (sidx >> 3) : row0;
+      const uint32_t kcore = narrow ? kcore0 + (sidx & 7) : kcore0 + sidx;
+      *reinterpret_cast<uint4*>(wsm + (static_cast<size_t>(kcore) * n_rows + row) * 16) =
+          make_uint4(pk[0], pk[1], pk[2], pk[3]);
     }
-    const uint32_t row = narrow ? row0 + 32 * (s >> 3) : row0;
-    const uint32_t kcore = narrow ? kcore0 + (s & 7) : kcore0 + s;
-    *reinterpret_cast<uint4*>(wsm + (static_cast<size_t>(kcore) * n_rows + row) * 16) =
-        make_uint4(pk[0], pk[1], pk[2], pk[3]);
+#pragma unroll
+    for (int i = 0; i + BITS < 4 * BITS; ++i) w[i] = w[i + BITS];
   }
 }
 

@@ -22,6 +22,17 @@ __device__ __forceinline__ uint32_t extract_index(const uint32_t (&w)[4 * BITS],
   return v & ((1u << BITS) - 1u);
 }
 
+// Same extraction from the first BITS words of a quantum (32 indexes).
+template <int BITS>
+__device__ __forceinline__ uint32_t extract_index_words(const uint32_t (&w)[BITS], int i) {
+  const int b = i * BITS;
+  const int word = b >> 5;
+  const int s = b & 31;
+  uint32_t v = w[word] >> s;
+  if (s + BITS > 32) v |= w[word + 1] << (32 - s);
+  return v & ((1u << BITS) - 1u);
+}
+
 __device__ __forceinline__ uint16_t bf16_bits(float f) {
   return __bfloat16_as_ushort(__float2bfloat16_rn(f));
 }

@@ -70,3 +70,25 @@ def test_tile_shapes_do_not_change_results_beyond_rounding():
     for tune in ("qkv_n=32,f1_n=32,o_group=1,f2_group=1", "qkv_n=64,f1_n=128,o_group=16,f2_group=4,f2_n=128,o_n=128"):
         y, _ = _run(work, {"STI_TUNE": tune})
         assert rel_err(y, ref) <= REL_TOL, tune
+
+
+def test_load_then_execute_order_gives_the_same_result():
+    """The Load&Exec order (every streamed layer copied before layer 0 starts) against the layerwise pipeline."""
+    from gpu_util import run_model
+    work = _workload()                                   # layers 2 and 3 streamed
+    with sti.Session(work) as s:                         # two ring slots = two streamed layers
+        piped = run_model(s, work)
+        sti.sti_plan_set_overlap(s.plan, False)
+        loaded_first = run_model(s, work)
+        again = run_model(s, work)
+        sti.sti_plan_set_overlap(s.plan, True)
+        back = run_model(s, work)
+    assert np.array_equal(piped, loaded_first) and np.array_equal(piped, again) and np.array_equal(piped, back)
+    # one slot per streamed layer is required: three streamed layers do not fit two slots
+    import dataclasses
+    attn = [[dataclasses.replace(u, resident=l < 1) for u in row] for l, row in enumerate(work.attn_plan)]
+    ffn = [[dataclasses.replace(u, resident=l < 1) for u in row] for l, row in enumerate(work.ffn_plan)]
+    with sti.Session(dataclasses.replace(work, attn_plan=attn, ffn_plan=ffn)) as s:
+        with pytest.raises(sti.StiError) as err:
+            sti.sti_plan_set_overlap(s.plan, False)
+        assert "state" in str(err.value)
