@@ -41,7 +41,7 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 # dram__bytes_read.sum + dram__bytes_write.sum per dequant-GEMM launch (mean over one layer's QKV, O, FFN1, FFN2
 # launches; BERT-large layer, batch 1, seq 256) from the ncu capture summarised in
 # profiles/dqgemm_bertlarge_seq256_ncu_full.md.  Set to None whenever dqgemm.cu changes after that capture.
-NCU_DRAM_BYTES_PER_GEMM_LAUNCH = 2534464
+NCU_DRAM_BYTES_PER_GEMM_LAUNCH = 2542016
 
 
 def load_peaks():
@@ -516,7 +516,7 @@ def run_baselines(args):
                 "bits_hist": {int(b): int((kept_bits == b).sum()) for b in np.unique(kept_bits)},
                 "predicted_ms": predicted_us * 1e-3, "measured_ms": ms, "meets_target": bool(ms <= target_ms * 1.02),
                 "device_bytes_resident": mem["preload_bytes"], "device_bytes_ring": mem["ring_bytes"],
-                "streamed_bytes": work.packed_bytes() - mem["preload_bytes"]}
+                "streamed_bytes": max(0, work.packed_bytes() - mem["preload_bytes"])}
 
     rows = []
     for target_ms in [float(t) for t in args.planner_targets_ms.split(",")]:

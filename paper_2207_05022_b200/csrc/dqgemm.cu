@@ -248,9 +248,41 @@ dqgemm_kernel(const __grid_constant__ CUtensorMap xmap, const Job* __restrict__ 
         const int t = static_cast<int>((blockIdx.y + ti * gridDim.y) * kTileM + q * 32 + lane);
         OutT* drow = out + (static_cast<size_t>(job.out_mat) * T + (t < T ? t : 0)) * ldo + job.out_col;
         const uint32_t taddr = tmem_base + ((q * 32) << 16) + buf * n_rows;
-        if (ncol >= 32) {
-          // 32 columns per step: each thread then writes 128 (fp32) or 64 (bf16) contiguous bytes of its row
+        if (my_mtiles <= 2) {
+          // 16 columns per step in a rolled loop: the epilogue runs once per tile, its code is fetched cold
+#pragma unroll 1
+          for (uint32_t col = half * ncol; col < (half + 1) * ncol; col += 16) {
+            uint32_t r[16];
+            tmem_ld_32x32b_x16(taddr + col, r);
+            tc_wait_ld();
+            if (t < T) {
+              float v[16];
+#pragma unroll
+              for (int i = 0; i < 16; ++i) {
+                const float a = __uint_as_float(r[i]) + bias_sm[col + i];
+                v[i] = GELU ? gelu_erf(a) : a;
+              }
+              store_row16<OutT>(drow + col, v);
+            }
+          }
+        } else {
+          // many tiles per CTA: 32 columns per step, unrolled (each thread writes 128 or 64 contiguous bytes)
           for (uint32_t col = half * ncol; col < (half + 1) * ncol; col += 32) {
+            if (col + 32 > (half + 1) * ncol) {            // 16-column tail of 32-row tiles
+              uint32_t r[16];
+              tmem_ld_32x32b_x16(taddr + col, r);
+              tc_wait_ld();
+              if (t < T) {
+                float v[16];
+#pragma unroll
+                for (int i = 0; i < 16; ++i) {
+                  const float a = __uint_as_float(r[i]) + bias_sm[col + i];
+                  v[i] = GELU ? gelu_erf(a) : a;
+                }
+                store_row16<OutT>(drow + col, v);
+              }
+              break;
+            }
             uint32_t r[32];
             tmem_ld_32x32b_x32(taddr + col, r);
             tc_wait_ld();
@@ -266,20 +298,6 @@ dqgemm_kernel(const __grid_constant__ CUtensorMap xmap, const Job* __restrict__ 
                 store_row16<OutT>(drow + col + h * 16, v);
               }
             }
-          }
-        } else {
-          const uint32_t col = half * ncol;      // 16 columns
-          uint32_t r[16];
-          tmem_ld_32x32b_x16(taddr + col, r);
-          tc_wait_ld();
-          if (t < T) {
-            float v[16];
-#pragma unroll
-            for (int i = 0; i < 16; ++i) {
-              const float a = __uint_as_float(r[i]) + bias_sm[col + i];
-              v[i] = GELU ? gelu_erf(a) : a;
-            }
-            store_row16<OutT>(drow + col, v);
           }
         }
         tc_fence_before_sync();
