@@ -11,5 +11,6 @@ from .binding import (  # noqa: F401
     sti_shard_upload, sti_plan_finalize, sti_layer_forward, sti_model_forward, sti_model_forward_host,
     sti_sync, sti_shard_decode, sti_plan_set_profiling, sti_plan_set_overlap, sti_get_stats, sti_plan_memory,
     sti_ctx_launch_count, sti_host_retile, sti_strerror, sti_matrix_decode_noalloc, sti_plan_auto, sti_preload_after_run,
+    sti_quantize_units, sti_quantize_workspace_bytes,
     Session,
 )

@@ -104,7 +104,7 @@ EXPORTED = ("sti_ctx_create", "sti_ctx_destroy", "sti_ctx_set_layer_params", "st
             "sti_model_forward", "sti_model_forward_host", "sti_sync", "sti_shard_decode",
             "sti_plan_set_profiling", "sti_plan_set_overlap", "sti_get_stats", "sti_plan_memory", "sti_ctx_launch_count",
             "sti_host_retile", "sti_strerror", "sti_matrix_decode_noalloc", "sti_plan_auto",
-            "sti_preload_after_run")
+            "sti_preload_after_run", "sti_quantize_units", "sti_quantize_workspace_bytes")
 
 
 def _check(status: int, where: str):
@@ -321,6 +321,27 @@ def sti_preload_after_run(keep, bits, shard_bytes, buffer_bytes: int):
                                      (C.c_uint64 * 6)(*[int(v) for v in shard_bytes]), int(buffer_bytes),
                                      _ptr(out), C.byref(used)), "sti_preload_after_run")
     return out, int(used.value)
+
+
+def sti_quantize_workspace_bytes(n_units: int, n_weights: int) -> int:
+    lib = load_library()
+    lib.sti_quantize_workspace_bytes.restype = C.c_size_t
+    lib.sti_quantize_workspace_bytes.argtypes = [C.c_uint32, C.c_uint32]
+    return int(lib.sti_quantize_workspace_bytes(n_units, n_weights))
+
+
+def sti_quantize_units(w_dev: int, n_units: int, n_weights: int, bits: int, codes_dev: int, centroids_dev: int,
+                       outlier_off_dev: int, outlier_val_dev: int, max_outliers: int, n_outliers_dev: int,
+                       workspace_dev: int, workspace_bytes: int, device: int = 0, stream: int = 0):
+    """Section 6 quantizer on the device; every buffer is a device address owned by the caller (see sti_quantize.h)."""
+    lib = load_library()
+    lib.sti_quantize_units.restype = C.c_int
+    lib.sti_quantize_units.argtypes = [C.c_int, C.c_void_p, C.c_void_p, C.c_uint32, C.c_uint32, C.c_int, C.c_void_p,
+                                       C.c_void_p, C.c_void_p, C.c_void_p, C.c_uint32, C.c_void_p, C.c_void_p, C.c_size_t]
+    _check(lib.sti_quantize_units(device, C.c_void_p(stream or None), C.c_void_p(w_dev), n_units, n_weights, int(bits),
+                                  C.c_void_p(codes_dev), C.c_void_p(centroids_dev), C.c_void_p(outlier_off_dev),
+                                  C.c_void_p(outlier_val_dev), max_outliers, C.c_void_p(n_outliers_dev),
+                                  C.c_void_p(workspace_dev), workspace_bytes), "sti_quantize_units")
 
 
 class Session:
