@@ -543,6 +543,73 @@ def run_baselines(args):
                       "t_io_us": t_io_us, "t_comp_us": t_comp_us[1:], "rows": rows}))
 
 
+def run_quantize(args):
+    """Section 6 on the device: every shard unit of `--layers` BERT-large layers (16 attention units of 262,144
+    weights and 16 FFN units of 524,288 weights per layer) quantized at `--baseline-bits` bits by
+    sti_quantize_units, timed with CUDA events, next to the CPU oracle on a sample of the same units."""
+    import workloads as W
+    from workloads.shards import ATTN, FFN, make_unit_weights
+    from oracle import sti_quantizer_oracle as Q
+    n_layers = args.layers or 4
+    bits = args.baseline_bits
+    shape = W.BERT_LARGE
+    groups = {}
+    for kind, name in ((ATTN, "attn"), (FFN, "ffn")):
+        groups[name] = np.stack([np.concatenate([m.reshape(-1) for m in make_unit_weights(shape, 0, l, kind, i)])
+                                 for l in range(n_layers) for i in range(shape.n_heads)])
+    t0 = time.perf_counter()
+    sample = [groups["attn"][0], groups["ffn"][0]]
+    for u in sample:
+        Q.quantize_unit(u, bits)
+    cpu_s = time.perf_counter() - t0
+    cpu_weights = sum(u.size for u in sample)
+    import torch
+    import paper_2207_05022_b200 as sti
+    from paper_2207_05022_b200 import build
+    build.build_library()
+    peaks, peak_src = load_peaks()
+    stream = torch.cuda.current_stream()
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
+    rows, total_ms, total_weights, total_bytes = [], 0.0, 0, 0
+    for name, units in groups.items():
+        n_units, n = units.shape
+        w = torch.from_numpy(units).cuda()
+        codes = torch.zeros((n_units, n * bits // 32), dtype=torch.int32, device="cuda")
+        cents = torch.zeros((n_units, 1 << bits), dtype=torch.float32, device="cuda")
+        off = torch.zeros((n_units, 4096), dtype=torch.int32, device="cuda")
+        val = torch.zeros((n_units, 4096), dtype=torch.float32, device="cuda")
+        cnt = torch.zeros(n_units, dtype=torch.int32, device="cuda")
+        ws_bytes = sti.sti_quantize_workspace_bytes(n_units, n)
+        ws = torch.empty(ws_bytes, dtype=torch.uint8, device="cuda")
+        ms = []
+        for i in range(args.warmup + args.steps):
+            flush.zero_()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(stream)
+            sti.sti_quantize_units(w.data_ptr(), n_units, n, bits, codes.data_ptr(), cents.data_ptr(), off.data_ptr(),
+                                   val.data_ptr(), 4096, cnt.data_ptr(), ws.data_ptr(), ws_bytes,
+                                   stream=stream.cuda_stream)
+            e1.record(stream)
+            stream.synchronize()
+            if i >= args.warmup:
+                ms.append(e0.elapsed_time(e1))
+        med = float(np.median(ms))
+        algo = n_units * (n * 4 + n * bits // 8 + (4 << bits))            # fp32 in, index stream + table out
+        rows.append({"units": name, "n_units": n_units, "weights_per_unit": n, "ms": med,
+                     "Mweights_per_s": n_units * n / med / 1e3, "algorithmic_GBps": algo / med / 1e6,
+                     "frac_of_hbm_peak": algo / med / 1e6 / peaks["hbm_gbs"], "workspace_bytes": ws_bytes,
+                     "outliers_mean": float(cnt.float().mean().item())})
+        total_ms += med; total_weights += n_units * n; total_bytes += algo
+    print(json.dumps({"quantize": f"Section 6 quantizer, {n_layers} BERT-large layers, {bits} bits", "rows": rows,
+                      "total_ms": total_ms, "Mweights_per_s": total_weights / total_ms / 1e3,
+                      "roofline": {"bound": "hbm", "achieved": total_bytes / total_ms / 1e6, "peak": peaks["hbm_gbs"],
+                                   "unit": "GB/s", "frac": total_bytes / total_ms / 1e6 / peaks["hbm_gbs"],
+                                   "traffic": None, "peak_source": f"hbm_gbs, {peak_src}",
+                                   "note": "one CTA per unit; four radix passes move 16 B per weight each inside the workspace"},
+                      "cpu_baseline": {"value": cpu_weights / cpu_s / 1e6, "unit": "Mweights/s", "cores": blas_threads(),
+                                       "kind": "oracle", "sample": "one attention unit and one FFN unit of layer 0"}}))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -563,6 +630,7 @@ def main():
                     help="preload buffer sizes of consecutive back-to-back executions at the last target")
     ap.add_argument("--baselines", action="store_true",
                     help="Load&Exec / StdPL-X / PreloadModel-X / planner comparison on the profiled device")
+    ap.add_argument("--quantize", action="store_true", help="time the device quantizer (Section 6) on BERT-large units")
     ap.add_argument("--baseline-bits", type=int, default=6, choices=[2, 3, 4, 5, 6])
     ap.add_argument("--planner-ring", type=int, default=24,
                     help="most streamed-layer buffers on the device (the IO budgets assume loading runs ahead freely)")
@@ -577,6 +645,10 @@ def main():
     if args.planner:
         args.steps = min(args.steps, 20)
         run_planner(args)
+        return
+    if args.quantize:
+        args.steps = min(args.steps, 10)
+        run_quantize(args)
         return
     if args.baselines:
         args.steps = min(args.steps, 20)

@@ -5,7 +5,9 @@
 //   2. outliers = weights whose log-likelihood is below -4: their (offset, value) pairs are written in
 //      ascending offset order by a stable compaction; the other weights become (sortable key, offset) pairs;
 //   3. a least-significant-digit radix sort (4 passes of 8 bits, stable, so equal weights keep their
-//      original order) of the pairs between two workspace buffers;
+//      original order) of the pairs between two workspace buffers, 4096 elements per step: every thread
+//      holds one element of each of four consecutive 1024-element stripes, ranks come from warp match
+//      masks plus a per-(stripe, warp, digit) count table in shared memory;
 //   4. 2^k clusters of equal population over the sorted order, cluster c = [floor(c n'/2^k), floor((c+1) n'/2^k)),
 //      centroid = arithmetic mean (fp64 sum, rounded once to fp32);
 //   5. every weight gets its cluster's k-bit index; an outlier's slot gets the nearest centroid's index
@@ -23,13 +25,18 @@ namespace {
 constexpr int kQThreads = 1024;
 constexpr int kQWarps = kQThreads / 32;
 
+constexpr int kItems = 4;             // elements per thread and chunk; a chunk is 4 stripes of 1024 consecutive elements
+constexpr int kSlots = kItems * kQWarps;   // (stripe, warp) pairs of a chunk, in element order
+
 struct QuantShared {
   double red[kQWarps];
   uint32_t hist[256];
   uint32_t base[2][256];
-  uint8_t wcount[kQWarps][256];      // per chunk: elements of digit d held by warp w
-  uint16_t woff[kQWarps][256];       // per chunk: elements of digit d held by warps before w
-  uint32_t wcnt_in[kQWarps], wcnt_out[kQWarps];
+  uint8_t wcount[kSlots][256];       // per chunk: elements of digit d held by (stripe, warp) slot q
+  uint16_t woff[kSlots][256];        // per chunk: elements of digit d held by the slots before q
+  uint32_t wcnt_in[kSlots], wcnt_out[kSlots];
+  uint32_t tot_in, tot_out;
+  uint16_t stripe_tot[kItems][256];  // per chunk: elements of digit d in stripe j
   uint32_t bounds[65];
   float cents[64];
 };
@@ -54,16 +61,30 @@ __device__ __forceinline__ uint32_t sort_key(float x) {
 __device__ __forceinline__ float key_value(uint32_t k) {
   return __uint_as_float((k & 0x80000000u) ? (k & 0x7fffffffu) : ~k);
 }
-__device__ __forceinline__ bool is_outlier(float x, double mu, double var, double c0) {
+// Lanes of the warp that hold the same 8-bit digit (valid lanes only): eight ballots, a fixed cost whatever
+// the number of distinct digits (a hardware match instruction walks the distinct values one by one).
+__device__ __forceinline__ uint32_t same_digit_lanes(uint32_t d, bool valid) {
+  uint32_t peers = __ballot_sync(0xffffffffu, valid);
+#pragma unroll
+  for (int b = 0; b < 8; ++b) {
+    const bool bit = (d >> b) & 1u;
+    const uint32_t bal = __ballot_sync(0xffffffffu, bit);
+    peers &= bit ? bal : ~bal;
+  }
+  return peers;
+}
+// inv2var = 1 / (2 var); with zero variance c0 is +inf and 0 * inf is NaN, which compares false: no outliers
+__device__ __forceinline__ bool is_outlier(float x, double mu, double inv2var, double c0) {
   const double d = static_cast<double>(x) - mu;
-  const double ll = c0 - d * d / (2.0 * var);        // NaN when the variance is zero: compares false
+  const double ll = c0 - d * d * inv2var;
   return ll < -4.0;
 }
 
 __global__ void __launch_bounds__(kQThreads, 1)
 quantize_units_kernel(const float* w_all, uint32_t n, int bits, uint32_t* codes_all, float* cent_all, uint32_t* ooff_all,
                       float* oval_all, uint32_t max_out, uint32_t* n_out_all, uint8_t* ws_all, size_t ws_per_unit) {
-  __shared__ QuantShared sm;
+  extern __shared__ __align__(16) uint8_t q_smem[];
+  QuantShared& sm = *reinterpret_cast<QuantShared*>(q_smem);
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const uint32_t unit = blockIdx.x;
   const uint32_t K = 1u << bits;
@@ -77,47 +98,89 @@ quantize_units_kernel(const float* w_all, uint32_t n, int bits, uint32_t* codes_
   uint32_t* idx[2] = {key[0] + n, key[1] + n};
   uint8_t* codes8 = ws + 16 * static_cast<size_t>(n);
 
-  // ---- 1. Gaussian fit
+  // ---- 1. Gaussian fit (eight independent loads in flight per thread: a single CTA has little else to hide latency)
   double s = 0.0;
-  for (uint32_t i = tid; i < n; i += kQThreads) s += static_cast<double>(w[i]);
+  for (uint32_t i0 = tid; i0 < n; i0 += 8 * kQThreads) {
+    float v[8];
+#pragma unroll
+    for (int u = 0; u < 8; ++u) { const uint32_t i = i0 + u * kQThreads; v[u] = i < n ? w[i] : 0.f; }
+#pragma unroll
+    for (int u = 0; u < 8; ++u) s += static_cast<double>(v[u]);
+  }
   const double mu = block_sum(s, sm, tid) / static_cast<double>(n);
   double q = 0.0;
-  for (uint32_t i = tid; i < n; i += kQThreads) {
-    const double d = static_cast<double>(w[i]) - mu;
-    q += d * d;
+  for (uint32_t i0 = tid; i0 < n; i0 += 8 * kQThreads) {
+    float v[8];
+#pragma unroll
+    for (int u = 0; u < 8; ++u) { const uint32_t i = i0 + u * kQThreads; v[u] = i < n ? w[i] : 0.f; }
+#pragma unroll
+    for (int u = 0; u < 8; ++u) {
+      const double d = static_cast<double>(v[u]) - mu;
+      if (i0 + u * kQThreads < n) q += d * d;
+    }
   }
   const double var = block_sum(q, sm, tid) / static_cast<double>(n);
   const double c0 = -0.5 * log(2.0 * 3.14159265358979323846 * var);
+  const double inv2var = 1.0 / (2.0 * var);
 
   // ---- 2. outliers out (ascending offsets), the rest as (key, offset) pairs, both by stable compaction
   uint32_t n_in = 0, n_out = 0;
   const uint32_t lt_mask = (1u << lane) - 1u;
-  for (uint32_t start = 0; start < n; start += kQThreads) {
-    const uint32_t i = start + tid;
-    const bool valid = i < n;
-    const float x = valid ? w[i] : 0.f;
-    const bool out = valid && is_outlier(x, mu, var, c0);
-    const bool in = valid && !out;
-    const uint32_t m_in = __ballot_sync(0xffffffffu, in), m_out = __ballot_sync(0xffffffffu, out);
-    if (lane == 0) { sm.wcnt_in[warp] = __popc(m_in); sm.wcnt_out[warp] = __popc(m_out); }
+  for (uint32_t start = 0; start < n; start += kItems * kQThreads) {
+    float x[kItems];
+    bool in[kItems], out[kItems];
+    uint32_t m_in[kItems], m_out[kItems];
+#pragma unroll
+    for (int j = 0; j < kItems; ++j) {
+      const uint32_t i = start + j * kQThreads + tid;
+      x[j] = i < n ? w[i] : 0.f;
+    }
+#pragma unroll
+    for (int j = 0; j < kItems; ++j) {
+      const uint32_t i = start + j * kQThreads + tid;
+      out[j] = i < n && is_outlier(x[j], mu, inv2var, c0);
+      in[j] = i < n && !out[j];
+      m_in[j] = __ballot_sync(0xffffffffu, in[j]);
+      m_out[j] = __ballot_sync(0xffffffffu, out[j]);
+      if (lane == 0) { sm.wcnt_in[j * kQWarps + warp] = __popc(m_in[j]); sm.wcnt_out[j * kQWarps + warp] = __popc(m_out[j]); }
+    }
     __syncthreads();
-    uint32_t pre_in = 0, pre_out = 0, tot_in = 0, tot_out = 0;
-    for (int ww = 0; ww < kQWarps; ++ww) {
-      const uint32_t a = sm.wcnt_in[ww], b = sm.wcnt_out[ww];
-      if (ww < warp) { pre_in += a; pre_out += b; }
-      tot_in += a; tot_out += b;
+    // exclusive prefix of the 128 slot counts in element order: warp 0, four slots per lane, one shuffle scan
+    if (warp == 0) {
+      uint32_t a[4], b[4], sa = 0, sb = 0;
+#pragma unroll
+      for (int e = 0; e < 4; ++e) { a[e] = sm.wcnt_in[4 * lane + e]; b[e] = sm.wcnt_out[4 * lane + e]; sa += a[e]; sb += b[e]; }
+      uint32_t ia = sa, ib = sb;
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) {
+        const uint32_t ta = __shfl_up_sync(0xffffffffu, ia, o), tb = __shfl_up_sync(0xffffffffu, ib, o);
+        if (lane >= o) { ia += ta; ib += tb; }
+      }
+      uint32_t ea = ia - sa, eb = ib - sb;
+#pragma unroll
+      for (int e = 0; e < 4; ++e) { sm.wcnt_in[4 * lane + e] = ea; sm.wcnt_out[4 * lane + e] = eb; ea += a[e]; eb += b[e]; }
+      if (lane == 31) { sm.tot_in = ia; sm.tot_out = ib; }
     }
-    if (in) {
-      const uint32_t dst = n_in + pre_in + __popc(m_in & lt_mask);
-      key[0][dst] = sort_key(x);
-      idx[0][dst] = i;
+    __syncthreads();
+    const uint32_t run_in = sm.tot_in, run_out = sm.tot_out;
+    uint32_t pre_in[kItems], pre_out[kItems];
+#pragma unroll
+    for (int j = 0; j < kItems; ++j) { pre_in[j] = sm.wcnt_in[j * kQWarps + warp]; pre_out[j] = sm.wcnt_out[j * kQWarps + warp]; }
+#pragma unroll
+    for (int j = 0; j < kItems; ++j) {
+      const uint32_t i = start + j * kQThreads + tid;
+      if (in[j]) {
+        const uint32_t dst = n_in + pre_in[j] + __popc(m_in[j] & lt_mask);
+        key[0][dst] = sort_key(x[j]);
+        idx[0][dst] = i;
+      }
+      if (out[j]) {
+        const uint32_t dst = n_out + pre_out[j] + __popc(m_out[j] & lt_mask);
+        if (dst < max_out) { ooff[dst] = i; oval[dst] = x[j]; }
+      }
     }
-    if (out) {
-      const uint32_t dst = n_out + pre_out + __popc(m_out & lt_mask);
-      if (dst < max_out) { ooff[dst] = i; oval[dst] = x; }
-    }
-    n_in += tot_in;
-    n_out += tot_out;
+    n_in += run_in;
+    n_out += run_out;
     __syncthreads();
   }
   if (tid == 0) n_out_all[unit] = n_out;
@@ -132,7 +195,20 @@ quantize_units_kernel(const float* w_all, uint32_t n, int bits, uint32_t* codes_
     uint32_t* idst = idx[cur ^ 1];
     if (tid < 256) sm.hist[tid] = 0;
     __syncthreads();
-    for (uint32_t i = tid; i < n_in; i += kQThreads) atomicAdd(&sm.hist[(ksrc[i] >> shift) & 255u], 1u);
+    // one shared-memory atomic per distinct digit of a warp (the high digits of weights fall into a few bins)
+    const uint32_t n_in_up = (n_in + 31u) & ~31u;          // whole warps take every iteration (match is warp-wide)
+    for (uint32_t i0 = tid; i0 < n_in_up; i0 += 8 * kQThreads) {
+      uint32_t kv[8];
+#pragma unroll
+      for (int u = 0; u < 8; ++u) { const uint32_t i = i0 + u * kQThreads; kv[u] = i < n_in ? ksrc[i] : 0u; }
+#pragma unroll
+      for (int u = 0; u < 8; ++u) {
+        const uint32_t i = i0 + u * kQThreads;
+        const uint32_t dg = (kv[u] >> shift) & 255u;
+        const uint32_t pm = same_digit_lanes(dg, i < n_in);
+        if (i < n_in && (pm & lt_mask) == 0) atomicAdd(&sm.hist[dg], static_cast<uint32_t>(__popc(pm)));
+      }
+    }
     __syncthreads();
     // exclusive prefix of the histogram -> first destination of every digit
     if (tid < 256) sm.base[0][tid] = sm.hist[tid];
@@ -147,36 +223,56 @@ quantize_units_kernel(const float* w_all, uint32_t n, int bits, uint32_t* codes_
     if (tid < 256) sm.base[0][tid] -= sm.hist[tid];
     __syncthreads();
     int bsel = 0;
-    for (uint32_t start = 0; start < n_in; start += kQThreads) {
-      const uint32_t i = start + tid;
-      const bool valid = i < n_in;
-      const uint32_t kk = valid ? ksrc[i] : 0u;
-      const uint32_t ii = valid ? isrc[i] : 0u;
-      const uint32_t d = (kk >> shift) & 255u;
-      // lanes holding the same digit; lanes past the end get a value of their own
-      const uint32_t peers = __match_any_sync(0xffffffffu, valid ? d : (256u + lane));
-      const uint32_t rank_w = __popc(peers & lt_mask);
-      reinterpret_cast<uint32_t*>(&sm.wcount[0][0])[tid] = 0u;
-      reinterpret_cast<uint32_t*>(&sm.wcount[0][0])[tid + kQThreads] = 0u;
+    for (uint32_t start = 0; start < n_in; start += kItems * kQThreads) {
+      uint32_t kk[kItems], ii[kItems], d[kItems], peers[kItems];
+      bool valid[kItems];
+#pragma unroll
+      for (int j = 0; j < kItems; ++j) {
+        const uint32_t i = start + j * kQThreads + tid;
+        valid[j] = i < n_in;
+        kk[j] = valid[j] ? ksrc[i] : 0u;
+        ii[j] = valid[j] ? isrc[i] : 0u;
+      }
+      for (int z = tid; z < kSlots * 256 / 4; z += kQThreads) reinterpret_cast<uint32_t*>(&sm.wcount[0][0])[z] = 0u;
+#pragma unroll
+      for (int j = 0; j < kItems; ++j) {
+        d[j] = (kk[j] >> shift) & 255u;
+        peers[j] = same_digit_lanes(d[j], valid[j]);
+      }
       __syncthreads();
-      if (valid && rank_w == 0) sm.wcount[warp][d] = static_cast<uint8_t>(__popc(peers));
+#pragma unroll
+      for (int j = 0; j < kItems; ++j)
+        if (valid[j] && (peers[j] & lt_mask) == 0) sm.wcount[j * kQWarps + warp][d[j]] = static_cast<uint8_t>(__popc(peers[j]));
       __syncthreads();
-      if (tid < 256) {
+      {
+        // thread (stripe sj, digit sd): prefix over the stripe's 32 warps; the four stripes run side by side
+        const int sj = tid >> 8, sd = tid & 255;
         uint32_t pre = 0;
         for (int ww = 0; ww < kQWarps; ++ww) {
-          sm.woff[ww][tid] = static_cast<uint16_t>(pre);
-          pre += sm.wcount[ww][tid];
+          sm.woff[sj * kQWarps + ww][sd] = static_cast<uint16_t>(pre);
+          pre += sm.wcount[sj * kQWarps + ww][sd];
         }
-        sm.base[bsel ^ 1][tid] = sm.base[bsel][tid] + pre;
+        sm.stripe_tot[sj][sd] = static_cast<uint16_t>(pre);
       }
       __syncthreads();
-      if (valid) {
-        const uint32_t dst = sm.base[bsel][d] + sm.woff[warp][d] + rank_w;
-        kdst[dst] = kk;
-        idst[dst] = ii;
+      if (tid < 256) {
+        uint32_t t = 0;
+#pragma unroll
+        for (int j = 0; j < kItems; ++j) t += sm.stripe_tot[j][tid];
+        sm.base[bsel ^ 1][tid] = sm.base[bsel][tid] + t;
+      }
+#pragma unroll
+      for (int j = 0; j < kItems; ++j) {
+        if (valid[j]) {
+          uint32_t dst = sm.base[bsel][d[j]] + sm.woff[j * kQWarps + warp][d[j]] + __popc(peers[j] & lt_mask);
+#pragma unroll
+          for (int jj = 0; jj < kItems; ++jj)
+            if (jj < j) dst += sm.stripe_tot[jj][d[j]];
+          kdst[dst] = kk[j];
+          idst[dst] = ii[j];
+        }
       }
       bsel ^= 1;
-      // the next chunk's zeroing of wcount is ordered after these reads by its own barrier below the zeroing
       __syncthreads();
     }
     cur ^= 1;
@@ -203,42 +299,61 @@ quantize_units_kernel(const float* w_all, uint32_t n, int bits, uint32_t* codes_
   __syncthreads();
 
   // ---- 5. indexes: the cluster of a weight's rank; for an outlier the nearest centroid
-  for (uint32_t r = tid; r < n_in; r += kQThreads) {
-    uint32_t c = static_cast<uint32_t>(static_cast<uint64_t>(r) * K / n_in);
-    while (c + 1 < K && sm.bounds[c + 1] <= r) ++c;
-    while (c > 0 && sm.bounds[c] > r) --c;
-    codes8[is[r]] = static_cast<uint8_t>(c);
+  for (uint32_t r0 = tid; r0 < n_in; r0 += 8 * kQThreads) {
+    uint32_t dst[8];
+#pragma unroll
+    for (int u = 0; u < 8; ++u) { const uint32_t r = r0 + u * kQThreads; dst[u] = r < n_in ? is[r] : 0u; }
+#pragma unroll
+    for (int u = 0; u < 8; ++u) {
+      const uint32_t r = r0 + u * kQThreads;
+      if (r >= n_in) continue;
+      uint32_t c = r * K / n_in;             // r < 2^26 and K <= 2^6: the product fits 32 bits
+      while (c + 1 < K && sm.bounds[c + 1] <= r) ++c;
+      while (c > 0 && sm.bounds[c] > r) --c;
+      codes8[dst[u]] = static_cast<uint8_t>(c);
+    }
   }
   if (n_out > 0) {
-    for (uint32_t i = tid; i < n; i += kQThreads) {
-      const float x = w[i];
-      if (!is_outlier(x, mu, var, c0)) continue;
-      uint32_t best = 0;
-      double bd = fabs(static_cast<double>(x) - static_cast<double>(sm.cents[0]));
-      for (uint32_t c = 1; c < K; ++c) {
-        const double dd = fabs(static_cast<double>(x) - static_cast<double>(sm.cents[c]));
-        if (dd < bd) { bd = dd; best = c; }
+    for (uint32_t i0 = tid; i0 < n; i0 += 8 * kQThreads) {
+      float v[8];
+#pragma unroll
+      for (int u = 0; u < 8; ++u) { const uint32_t i = i0 + u * kQThreads; v[u] = i < n ? w[i] : 0.f; }
+#pragma unroll
+      for (int u = 0; u < 8; ++u) {
+        const uint32_t i = i0 + u * kQThreads;
+        if (i >= n || !is_outlier(v[u], mu, inv2var, c0)) continue;
+        uint32_t best = 0;
+        double bd = fabs(static_cast<double>(v[u]) - static_cast<double>(sm.cents[0]));
+        for (uint32_t c = 1; c < K; ++c) {
+          const double dd = fabs(static_cast<double>(v[u]) - static_cast<double>(sm.cents[c]));
+          if (dd < bd) { bd = dd; best = c; }
+        }
+        codes8[i] = static_cast<uint8_t>(best);
       }
-      codes8[i] = static_cast<uint8_t>(best);
     }
   }
   __syncthreads();
 
-  // ---- 6. the index stream: word j holds stream bits [32 j, 32 j + 32)
-  const uint32_t n_words = static_cast<uint32_t>(static_cast<uint64_t>(n) * bits / 32);
-  for (uint32_t j = tid; j < n_words; j += kQThreads) {
-    const uint32_t bit0 = 32u * j;
-    uint32_t i = bit0 / bits;
-    const uint32_t used = bit0 - i * bits;             // bits of index i that belong to the previous word
-    uint32_t word = static_cast<uint32_t>(codes8[i]) >> used;
-    uint32_t pos = bits - used;
-    ++i;
-    while (pos < 32u) {
-      word |= static_cast<uint32_t>(codes8[i]) << pos;
-      pos += bits;
-      ++i;
+  // ---- 6. the index stream: 32 consecutive indexes are exactly `bits` words; a thread reads them as two 16-byte
+  //         loads and shifts them into a 64-bit window, emitting a word whenever 32 bits are complete
+  const uint32_t n_groups = n / 32;
+  for (uint32_t gidx = tid; gidx < n_groups; gidx += kQThreads) {
+    const uint4 a = *reinterpret_cast<const uint4*>(codes8 + static_cast<size_t>(gidx) * 32);
+    const uint4 b = *reinterpret_cast<const uint4*>(codes8 + static_cast<size_t>(gidx) * 32 + 16);
+    const uint32_t src[8] = {a.x, a.y, a.z, a.w, b.x, b.y, b.z, b.w};
+    uint64_t window = 0;
+    uint32_t fill = 0, out_w = gidx * bits;
+#pragma unroll
+    for (int e = 0; e < 32; ++e) {
+      const uint32_t code = (src[e >> 2] >> (8 * (e & 3))) & 255u;
+      window |= static_cast<uint64_t>(code) << fill;
+      fill += bits;
+      if (fill >= 32u) {
+        codes[out_w++] = static_cast<uint32_t>(window);
+        window >>= 32;
+        fill -= 32u;
+      }
     }
-    codes[j] = word;
   }
 }
 
@@ -268,7 +383,10 @@ sti_status sti_quantize_units(int device, void* stream, const float* w_dev, uint
     return STI_ERR_CUDA;
   }
   if (cudaSetDevice(device) != cudaSuccess) return STI_ERR_CUDA;
-  quantize_units_kernel<<<n_units, kQThreads, 0, static_cast<cudaStream_t>(stream)>>>(
+  if (cudaFuncSetAttribute(quantize_units_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                           static_cast<int>(sizeof(QuantShared))) != cudaSuccess)
+    return STI_ERR_CUDA;
+  quantize_units_kernel<<<n_units, kQThreads, sizeof(QuantShared), static_cast<cudaStream_t>(stream)>>>(
       w_dev, n_weights, bits, codes_dev, centroids_dev, outlier_off_dev, outlier_val_dev, max_outliers, n_outliers_dev,
       static_cast<uint8_t*>(workspace_dev), ws_per_unit_bytes(n_weights));
   return cudaGetLastError() == cudaSuccess ? STI_OK : STI_ERR_CUDA;
