@@ -18,6 +18,8 @@
 #include <cuda.h>
 #include <cuda_bf16.h>
 
+#include <type_traits>
+
 #include "gemm_device.cuh"
 
 namespace sti {
@@ -27,12 +29,70 @@ namespace {
 // ---------------------------------------------------------------------------------------
 // The kernel
 // ---------------------------------------------------------------------------------------
+// One accumulator tile's columns [half * ncol, (half + 1) * ncol) of this warp's 32 token rows: TMEM -> bias / erf-GELU -> global.
+template <typename OutT, bool GELU>
+__device__ __forceinline__ void epilogue_tile(uint32_t taddr, uint32_t half, uint32_t ncol, const float* bias_sm, OutT* drow,
+                                              bool row_ok, bool few_tiles) {
+    if (few_tiles) {
+      // 16 columns per step in a rolled loop: the epilogue runs once per tile, its code is fetched cold
+#pragma unroll 1
+      for (uint32_t col = half * ncol; col < (half + 1) * ncol; col += 16) {
+        uint32_t r[16];
+        tmem_ld_32x32b_x16(taddr + col, r);
+        tc_wait_ld();
+        if (row_ok) {
+          float v[16];
+#pragma unroll
+          for (int i = 0; i < 16; ++i) {
+            const float a = __uint_as_float(r[i]) + bias_sm[col + i];
+            v[i] = GELU ? gelu_erf(a) : a;
+          }
+          store_row16<OutT>(drow + col, v);
+        }
+      }
+    } else {
+      // many tiles per CTA: 32 columns per step, unrolled (each thread writes 128 or 64 contiguous bytes)
+      for (uint32_t col = half * ncol; col < (half + 1) * ncol; col += 32) {
+        if (col + 32 > (half + 1) * ncol) {            // 16-column tail of 32-row tiles
+          uint32_t r[16];
+          tmem_ld_32x32b_x16(taddr + col, r);
+          tc_wait_ld();
+          if (row_ok) {
+            float v[16];
+#pragma unroll
+            for (int i = 0; i < 16; ++i) {
+              const float a = __uint_as_float(r[i]) + bias_sm[col + i];
+              v[i] = GELU ? gelu_erf(a) : a;
+            }
+            store_row16<OutT>(drow + col, v);
+          }
+          break;
+        }
+        uint32_t r[32];
+        tmem_ld_32x32b_x32(taddr + col, r);
+        tc_wait_ld();
+        if (row_ok) {
+#pragma unroll
+          for (int h = 0; h < 2; ++h) {
+            float v[16];
+#pragma unroll
+            for (int i = 0; i < 16; ++i) {
+              const float a = __uint_as_float(r[h * 16 + i]) + bias_sm[col + h * 16 + i];
+              v[i] = GELU ? gelu_erf(a) : a;
+            }
+            store_row16<OutT>(drow + col + h * 16, v);
+          }
+        }
+      }
+    }
+}
+
 template <typename OutT, bool GELU, bool SIMT>
 __global__ void __launch_bounds__(kThreads, 1)
 dqgemm_kernel(const __grid_constant__ CUtensorMap xmap, const Job* __restrict__ jobs, const Seg* __restrict__ segs,
               const __nv_bfloat16* __restrict__ x, int ldx, int T, OutT* __restrict__ out, int ldo,
               const float* __restrict__ bias, int* __restrict__ err, uint32_t n_stages, uint32_t bps,
-              uint32_t w_bytes, uint32_t hdr_bytes, uint32_t seg_stride, PrefetchRanges pf) {
+              uint32_t w_bytes, uint32_t hdr_bytes, uint32_t seg_stride, PrefetchRanges pf, int kind) {
   extern __shared__ __align__(1024) uint8_t smem_raw[];
   uint8_t* smem = smem_raw;
   const uint32_t tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -246,59 +306,19 @@ dqgemm_kernel(const __grid_constant__ CUtensorMap xmap, const Job* __restrict__ 
         if (!ok) { failed = true; break; }
         tc_fence_after_sync();
         const int t = static_cast<int>((blockIdx.y + ti * gridDim.y) * kTileM + q * 32 + lane);
-        OutT* drow = out + (static_cast<size_t>(job.out_mat) * T + (t < T ? t : 0)) * ldo + job.out_col;
+        const size_t row_off = (static_cast<size_t>(job.out_mat) * T + (t < T ? t : 0)) * ldo + job.out_col;
         const uint32_t taddr = tmem_base + ((q * 32) << 16) + buf * n_rows;
-        if (my_mtiles <= 2) {
-          // 16 columns per step in a rolled loop: the epilogue runs once per tile, its code is fetched cold
-#pragma unroll 1
-          for (uint32_t col = half * ncol; col < (half + 1) * ncol; col += 16) {
-            uint32_t r[16];
-            tmem_ld_32x32b_x16(taddr + col, r);
-            tc_wait_ld();
-            if (t < T) {
-              float v[16];
-#pragma unroll
-              for (int i = 0; i < 16; ++i) {
-                const float a = __uint_as_float(r[i]) + bias_sm[col + i];
-                v[i] = GELU ? gelu_erf(a) : a;
-              }
-              store_row16<OutT>(drow + col, v);
-            }
-          }
+        if constexpr (std::is_void<OutT>::value) {
+          // one kernel for every GEMM of a layer: the output kind is a launch parameter, the code stays in the
+          // instruction caches from launch to launch
+          if (kind == GEMM_BF16_TO_F32)
+            epilogue_tile<float, false>(taddr, half, ncol, bias_sm, static_cast<float*>(out) + row_off, t < T, my_mtiles <= 2);
+          else if (kind == GEMM_BF16_TO_BF16_GELU)
+            epilogue_tile<__nv_bfloat16, true>(taddr, half, ncol, bias_sm, static_cast<__nv_bfloat16*>(out) + row_off, t < T, my_mtiles <= 2);
+          else
+            epilogue_tile<__nv_bfloat16, false>(taddr, half, ncol, bias_sm, static_cast<__nv_bfloat16*>(out) + row_off, t < T, my_mtiles <= 2);
         } else {
-          // many tiles per CTA: 32 columns per step, unrolled (each thread writes 128 or 64 contiguous bytes)
-          for (uint32_t col = half * ncol; col < (half + 1) * ncol; col += 32) {
-            if (col + 32 > (half + 1) * ncol) {            // 16-column tail of 32-row tiles
-              uint32_t r[16];
-              tmem_ld_32x32b_x16(taddr + col, r);
-              tc_wait_ld();
-              if (t < T) {
-                float v[16];
-#pragma unroll
-                for (int i = 0; i < 16; ++i) {
-                  const float a = __uint_as_float(r[i]) + bias_sm[col + i];
-                  v[i] = GELU ? gelu_erf(a) : a;
-                }
-                store_row16<OutT>(drow + col, v);
-              }
-              break;
-            }
-            uint32_t r[32];
-            tmem_ld_32x32b_x32(taddr + col, r);
-            tc_wait_ld();
-            if (t < T) {
-#pragma unroll
-              for (int h = 0; h < 2; ++h) {
-                float v[16];
-#pragma unroll
-                for (int i = 0; i < 16; ++i) {
-                  const float a = __uint_as_float(r[h * 16 + i]) + bias_sm[col + h * 16 + i];
-                  v[i] = GELU ? gelu_erf(a) : a;
-                }
-                store_row16<OutT>(drow + col + h * 16, v);
-              }
-            }
-          }
+          epilogue_tile<OutT, GELU>(taddr, half, ncol, bias_sm, out + row_off, t < T, my_mtiles <= 2);
         }
         tc_fence_before_sync();
         __syncwarp();
@@ -599,9 +619,14 @@ cudaError_t launch_t(const GemmLaunch& p, cudaStream_t s) {
   dim3 grid(p.n_jobs, p.m_ctas), block(kThreads);
   PrefetchRanges pf;
   for (int r = 0; r < 4; ++r) { pf.ptr[r] = p.pf_ptr[r]; pf.bytes[r] = p.pf_bytes[r]; }
+  const int kind = sizeof(OutT) == 4 ? GEMM_BF16_TO_F32 : (GELU ? GEMM_BF16_TO_BF16_GELU : GEMM_BF16_TO_BF16);
   if (p.simt_debug)
-    return launch_kernel(dqgemm_kernel<OutT, GELU, true>, grid, block, p.smem_bytes, s, p.pdl, p.xmap, p.jobs, p.segs, x, p.ldx, p.T, static_cast<OutT*>(p.out), p.ldo, p.bias, p.err, p.n_stages, p.bps, p.w_bytes, p.hdr_bytes, p.seg_stride, pf);
-  return launch_kernel(dqgemm_kernel<OutT, GELU, false>, grid, block, p.smem_bytes, s, p.pdl, p.xmap, p.jobs, p.segs, x, p.ldx, p.T, static_cast<OutT*>(p.out), p.ldo, p.bias, p.err, p.n_stages, p.bps, p.w_bytes, p.hdr_bytes, p.seg_stride, pf);
+    return launch_kernel(dqgemm_kernel<OutT, GELU, true>, grid, block, p.smem_bytes, s, p.pdl, p.xmap, p.jobs, p.segs, x, p.ldx,
+                         p.T, static_cast<OutT*>(p.out), p.ldo, p.bias, p.err, p.n_stages, p.bps, p.w_bytes, p.hdr_bytes,
+                         p.seg_stride, pf, kind);
+  // every output kind runs the same kernel (the kind is a parameter): one copy of the code for a layer's four GEMMs
+  return launch_kernel(dqgemm_kernel<void, false, false>, grid, block, p.smem_bytes, s, p.pdl, p.xmap, p.jobs, p.segs, x, p.ldx,
+                       p.T, p.out, p.ldo, p.bias, p.err, p.n_stages, p.bps, p.w_bytes, p.hdr_bytes, p.seg_stride, pf, kind);
 }
 
 template <typename K>
@@ -635,9 +660,9 @@ bool gemm_pick_ring(uint32_t w_bytes, uint32_t k_total, uint32_t hdr_bytes, uint
 cudaError_t gemm_configure() {
   cudaError_t e;
 #define STI_SET(OutT, G)                                                  \
-  if ((e = set_smem(dqgemm_kernel<OutT, G, false>)) != cudaSuccess) return e; \
   if ((e = set_smem(dqgemm_kernel<OutT, G, true>)) != cudaSuccess) return e;  \
   if ((e = set_smem(dqgemm_pair_kernel<OutT, G>)) != cudaSuccess) return e;
+  if ((e = set_smem(dqgemm_kernel<void, false, false>)) != cudaSuccess) return e;
   STI_SET(__nv_bfloat16, false)
   STI_SET(__nv_bfloat16, true)
   STI_SET(float, false)
