@@ -117,3 +117,30 @@ def test_argument_checks():
     with pytest.raises(sti.StiError) as e:
         sti.sti_quantize_units(w.data_ptr(), 1, 64, 4, p, p, p, p, 4, p, p, 100)
     assert e.value.status == 4
+
+
+def test_device_quantized_units_run_through_the_layer():
+    """fp32 weights -> sti_quantize_units -> sti_shard_upload -> sti_layer_forward, against the oracle's forward
+    on the oracle's own quantization of the same weights."""
+    from gpu_util import run_layer, rel_err, REL_TOL
+    from oracle import sti_oracle as O
+    from workloads.shards import ShardBlob
+    shape = W.ModelShape(n_layers=1, hidden=256, n_heads=4, head_dim=64, ffn=1024, n_ffn_slices=4)
+    bits_of = {ATTN: [2, 3, 5, 6], FFN: [4, 6, 3, 2]}
+    attn = [[W.UnitPlan(True, bits_of[ATTN][i], True) for i in range(4)]]
+    ffn = [[W.UnitPlan(True, bits_of[FFN][i], True) for i in range(4)]]
+    work = W.build_workload("quantized_on_device", shape, 1, 96, "f32", attn, ffn, seed=19, ring_slots=2)
+    blobs = {}
+    for (l, kind, idx), ref_blob in work.blobs.items():
+        flat = np.concatenate([m.reshape(-1) for m in make_unit_weights(shape, 19, l, kind, idx)])[None, :]
+        words, cents, off, val, cnt = _run(flat, ref_blob.bits)
+        n_out = int(cnt[0])
+        blobs[(l, kind, idx)] = ShardBlob(bits=ref_blob.bits, codes=words[0].copy(), centroids=cents[0].copy(),
+                                          outlier_off=off[0, :n_out].copy(), outlier_val=val[0, :n_out].copy())
+        assert np.array_equal(words[0], ref_blob.codes)          # the generator's blob is the same quantization
+    import dataclasses
+    work_dev = dataclasses.replace(work, blobs=blobs)
+    ref = O.run_workload(work)
+    with sti.Session(work_dev) as s:
+        y = run_layer(s, work_dev, 0)
+    assert rel_err(y, ref) <= REL_TOL
