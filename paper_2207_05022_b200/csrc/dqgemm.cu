@@ -30,13 +30,38 @@ namespace {
 // The kernel
 // ---------------------------------------------------------------------------------------
 // One accumulator tile's columns [half * ncol, (half + 1) * ncol) of this warp's 32 token rows: TMEM -> bias / erf-GELU -> global.
-template <typename OutT, bool GELU>
+// FEW (at most two token tiles per CTA): eight columns per step in a rolled loop - the epilogue then runs once or twice
+// per CTA, its instructions are fetched cold, and the kernel's code size is what it costs.  Otherwise 32 columns per step,
+// unrolled (each thread writes 128 or 64 contiguous bytes of its row).
+template <typename OutT, bool GELU, bool FEW>
 __device__ __forceinline__ void epilogue_tile(uint32_t taddr, uint32_t half, uint32_t ncol, const float* bias_sm, OutT* drow,
-                                              bool row_ok, bool few_tiles) {
-    if (few_tiles) {
-      // 16 columns per step in a rolled loop: the epilogue runs once per tile, its code is fetched cold
+                                              bool row_ok) {
+  if constexpr (FEW) {
 #pragma unroll 1
-      for (uint32_t col = half * ncol; col < (half + 1) * ncol; col += 16) {
+    for (uint32_t col = half * ncol; col < (half + 1) * ncol; col += 8) {
+      uint32_t r[8];
+      tmem_ld_32x32b_x8(taddr + col, r);
+      tc_wait_ld();
+      float v[8];
+#pragma unroll
+      for (int i = 0; i < 8; ++i) {
+        const float a = __uint_as_float(r[i]) + bias_sm[col + i];
+        v[i] = GELU ? gelu_erf(a) : a;
+      }
+      if constexpr (sizeof(OutT) == 2) {
+        const uint4 o = make_uint4(pack_bf16x2(v[0], v[1]), pack_bf16x2(v[2], v[3]), pack_bf16x2(v[4], v[5]),
+                                   pack_bf16x2(v[6], v[7]));
+        if (row_ok) *reinterpret_cast<uint4*>(drow + col) = o;
+      } else {
+        if (row_ok) {
+          reinterpret_cast<float4*>(drow + col)[0] = make_float4(v[0], v[1], v[2], v[3]);
+          reinterpret_cast<float4*>(drow + col)[1] = make_float4(v[4], v[5], v[6], v[7]);
+        }
+      }
+    }
+  } else {
+    for (uint32_t col = half * ncol; col < (half + 1) * ncol; col += 32) {
+      if (col + 32 > (half + 1) * ncol) {            // 16-column tail of 32-row tiles
         uint32_t r[16];
         tmem_ld_32x32b_x16(taddr + col, r);
         tc_wait_ld();
@@ -49,45 +74,28 @@ __device__ __forceinline__ void epilogue_tile(uint32_t taddr, uint32_t half, uin
           }
           store_row16<OutT>(drow + col, v);
         }
+        break;
       }
-    } else {
-      // many tiles per CTA: 32 columns per step, unrolled (each thread writes 128 or 64 contiguous bytes)
-      for (uint32_t col = half * ncol; col < (half + 1) * ncol; col += 32) {
-        if (col + 32 > (half + 1) * ncol) {            // 16-column tail of 32-row tiles
-          uint32_t r[16];
-          tmem_ld_32x32b_x16(taddr + col, r);
-          tc_wait_ld();
-          if (row_ok) {
-            float v[16];
+      uint32_t r[32];
+      tmem_ld_32x32b_x32(taddr + col, r);
+      tc_wait_ld();
+      if (row_ok) {
 #pragma unroll
-            for (int i = 0; i < 16; ++i) {
-              const float a = __uint_as_float(r[i]) + bias_sm[col + i];
-              v[i] = GELU ? gelu_erf(a) : a;
-            }
-            store_row16<OutT>(drow + col, v);
+        for (int h = 0; h < 2; ++h) {
+          float v[16];
+#pragma unroll
+          for (int i = 0; i < 16; ++i) {
+            const float a = __uint_as_float(r[h * 16 + i]) + bias_sm[col + h * 16 + i];
+            v[i] = GELU ? gelu_erf(a) : a;
           }
-          break;
-        }
-        uint32_t r[32];
-        tmem_ld_32x32b_x32(taddr + col, r);
-        tc_wait_ld();
-        if (row_ok) {
-#pragma unroll
-          for (int h = 0; h < 2; ++h) {
-            float v[16];
-#pragma unroll
-            for (int i = 0; i < 16; ++i) {
-              const float a = __uint_as_float(r[h * 16 + i]) + bias_sm[col + h * 16 + i];
-              v[i] = GELU ? gelu_erf(a) : a;
-            }
-            store_row16<OutT>(drow + col + h * 16, v);
-          }
+          store_row16<OutT>(drow + col + h * 16, v);
         }
       }
     }
+  }
 }
 
-template <typename OutT, bool GELU, bool SIMT>
+template <typename OutT, bool GELU, bool SIMT, bool FEW>
 __global__ void __launch_bounds__(kThreads, 1)
 dqgemm_kernel(const __grid_constant__ CUtensorMap xmap, const Job* __restrict__ jobs, const Seg* __restrict__ segs,
               const __nv_bfloat16* __restrict__ x, int ldx, int T, OutT* __restrict__ out, int ldo,
@@ -312,13 +320,13 @@ dqgemm_kernel(const __grid_constant__ CUtensorMap xmap, const Job* __restrict__ 
           // one kernel for every GEMM of a layer: the output kind is a launch parameter, the code stays in the
           // instruction caches from launch to launch
           if (kind == GEMM_BF16_TO_F32)
-            epilogue_tile<float, false>(taddr, half, ncol, bias_sm, static_cast<float*>(out) + row_off, t < T, my_mtiles <= 2);
+            epilogue_tile<float, false, FEW>(taddr, half, ncol, bias_sm, static_cast<float*>(out) + row_off, t < T);
           else if (kind == GEMM_BF16_TO_BF16_GELU)
-            epilogue_tile<__nv_bfloat16, true>(taddr, half, ncol, bias_sm, static_cast<__nv_bfloat16*>(out) + row_off, t < T, my_mtiles <= 2);
+            epilogue_tile<__nv_bfloat16, true, FEW>(taddr, half, ncol, bias_sm, static_cast<__nv_bfloat16*>(out) + row_off, t < T);
           else
-            epilogue_tile<__nv_bfloat16, false>(taddr, half, ncol, bias_sm, static_cast<__nv_bfloat16*>(out) + row_off, t < T, my_mtiles <= 2);
+            epilogue_tile<__nv_bfloat16, false, FEW>(taddr, half, ncol, bias_sm, static_cast<__nv_bfloat16*>(out) + row_off, t < T);
         } else {
-          epilogue_tile<OutT, GELU>(taddr, half, ncol, bias_sm, out + row_off, t < T, my_mtiles <= 2);
+          epilogue_tile<OutT, GELU, FEW>(taddr, half, ncol, bias_sm, out + row_off, t < T);
         }
         tc_fence_before_sync();
         __syncwarp();
@@ -621,12 +629,18 @@ cudaError_t launch_t(const GemmLaunch& p, cudaStream_t s) {
   for (int r = 0; r < 4; ++r) { pf.ptr[r] = p.pf_ptr[r]; pf.bytes[r] = p.pf_bytes[r]; }
   const int kind = sizeof(OutT) == 4 ? GEMM_BF16_TO_F32 : (GELU ? GEMM_BF16_TO_BF16_GELU : GEMM_BF16_TO_BF16);
   if (p.simt_debug)
-    return launch_kernel(dqgemm_kernel<OutT, GELU, true>, grid, block, p.smem_bytes, s, p.pdl, p.xmap, p.jobs, p.segs, x, p.ldx,
+    return launch_kernel(dqgemm_kernel<OutT, GELU, true, false>, grid, block, p.smem_bytes, s, p.pdl, p.xmap, p.jobs, p.segs, x, p.ldx,
                          p.T, static_cast<OutT*>(p.out), p.ldo, p.bias, p.err, p.n_stages, p.bps, p.w_bytes, p.hdr_bytes,
                          p.seg_stride, pf, kind);
-  // every output kind runs the same kernel (the kind is a parameter): one copy of the code for a layer's four GEMMs
-  return launch_kernel(dqgemm_kernel<void, false, false>, grid, block, p.smem_bytes, s, p.pdl, p.xmap, p.jobs, p.segs, x, p.ldx,
-                       p.T, p.out, p.ldo, p.bias, p.err, p.n_stages, p.bps, p.w_bytes, p.hdr_bytes, p.seg_stride, pf, kind);
+  // every output kind runs the same kernel (the kind is a parameter): one copy of the code for a layer's four GEMMs;
+  // two builds of it, for few and for many token tiles per CTA (they differ in the epilogue's shape)
+  const int n_mtiles = (p.T + kTileM - 1) / kTileM;
+  const bool few = (n_mtiles + p.m_ctas - 1) / p.m_ctas <= 2;
+  if (few)
+    return launch_kernel(dqgemm_kernel<void, false, false, true>, grid, block, p.smem_bytes, s, p.pdl, p.xmap, p.jobs, p.segs, x,
+                         p.ldx, p.T, p.out, p.ldo, p.bias, p.err, p.n_stages, p.bps, p.w_bytes, p.hdr_bytes, p.seg_stride, pf, kind);
+  return launch_kernel(dqgemm_kernel<void, false, false, false>, grid, block, p.smem_bytes, s, p.pdl, p.xmap, p.jobs, p.segs, x,
+                       p.ldx, p.T, p.out, p.ldo, p.bias, p.err, p.n_stages, p.bps, p.w_bytes, p.hdr_bytes, p.seg_stride, pf, kind);
 }
 
 template <typename K>
@@ -660,9 +674,10 @@ bool gemm_pick_ring(uint32_t w_bytes, uint32_t k_total, uint32_t hdr_bytes, uint
 cudaError_t gemm_configure() {
   cudaError_t e;
 #define STI_SET(OutT, G)                                                  \
-  if ((e = set_smem(dqgemm_kernel<OutT, G, true>)) != cudaSuccess) return e;  \
+  if ((e = set_smem(dqgemm_kernel<OutT, G, true, false>)) != cudaSuccess) return e;  \
   if ((e = set_smem(dqgemm_pair_kernel<OutT, G>)) != cudaSuccess) return e;
-  if ((e = set_smem(dqgemm_kernel<void, false, false>)) != cudaSuccess) return e;
+  if ((e = set_smem(dqgemm_kernel<void, false, false, true>)) != cudaSuccess) return e;
+  if ((e = set_smem(dqgemm_kernel<void, false, false, false>)) != cudaSuccess) return e;
   STI_SET(__nv_bfloat16, false)
   STI_SET(__nv_bfloat16, true)
   STI_SET(float, false)

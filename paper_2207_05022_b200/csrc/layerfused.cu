@@ -76,7 +76,7 @@ __device__ __forceinline__ bool grid_wait(unsigned int* ctr, unsigned int target
 // GEMM step, part 1: tables, bias and the decoded weight tile of this CTA's job.
 // Reads only weights, descriptors and parameters - may run before the data dependency is met.
 // ---------------------------------------------------------------------------------------
-__device__ __forceinline__ void gemm_prologue(const FusedGemm& g, int gi, uint32_t cta, uint8_t* smem, uint32_t slot_off,
+__device__ __noinline__ void gemm_prologue(const FusedGemm& g, int gi, uint32_t cta, uint8_t* smem, uint32_t slot_off,
                                               int* err, uint32_t tid) {
   FusedScratch* sc = reinterpret_cast<FusedScratch*>(smem + 256);
   const uint32_t n_items = static_cast<uint32_t>(g.n_jobs) * static_cast<uint32_t>(g.m_ctas);
@@ -123,7 +123,7 @@ __device__ __forceinline__ void drain_tile(uint32_t taddr, uint32_t col0, uint32
 }
 
 // Returns false when a bounded wait ran out.
-__device__ __forceinline__ bool gemm_main(const FusedGemm& g, int gi, uint32_t cta, int T, uint8_t* smem, uint32_t slot_off,
+__device__ __noinline__ bool gemm_main(const FusedGemm& g, int gi, uint32_t cta, int T, uint8_t* smem, uint32_t slot_off,
                                           uint32_t tmem_base, uint32_t tid, const FusedLayerParams* pf = nullptr) {
   SmemHeader* hdr = reinterpret_cast<SmemHeader*>(smem);
   FusedScratch* sc = reinterpret_cast<FusedScratch*>(smem + 256);
@@ -312,7 +312,7 @@ __device__ __forceinline__ float group_sum(float v, float* red, int gt, int n_wa
   return t;
 }
 
-__device__ __forceinline__ void layernorm_step(const LnLaunch& p, uint32_t cta, uint32_t n_ctas, uint8_t* smem, uint32_t tid) {
+__device__ __noinline__ void layernorm_step(const LnLaunch& p, uint32_t cta, uint32_t n_ctas, uint8_t* smem, uint32_t tid) {
   FusedScratch* sc = reinterpret_cast<FusedScratch*>(smem + 256);
   const int tpr = p.d / 4;                               // threads per row (a multiple of 32)
   const int groups = kThreads / tpr >= 2 ? 2 : 1;        // row groups per CTA

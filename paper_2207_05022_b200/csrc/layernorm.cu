@@ -16,6 +16,7 @@ __device__ __forceinline__ float block_sum(float v, float* red, int tid, int n_w
   if ((tid & 31) == 0) red[tid >> 5] = v;
   __syncthreads();
   float t = 0.f;
+#pragma unroll 1
   for (int w = 0; w < n_warps; ++w) t += red[w];
   __syncthreads();
   return t;
@@ -43,6 +44,7 @@ layernorm_kernel(LnLaunch p) {
   }
   const size_t pstride = static_cast<size_t>(p.T) * p.d;
   int q = 0;
+#pragma unroll 1
   for (; q + 4 <= p.n_partial; q += 4) {          // four independent loads at a time
     const float4 s0 = __ldg(reinterpret_cast<const float4*>(p.partial + (q + 0) * pstride + row + c));
     const float4 s1 = __ldg(reinterpret_cast<const float4*>(p.partial + (q + 1) * pstride + row + c));
@@ -51,6 +53,7 @@ layernorm_kernel(LnLaunch p) {
     a.x += (s0.x + s1.x) + (s2.x + s3.x); a.y += (s0.y + s1.y) + (s2.y + s3.y);
     a.z += (s0.z + s1.z) + (s2.z + s3.z); a.w += (s0.w + s1.w) + (s2.w + s3.w);
   }
+#pragma unroll 1
   for (; q < p.n_partial; ++q) {
     const float4 s = __ldg(reinterpret_cast<const float4*>(p.partial + q * pstride + row + c));
     a.x += s.x; a.y += s.y; a.z += s.z; a.w += s.w;
