@@ -33,6 +33,7 @@ struct Tuning {
   int qkv_n = 32, f1_n = 64, o_n = 64, o_group = 4, f2_n = 64, f2_group = 2;
   int cta_budget = 148;                // CTAs a GEMM launch may use when it splits the token tiles over CTAs
   int pair_min_tiles = 8;              // two-CTA GEMM from this many 128-token tiles on (0 = never)
+  int ln1_ctas = -1, ln2_ctas = -1;    // LayerNorm CTA counts: -1 = chosen per launch (see ln_ctas_hint), 0 = one row per CTA
   int fused_max_tokens = 0;            // whole-layer kernel up to this many tokens (0 = never; STI_TUNE turns it on)
 };
 
@@ -192,6 +193,8 @@ void parse_tuning(Tuning* t, int tmax, const sti_model_desc& d) {
         else if (k == "pair_min_tiles") t->pair_min_tiles = v;
         else if (k == "cta_budget") t->cta_budget = std::max(1, v);
         else if (k == "fused_max_tokens") t->fused_max_tokens = std::max(0, v);
+        else if (k == "ln1_ctas") t->ln1_ctas = std::max(-1, v);
+        else if (k == "ln2_ctas") t->ln2_ctas = std::max(-1, v);
       }
       pos = end + 1;
     }
@@ -473,6 +476,18 @@ sti_status enqueue_layer_fused(sti_plan* p, int li, const void* xq, const void* 
   return STI_OK;
 }
 
+// How many CTAs a LayerNorm launch should use, given the GEMM that follows it.  A GEMM CTA needs a whole SM and its
+// CTAs are launched while the LayerNorm runs (they decode their weights meanwhile) - on SMs that hold no LayerNorm
+// CTA.  With one row per CTA the LayerNorm of a few hundred tokens spreads over about 64 SMs; when the next GEMM
+// wants more than the other 84, its last CTAs start late and their decode lands on the critical path.  Then the
+// rows are packed into fewer CTAs (measured: 54.6 -> 50.9 us per BERT-large layer at 256 tokens).  Otherwise, and
+// for many tokens, one row per CTA is faster.
+int ln_ctas_hint(int tuned, int T, int next_gemm_ctas) {
+  if (tuned >= 0) return tuned;
+  if (T > 512 || next_gemm_ctas <= 84) return 0;
+  return std::max(32, 148 - next_gemm_ctas);
+}
+
 // The seven kernels of one layer on the compute stream.
 // `x_ready_bf16`: the bf16 copy of x already sits in p->x_bf16 (written by the previous layer's LayerNorm);
 // `want_next_bf16`: this layer's last kernel also writes y as bf16 into p->x_bf16 for the next layer.
@@ -528,6 +543,7 @@ sti_status enqueue_layer(sti_plan* p, int li, const void* x, void* y, int batch,
   ln.bias = dense + c->off_bo; ln.resid = x; ln.resid_bf16 = bf16_act ? 1 : 0;
   ln.gamma = dense + c->off_ln1g; ln.beta = dense + c->off_ln1b; ln.eps = d.ln_eps; ln.T = T; ln.d = d.hidden;
   ln.out_f32 = p->h1_f32; ln.out_bf16 = p->h1_bf16;
+  ln.ctas_hint = ln_ctas_hint(p->tune.ln1_ctas, T, ns > 0 ? L.f1.n_jobs * m_ctas_for(L.f1.n_jobs, T, p->tune.cta_budget) : 0);
   CUDA_TRY(launch_layernorm(ln, c->compute, c->pdl));
   c->launches++;
   L.k_ran[3] = true;
@@ -549,6 +565,14 @@ sti_status enqueue_layer(sti_plan* p, int li, const void* x, void* y, int batch,
   l2.gamma = dense + c->off_ln2g; l2.beta = dense + c->off_ln2b; l2.eps = d.ln_eps; l2.T = T; l2.d = d.hidden;
   l2.out_f32 = bf16_act ? nullptr : static_cast<float*>(y);
   l2.out_bf16 = bf16_act ? static_cast<uint16_t*>(y) : (want_next_bf16 ? p->x_bf16 : nullptr);
+  {
+    int next_ctas = 0;
+    if (next_layer >= 0 && next_layer < static_cast<int>(p->layers.size())) {
+      const GemmTable& q = p->layers[next_layer].qkv;
+      next_ctas = q.n_jobs * m_ctas_for(q.n_jobs, T, p->tune.cta_budget);
+    }
+    l2.ctas_hint = ln_ctas_hint(p->tune.ln2_ctas, T, next_ctas);
+  }
   CUDA_TRY(launch_layernorm(l2, c->compute, c->pdl));
   c->launches++;
   L.k_ran[6] = true;

@@ -2,6 +2,8 @@
 // (Section 2.1; Section 6: biases and layernorm parameters stay in fp32).
 // One CTA per token row, one float4 per thread (hidden / 4 threads): every load of a row is in
 // flight at once; mean and variance are two-pass over registers with a block reduction.
+#include <algorithm>
+
 #include <cuda_bf16.h>
 
 #include "sti_device.cuh"
@@ -70,6 +72,101 @@ layernorm_kernel(LnLaunch p) {
     *reinterpret_cast<uint2*>(p.out_bf16 + row + c) = make_uint2(pack_bf16x2(y.x, y.y), pack_bf16x2(y.z, y.w));
 }
 
+// Few tokens: the same arithmetic with several rows per CTA and several float4 per thread, so that the kernel
+// sits on a handful of SMs only.  A GEMM CTA needs a whole SM; the CTAs of the GEMM that follows are launched while
+// this kernel runs (programmatic dependent launch) and decode their weights meanwhile - but only on SMs that hold
+// none of this kernel's CTAs.  A row is handled by `wpr` warps (named barrier = row slot, 0..15; the kernel uses
+// no CTA-wide barrier), thread t of the row holds float4 number t, t + tpr, ... of it.
+constexpr int kLnMaxV = 4;
+template <int V>
+__global__ void __launch_bounds__(1024)
+layernorm_rows_kernel(LnLaunch p, int tpr, int rows_per_cta) {
+  __shared__ float red_all[16][16];
+  const int slot = threadIdx.x / tpr, tid = threadIdx.x % tpr;
+  const int n_warps = tpr >> 5;
+  const int r = blockIdx.x * rows_per_cta + slot;
+  pdl_launch_dependents();
+  if (slot >= rows_per_cta || r >= p.T) {      // whole warps: tpr is a multiple of 32
+    pdl_wait();
+    return;
+  }
+  float* red = red_all[slot];
+  const size_t row = static_cast<size_t>(r) * p.d;
+  float4 a[V];
+#pragma unroll
+  for (int v = 0; v < V; ++v) a[v] = __ldg(reinterpret_cast<const float4*>(p.bias + (tid + v * tpr) * 4));
+  pdl_wait();
+  const size_t pstride = static_cast<size_t>(p.T) * p.d;
+#pragma unroll
+  for (int v = 0; v < V; ++v) {
+    {
+      const int c = (tid + v * tpr) * 4;
+      if (p.resid_bf16) {
+        const uint2 rr = __ldg(reinterpret_cast<const uint2*>(static_cast<const uint16_t*>(p.resid) + row + c));
+        a[v].x += __uint_as_float(rr.x << 16); a[v].y += __uint_as_float(rr.x & 0xffff0000u);
+        a[v].z += __uint_as_float(rr.y << 16); a[v].w += __uint_as_float(rr.y & 0xffff0000u);
+      } else {
+        const float4 rr = __ldg(reinterpret_cast<const float4*>(static_cast<const float*>(p.resid) + row + c));
+        a[v].x += rr.x; a[v].y += rr.y; a[v].z += rr.z; a[v].w += rr.w;
+      }
+      int q = 0;
+#pragma unroll 1
+      for (; q + 4 <= p.n_partial; q += 4) {          // same grouping of the partial sums as the one-row kernel
+        const float4 s0 = __ldg(reinterpret_cast<const float4*>(p.partial + (q + 0) * pstride + row + c));
+        const float4 s1 = __ldg(reinterpret_cast<const float4*>(p.partial + (q + 1) * pstride + row + c));
+        const float4 s2 = __ldg(reinterpret_cast<const float4*>(p.partial + (q + 2) * pstride + row + c));
+        const float4 s3 = __ldg(reinterpret_cast<const float4*>(p.partial + (q + 3) * pstride + row + c));
+        a[v].x += (s0.x + s1.x) + (s2.x + s3.x); a[v].y += (s0.y + s1.y) + (s2.y + s3.y);
+        a[v].z += (s0.z + s1.z) + (s2.z + s3.z); a[v].w += (s0.w + s1.w) + (s2.w + s3.w);
+      }
+#pragma unroll 1
+      for (; q < p.n_partial; ++q) {
+        const float4 s = __ldg(reinterpret_cast<const float4*>(p.partial + q * pstride + row + c));
+        a[v].x += s.x; a[v].y += s.y; a[v].z += s.z; a[v].w += s.w;
+      }
+    }
+  }
+  auto row_sum = [&](float v) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    if ((tid & 31) == 0) red[tid >> 5] = v;
+    asm volatile("bar.sync %0, %1;" ::"r"(slot), "r"(tpr) : "memory");
+    float t = 0.f;
+#pragma unroll 1
+    for (int w = 0; w < n_warps; ++w) t += red[w];
+    asm volatile("bar.sync %0, %1;" ::"r"(slot), "r"(tpr) : "memory");
+    return t;
+  };
+  float part = 0.f;
+#pragma unroll
+  for (int v = 0; v < V; ++v) part += a[v].x + a[v].y + a[v].z + a[v].w;
+  const float mean = row_sum(part) / static_cast<float>(p.d);
+  part = 0.f;
+#pragma unroll
+  for (int v = 0; v < V; ++v) {
+    {
+      a[v].x -= mean; a[v].y -= mean; a[v].z -= mean; a[v].w -= mean;
+      part += a[v].x * a[v].x + a[v].y * a[v].y + a[v].z * a[v].z + a[v].w * a[v].w;
+    }
+  }
+  const float var = row_sum(part) / static_cast<float>(p.d);
+  const float rstd = rsqrtf(var + p.eps);
+#pragma unroll
+  for (int v = 0; v < V; ++v) {
+    {
+      const int c = (tid + v * tpr) * 4;
+      const float4 g = __ldg(reinterpret_cast<const float4*>(p.gamma + c));
+      const float4 b = __ldg(reinterpret_cast<const float4*>(p.beta + c));
+      float4 y;
+      y.x = a[v].x * rstd * g.x + b.x; y.y = a[v].y * rstd * g.y + b.y;
+      y.z = a[v].z * rstd * g.z + b.z; y.w = a[v].w * rstd * g.w + b.w;
+      if (p.out_f32) *reinterpret_cast<float4*>(p.out_f32 + row + c) = y;
+      if (p.out_bf16)
+        *reinterpret_cast<uint2*>(p.out_bf16 + row + c) = make_uint2(pack_bf16x2(y.x, y.y), pack_bf16x2(y.z, y.w));
+    }
+  }
+}
+
 __global__ void cast_bf16_kernel(const float* __restrict__ in, uint16_t* __restrict__ out, size_t n4) {
   const size_t i = static_cast<size_t>(blockIdx.x) * blockDim.x + threadIdx.x;
   pdl_launch_dependents();
@@ -84,6 +181,27 @@ __global__ void cast_bf16_kernel(const float* __restrict__ in, uint16_t* __restr
 cudaError_t launch_layernorm(const LnLaunch& p, cudaStream_t s, bool pdl) {
   if (p.T <= 0) return cudaSuccess;
   if (p.d % 128 != 0 || p.d > 2048) return cudaErrorInvalidValue;     // d / 4 threads, whole warps
+  if (p.ctas_hint > 0 && p.ctas_hint < p.T) {
+    // the widest row group (fewest float4 per thread) whose CTA count stays within the hint
+    const int n4 = p.d / 4;
+    int tpr = 0;
+    for (int cand = n4; cand >= 32; cand -= 32) {
+      if (n4 % cand != 0 || (n4 / cand != 1 && n4 / cand != 2 && n4 / cand != 4)) continue;
+      const int rows = std::min(16, 1024 / cand);
+      tpr = cand;
+      if ((p.T + rows - 1) / rows <= p.ctas_hint) break;
+    }
+    if (tpr > 0) {
+      const int rows = std::min(16, 1024 / tpr);
+      const dim3 grid((p.T + rows - 1) / rows), block(rows * tpr);
+      switch (n4 / tpr) {
+        case 1: return launch_kernel(layernorm_rows_kernel<1>, grid, block, 0, s, pdl, p, tpr, rows);
+        case 2: return launch_kernel(layernorm_rows_kernel<2>, grid, block, 0, s, pdl, p, tpr, rows);
+        case 4: return launch_kernel(layernorm_rows_kernel<4>, grid, block, 0, s, pdl, p, tpr, rows);
+        default: break;
+      }
+    }
+  }
   return launch_kernel(layernorm_kernel, dim3(p.T), dim3(p.d / 4), 0, s, pdl, p);
 }
 

@@ -93,6 +93,7 @@ struct LnLaunch {
   int T, d;
   float* out_f32;           // optional
   uint16_t* out_bf16;       // optional
+  int ctas_hint;            // > 0: pack rows so that about this many CTAs are launched (few tokens); 0: one row per CTA
 };
 cudaError_t launch_layernorm(const LnLaunch& p, cudaStream_t s, bool pdl);
 
