@@ -480,11 +480,11 @@ sti_status enqueue_layer_fused(sti_plan* p, int li, const void* xq, const void* 
 // CTAs are launched while the LayerNorm runs (they decode their weights meanwhile) - on SMs that hold no LayerNorm
 // CTA.  With one row per CTA the LayerNorm of a few hundred tokens spreads over about 64 SMs; when the next GEMM
 // wants more than the other 84, its last CTAs start late and their decode lands on the critical path.  Then the
-// rows are packed into fewer CTAs (measured: 54.6 -> 50.9 us per BERT-large layer at 256 tokens).  Otherwise, and
-// for many tokens, one row per CTA is faster.
+// rows are packed into fewer CTAs (measured: 54.6 -> 50.5 us per BERT-large layer at 256 tokens; at 512 tokens
+// packing loses 1-3 us, at BERT-base sizes it changes nothing).  Otherwise one row per CTA.
 int ln_ctas_hint(int tuned, int T, int next_gemm_ctas) {
   if (tuned >= 0) return tuned;
-  if (T > 512 || next_gemm_ctas <= 84) return 0;
+  if (T > 256 || next_gemm_ctas <= 84) return 0;      // at 512 tokens the packed LayerNorm itself costs more than it frees
   return std::max(32, 148 - next_gemm_ctas);
 }
 
