@@ -93,3 +93,23 @@ def test_key_split_attention_long_sequence_and_mask():
     with sti.Session(work) as s:
         y = run_model(s, work, lens=lens)
     assert rel_err(y, ref) <= REL_TOL
+
+
+@pytest.mark.parametrize("hint", ["ln1_ctas=8,ln2_ctas=8", "ln1_ctas=20,ln2_ctas=64"])
+def test_packed_layernorm_on_bert_base_width(hint):
+    """hidden 768: 192 float4 per row, packed as 5 rows x 192 threads or 10 rows x 96 threads (two float4 per thread)."""
+    from gpu_util import run_model, rel_err, REL_TOL
+    shape = W.ModelShape(n_layers=2, hidden=768, n_heads=12, head_dim=64, ffn=3072, n_ffn_slices=12)
+    attn = [[W.UnitPlan(i % 3 != 2, 2 + (i + l) % 5, True) for i in range(12)] for l in range(2)]
+    ffn = [[W.UnitPlan(i % 4 != 1, 2 + (2 * i + l) % 5, True) for i in range(12)] for l in range(2)]
+    work = W.build_workload("ln_packed", shape, 1, 100, "bf16", attn, ffn, seed=53, ring_slots=2, workers=2)
+    ref = O.run_workload(work)
+
+    def run():
+        with sti.Session(work) as s:
+            return run_model(s, work)
+
+    y = _with_env({"STI_TUNE": hint}, run)
+    y_plain = _with_env({"STI_TUNE": "ln1_ctas=0,ln2_ctas=0"}, run)
+    assert rel_err(y, ref) <= REL_TOL
+    assert rel_err(y, y_plain) <= 5e-3

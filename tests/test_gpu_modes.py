@@ -67,7 +67,9 @@ def test_tile_shapes_do_not_change_results_beyond_rounding():
     from gpu_util import rel_err, REL_TOL
     work = _workload()
     ref = O.run_workload(work)
-    for tune in ("qkv_n=32,f1_n=32,o_group=1,f2_group=1", "qkv_n=64,f1_n=128,o_group=16,f2_group=4,f2_n=128,o_n=128"):
+    for tune in ("qkv_n=32,f1_n=32,o_group=1,f2_group=1", "qkv_n=64,f1_n=128,o_group=16,f2_group=4,f2_n=128,o_n=128",
+                 "ln1_ctas=1,ln2_ctas=40",        # LayerNorm rows packed 16 per CTA / two float4 per thread
+                 "ln1_ctas=0,ln2_ctas=0"):        # one row per CTA
         y, _ = _run(work, {"STI_TUNE": tune})
         assert rel_err(y, ref) <= REL_TOL, tune
 
