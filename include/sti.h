@@ -173,11 +173,52 @@ sti_status sti_sync(sti_ctx* ctx);
 sti_status sti_shard_decode(sti_plan* plan, int layer, sti_kind kind, int index, int matrix,
                             float* w_dev, uint8_t* codes_dev, uint16_t* wbf16_dev);
 
+/* Section 4.2 (decompression feeds the layer's linear maps directly): runs ONE of a layer's four fused
+ * dequant-GEMMs by itself, on activations the caller supplies, with the tile tables, the decode routine and
+ * the kernel that a forward uses: out = x W^T, no bias, no activation function.  It is the parity hook for
+ * the decode that lives inside the GEMM: with x = the identity matrix the output holds, bit for bit, the
+ * bf16 (round-to-nearest-even) dequantized weights the tensor cores were given (each output element is one
+ * exact product 1 * w).
+ *   gemm       : 0 = QKV, 1 = O projection, 2 = FFN1, 3 = FFN2, over the layer's kept units in index order
+ *   x_bf16_dev : DEVICE, [tokens, K] bf16 row-major, 16-byte aligned; K = hidden (QKV, FFN1),
+ *                64 * kept heads (O), f * kept slices (FFN2); tokens need not respect max_batch * max_seq
+ *   out_dev    : DEVICE, 16-byte aligned, caller-owned:
+ *                QKV  bf16 [(kept head * 3 + {Q,K,V})][tokens][64]
+ *                FFN1 bf16 [tokens][kept slices * f]
+ *                O, FFN2  fp32 [n_partials][tokens][hidden]: the K range is split over n_partials groups of
+ *                         units, each group writes its own partial sum (the caller adds them up)
+ *   out_capacity_bytes : size of out_dev; STI_ERR_SIZE when the result would not fit
+ *   variant    : 0 = the kernel a forward would choose for this token count, 1 = the one-CTA kernel,
+ *                2 = the two-CTA (cta_group::2) kernel, STI_ERR_STATE when the tiling does not allow it,
+ *                3 = the one-CTA kernel on the tile tables that the O projection and FFN2 use when bias,
+ *                    residual and LayerNorm run in their epilogue (same fp32 partial output as 1)
+ *   n_partials : optional out
+ * STI_ERR_STATE when no kept unit feeds the GEMM.  A streamed layer is copied first.  Asynchronous. */
+sti_status sti_gemm_probe(sti_plan* plan, int layer, int gemm, const void* x_bf16_dev, int tokens, void* out_dev,
+                          size_t out_capacity_bytes, int variant, int32_t* n_partials);
+
 /* Section 5.2 (profiling of IO and compute delays): per-layer timings of the last
  * sti_model_forward.  Enable with sti_plan_set_profiling before that forward: level 0 = off,
- * 1 = per-layer events, 2 = additionally events around every kernel (slightly slower). */
+ * 1 = per-layer events, 2 = additionally events around every kernel (slightly slower; levels 1 and 2 launch
+ * the kernels one by one instead of replaying a CUDA graph), 3 = device-timer stamps written by the kernels
+ * themselves (read with sti_get_kernel_stamps; sti_get_stats has nothing to report at this level). */
 sti_status sti_plan_set_profiling(sti_plan* plan, int level);
 sti_status sti_get_stats(sti_plan* plan, sti_stats* out);
+
+/* Section 5.2, kernel by kernel and in the execution mode that is timed: with profiling level 3 a forward runs as
+ * usual (CUDA graph replay, kernels launched ahead of their predecessors' end) and every kernel additionally
+ * stamps the device's nanosecond timer into a record of its own.  sti_get_kernel_stamps waits for the context and
+ * copies the records of the last such forward to `out` (HOST): [layer][kernel][word], STI_STAMP_KERNELS kernels per
+ * layer in execution order (fp32->bf16 cast of the model input, QKV, attention, O projection, LayerNorm 1, FFN1,
+ * FFN2, LayerNorm 2), STI_STAMP_WORDS words per kernel, times in ns on the device timer, 0 = not stamped (the
+ * kernel did not run: dropped units, LayerNorm merged into the preceding GEMM):
+ *   word 0 first CTA started          1 first CTA past the wait for the preceding kernel   2 last CTA finished
+ *   word 3 last weight tile decoded   4 last CTA started      5 accumulators complete      6 row statistics exchanged
+ *   (3: dequant-GEMMs only; 5, 6: dequant-GEMMs with the LayerNorm epilogue only; 7 unused)
+ * capacity_words must be at least n_layers * STI_STAMP_KERNELS * STI_STAMP_WORDS (STI_ERR_SIZE otherwise). */
+#define STI_STAMP_KERNELS 8
+#define STI_STAMP_WORDS 8
+sti_status sti_get_kernel_stamps(sti_plan* plan, uint64_t* out, size_t capacity_words, int32_t* n_layers);
 
 /* Section 7.1 (the Load&Exec baseline "loads model as a whole and executes it"): with overlap = 0 a model
  * forward first copies every streamed layer into its ring slot and only then starts layer 0, so IO and

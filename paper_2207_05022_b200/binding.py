@@ -81,7 +81,9 @@ def load_library():
         "sti_model_forward_host": ([vp, vp, vp, i32, i32, vp], i32),
         "sti_sync": ([vp], i32),
         "sti_shard_decode": ([vp, i32, i32, i32, i32, vp, vp, vp], i32),
+        "sti_gemm_probe": ([vp, i32, i32, vp, i32, vp, C.c_size_t, i32, C.POINTER(C.c_int32)], i32),
         "sti_plan_set_profiling": ([vp, i32], i32),
+        "sti_get_kernel_stamps": ([vp, vp, C.c_size_t, C.POINTER(C.c_int32)], i32),
         "sti_plan_set_overlap": ([vp, i32], i32),
         "sti_get_stats": ([vp, C.POINTER(StiStats)], i32),
         "sti_plan_memory": ([vp, u64p, u64p, u64p], i32),
@@ -101,7 +103,7 @@ def load_library():
 
 EXPORTED = ("sti_ctx_create", "sti_ctx_destroy", "sti_ctx_set_layer_params", "sti_plan_create",
             "sti_plan_destroy", "sti_shard_upload", "sti_plan_finalize", "sti_layer_forward",
-            "sti_model_forward", "sti_model_forward_host", "sti_sync", "sti_shard_decode",
+            "sti_model_forward", "sti_model_forward_host", "sti_sync", "sti_shard_decode", "sti_gemm_probe", "sti_get_kernel_stamps",
             "sti_plan_set_profiling", "sti_plan_set_overlap", "sti_get_stats", "sti_plan_memory", "sti_ctx_launch_count",
             "sti_host_retile", "sti_strerror", "sti_matrix_decode_noalloc", "sti_plan_auto",
             "sti_preload_after_run", "sti_quantize_units", "sti_quantize_workspace_bytes")
@@ -205,9 +207,30 @@ def sti_shard_decode(plan: int, layer: int, kind: int, index: int, matrix: int, 
            "sti_shard_decode")
 
 
+def sti_gemm_probe(plan: int, layer: int, gemm: int, x_bf16_dev: int, tokens: int, out_dev: int,
+                   out_capacity_bytes: int, variant: int = 0) -> int:
+    """One fused dequant-GEMM of a layer on the caller's activations (see sti.h); returns n_partials."""
+    n = C.c_int32(0)
+    _check(load_library().sti_gemm_probe(C.c_void_p(plan), layer, gemm, C.c_void_p(x_bf16_dev), tokens,
+                                         C.c_void_p(out_dev), out_capacity_bytes, variant, C.byref(n)), "sti_gemm_probe")
+    return int(n.value)
+
+
 def sti_plan_set_profiling(plan: int, level: int):
     """0 = off, 1 = per-layer events, 2 = events around every kernel."""
     _check(load_library().sti_plan_set_profiling(C.c_void_p(plan), int(level)), "sti_plan_set_profiling")
+
+
+STI_STAMP_KERNELS, STI_STAMP_WORDS = 8, 8
+STAMP_KERNEL_NAMES = ("cast", "qkv", "attention", "o_proj", "layernorm1", "ffn1", "ffn2", "layernorm2")
+
+
+def sti_get_kernel_stamps(plan: int, n_layers: int) -> np.ndarray:
+    """uint64 [n_layers, STI_STAMP_KERNELS, STI_STAMP_WORDS] of the last forward run at profiling level 3 (see sti.h)."""
+    out = np.zeros((n_layers, STI_STAMP_KERNELS, STI_STAMP_WORDS), np.uint64)
+    n = C.c_int32(0)
+    _check(load_library().sti_get_kernel_stamps(C.c_void_p(plan), _ptr(out), out.size, C.byref(n)), "sti_get_kernel_stamps")
+    return out[:n.value]
 
 
 def sti_plan_set_overlap(plan: int, overlap: bool):

@@ -20,6 +20,10 @@ namespace {
 
 constexpr int kMaxLayersStats = 64;
 constexpr size_t kMaxSmem = 227 * 1024;
+constexpr int kStampKernels = 8;       // per layer: cast, QKV, attention, O projection, LayerNorm 1, FFN1, FFN2, LayerNorm 2
+constexpr int kStampRecord = 8;        // 64-bit words per kernel launch (kStampWords of the device code)
+constexpr int kLnCounters = 64;        // arrival counters per LayerNorm epilogue launch (token-tile groups x cluster ranks)
+constexpr int kLnMaxTiles = 32;        // most column tiles of a row (hidden <= 2048, 64-feature tiles)
 
 inline size_t align16(size_t v) { return (v + 15) & ~static_cast<size_t>(15); }
 inline size_t align256(size_t v) { return (v + 255) & ~static_cast<size_t>(255); }
@@ -34,7 +38,8 @@ struct Tuning {
   int cta_budget = 148;                // CTAs a GEMM launch may use when it splits the token tiles over CTAs
   int pair_min_tiles = 8;              // two-CTA GEMM from this many 128-token tiles on (0 = never)
   int ln1_ctas = -1, ln2_ctas = -1;    // LayerNorm CTA counts: -1 = chosen per launch (see ln_ctas_hint), 0 = one row per CTA
-  int fused_max_tokens = 0;            // whole-layer kernel up to this many tokens (0 = never; STI_TUNE turns it on)
+  int ln_fuse = 0;                     // residual + LayerNorm in the epilogue of the O projection and of FFN2 (few tokens)
+  int ln_o_split = 8, ln_f2_split = 8; // most K splits (= CTAs per cluster) of a column tile in that form
 };
 
 struct Unit {
@@ -56,7 +61,6 @@ struct GemmTable {
   uint32_t w_bytes = 0, n_stages = 0, bps = 1, k_max = 0, hdr_bytes = 0, seg_stride = 0;
   bool pair_ok = false;                // consecutive jobs can share two-CTA MMAs (64-row tiles, same K range)
   int n_split = 0;
-  uint32_t f_stages = 0, f_bps = 0;    // activation ring inside the whole-layer kernel (0: the tile does not fit there)
 };
 
 struct Layer {
@@ -68,6 +72,7 @@ struct Layer {
   int slot = -1;                       // ring slot of the streamed part
   size_t tables_off = 0, tables_bytes = 0;   // this layer's tile-job descriptors inside the plan's table buffer
   GemmTable qkv, o, f1, f2;
+  GemmTable o_ln, f2_ln;               // O projection / FFN2 tiled for the LayerNorm epilogue (K splits of a column tile adjacent)
   cudaEvent_t ev_loaded = nullptr, ev_done = nullptr, ev_copy_start = nullptr, ev_comp_start = nullptr;
   cudaEvent_t g_ev_loaded = nullptr;   // the same role inside graph capture (captured events cannot be reused outside)
   cudaEvent_t ev_k[8] = {};           // boundaries of the seven kernels (kernel-level profiling)
@@ -89,6 +94,8 @@ struct sti_ctx {
   uint64_t launches = 0;
   bool simt_debug = false;
   bool pdl = true;                     // programmatic dependent launch between the kernels of a layer
+  int sm_count = 0;
+  int max_clusters[9] = {};            // clusters of 1..8 full-shared-memory GEMM CTAs the device holds at once
   sti_status async_error = STI_OK;
   MatrixInfo attn_m[4]{}, ffn_m[2]{};
   uint32_t attn_weights = 0, ffn_weights = 0;
@@ -100,8 +107,9 @@ struct ForwardKey {
   const int32_t* lens = nullptr;                         // device
   int batch = 0, seq = 0;
   int layer = -1;                                        // >= 0: a single layer (sti_layer_forward)
+  bool stamps = false;                                   // kernels write profiling stamps (profiling level 3)
   bool operator==(const ForwardKey& o) const {
-    return layer == o.layer && x == o.x && y == o.y && x_host == o.x_host && y_host == o.y_host && lens == o.lens && batch == o.batch &&
+    return stamps == o.stamps && layer == o.layer && x == o.x && y == o.y && x_host == o.x_host && y_host == o.y_host && lens == o.lens && batch == o.batch &&
            seq == o.seq;
   }
 };
@@ -132,8 +140,13 @@ struct sti_plan {
   void* buf[2] = {nullptr, nullptr};
   void* x_in = nullptr; void* y_out = nullptr; int32_t* lens_dev = nullptr;
   int max_partial = 1;
-  unsigned int* fused_ctr = nullptr;   // one grid-barrier counter per layer, zeroed at the start of every forward
-  bool fused_off = false;
+  float* zero_bias = nullptr;          // all-zero bias vector of sti_gemm_probe (allocated by its first call)
+  // LayerNorm epilogue scratch: arrival counters (per layer and LayerNorm, zeroed at the start of every forward) and the
+  // per-column-tile row statistics of the two LayerNorms
+  unsigned int* ln_ctr = nullptr;
+  unsigned long long* stamps = nullptr;   // [layer][kStampKernels][kStampWords] device, profiling level 3
+  bool stamping = false;               // the forward being enqueued writes stamps
+  float2* ln_stats[2] = {nullptr, nullptr};
   bool overlap = true;                 // false: load every streamed layer, then execute (Load&Exec)
   int n_streamed_layers = 0;
   bool stats_valid = false;
@@ -164,9 +177,10 @@ size_t matrix_code_bytes(const MatrixInfo& m, int bits) {
   return static_cast<size_t>(m.rows) * m.kc * bits / 8;
 }
 
-void parse_tuning(Tuning* t, int tmax, const sti_model_desc& d) {
-  // more, smaller tiles when there are few tokens (spread the decode over all SMs);
-  // wider tiles when each decoded weight is reused by many token tiles
+void parse_tuning(Tuning* t, int tmax, const sti_model_desc& d, int sm_count) {
+  t->cta_budget = sm_count;
+  // few tokens: K groups of 8 heads / 2 FFN slices, one CTA per token tile (the decode is spread over the SMs, MMA
+  // chains stay short); many tokens: wide K groups, each CTA walks many token tiles with its decoded weights
   if (tmax > 1024) {
     t->qkv_n = 64; t->f1_n = 64; t->o_n = 64; t->o_group = 16; t->f2_n = 64; t->f2_group = 4;
   } else {
@@ -192,7 +206,9 @@ void parse_tuning(Tuning* t, int tmax, const sti_model_desc& d) {
         else if (k == "f2_group") t->f2_group = v;
         else if (k == "pair_min_tiles") t->pair_min_tiles = v;
         else if (k == "cta_budget") t->cta_budget = std::max(1, v);
-        else if (k == "fused_max_tokens") t->fused_max_tokens = std::max(0, v);
+        else if (k == "ln_fuse") t->ln_fuse = v != 0;
+        else if (k == "ln_o_split") t->ln_o_split = std::max(1, std::min(8, v));
+        else if (k == "ln_f2_split") t->ln_f2_split = std::max(1, std::min(8, v));
         else if (k == "ln1_ctas") t->ln1_ctas = std::max(-1, v);
         else if (k == "ln2_ctas") t->ln2_ctas = std::max(-1, v);
       }
@@ -275,7 +291,7 @@ struct TableBuilder {
   }
 };
 
-void build_layer_tables(sti_plan* p, Layer& L, TableBuilder tb[4]) {
+void build_layer_tables(sti_plan* p, Layer& L, TableBuilder tb[6]) {
   const sti_ctx* c = p->ctx;
   const sti_model_desc& d = c->desc;
   const Tuning& t = p->tune;
@@ -333,6 +349,35 @@ void build_layer_tables(sti_plan* p, Layer& L, TableBuilder tb[4]) {
       tb[3].add(j, ss);
     }
   }
+  // The same two GEMMs tiled for the LayerNorm epilogue: the K splits of a column tile are adjacent jobs (one
+  // thread-block cluster), at most 8 of them, and column tiles times splits stay within the CTA budget.
+  auto ln_tables = [&](TableBuilder& out, GemmTable& gt, const std::vector<int>& kept, std::vector<Unit>& units,
+                       sti_kind kind, int matrix, uint32_t tile_n, uint32_t unit_k, int max_split) {
+    const int n = static_cast<int>(kept.size());
+    gt.n_split = 0;
+    if (n == 0 || (tile_n != 64 && tile_n != 128)) return;
+    const int n_nt = d.hidden / static_cast<int>(tile_n);
+    int c_target = std::max(1, std::min(std::min(8, max_split), t.cta_budget / std::max(1, n_nt)));
+    while (c_target > 1 && c->max_clusters[c_target] < n_nt) --c_target;     // every column tile's cluster resident at once
+    int group = (n + c_target - 1) / c_target;
+    // the tile of one split must fit in shared memory next to a small activation ring
+    while (group > 1 && gemm_weight_bytes(tile_n, group * unit_k) > 128 * 1024) --group;
+    gt.n_split = (n + group - 1) / group;
+    if (gt.n_split > 8) { gt.n_split = 0; return; }
+    for (uint32_t n0 = 0; n0 < static_cast<uint32_t>(d.hidden); n0 += tile_n)
+      for (int sp = 0; sp < gt.n_split; ++sp) {
+        const int first = sp * group, cnt = std::min(group, n - first);
+        Job j{};
+        j.n_rows = tile_n; j.k_total = cnt * unit_k; j.x_koff = first * unit_k;
+        j.out_mat = sp; j.out_col = n0; j.bias_off = -1;
+        std::vector<Seg> ss;
+        for (int i = 0; i < cnt; ++i)
+          ss.push_back(make_seg(c, units[kept[first + i]], kind, matrix, n0, tile_n, i * unit_k));
+        out.add(j, ss);
+      }
+  };
+  ln_tables(tb[4], L.o_ln, L.kept_heads, L.attn, STI_ATTN, 3, t.o_n, 64, t.ln_o_split);
+  ln_tables(tb[5], L.f2_ln, L.kept_slices, L.ffn, STI_FFN, 1, std::max(64, t.f2_n), f, t.ln_f2_split);
 }
 
 sti_status check_async(sti_ctx* c) {
@@ -396,13 +441,46 @@ void layer_ranges(const sti_plan* p, int li, const uint8_t* ptr[4], uint32_t byt
   bytes[3] = static_cast<uint32_t>(p->ctx->dense_stride * sizeof(float));
 }
 
+// Can this table run with the LayerNorm epilogue for T tokens?  Every CTA of the launch must be resident at the same
+// time (the column tiles of a row wait for one another), a CTA's token tiles must all fit in tensor memory, and the
+// exchange buffer in shared memory.
+// CTAs along the token dimension for a table in the LayerNorm form: as many as the CTA budget allows while the
+// whole launch (column tiles x token groups clusters of n_split CTAs) can be resident at once.
+int ln_m_ctas(const sti_plan* p, const GemmTable& tab, int T) {
+  const int n_nt = tab.n_jobs / tab.n_split;
+  const int by_clusters = tab.n_split <= 8 ? p->ctx->max_clusters[tab.n_split] / std::max(1, n_nt) : 0;
+  return std::max(1, std::min(m_ctas_for(tab.n_jobs, T, p->tune.cta_budget), by_clusters));
+}
+
+bool ln_form_fits(const sti_plan* p, const GemmTable& tab, int T) {
+  if (tab.n_jobs == 0 || tab.n_split < 1 || !p->tune.ln_fuse || p->ctx->simt_debug) return false;
+  const int m_ctas = ln_m_ctas(p, tab, T);
+  const int n_mtiles = (T + 127) / 128;
+  const int my_mtiles = (n_mtiles + m_ctas - 1) / m_ctas;
+  const uint32_t n_rows = static_cast<uint32_t>(p->ctx->desc.hidden / (tab.n_jobs / tab.n_split));
+  if (tab.n_split > 8 || (tab.n_jobs / tab.n_split) * m_ctas > p->ctx->max_clusters[tab.n_split] ||
+      m_ctas * tab.n_split > kLnCounters)
+    return false;
+  if (my_mtiles * n_rows > 512) return false;
+  return tab.hdr_bytes + gemm_ln_exchange_bytes(my_mtiles, n_rows) <= kMaxSmem;
+}
+
+// `force_pair`: -1 = the two-CTA kernel from pair_min_tiles token tiles on, 0 = never, 1 = always (the table must allow it).
+// `ln`: the LayerNorm epilogue's parameters (kind GEMM_BF16_TO_LN; the table is in that form and ln_form_fits said yes).
 sti_status run_gemm(sti_plan* p, GemmKind kind, const GemmTable& tab, const void* x, int ldx, int T, void* out,
-                    int ldo, const float* bias, int prefetch_layer = -1) {
+                    int ldo, const float* bias, int prefetch_layer = -1, int force_pair = -1, const LnEpilogue* ln = nullptr,
+                    unsigned long long* stamps = nullptr) {
   if (tab.n_jobs == 0) return STI_OK;
   GemmLaunch g{};
+  g.stamps = stamps;
   g.jobs = tab.jobs; g.segs = tab.segs; g.n_jobs = tab.n_jobs; g.m_ctas = m_ctas_for(tab.n_jobs, T, p->tune.cta_budget);
   const int n_mtiles = (T + 127) / 128;
-  g.pair = tab.pair_ok && p->tune.pair_min_tiles > 0 && n_mtiles >= p->tune.pair_min_tiles;
+  g.pair = !ln && tab.pair_ok && p->tune.pair_min_tiles > 0 && n_mtiles >= p->tune.pair_min_tiles;
+  if (force_pair == 0) g.pair = false;
+  if (force_pair == 1) {
+    if (!tab.pair_ok) return STI_ERR_STATE;
+    g.pair = true;
+  }
   if (g.pair) {      // a pair of CTAs takes two token tiles at a time
     const int n_mpairs = (n_mtiles + 1) / 2;
     g.m_ctas = std::max(1, std::min(n_mpairs, p->tune.cta_budget / tab.n_jobs));
@@ -411,81 +489,35 @@ sti_status run_gemm(sti_plan* p, GemmKind kind, const GemmTable& tab, const void
   layer_ranges(p, prefetch_layer, g.pf_ptr, g.pf_bytes);
   g.x = x; g.ldx = ldx; g.T = T; g.out = out; g.ldo = ldo; g.bias = bias; g.err = p->ctx->err_dev;
   g.smem_bytes = tab.smem; g.n_stages = tab.n_stages; g.bps = tab.bps; g.w_bytes = tab.w_bytes; g.hdr_bytes = tab.hdr_bytes; g.seg_stride = tab.seg_stride; g.simt_debug = p->ctx->simt_debug; g.pdl = p->ctx->pdl;
+  if (ln) {
+    if (kind != GEMM_BF16_TO_LN) return STI_ERR_ARG;
+    g.ln = *ln;
+    g.m_ctas = ln_m_ctas(p, tab, T);
+    // the exchange buffer reuses the activation ring and the weight tile; widen the latter if they are too small
+    const uint32_t n_rows = static_cast<uint32_t>(ln->d / ln->n_ntiles);
+    const size_t need = gemm_ln_exchange_bytes((n_mtiles + g.m_ctas - 1) / g.m_ctas, n_rows);
+    const size_t have = gemm_smem_bytes(g.w_bytes, g.n_stages, g.bps, 0);
+    if (need > have) {
+      g.w_bytes += static_cast<uint32_t>(need - have);
+      g.smem_bytes = gemm_smem_bytes(g.w_bytes, g.n_stages, g.bps, g.hdr_bytes);
+    }
+    if (g.smem_bytes > kMaxSmem) return STI_ERR_SHAPE;
+  }
   CUDA_TRY(launch_gemm(kind, g, p->ctx->compute));
   p->ctx->launches++;
-  return STI_OK;
-}
-
-// One launch for the whole layer (few tokens): returns STI_OK and sets *done when the layer was enqueued
-// through the whole-layer kernel, leaves *done false when the shapes call for the seven-kernel path.
-sti_status enqueue_layer_fused(sti_plan* p, int li, const void* xq, const void* x, void* y, int batch, int seq,
-                               const int32_t* lens, bool want_next_bf16, int next_layer, bool* done) {
-  *done = false;
-  sti_ctx* c = p->ctx;
-  const sti_model_desc& d = c->desc;
-  Layer& L = p->layers[li];
-  const int T = batch * seq;
-  const int nh = static_cast<int>(L.kept_heads.size()), ns = static_cast<int>(L.kept_slices.size());
-  if (p->fused_off || c->simt_debug || p->profiling >= 2 || nh == 0 || ns == 0 || T > p->tune.fused_max_tokens) return STI_OK;
-  const GemmTable* gt[4] = {&L.qkv, &L.o, &L.f1, &L.f2};
-  int grid = 1;
-  for (const GemmTable* t : gt) {
-    if (t->f_stages == 0 || t->n_jobs < 1 || t->n_jobs > kFusedMaxCtas) return STI_OK;
-    grid = std::max(grid, t->n_jobs * m_ctas_for(t->n_jobs, T, kFusedMaxCtas));
-  }
-  const size_t top = fused_smem_total(), attn_end = fused_low_offset() + fused_attention_bytes(seq);
-  if (attn_end > top) return STI_OK;
-  const float* dense = c->dense + static_cast<size_t>(li) * c->dense_stride;
-  const bool bf16_act = d.act_dtype == STI_BF16;
-  const int f = d.ffn / d.n_ffn_slices;
-  FusedLayerParams fp{};
-  const void* xs[4] = {xq, p->attn_out, p->h1_bf16, p->u};
-  const int ldx[4] = {d.hidden, nh * 64, d.hidden, ns * f};
-  void* outs[4] = {p->qkv, p->partial, p->u, p->partial};
-  const int ldo[4] = {64, d.hidden, ns * f, d.hidden};
-  const float* bias[4] = {dense + c->off_bq, nullptr, dense + c->off_b1, nullptr};
-  const int kinds[4] = {GEMM_BF16_TO_BF16, GEMM_BF16_TO_F32, GEMM_BF16_TO_BF16_GELU, GEMM_BF16_TO_F32};
-  for (int i = 0; i < 4; ++i) {
-    FusedGemm& g = fp.g[i];
-    if (!make_xmap(&g.xmap, xs[i], ldx[i], T)) return STI_ERR_CUDA;
-    g.jobs = gt[i]->jobs; g.segs = gt[i]->segs; g.out = outs[i]; g.bias = bias[i];
-    g.n_jobs = gt[i]->n_jobs; g.m_ctas = m_ctas_for(gt[i]->n_jobs, T, kFusedMaxCtas);
-    g.ldo = ldo[i]; g.kind = kinds[i];
-    g.n_stages = gt[i]->f_stages; g.bps = gt[i]->f_bps; g.w_bytes = gt[i]->w_bytes; g.seg_stride = gt[i]->seg_stride;
-    g.ahead = 1;
-  }
-  fp.g[0].ahead = 0;
-  fp.g[1].ahead = attn_end + L.o.w_bytes <= top ? 1 : 0;    // the O tile must fit above the attention buffers
-  LnLaunch& l1 = fp.ln[0];
-  l1.partial = p->partial; l1.n_partial = L.o.n_split; l1.bias = dense + c->off_bo; l1.resid = x;
-  l1.resid_bf16 = bf16_act ? 1 : 0; l1.gamma = dense + c->off_ln1g; l1.beta = dense + c->off_ln1b; l1.eps = d.ln_eps;
-  l1.T = T; l1.d = d.hidden; l1.out_f32 = p->h1_f32; l1.out_bf16 = p->h1_bf16;
-  LnLaunch& l2 = fp.ln[1];
-  l2.partial = p->partial; l2.n_partial = L.f2.n_split; l2.bias = dense + c->off_b2; l2.resid = p->h1_f32;
-  l2.resid_bf16 = 0; l2.gamma = dense + c->off_ln2g; l2.beta = dense + c->off_ln2b; l2.eps = d.ln_eps;
-  l2.T = T; l2.d = d.hidden;
-  l2.out_f32 = bf16_act ? nullptr : static_cast<float*>(y);
-  l2.out_bf16 = bf16_act ? static_cast<uint16_t*>(y) : (want_next_bf16 ? p->x_bf16 : nullptr);
-  fp.qkv = p->qkv; fp.attn_out = p->attn_out; fp.seq_lens = lens;
-  fp.n_kept_heads = nh; fp.batch = batch; fp.seq = seq; fp.T = T;
-  fp.barrier = p->fused_ctr + li; fp.err = c->err_dev;
-  layer_ranges(p, next_layer, fp.pf_ptr, fp.pf_bytes);
-  CUDA_TRY(launch_fused_layer(fp, grid, c->compute, c->pdl));
-  c->launches++;
-  *done = true;
   return STI_OK;
 }
 
 // How many CTAs a LayerNorm launch should use, given the GEMM that follows it.  A GEMM CTA needs a whole SM and its
 // CTAs are launched while the LayerNorm runs (they decode their weights meanwhile) - on SMs that hold no LayerNorm
 // CTA.  With one row per CTA the LayerNorm of a few hundred tokens spreads over about 64 SMs; when the next GEMM
-// wants more than the other 84, its last CTAs start late and their decode lands on the critical path.  Then the
+// wants more than the SMs it leaves free (84 of 148), its last CTAs start late and their decode lands on the critical path.  Then the
 // rows are packed into fewer CTAs (measured: 54.6 -> 50.5 us per BERT-large layer at 256 tokens; at 512 tokens
 // packing loses 1-3 us, at BERT-base sizes it changes nothing).  Otherwise one row per CTA.
-int ln_ctas_hint(int tuned, int T, int next_gemm_ctas) {
+int ln_ctas_hint(int tuned, int T, int next_gemm_ctas, int sm_count) {
   if (tuned >= 0) return tuned;
-  if (T > 256 || next_gemm_ctas <= 84) return 0;      // at 512 tokens the packed LayerNorm itself costs more than it frees
-  return std::max(32, 148 - next_gemm_ctas);
+  if (T > 256 || next_gemm_ctas <= sm_count - 64) return 0;      // at 512 tokens the packed LayerNorm itself costs more than it frees
+  return std::max(32, sm_count - next_gemm_ctas);
 }
 
 // The seven kernels of one layer on the compute stream.
@@ -505,6 +537,18 @@ sti_status enqueue_layer(sti_plan* p, int li, const void* x, void* y, int batch,
   const bool kprof = p->profiling >= 2;
   auto mark = [&](int i) -> cudaError_t { return kprof ? cudaEventRecord(L.ev_k[i], c->compute) : cudaSuccess; };
   for (bool& r : L.k_ran) r = false;
+  const bool ln1_fused = nh > 0 && ln_form_fits(p, L.o_ln, T), ln2_fused = ns > 0 && ln_form_fits(p, L.f2_ln, T);
+  auto stamp = [&](int kernel) -> unsigned long long* {
+    return p->stamping ? p->stamps + (static_cast<size_t>(li) * kStampKernels + kernel) * kStampRecord : nullptr;
+  };
+  auto ln_params = [&](const GemmTable& tab, int which) {
+    LnEpilogue e{};
+    e.stats = p->ln_stats[which];
+    e.counters = p->ln_ctr + (static_cast<size_t>(li) * 2 + which) * kLnCounters;
+    e.eps = d.ln_eps; e.d = d.hidden;
+    e.n_ntiles = tab.n_jobs / tab.n_split; e.cluster = tab.n_split;
+    return e;
+  };
   CUDA_TRY(mark(0));
   if (nh > 0) {
     const void* xq = x;
@@ -512,25 +556,27 @@ sti_status enqueue_layer(sti_plan* p, int li, const void* x, void* y, int batch,
       // the GEMMs take bf16 operands: fp32 activations are rounded once (round-to-nearest-even)
       if (!x_ready_bf16) {
         CUDA_TRY(launch_cast_bf16(static_cast<const float*>(x), p->x_bf16, static_cast<size_t>(T) * d.hidden,
-                                  c->compute, c->pdl));
+                                  c->compute, c->pdl, stamp(0)));
         c->launches++;
       }
       xq = p->x_bf16;
     }
-    bool fused = false;
-    st = enqueue_layer_fused(p, li, xq, x, y, batch, seq, lens, want_next_bf16, next_layer, &fused);
-    if (st != STI_OK) return st;
-    if (fused) {
-      for (int i = 1; i <= 7; ++i) CUDA_TRY(mark(i));
-      return STI_OK;
-    }
-    st = run_gemm(p, GEMM_BF16_TO_BF16, L.qkv, xq, d.hidden, T, p->qkv, 64, dense + c->off_bq, next_layer);
+    st = run_gemm(p, GEMM_BF16_TO_BF16, L.qkv, xq, d.hidden, T, p->qkv, 64, dense + c->off_bq, next_layer, -1, nullptr, stamp(1));
     if (st != STI_OK) return st;
     CUDA_TRY(mark(1));
-    CUDA_TRY(launch_attention(p->qkv, p->attn_out, nh, batch, seq, lens, c->compute, c->pdl));
+    CUDA_TRY(launch_attention(p->qkv, p->attn_out, nh, batch, seq, lens, c->compute, c->pdl, stamp(2)));
     c->launches++;
     CUDA_TRY(mark(2));
-    st = run_gemm(p, GEMM_BF16_TO_F32, L.o, p->attn_out, nh * 64, T, p->partial, d.hidden, nullptr);
+    if (ln1_fused) {
+      // O projection + bias + residual + LayerNorm in one launch (no partial sums in global memory)
+      LnEpilogue e = ln_params(L.o_ln, 0);
+      e.bias = dense + c->off_bo; e.resid = x; e.resid_bf16 = bf16_act ? 1 : 0;
+      e.gamma = dense + c->off_ln1g; e.beta = dense + c->off_ln1b;
+      e.out_f32 = p->h1_f32; e.out_bf16 = p->h1_bf16;
+      st = run_gemm(p, GEMM_BF16_TO_LN, L.o_ln, p->attn_out, nh * 64, T, nullptr, d.hidden, nullptr, -1, 0, &e, stamp(3));
+    } else {
+      st = run_gemm(p, GEMM_BF16_TO_F32, L.o, p->attn_out, nh * 64, T, p->partial, d.hidden, nullptr, -1, -1, nullptr, stamp(3));
+    }
     if (st != STI_OK) return st;
     L.k_ran[0] = L.k_ran[1] = L.k_ran[2] = true;
   } else {
@@ -538,27 +584,43 @@ sti_status enqueue_layer(sti_plan* p, int li, const void* x, void* y, int batch,
     CUDA_TRY(mark(2));
   }
   CUDA_TRY(mark(3));
-  LnLaunch ln{};
-  ln.partial = p->partial; ln.n_partial = nh > 0 ? L.o.n_split : 0;
-  ln.bias = dense + c->off_bo; ln.resid = x; ln.resid_bf16 = bf16_act ? 1 : 0;
-  ln.gamma = dense + c->off_ln1g; ln.beta = dense + c->off_ln1b; ln.eps = d.ln_eps; ln.T = T; ln.d = d.hidden;
-  ln.out_f32 = p->h1_f32; ln.out_bf16 = p->h1_bf16;
-  ln.ctas_hint = ln_ctas_hint(p->tune.ln1_ctas, T, ns > 0 ? L.f1.n_jobs * m_ctas_for(L.f1.n_jobs, T, p->tune.cta_budget) : 0);
-  CUDA_TRY(launch_layernorm(ln, c->compute, c->pdl));
-  c->launches++;
-  L.k_ran[3] = true;
+  if (!ln1_fused) {
+    LnLaunch ln{};
+    ln.partial = p->partial; ln.n_partial = nh > 0 ? L.o.n_split : 0;
+    ln.bias = dense + c->off_bo; ln.resid = x; ln.resid_bf16 = bf16_act ? 1 : 0;
+    ln.gamma = dense + c->off_ln1g; ln.beta = dense + c->off_ln1b; ln.eps = d.ln_eps; ln.T = T; ln.d = d.hidden;
+    ln.out_f32 = p->h1_f32; ln.out_bf16 = p->h1_bf16;
+    ln.ctas_hint = ln_ctas_hint(p->tune.ln1_ctas, T, ns > 0 ? L.f1.n_jobs * m_ctas_for(L.f1.n_jobs, T, p->tune.cta_budget) : 0, c->sm_count);
+    ln.stamps = stamp(4);
+    CUDA_TRY(launch_layernorm(ln, c->compute, c->pdl));
+    c->launches++;
+    L.k_ran[3] = true;
+  }
   CUDA_TRY(mark(4));
   if (ns > 0) {
-    st = run_gemm(p, GEMM_BF16_TO_BF16_GELU, L.f1, p->h1_bf16, d.hidden, T, p->u, ns * f, dense + c->off_b1);
+    st = run_gemm(p, GEMM_BF16_TO_BF16_GELU, L.f1, p->h1_bf16, d.hidden, T, p->u, ns * f, dense + c->off_b1, -1, -1, nullptr, stamp(5));
     if (st != STI_OK) return st;
     CUDA_TRY(mark(5));
-    st = run_gemm(p, GEMM_BF16_TO_F32, L.f2, p->u, ns * f, T, p->partial, d.hidden, nullptr);
+    if (ln2_fused) {
+      LnEpilogue e = ln_params(L.f2_ln, 1);
+      e.bias = dense + c->off_b2; e.resid = p->h1_f32; e.resid_bf16 = 0;
+      e.gamma = dense + c->off_ln2g; e.beta = dense + c->off_ln2b;
+      e.out_f32 = bf16_act ? nullptr : static_cast<float*>(y);
+      e.out_bf16 = bf16_act ? static_cast<uint16_t*>(y) : (want_next_bf16 ? p->x_bf16 : nullptr);
+      st = run_gemm(p, GEMM_BF16_TO_LN, L.f2_ln, p->u, ns * f, T, nullptr, d.hidden, nullptr, -1, 0, &e, stamp(6));
+    } else {
+      st = run_gemm(p, GEMM_BF16_TO_F32, L.f2, p->u, ns * f, T, p->partial, d.hidden, nullptr, -1, -1, nullptr, stamp(6));
+    }
     if (st != STI_OK) return st;
     L.k_ran[4] = L.k_ran[5] = true;
   } else {
     CUDA_TRY(mark(5));
   }
   CUDA_TRY(mark(6));
+  if (ln2_fused) {
+    CUDA_TRY(mark(7));
+    return STI_OK;
+  }
   LnLaunch l2{};
   l2.partial = p->partial; l2.n_partial = ns > 0 ? L.f2.n_split : 0;
   l2.bias = dense + c->off_b2; l2.resid = p->h1_f32; l2.resid_bf16 = 0;
@@ -571,7 +633,8 @@ sti_status enqueue_layer(sti_plan* p, int li, const void* x, void* y, int batch,
       const GemmTable& q = p->layers[next_layer].qkv;
       next_ctas = q.n_jobs * m_ctas_for(q.n_jobs, T, p->tune.cta_budget);
     }
-    l2.ctas_hint = ln_ctas_hint(p->tune.ln2_ctas, T, next_ctas);
+    l2.ctas_hint = ln_ctas_hint(p->tune.ln2_ctas, T, next_ctas, c->sm_count);
+    l2.stamps = stamp(7);
   }
   CUDA_TRY(launch_layernorm(l2, c->compute, c->pdl));
   c->launches++;
@@ -681,8 +744,11 @@ sti_status enqueue_forward_io(sti_plan* p, const ForwardKey& k, bool capturing) 
     x = p->x_in;
     y = p->y_out;
   }
-  // grid-barrier counters of the whole-layer kernels start every forward at zero
-  CUDA_TRY(cudaMemsetAsync(p->fused_ctr, 0, p->layers.size() * sizeof(unsigned int), c->compute));
+  // the arrival counters of the LayerNorm epilogues start every forward at zero
+  CUDA_TRY(cudaMemsetAsync(p->ln_ctr, 0, p->layers.size() * 2 * kLnCounters * sizeof(unsigned int), c->compute));
+  p->stamping = k.stamps;
+  if (k.stamps)
+    CUDA_TRY(cudaMemsetAsync(p->stamps, 0xff, p->layers.size() * kStampKernels * kStampRecord * sizeof(unsigned long long), c->compute));
   sti_status st;
   if (k.layer >= 0) {
     // a single layer: its IO job (if it has streamed units) runs on the compute stream, not overlapped
@@ -705,7 +771,7 @@ sti_status enqueue_forward_io(sti_plan* p, const ForwardKey& k, bool capturing) 
 // ~7 per layer, no per-kernel host work); anything else is captured anew.  Profiling runs ungraphed.
 sti_status model_forward_impl(sti_plan* p, const ForwardKey& k) {
   sti_ctx* c = p->ctx;
-  if (p->profiling || p->graph_off) return enqueue_forward_io(p, k, false);
+  if ((p->profiling && p->profiling < 3) || p->graph_off) return enqueue_forward_io(p, k, false);
   sti_plan::CachedGraph* hit = nullptr;
   for (auto& g : p->graphs) if (g.exec && g.key == k) hit = &g;
   if (!hit) {
@@ -762,7 +828,8 @@ void free_plan_device(sti_plan* p) {
   cudaFree(p->qkv); cudaFree(p->attn_out); cudaFree(p->partial); cudaFree(p->h1_f32); cudaFree(p->h1_bf16);
   cudaFree(p->u); cudaFree(p->x_bf16); cudaFree(p->buf[0]); cudaFree(p->buf[1]); cudaFree(p->x_in); cudaFree(p->y_out);
   cudaFree(p->lens_dev);
-  cudaFree(p->fused_ctr);
+  cudaFree(p->ln_ctr); cudaFree(p->ln_stats[0]); cudaFree(p->ln_stats[1]); cudaFree(p->stamps);
+  cudaFree(p->zero_bias);
   for (auto& L : p->layers) {
     if (L.ev_loaded) cudaEventDestroy(L.ev_loaded);
     if (L.g_ev_loaded) cudaEventDestroy(L.g_ev_loaded);
@@ -855,8 +922,16 @@ sti_status sti_ctx_create(const sti_model_desc* desc, int device, void* compute_
   if (cudaMemset(c->dense, 0, c->dense_stride * d.n_layers * sizeof(float)) != cudaSuccess) return fail(STI_ERR_CUDA);
   if (cudaMalloc(&c->err_dev, sizeof(int)) != cudaSuccess) return fail(STI_ERR_OOM);
   if (cudaMemset(c->err_dev, 0, sizeof(int)) != cudaSuccess) return fail(STI_ERR_CUDA);
-  if (gemm_configure() != cudaSuccess || attention_configure() != cudaSuccess || fused_configure() != cudaSuccess)
+  if (gemm_configure() != cudaSuccess || attention_configure() != cudaSuccess)
     return fail(STI_ERR_CUDA);
+  if (cudaDeviceGetAttribute(&c->sm_count, cudaDevAttrMultiProcessorCount, device) != cudaSuccess || c->sm_count < 1)
+    return fail(STI_ERR_CUDA);
+  for (unsigned cx = 1; cx <= 8; ++cx) c->max_clusters[cx] = gemm_max_active_clusters(cx, kMaxSmem);
+  if (getenv("STI_VERBOSE")) {
+    fprintf(stderr, "sti: %d SMs; resident clusters of 1..8 GEMM CTAs:", c->sm_count);
+    for (int cx = 1; cx <= 8; ++cx) fprintf(stderr, " %d", c->max_clusters[cx]);
+    fprintf(stderr, "\n");
+  }
   const char* dbg = getenv("STI_DEBUG_SIMT");
   c->simt_debug = dbg && dbg[0] == '1';
   const char* nopdl = getenv("STI_NO_PDL");
@@ -924,7 +999,7 @@ sti_status sti_plan_create(sti_ctx* c, const sti_shard_cfg* attn, const sti_shar
       if (L.ffn[s].cfg.keep) L.kept_slices.push_back(s);
     }
   }
-  parse_tuning(&p->tune, d.max_batch * d.max_seq, d);
+  parse_tuning(&p->tune, d.max_batch * d.max_seq, d, c->sm_count);
   *out = p;
   return STI_OK;
 }
@@ -1049,30 +1124,29 @@ sti_status sti_plan_finalize(sti_plan* p) {
   std::vector<Fix> fixes;
   p->max_partial = 1;
   for (auto& L : p->layers) {
-    TableBuilder tb[4];
+    TableBuilder tb[6];
     L.tables_off = align16(host_tables.size());
     build_layer_tables(p, L, tb);
-    GemmTable* gt[4] = {&L.qkv, &L.o, &L.f1, &L.f2};
-    for (int i = 0; i < 4; ++i) {
+    GemmTable* gt[6] = {&L.qkv, &L.o, &L.f1, &L.f2, &L.o_ln, &L.f2_ln};
+    for (int i = 0; i < 6; ++i) {
       tb[i].finish();
       gt[i]->seg_stride = tb[i].seg_stride;
       gt[i]->n_jobs = static_cast<int>(tb[i].jobs.size());
       gt[i]->w_bytes = tb[i].w_bytes;
       gt[i]->n_stages = 2; gt[i]->bps = 1;
       gt[i]->hdr_bytes = gemm_header_bytes();
-      gt[i]->pair_ok = !tb[i].jobs.empty() && tb[i].jobs.size() % 2 == 0;
+      gt[i]->pair_ok = i < 4 && !tb[i].jobs.empty() && tb[i].jobs.size() % 2 == 0;
       for (size_t j = 0; gt[i]->pair_ok && j < tb[i].jobs.size(); j += 2) {
         const Job &a = tb[i].jobs[j], &b = tb[i].jobs[j + 1];
         gt[i]->pair_ok = a.n_rows == 64 && b.n_rows == 64 && a.k_total == b.k_total && a.x_koff == b.x_koff;
       }
       if (!tb[i].jobs.empty() &&
-          !gemm_pick_ring(tb[i].w_bytes, tb[i].k_max, gt[i]->hdr_bytes, &gt[i]->n_stages, &gt[i]->bps))
-        return STI_ERR_SHAPE;
+          !gemm_pick_ring(tb[i].w_bytes, tb[i].k_max, gt[i]->hdr_bytes, &gt[i]->n_stages, &gt[i]->bps)) {
+        if (i < 4) return STI_ERR_SHAPE;
+        tb[i] = TableBuilder();          // the LayerNorm form is optional: fall back to partial sums + LayerNorm kernel
+        gt[i]->n_jobs = 0; gt[i]->n_split = 0;
+      }
       gt[i]->smem = gemm_smem_bytes(tb[i].w_bytes, gt[i]->n_stages, gt[i]->bps, gt[i]->hdr_bytes);
-      // the whole-layer kernel keeps both header slots resident: its activation ring starts further up
-      if (tb[i].jobs.empty() || tb[i].seg_stride > 16 ||
-          !gemm_pick_ring(tb[i].w_bytes, tb[i].k_max, static_cast<uint32_t>(fused_low_offset()), &gt[i]->f_stages, &gt[i]->f_bps))
-        gt[i]->f_stages = gt[i]->f_bps = 0;
       if (gt[i]->smem > kMaxSmem && !tb[i].jobs.empty()) return STI_ERR_SHAPE;
       Fix fx{gt[i], 0, 0};
       fx.jobs_off = align16(host_tables.size());
@@ -1109,8 +1183,10 @@ sti_status sti_plan_finalize(sti_plan* p) {
   CUDA_TRY(cudaMalloc(&p->x_in, Tmax * d.hidden * act_size(c)));
   CUDA_TRY(cudaMalloc(&p->y_out, Tmax * d.hidden * act_size(c)));
   CUDA_TRY(cudaMalloc(&p->lens_dev, static_cast<size_t>(d.max_batch) * 4));
-  CUDA_TRY(cudaMalloc(&p->fused_ctr, static_cast<size_t>(d.n_layers) * sizeof(unsigned int)));
-  CUDA_TRY(cudaMemset(p->fused_ctr, 0, static_cast<size_t>(d.n_layers) * sizeof(unsigned int)));
+  CUDA_TRY(cudaMalloc(&p->ln_ctr, static_cast<size_t>(d.n_layers) * 2 * kLnCounters * sizeof(unsigned int)));
+  CUDA_TRY(cudaMemset(p->ln_ctr, 0, static_cast<size_t>(d.n_layers) * 2 * kLnCounters * sizeof(unsigned int)));
+  for (auto& st : p->ln_stats) CUDA_TRY(cudaMalloc(&st, Tmax * kLnMaxTiles * sizeof(float2)));
+  CUDA_TRY(cudaMalloc(&p->stamps, static_cast<size_t>(d.n_layers) * kStampKernels * kStampRecord * sizeof(unsigned long long)));
   // 5. events
   const unsigned flags = cudaEventDefault;     // timing-capable; only recorded when profiling
   for (auto& L : p->layers) {
@@ -1132,7 +1208,6 @@ sti_status sti_plan_finalize(sti_plan* p) {
   p->g_slot_free.resize(p->ring_slots);
   for (auto& e : p->g_slot_free) CUDA_TRY(cudaEventCreateWithFlags(&e, cudaEventDisableTiming));
   { const char* ng = getenv("STI_NO_GRAPH"); p->graph_off = ng && ng[0] == '1'; }
-  { const char* nf = getenv("STI_NO_FUSED"); p->fused_off = nf && nf[0] == '1'; }
   CUDA_TRY(cudaEventCreateWithFlags(&p->ev_begin, flags));
   CUDA_TRY(cudaEventCreateWithFlags(&p->ev_end, flags));
   p->finalized = true;
@@ -1153,6 +1228,7 @@ sti_status sti_layer_forward(sti_plan* p, int layer, const void* x, void* y, int
   }
   ForwardKey k;
   k.x = x; k.y = y; k.lens = lens; k.batch = batch; k.seq = seq; k.layer = layer;
+  k.stamps = p->profiling == 3;
   return model_forward_impl(p, k);
 }
 
@@ -1163,6 +1239,7 @@ sti_status sti_model_forward(sti_plan* p, const void* x, void* y, int batch, int
   CUDA_TRY(cudaSetDevice(p->ctx->device));
   ForwardKey k;
   k.x = x; k.y = y; k.lens = lens; k.batch = batch; k.seq = seq;
+  k.stamps = p->profiling == 3;
   return model_forward_impl(p, k);
 }
 
@@ -1180,6 +1257,7 @@ sti_status sti_model_forward_host(sti_plan* p, const void* x_host, void* y_host,
     CUDA_TRY(cudaMemcpyAsync(p->lens_dev, lens_host, static_cast<size_t>(batch) * 4, cudaMemcpyHostToDevice, c->compute));
     k.lens = p->lens_dev;
   }
+  k.stamps = p->profiling == 3;
   return model_forward_impl(p, k);
 }
 
@@ -1220,9 +1298,53 @@ sti_status sti_shard_decode(sti_plan* p, int layer, sti_kind kind, int index, in
   return STI_OK;
 }
 
+sti_status sti_gemm_probe(sti_plan* p, int layer, int gemm, const void* x_bf16_dev, int tokens, void* out_dev,
+                          size_t out_capacity_bytes, int variant, int32_t* n_partials) {
+  if (!p || !x_bf16_dev || !out_dev || gemm < 0 || gemm > 3 || variant < 0 || variant > 3) return STI_ERR_ARG;
+  if (layer < 0 || layer >= static_cast<int>(p->layers.size())) return STI_ERR_ARG;
+  if (tokens < 1 || tokens > 65536) return STI_ERR_SHAPE;
+  if ((reinterpret_cast<uintptr_t>(x_bf16_dev) & 15) || (reinterpret_cast<uintptr_t>(out_dev) & 15)) return STI_ERR_ARG;
+  sti_status st = sti_plan_finalize(p);
+  if (st != STI_OK) return st;
+  sti_ctx* c = p->ctx;
+  const sti_model_desc& d = c->desc;
+  CUDA_TRY(cudaSetDevice(c->device));
+  Layer& L = p->layers[layer];
+  const int nh = static_cast<int>(L.kept_heads.size()), ns = static_cast<int>(L.kept_slices.size());
+  const int f = d.ffn / d.n_ffn_slices;
+  // variant 3: the O projection / FFN2 tile tables of the LayerNorm-epilogue form (QKV and FFN1 have one form only)
+  const bool ln_tables = variant == 3 && (gemm == 1 || gemm == 3);
+  const GemmTable* tabs[4] = {&L.qkv, ln_tables ? &L.o_ln : &L.o, &L.f1, ln_tables ? &L.f2_ln : &L.f2};
+  const GemmTable& tab = *tabs[gemm];
+  if (tab.n_jobs == 0) return STI_ERR_STATE;               // no kept unit feeds this GEMM (or the form is not available)
+  const int ldx[4] = {d.hidden, nh * 64, d.hidden, ns * f};
+  const int ldo[4] = {64, d.hidden, ns * f, d.hidden};
+  const int parts[4] = {1, tabs[1]->n_split, 1, tabs[3]->n_split};
+  const size_t out_elems[4] = {static_cast<size_t>(3) * nh * tokens * 64, static_cast<size_t>(parts[1]) * tokens * d.hidden,
+                               static_cast<size_t>(tokens) * ns * f, static_cast<size_t>(parts[3]) * tokens * d.hidden};
+  const size_t need = out_elems[gemm] * ((gemm == 1 || gemm == 3) ? 4 : 2);
+  if (out_capacity_bytes < need) return STI_ERR_SIZE;
+  if (!p->zero_bias) {
+    const size_t n = static_cast<size_t>(3) * d.n_heads * 64 + d.ffn;
+    CUDA_TRY(cudaMalloc(&p->zero_bias, n * sizeof(float)));
+    CUDA_TRY(cudaMemset(p->zero_bias, 0, n * sizeof(float)));
+  }
+  if (L.str_bytes > 0) {           // a streamed layer is brought into its ring slot first (not overlapped)
+    if (p->copy_tail_valid) CUDA_TRY(cudaStreamWaitEvent(c->compute, p->ev_copy_tail, 0));
+    if ((st = enqueue_layer_copy(p, layer, c->compute)) != STI_OK) return st;
+  }
+  const GemmKind kind = (gemm == 1 || gemm == 3) ? GEMM_BF16_TO_F32 : GEMM_BF16_TO_BF16;
+  st = run_gemm(p, kind, tab, x_bf16_dev, ldx[gemm], tokens, out_dev, ldo[gemm], p->zero_bias, -1,
+                variant == 0 ? -1 : (variant == 3 ? 0 : variant - 1));
+  if (st != STI_OK) return st;
+  if (L.str_bytes > 0) CUDA_TRY(cudaEventRecord(p->slot_free[L.slot], c->compute));
+  if (n_partials) *n_partials = parts[gemm];
+  return STI_OK;
+}
+
 sti_status sti_plan_set_profiling(sti_plan* p, int enabled) {
   if (!p) return STI_ERR_ARG;
-  p->profiling = enabled < 0 ? 0 : (enabled > 2 ? 2 : enabled);
+  p->profiling = enabled < 0 ? 0 : (enabled > 3 ? 3 : enabled);
   p->stats_valid = false;
   return STI_OK;
 }
@@ -1269,6 +1391,27 @@ sti_status sti_get_stats(sti_plan* p, sti_stats* out) {
   CUDA_TRY(cudaEventElapsedTime(&tot, p->ev_begin, p->ev_end));
   s.total_us = tot * 1e3f;
   *out = s;
+  return STI_OK;
+}
+
+sti_status sti_get_kernel_stamps(sti_plan* p, uint64_t* out, size_t capacity_words, int32_t* n_layers) {
+  if (!p || !out) return STI_ERR_ARG;
+  if (!p->finalized) return STI_ERR_STATE;
+  const size_t n = p->layers.size() * kStampKernels * kStampRecord;
+  if (capacity_words < n) return STI_ERR_SIZE;
+  sti_ctx* c = p->ctx;
+  CUDA_TRY(cudaSetDevice(c->device));
+  CUDA_TRY(cudaStreamSynchronize(c->copy));
+  CUDA_TRY(cudaStreamSynchronize(c->compute));
+  std::vector<unsigned long long> raw(n);
+  CUDA_TRY(cudaMemcpy(raw.data(), p->stamps, n * sizeof(unsigned long long), cudaMemcpyDeviceToHost));
+  for (size_t i = 0; i < n; ++i) {
+    const size_t slot = i % kStampRecord;
+    const bool is_min = slot == 0 || slot == 1;          // the other slots hold complemented maxima
+    const unsigned long long v = raw[i];
+    out[i] = v == ~0ull ? 0 : (is_min ? v : ~v);
+  }
+  if (n_layers) *n_layers = static_cast<int32_t>(p->layers.size());
   return STI_OK;
 }
 

@@ -21,7 +21,7 @@ constexpr int kKStride = kAttnKStride;
 template <int WARPS>      // 16 query rows per warp; K and V of the sequence are shared by the CTA's warps
 __global__ void __launch_bounds__(32 * WARPS)
 attention_kernel(const uint16_t* __restrict__ qkv, uint16_t* __restrict__ out, int n_kept, int batch, int L,
-                 const int32_t* __restrict__ seq_lens) {
+                 const int32_t* __restrict__ seq_lens, unsigned long long* stamps) {
   extern __shared__ __align__(16) uint8_t smem[];
   const int qt = blockIdx.x, hi = blockIdx.y, b = blockIdx.z;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -36,7 +36,9 @@ attention_kernel(const uint16_t* __restrict__ qkv, uint16_t* __restrict__ out, i
   const uint16_t* Vg = qkv + (static_cast<size_t>(hi * 3 + 2) * T + static_cast<size_t>(b) * L) * kHeadDim;
 
   pdl_launch_dependents();
+  if (tid == 0) { stamp_min(stamps, STAMP_FIRST_START); stamp_max(stamps, STAMP_LAST_START); }
   pdl_wait();          // q, k, v (and possibly seq_lens) come from the preceding kernels
+  if (tid == 0) stamp_min(stamps, STAMP_RELEASE);
   int valid = L;
   if (seq_lens != nullptr) {
     valid = seq_lens[b];
@@ -162,6 +164,10 @@ attention_kernel(const uint16_t* __restrict__ qkv, uint16_t* __restrict__ out, i
         *reinterpret_cast<uint32_t*>(dst + jd * 8) = pack_bf16x2(o[jd][2 * r] * inv[r], o[jd][2 * r + 1] * inv[r]);
     }
   }
+  if (stamps != nullptr) {
+    __syncthreads();
+    if (tid == 0) stamp_max(stamps, STAMP_LAST_END);
+  }
 }
 
 // Few tokens: one CTA of 16 warps per (64-query tile, kept head, sequence), keys split four ways inside the
@@ -170,8 +176,14 @@ __global__ void __launch_bounds__(kAttnThreads)
 attention_split_kernel(AttnArgs p) {
   extern __shared__ __align__(16) uint8_t smem[];
   pdl_launch_dependents();
+  if (threadIdx.x == 0) { stamp_min(p.stamps, STAMP_FIRST_START); stamp_max(p.stamps, STAMP_LAST_START); }
   pdl_wait();          // q, k, v (and possibly seq_lens) come from the preceding kernels
+  if (threadIdx.x == 0) stamp_min(p.stamps, STAMP_RELEASE);
   attention_step(p, blockIdx.x, gridDim.x, smem, threadIdx.x);
+  if (p.stamps != nullptr) {
+    __syncthreads();
+    if (threadIdx.x == 0) stamp_max(p.stamps, STAMP_LAST_END);
+  }
 }
 
 size_t attn_split_smem_bytes(int L) {
@@ -198,24 +210,24 @@ cudaError_t attention_configure() {
 }
 
 cudaError_t launch_attention(const uint16_t* qkv, uint16_t* out, int n_kept, int batch, int seq,
-                             const int32_t* seq_lens, cudaStream_t s, bool pdl) {
+                             const int32_t* seq_lens, cudaStream_t s, bool pdl, unsigned long long* stamps) {
   if (n_kept <= 0) return cudaSuccess;
   // 128-query CTAs when there are enough of them to fill the GPU (fewer K/V re-reads per head), 64 otherwise
   const long ctas128 = static_cast<long>((seq + 127) / 128) * n_kept * batch;
   if (seq >= 128 && ctas128 >= 148) {
     dim3 grid((seq + 127) / 128, n_kept, batch);
     return launch_kernel(attention_kernel<8>, grid, dim3(256), attn_smem_bytes(seq), s, pdl, qkv, out, n_kept, batch,
-                         seq, seq_lens);
+                         seq, seq_lens, stamps);
   }
   const long items = static_cast<long>((seq + 63) / 64) * n_kept * batch;
   if (items <= 2 * 148 && seq > 64) {          // too few CTAs to fill the GPU: shorten each CTA's key loop instead
-    AttnArgs a{qkv, out, seq_lens, n_kept, batch, seq, batch * seq};
+    AttnArgs a{qkv, out, seq_lens, n_kept, batch, seq, batch * seq, stamps};
     return launch_kernel(attention_split_kernel, dim3(static_cast<unsigned>(items)), dim3(kAttnThreads),
                          attn_split_smem_bytes(seq), s, pdl, a);
   }
   dim3 grid((seq + 63) / 64, n_kept, batch);
   return launch_kernel(attention_kernel<4>, grid, dim3(128), attn_smem_bytes(seq), s, pdl, qkv, out, n_kept, batch, seq,
-                       seq_lens);
+                       seq_lens, stamps);
 }
 
 }  // namespace sti

@@ -17,6 +17,7 @@ struct AttnArgs {
   uint16_t* out;            // [T][n_kept * 64] bf16
   const int32_t* seq_lens;  // optional, per sequence
   int n_kept, batch, seq, T;
+  unsigned long long* stamps;   // profiling record or null
 };
 
 // ---------------------------------------------------------------------------------------

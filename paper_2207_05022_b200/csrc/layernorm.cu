@@ -32,10 +32,12 @@ layernorm_kernel(LnLaunch p) {
   const size_t row = static_cast<size_t>(blockIdx.x) * p.d;
   const int c = tid * 4;
   pdl_launch_dependents();
+  if (tid == 0) { stamp_min(p.stamps, STAMP_FIRST_START); stamp_max(p.stamps, STAMP_LAST_START); }
   float4 a = __ldg(reinterpret_cast<const float4*>(p.bias + c));      // parameters: not written by any kernel
   const float4 g = __ldg(reinterpret_cast<const float4*>(p.gamma + c));
   const float4 b = __ldg(reinterpret_cast<const float4*>(p.beta + c));
   pdl_wait();                                                          // residual and partial sums are
+  if (tid == 0) stamp_min(p.stamps, STAMP_RELEASE);                    // the preceding kernels' output
   if (p.resid_bf16) {
     const uint2 r = __ldg(reinterpret_cast<const uint2*>(static_cast<const uint16_t*>(p.resid) + row + c));
     a.x += __uint_as_float(r.x << 16); a.y += __uint_as_float(r.x & 0xffff0000u);
@@ -70,6 +72,10 @@ layernorm_kernel(LnLaunch p) {
   if (p.out_f32) *reinterpret_cast<float4*>(p.out_f32 + row + c) = y;
   if (p.out_bf16)
     *reinterpret_cast<uint2*>(p.out_bf16 + row + c) = make_uint2(pack_bf16x2(y.x, y.y), pack_bf16x2(y.z, y.w));
+  if (p.stamps != nullptr) {
+    __syncthreads();
+    if (tid == 0) stamp_max(p.stamps, STAMP_LAST_END);
+  }
 }
 
 // Few tokens: the same arithmetic with several rows per CTA and several float4 per thread, so that the kernel
@@ -86,6 +92,7 @@ layernorm_rows_kernel(LnLaunch p, int tpr, int rows_per_cta) {
   const int n_warps = tpr >> 5;
   const int r = blockIdx.x * rows_per_cta + slot;
   pdl_launch_dependents();
+  if (threadIdx.x == 0) { stamp_min(p.stamps, STAMP_FIRST_START); stamp_max(p.stamps, STAMP_LAST_START); }
   if (slot >= rows_per_cta || r >= p.T) {      // whole warps: tpr is a multiple of 32
     pdl_wait();
     return;
@@ -96,6 +103,7 @@ layernorm_rows_kernel(LnLaunch p, int tpr, int rows_per_cta) {
 #pragma unroll
   for (int v = 0; v < V; ++v) a[v] = __ldg(reinterpret_cast<const float4*>(p.bias + (tid + v * tpr) * 4));
   pdl_wait();
+  if (tid == 0) stamp_min(p.stamps, STAMP_RELEASE);
   const size_t pstride = static_cast<size_t>(p.T) * p.d;
 #pragma unroll
   for (int v = 0; v < V; ++v) {
@@ -165,15 +173,27 @@ layernorm_rows_kernel(LnLaunch p, int tpr, int rows_per_cta) {
         *reinterpret_cast<uint2*>(p.out_bf16 + row + c) = make_uint2(pack_bf16x2(y.x, y.y), pack_bf16x2(y.z, y.w));
     }
   }
+  if (p.stamps != nullptr) {
+    asm volatile("bar.sync %0, %1;" ::"r"(slot), "r"(tpr) : "memory");
+    if (tid == 0) stamp_max(p.stamps, STAMP_LAST_END);
+  }
 }
 
-__global__ void cast_bf16_kernel(const float* __restrict__ in, uint16_t* __restrict__ out, size_t n4) {
+__global__ void cast_bf16_kernel(const float* __restrict__ in, uint16_t* __restrict__ out, size_t n4,
+                                 unsigned long long* stamps) {
   const size_t i = static_cast<size_t>(blockIdx.x) * blockDim.x + threadIdx.x;
   pdl_launch_dependents();
+  if (threadIdx.x == 0) { stamp_min(stamps, STAMP_FIRST_START); stamp_max(stamps, STAMP_LAST_START); }
   pdl_wait();
-  if (i >= n4) return;
-  const float4 v = __ldg(reinterpret_cast<const float4*>(in) + i);
-  reinterpret_cast<uint2*>(out)[i] = make_uint2(pack_bf16x2(v.x, v.y), pack_bf16x2(v.z, v.w));
+  if (threadIdx.x == 0) stamp_min(stamps, STAMP_RELEASE);
+  if (i < n4) {
+    const float4 v = __ldg(reinterpret_cast<const float4*>(in) + i);
+    reinterpret_cast<uint2*>(out)[i] = make_uint2(pack_bf16x2(v.x, v.y), pack_bf16x2(v.z, v.w));
+  }
+  if (stamps != nullptr) {
+    __syncthreads();
+    if (threadIdx.x == 0) stamp_max(stamps, STAMP_LAST_END);
+  }
 }
 
 }  // namespace
@@ -205,11 +225,11 @@ cudaError_t launch_layernorm(const LnLaunch& p, cudaStream_t s, bool pdl) {
   return launch_kernel(layernorm_kernel, dim3(p.T), dim3(p.d / 4), 0, s, pdl, p);
 }
 
-cudaError_t launch_cast_bf16(const float* in, uint16_t* out, size_t n, cudaStream_t s, bool pdl) {
+cudaError_t launch_cast_bf16(const float* in, uint16_t* out, size_t n, cudaStream_t s, bool pdl, unsigned long long* stamps) {
   if (n == 0) return cudaSuccess;
   if (n % 4) return cudaErrorInvalidValue;
   const size_t n4 = n / 4;
-  return launch_kernel(cast_bf16_kernel, dim3(static_cast<unsigned>((n4 + 255) / 256)), dim3(256), 0, s, pdl, in, out, n4);
+  return launch_kernel(cast_bf16_kernel, dim3(static_cast<unsigned>((n4 + 255) / 256)), dim3(256), 0, s, pdl, in, out, n4, stamps);
 }
 
 }  // namespace sti

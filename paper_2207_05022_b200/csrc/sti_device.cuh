@@ -53,6 +53,29 @@ __device__ __forceinline__ uint64_t global_timer_ns() {
 }
 
 // ---------------------------------------------------------------------------------------
+// Profiling stamps (Section 5.2: the delays the planner works with are measured on the device in use).
+// One record of kStampWords 64-bit words per kernel launch, every word 0xff..ff before the forward.  A slot that
+// holds a minimum over the launch's CTAs stores the time, a slot that holds a maximum stores its complement, so
+// both are one atomicMin.  One thread per CTA stamps; a null record switches stamping off.
+// ---------------------------------------------------------------------------------------
+constexpr int kStampWords = 8;
+enum StampSlot : int {
+  STAMP_FIRST_START = 0,   // min: the launch's first CTA starts
+  STAMP_RELEASE = 1,       // min: first CTA past the wait for the preceding kernel
+  STAMP_LAST_END = 2,      // max: the last CTA is done
+  STAMP_DECODED = 3,       // max: weight tiles decoded (dequant-GEMM)
+  STAMP_LAST_START = 4,    // max: the launch's last CTA starts
+  STAMP_ACC = 5,           // max: accumulators complete (dequant-GEMM with the LayerNorm epilogue)
+  STAMP_EXCHANGED = 6      // max: row statistics of all column tiles have arrived (same)
+};
+__device__ __forceinline__ void stamp_min(unsigned long long* rec, int slot) {
+  if (rec != nullptr) atomicMin(rec + slot, static_cast<unsigned long long>(global_timer_ns()));
+}
+__device__ __forceinline__ void stamp_max(unsigned long long* rec, int slot) {
+  if (rec != nullptr) atomicMin(rec + slot, ~static_cast<unsigned long long>(global_timer_ns()));
+}
+
+// ---------------------------------------------------------------------------------------
 // mbarrier
 // ---------------------------------------------------------------------------------------
 __device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {

@@ -39,7 +39,29 @@ struct Job {
 enum GemmKind : int {
   GEMM_BF16_TO_BF16 = 1,      // bf16 in, bf16 out (+bias)                     : QKV
   GEMM_BF16_TO_BF16_GELU = 2, // bf16 in, bf16 out, +bias, erf-GELU            : FFN1
-  GEMM_BF16_TO_F32 = 3        // bf16 in, fp32 partial sums out, no bias       : O projection, FFN2
+  GEMM_BF16_TO_F32 = 3,       // bf16 in, fp32 partial sums out, no bias       : O projection, FFN2 (many tokens, probes)
+  GEMM_BF16_TO_LN = 4         // bf16 in, + bias + residual, LayerNorm, fp32 and/or bf16 out : O projection, FFN2
+};
+
+// Epilogue of GEMM_BF16_TO_LN: out = LayerNorm(x W^T + bias + resid) * gamma + beta with the K range of every
+// 64- or 128-feature column tile split over the CTAs of one thread-block cluster.  The partial sums of a cluster
+// meet in distributed shared memory; the per-row (mean, sum of squared deviations) of every column tile meet in
+// `stats`, counted in `counters` (zero before the launch), so that no partial sum reaches global memory and no
+// separate LayerNorm launch is needed.  Jobs of one column tile are consecutive (cluster rank = K split).
+struct LnEpilogue {
+  const float* bias;        // [d]
+  const void* resid;        // [T][d], fp32 or bf16
+  const float* gamma;
+  const float* beta;
+  float* out_f32;           // optional
+  uint16_t* out_bf16;       // optional
+  float2* stats;            // [T][n_ntiles] scratch
+  unsigned int* counters;   // [m_ctas * cluster] scratch, zero at launch
+  float eps;
+  int resid_bf16;
+  int d;
+  int n_ntiles;             // column tiles = clusters that share a token row
+  int cluster;              // CTAs per cluster = K splits per column tile (1..8)
 };
 
 struct GemmLaunch {
@@ -66,19 +88,24 @@ struct GemmLaunch {
   bool simt_debug;          // compute the products on the plain ALUs instead of the tensor cores
   bool pdl;                 // launch with programmatic dependent launch
   bool pair;                // two-CTA clusters (cta_group::2): jobs 2i and 2i+1 share one M=256 x N=128 MMA
+  LnEpilogue ln;            // GEMM_BF16_TO_LN only
+  unsigned long long* stamps;   // this launch's profiling record (see sti_device.cuh), or null
 };
 
 size_t gemm_weight_bytes(uint32_t n_rows, uint32_t k_total);
 uint32_t gemm_header_bytes();
 bool gemm_pick_ring(uint32_t w_bytes, uint32_t k_total, uint32_t hdr_bytes, uint32_t* n_stages, uint32_t* bps);   // false: does not fit
 size_t gemm_smem_bytes(uint32_t w_bytes, uint32_t n_stages, uint32_t bps, uint32_t hdr_bytes);
+// Shared memory (beyond the header) the LayerNorm epilogue needs for a CTA that owns `m_tiles` token tiles of `n_rows` features.
+size_t gemm_ln_exchange_bytes(uint32_t m_tiles, uint32_t n_rows);
 cudaError_t gemm_configure();   // opt in to large dynamic shared memory (once per device)
+int gemm_max_active_clusters(unsigned cluster_x, size_t smem_bytes);
 cudaError_t launch_gemm(GemmKind kind, const GemmLaunch& p, cudaStream_t s);
 
 // Per-head attention over kept heads.  qkv: [(kept*3 + which)][T][64] bf16; out: [T][n_kept*64] bf16.
 cudaError_t attention_configure();
 cudaError_t launch_attention(const uint16_t* qkv, uint16_t* out, int n_kept, int batch, int seq,
-                             const int32_t* seq_lens, cudaStream_t s, bool pdl);
+                             const int32_t* seq_lens, cudaStream_t s, bool pdl, unsigned long long* stamps);
 
 // out = LayerNorm(sum_p partial[p] + bias + resid) * gamma + beta, one warp per token row.
 struct LnLaunch {
@@ -94,11 +121,12 @@ struct LnLaunch {
   float* out_f32;           // optional
   uint16_t* out_bf16;       // optional
   int ctas_hint;            // > 0: pack rows so that about this many CTAs are launched (few tokens); 0: one row per CTA
+  unsigned long long* stamps;   // profiling record or null
 };
 cudaError_t launch_layernorm(const LnLaunch& p, cudaStream_t s, bool pdl);
 
 // fp32 -> bf16 (round-to-nearest-even) copy of the activations the first GEMM reads.
-cudaError_t launch_cast_bf16(const float* in, uint16_t* out, size_t n, cudaStream_t s, bool pdl);
+cudaError_t launch_cast_bf16(const float* in, uint16_t* out, size_t n, cudaStream_t s, bool pdl, unsigned long long* stamps);
 
 // Stand-alone decode of one matrix (inspection / parity).
 struct DecodeLaunch {
@@ -115,68 +143,37 @@ struct DecodeLaunch {
 };
 cudaError_t launch_decode(const DecodeLaunch& p, cudaStream_t s);
 
-// ---------------------------------------------------------------------------------------
-// Whole-layer kernel for few tokens (one launch per layer instead of seven).
-// A grid of at most one CTA per SM runs the layer's seven steps one after the other - QKV GEMM,
-// attention, O projection, residual + LayerNorm, FFN1 + GELU, FFN2, residual + LayerNorm - with a
-// grid-wide barrier between steps.  Between arriving at a barrier and waiting on it a CTA decodes the
-// weight tile of its next GEMM step (weights depend on no activation), so shard decode never sits on
-// the critical path, and the barriers replace the kernel boundaries.
-// ---------------------------------------------------------------------------------------
-struct FusedGemm {
-  CUtensorMap xmap;         // activation operand of this step: [T, ld] bf16, box 64 x 128, 128-byte swizzle
-  const Job* jobs;
-  const Seg* segs;          // the segments of job j start at segs[j * seg_stride]
-  void* out;
-  const float* bias;
-  int n_jobs;
-  int m_ctas;               // CTAs per job along the token dimension; n_jobs * m_ctas <= grid
-  int ldo;
-  int kind;                 // GemmKind
-  uint32_t n_stages, bps;   // activation ring: stages, 16 KB boxes per stage
-  uint32_t w_bytes;         // shared memory of the largest weight tile of this step
-  uint32_t seg_stride;
-  uint32_t ahead;           // 1: the tile is decoded before the preceding barrier wait (its shared memory is free then)
-};
-
-struct FusedLayerParams {
-  FusedGemm g[4];           // QKV, O projection, FFN1, FFN2
-  LnLaunch ln[2];           // after the O projection, after FFN2
-  const uint16_t* qkv;      // attention operands / result, as in launch_attention
-  uint16_t* attn_out;
-  const int32_t* seq_lens;
-  int n_kept_heads, batch, seq, T;
-  unsigned int* barrier;    // one counter per launch, zero when the kernel starts
-  const uint8_t* pf_ptr[4]; // the next layer's packed shards, tile descriptors and dense parameters,
-  uint32_t pf_bytes[4];     // pulled into L2 while this layer computes
-  int* err;
-};
-
-constexpr int kFusedMaxCtas = 148;
-cudaError_t fused_configure();
-// Shared memory the attention step needs for sequences of `seq` tokens, counted from the start of the
-// activation area; the O-projection tile may be decoded ahead only if it fits above that.
-size_t fused_attention_bytes(int seq);
-size_t fused_smem_total();      // dynamic shared memory of the kernel
-size_t fused_low_offset();      // where the activation stages / attention buffers start
-cudaError_t launch_fused_layer(const FusedLayerParams& p, int grid, cudaStream_t s, bool pdl);
-
 // Launch with or without the programmatic-dependent-launch attribute (every kernel of the layer calls
 // pdl_wait before it reads what its predecessor wrote, so consecutive kernels may overlap their prologues).
+// `cluster_x` > 1 groups that many consecutive CTAs along x into one thread-block cluster.
 template <typename... KArgs, typename... Args>
-inline cudaError_t launch_kernel(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t s, bool pdl,
-                                 Args... args) {
+inline cudaError_t launch_kernel_cluster(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t s,
+                                         bool pdl, unsigned cluster_x, Args... args) {
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = grid;
   cfg.blockDim = block;
   cfg.dynamicSmemBytes = smem;
   cfg.stream = s;
-  cudaLaunchAttribute attr[1];
-  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cudaLaunchAttribute attr[2];
+  unsigned n = 0;
+  if (pdl) {
+    attr[n].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[n].val.programmaticStreamSerializationAllowed = 1;
+    ++n;
+  }
+  if (cluster_x > 1) {
+    attr[n].id = cudaLaunchAttributeClusterDimension;
+    attr[n].val.clusterDim.x = cluster_x; attr[n].val.clusterDim.y = 1; attr[n].val.clusterDim.z = 1;
+    ++n;
+  }
   cfg.attrs = attr;
-  cfg.numAttrs = pdl ? 1 : 0;
+  cfg.numAttrs = n;
   return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_kernel(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t s, bool pdl,
+                                 Args... args) {
+  return launch_kernel_cluster(kernel, grid, block, smem, s, pdl, 1u, args...);
 }
 
 constexpr int ERR_NONE = 0;
