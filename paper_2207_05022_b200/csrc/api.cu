@@ -22,8 +22,6 @@ constexpr int kMaxLayersStats = 64;
 constexpr size_t kMaxSmem = 227 * 1024;
 constexpr int kStampKernels = 8;       // per layer: cast, QKV, attention, O projection, LayerNorm 1, FFN1, FFN2, LayerNorm 2
 constexpr int kStampRecord = 8;        // 64-bit words per kernel launch (kStampWords of the device code)
-constexpr int kLnCounters = 64;        // arrival counters per LayerNorm epilogue launch (token-tile groups x cluster ranks)
-constexpr int kLnMaxTiles = 32;        // most column tiles of a row (hidden <= 2048, 64-feature tiles)
 
 inline size_t align16(size_t v) { return (v + 15) & ~static_cast<size_t>(15); }
 inline size_t align256(size_t v) { return (v + 255) & ~static_cast<size_t>(255); }
@@ -38,8 +36,6 @@ struct Tuning {
   int cta_budget = 148;                // CTAs a GEMM launch may use when it splits the token tiles over CTAs
   int pair_min_tiles = 8;              // two-CTA GEMM from this many 128-token tiles on (0 = never)
   int ln1_ctas = -1, ln2_ctas = -1;    // LayerNorm CTA counts: -1 = chosen per launch (see ln_ctas_hint), 0 = one row per CTA
-  int ln_fuse = 0;                     // residual + LayerNorm in the epilogue of the O projection and of FFN2 (few tokens)
-  int ln_o_split = 8, ln_f2_split = 8; // most K splits (= CTAs per cluster) of a column tile in that form
 };
 
 struct Unit {
@@ -72,7 +68,6 @@ struct Layer {
   int slot = -1;                       // ring slot of the streamed part
   size_t tables_off = 0, tables_bytes = 0;   // this layer's tile-job descriptors inside the plan's table buffer
   GemmTable qkv, o, f1, f2;
-  GemmTable o_ln, f2_ln;               // O projection / FFN2 tiled for the LayerNorm epilogue (K splits of a column tile adjacent)
   cudaEvent_t ev_loaded = nullptr, ev_done = nullptr, ev_copy_start = nullptr, ev_comp_start = nullptr;
   cudaEvent_t g_ev_loaded = nullptr;   // the same role inside graph capture (captured events cannot be reused outside)
   cudaEvent_t ev_k[8] = {};           // boundaries of the seven kernels (kernel-level profiling)
@@ -95,7 +90,6 @@ struct sti_ctx {
   bool simt_debug = false;
   bool pdl = true;                     // programmatic dependent launch between the kernels of a layer
   int sm_count = 0;
-  int max_clusters[9] = {};            // clusters of 1..8 full-shared-memory GEMM CTAs the device holds at once
   sti_status async_error = STI_OK;
   MatrixInfo attn_m[4]{}, ffn_m[2]{};
   uint32_t attn_weights = 0, ffn_weights = 0;
@@ -141,12 +135,8 @@ struct sti_plan {
   void* x_in = nullptr; void* y_out = nullptr; int32_t* lens_dev = nullptr;
   int max_partial = 1;
   float* zero_bias = nullptr;          // all-zero bias vector of sti_gemm_probe (allocated by its first call)
-  // LayerNorm epilogue scratch: arrival counters (per layer and LayerNorm, zeroed at the start of every forward) and the
-  // per-column-tile row statistics of the two LayerNorms
-  unsigned int* ln_ctr = nullptr;
   unsigned long long* stamps = nullptr;   // [layer][kStampKernels][kStampWords] device, profiling level 3
   bool stamping = false;               // the forward being enqueued writes stamps
-  float2* ln_stats[2] = {nullptr, nullptr};
   bool overlap = true;                 // false: load every streamed layer, then execute (Load&Exec)
   int n_streamed_layers = 0;
   bool stats_valid = false;
@@ -206,9 +196,6 @@ void parse_tuning(Tuning* t, int tmax, const sti_model_desc& d, int sm_count) {
         else if (k == "f2_group") t->f2_group = v;
         else if (k == "pair_min_tiles") t->pair_min_tiles = v;
         else if (k == "cta_budget") t->cta_budget = std::max(1, v);
-        else if (k == "ln_fuse") t->ln_fuse = v != 0;
-        else if (k == "ln_o_split") t->ln_o_split = std::max(1, std::min(8, v));
-        else if (k == "ln_f2_split") t->ln_f2_split = std::max(1, std::min(8, v));
         else if (k == "ln1_ctas") t->ln1_ctas = std::max(-1, v);
         else if (k == "ln2_ctas") t->ln2_ctas = std::max(-1, v);
       }
@@ -291,7 +278,7 @@ struct TableBuilder {
   }
 };
 
-void build_layer_tables(sti_plan* p, Layer& L, TableBuilder tb[6]) {
+void build_layer_tables(sti_plan* p, Layer& L, TableBuilder tb[4]) {
   const sti_ctx* c = p->ctx;
   const sti_model_desc& d = c->desc;
   const Tuning& t = p->tune;
@@ -349,35 +336,6 @@ void build_layer_tables(sti_plan* p, Layer& L, TableBuilder tb[6]) {
       tb[3].add(j, ss);
     }
   }
-  // The same two GEMMs tiled for the LayerNorm epilogue: the K splits of a column tile are adjacent jobs (one
-  // thread-block cluster), at most 8 of them, and column tiles times splits stay within the CTA budget.
-  auto ln_tables = [&](TableBuilder& out, GemmTable& gt, const std::vector<int>& kept, std::vector<Unit>& units,
-                       sti_kind kind, int matrix, uint32_t tile_n, uint32_t unit_k, int max_split) {
-    const int n = static_cast<int>(kept.size());
-    gt.n_split = 0;
-    if (n == 0 || (tile_n != 64 && tile_n != 128)) return;
-    const int n_nt = d.hidden / static_cast<int>(tile_n);
-    int c_target = std::max(1, std::min(std::min(8, max_split), t.cta_budget / std::max(1, n_nt)));
-    while (c_target > 1 && c->max_clusters[c_target] < n_nt) --c_target;     // every column tile's cluster resident at once
-    int group = (n + c_target - 1) / c_target;
-    // the tile of one split must fit in shared memory next to a small activation ring
-    while (group > 1 && gemm_weight_bytes(tile_n, group * unit_k) > 128 * 1024) --group;
-    gt.n_split = (n + group - 1) / group;
-    if (gt.n_split > 8) { gt.n_split = 0; return; }
-    for (uint32_t n0 = 0; n0 < static_cast<uint32_t>(d.hidden); n0 += tile_n)
-      for (int sp = 0; sp < gt.n_split; ++sp) {
-        const int first = sp * group, cnt = std::min(group, n - first);
-        Job j{};
-        j.n_rows = tile_n; j.k_total = cnt * unit_k; j.x_koff = first * unit_k;
-        j.out_mat = sp; j.out_col = n0; j.bias_off = -1;
-        std::vector<Seg> ss;
-        for (int i = 0; i < cnt; ++i)
-          ss.push_back(make_seg(c, units[kept[first + i]], kind, matrix, n0, tile_n, i * unit_k));
-        out.add(j, ss);
-      }
-  };
-  ln_tables(tb[4], L.o_ln, L.kept_heads, L.attn, STI_ATTN, 3, t.o_n, 64, t.ln_o_split);
-  ln_tables(tb[5], L.f2_ln, L.kept_slices, L.ffn, STI_FFN, 1, std::max(64, t.f2_n), f, t.ln_f2_split);
 }
 
 sti_status check_async(sti_ctx* c) {
@@ -441,41 +399,16 @@ void layer_ranges(const sti_plan* p, int li, const uint8_t* ptr[4], uint32_t byt
   bytes[3] = static_cast<uint32_t>(p->ctx->dense_stride * sizeof(float));
 }
 
-// Can this table run with the LayerNorm epilogue for T tokens?  Every CTA of the launch must be resident at the same
-// time (the column tiles of a row wait for one another), a CTA's token tiles must all fit in tensor memory, and the
-// exchange buffer in shared memory.
-// CTAs along the token dimension for a table in the LayerNorm form: as many as the CTA budget allows while the
-// whole launch (column tiles x token groups clusters of n_split CTAs) can be resident at once.
-int ln_m_ctas(const sti_plan* p, const GemmTable& tab, int T) {
-  const int n_nt = tab.n_jobs / tab.n_split;
-  const int by_clusters = tab.n_split <= 8 ? p->ctx->max_clusters[tab.n_split] / std::max(1, n_nt) : 0;
-  return std::max(1, std::min(m_ctas_for(tab.n_jobs, T, p->tune.cta_budget), by_clusters));
-}
-
-bool ln_form_fits(const sti_plan* p, const GemmTable& tab, int T) {
-  if (tab.n_jobs == 0 || tab.n_split < 1 || !p->tune.ln_fuse || p->ctx->simt_debug) return false;
-  const int m_ctas = ln_m_ctas(p, tab, T);
-  const int n_mtiles = (T + 127) / 128;
-  const int my_mtiles = (n_mtiles + m_ctas - 1) / m_ctas;
-  const uint32_t n_rows = static_cast<uint32_t>(p->ctx->desc.hidden / (tab.n_jobs / tab.n_split));
-  if (tab.n_split > 8 || (tab.n_jobs / tab.n_split) * m_ctas > p->ctx->max_clusters[tab.n_split] ||
-      m_ctas * tab.n_split > kLnCounters)
-    return false;
-  if (my_mtiles * n_rows > 512) return false;
-  return tab.hdr_bytes + gemm_ln_exchange_bytes(my_mtiles, n_rows) <= kMaxSmem;
-}
-
 // `force_pair`: -1 = the two-CTA kernel from pair_min_tiles token tiles on, 0 = never, 1 = always (the table must allow it).
-// `ln`: the LayerNorm epilogue's parameters (kind GEMM_BF16_TO_LN; the table is in that form and ln_form_fits said yes).
 sti_status run_gemm(sti_plan* p, GemmKind kind, const GemmTable& tab, const void* x, int ldx, int T, void* out,
-                    int ldo, const float* bias, int prefetch_layer = -1, int force_pair = -1, const LnEpilogue* ln = nullptr,
+                    int ldo, const float* bias, int prefetch_layer = -1, int force_pair = -1,
                     unsigned long long* stamps = nullptr) {
   if (tab.n_jobs == 0) return STI_OK;
   GemmLaunch g{};
   g.stamps = stamps;
   g.jobs = tab.jobs; g.segs = tab.segs; g.n_jobs = tab.n_jobs; g.m_ctas = m_ctas_for(tab.n_jobs, T, p->tune.cta_budget);
   const int n_mtiles = (T + 127) / 128;
-  g.pair = !ln && tab.pair_ok && p->tune.pair_min_tiles > 0 && n_mtiles >= p->tune.pair_min_tiles;
+  g.pair = tab.pair_ok && p->tune.pair_min_tiles > 0 && n_mtiles >= p->tune.pair_min_tiles;
   if (force_pair == 0) g.pair = false;
   if (force_pair == 1) {
     if (!tab.pair_ok) return STI_ERR_STATE;
@@ -489,20 +422,6 @@ sti_status run_gemm(sti_plan* p, GemmKind kind, const GemmTable& tab, const void
   layer_ranges(p, prefetch_layer, g.pf_ptr, g.pf_bytes);
   g.x = x; g.ldx = ldx; g.T = T; g.out = out; g.ldo = ldo; g.bias = bias; g.err = p->ctx->err_dev;
   g.smem_bytes = tab.smem; g.n_stages = tab.n_stages; g.bps = tab.bps; g.w_bytes = tab.w_bytes; g.hdr_bytes = tab.hdr_bytes; g.seg_stride = tab.seg_stride; g.simt_debug = p->ctx->simt_debug; g.pdl = p->ctx->pdl;
-  if (ln) {
-    if (kind != GEMM_BF16_TO_LN) return STI_ERR_ARG;
-    g.ln = *ln;
-    g.m_ctas = ln_m_ctas(p, tab, T);
-    // the exchange buffer reuses the activation ring and the weight tile; widen the latter if they are too small
-    const uint32_t n_rows = static_cast<uint32_t>(ln->d / ln->n_ntiles);
-    const size_t need = gemm_ln_exchange_bytes((n_mtiles + g.m_ctas - 1) / g.m_ctas, n_rows);
-    const size_t have = gemm_smem_bytes(g.w_bytes, g.n_stages, g.bps, 0);
-    if (need > have) {
-      g.w_bytes += static_cast<uint32_t>(need - have);
-      g.smem_bytes = gemm_smem_bytes(g.w_bytes, g.n_stages, g.bps, g.hdr_bytes);
-    }
-    if (g.smem_bytes > kMaxSmem) return STI_ERR_SHAPE;
-  }
   CUDA_TRY(launch_gemm(kind, g, p->ctx->compute));
   p->ctx->launches++;
   return STI_OK;
@@ -537,17 +456,8 @@ sti_status enqueue_layer(sti_plan* p, int li, const void* x, void* y, int batch,
   const bool kprof = p->profiling >= 2;
   auto mark = [&](int i) -> cudaError_t { return kprof ? cudaEventRecord(L.ev_k[i], c->compute) : cudaSuccess; };
   for (bool& r : L.k_ran) r = false;
-  const bool ln1_fused = nh > 0 && ln_form_fits(p, L.o_ln, T), ln2_fused = ns > 0 && ln_form_fits(p, L.f2_ln, T);
   auto stamp = [&](int kernel) -> unsigned long long* {
     return p->stamping ? p->stamps + (static_cast<size_t>(li) * kStampKernels + kernel) * kStampRecord : nullptr;
-  };
-  auto ln_params = [&](const GemmTable& tab, int which) {
-    LnEpilogue e{};
-    e.stats = p->ln_stats[which];
-    e.counters = p->ln_ctr + (static_cast<size_t>(li) * 2 + which) * kLnCounters;
-    e.eps = d.ln_eps; e.d = d.hidden;
-    e.n_ntiles = tab.n_jobs / tab.n_split; e.cluster = tab.n_split;
-    return e;
   };
   CUDA_TRY(mark(0));
   if (nh > 0) {
@@ -561,22 +471,13 @@ sti_status enqueue_layer(sti_plan* p, int li, const void* x, void* y, int batch,
       }
       xq = p->x_bf16;
     }
-    st = run_gemm(p, GEMM_BF16_TO_BF16, L.qkv, xq, d.hidden, T, p->qkv, 64, dense + c->off_bq, next_layer, -1, nullptr, stamp(1));
+    st = run_gemm(p, GEMM_BF16_TO_BF16, L.qkv, xq, d.hidden, T, p->qkv, 64, dense + c->off_bq, next_layer, -1, stamp(1));
     if (st != STI_OK) return st;
     CUDA_TRY(mark(1));
     CUDA_TRY(launch_attention(p->qkv, p->attn_out, nh, batch, seq, lens, c->compute, c->pdl, stamp(2)));
     c->launches++;
     CUDA_TRY(mark(2));
-    if (ln1_fused) {
-      // O projection + bias + residual + LayerNorm in one launch (no partial sums in global memory)
-      LnEpilogue e = ln_params(L.o_ln, 0);
-      e.bias = dense + c->off_bo; e.resid = x; e.resid_bf16 = bf16_act ? 1 : 0;
-      e.gamma = dense + c->off_ln1g; e.beta = dense + c->off_ln1b;
-      e.out_f32 = p->h1_f32; e.out_bf16 = p->h1_bf16;
-      st = run_gemm(p, GEMM_BF16_TO_LN, L.o_ln, p->attn_out, nh * 64, T, nullptr, d.hidden, nullptr, -1, 0, &e, stamp(3));
-    } else {
-      st = run_gemm(p, GEMM_BF16_TO_F32, L.o, p->attn_out, nh * 64, T, p->partial, d.hidden, nullptr, -1, -1, nullptr, stamp(3));
-    }
+    st = run_gemm(p, GEMM_BF16_TO_F32, L.o, p->attn_out, nh * 64, T, p->partial, d.hidden, nullptr, -1, -1, stamp(3));
     if (st != STI_OK) return st;
     L.k_ran[0] = L.k_ran[1] = L.k_ran[2] = true;
   } else {
@@ -584,7 +485,7 @@ sti_status enqueue_layer(sti_plan* p, int li, const void* x, void* y, int batch,
     CUDA_TRY(mark(2));
   }
   CUDA_TRY(mark(3));
-  if (!ln1_fused) {
+  {
     LnLaunch ln{};
     ln.partial = p->partial; ln.n_partial = nh > 0 ? L.o.n_split : 0;
     ln.bias = dense + c->off_bo; ln.resid = x; ln.resid_bf16 = bf16_act ? 1 : 0;
@@ -598,29 +499,16 @@ sti_status enqueue_layer(sti_plan* p, int li, const void* x, void* y, int batch,
   }
   CUDA_TRY(mark(4));
   if (ns > 0) {
-    st = run_gemm(p, GEMM_BF16_TO_BF16_GELU, L.f1, p->h1_bf16, d.hidden, T, p->u, ns * f, dense + c->off_b1, -1, -1, nullptr, stamp(5));
+    st = run_gemm(p, GEMM_BF16_TO_BF16_GELU, L.f1, p->h1_bf16, d.hidden, T, p->u, ns * f, dense + c->off_b1, -1, -1, stamp(5));
     if (st != STI_OK) return st;
     CUDA_TRY(mark(5));
-    if (ln2_fused) {
-      LnEpilogue e = ln_params(L.f2_ln, 1);
-      e.bias = dense + c->off_b2; e.resid = p->h1_f32; e.resid_bf16 = 0;
-      e.gamma = dense + c->off_ln2g; e.beta = dense + c->off_ln2b;
-      e.out_f32 = bf16_act ? nullptr : static_cast<float*>(y);
-      e.out_bf16 = bf16_act ? static_cast<uint16_t*>(y) : (want_next_bf16 ? p->x_bf16 : nullptr);
-      st = run_gemm(p, GEMM_BF16_TO_LN, L.f2_ln, p->u, ns * f, T, nullptr, d.hidden, nullptr, -1, 0, &e, stamp(6));
-    } else {
-      st = run_gemm(p, GEMM_BF16_TO_F32, L.f2, p->u, ns * f, T, p->partial, d.hidden, nullptr, -1, -1, nullptr, stamp(6));
-    }
+    st = run_gemm(p, GEMM_BF16_TO_F32, L.f2, p->u, ns * f, T, p->partial, d.hidden, nullptr, -1, -1, stamp(6));
     if (st != STI_OK) return st;
     L.k_ran[4] = L.k_ran[5] = true;
   } else {
     CUDA_TRY(mark(5));
   }
   CUDA_TRY(mark(6));
-  if (ln2_fused) {
-    CUDA_TRY(mark(7));
-    return STI_OK;
-  }
   LnLaunch l2{};
   l2.partial = p->partial; l2.n_partial = ns > 0 ? L.f2.n_split : 0;
   l2.bias = dense + c->off_b2; l2.resid = p->h1_f32; l2.resid_bf16 = 0;
@@ -744,8 +632,6 @@ sti_status enqueue_forward_io(sti_plan* p, const ForwardKey& k, bool capturing) 
     x = p->x_in;
     y = p->y_out;
   }
-  // the arrival counters of the LayerNorm epilogues start every forward at zero
-  CUDA_TRY(cudaMemsetAsync(p->ln_ctr, 0, p->layers.size() * 2 * kLnCounters * sizeof(unsigned int), c->compute));
   p->stamping = k.stamps;
   if (k.stamps)
     CUDA_TRY(cudaMemsetAsync(p->stamps, 0xff, p->layers.size() * kStampKernels * kStampRecord * sizeof(unsigned long long), c->compute));
@@ -828,7 +714,7 @@ void free_plan_device(sti_plan* p) {
   cudaFree(p->qkv); cudaFree(p->attn_out); cudaFree(p->partial); cudaFree(p->h1_f32); cudaFree(p->h1_bf16);
   cudaFree(p->u); cudaFree(p->x_bf16); cudaFree(p->buf[0]); cudaFree(p->buf[1]); cudaFree(p->x_in); cudaFree(p->y_out);
   cudaFree(p->lens_dev);
-  cudaFree(p->ln_ctr); cudaFree(p->ln_stats[0]); cudaFree(p->ln_stats[1]); cudaFree(p->stamps);
+  cudaFree(p->stamps);
   cudaFree(p->zero_bias);
   for (auto& L : p->layers) {
     if (L.ev_loaded) cudaEventDestroy(L.ev_loaded);
@@ -926,12 +812,6 @@ sti_status sti_ctx_create(const sti_model_desc* desc, int device, void* compute_
     return fail(STI_ERR_CUDA);
   if (cudaDeviceGetAttribute(&c->sm_count, cudaDevAttrMultiProcessorCount, device) != cudaSuccess || c->sm_count < 1)
     return fail(STI_ERR_CUDA);
-  for (unsigned cx = 1; cx <= 8; ++cx) c->max_clusters[cx] = gemm_max_active_clusters(cx, kMaxSmem);
-  if (getenv("STI_VERBOSE")) {
-    fprintf(stderr, "sti: %d SMs; resident clusters of 1..8 GEMM CTAs:", c->sm_count);
-    for (int cx = 1; cx <= 8; ++cx) fprintf(stderr, " %d", c->max_clusters[cx]);
-    fprintf(stderr, "\n");
-  }
   const char* dbg = getenv("STI_DEBUG_SIMT");
   c->simt_debug = dbg && dbg[0] == '1';
   const char* nopdl = getenv("STI_NO_PDL");
@@ -1124,28 +1004,25 @@ sti_status sti_plan_finalize(sti_plan* p) {
   std::vector<Fix> fixes;
   p->max_partial = 1;
   for (auto& L : p->layers) {
-    TableBuilder tb[6];
+    TableBuilder tb[4];
     L.tables_off = align16(host_tables.size());
     build_layer_tables(p, L, tb);
-    GemmTable* gt[6] = {&L.qkv, &L.o, &L.f1, &L.f2, &L.o_ln, &L.f2_ln};
-    for (int i = 0; i < 6; ++i) {
+    GemmTable* gt[4] = {&L.qkv, &L.o, &L.f1, &L.f2};
+    for (int i = 0; i < 4; ++i) {
       tb[i].finish();
       gt[i]->seg_stride = tb[i].seg_stride;
       gt[i]->n_jobs = static_cast<int>(tb[i].jobs.size());
       gt[i]->w_bytes = tb[i].w_bytes;
       gt[i]->n_stages = 2; gt[i]->bps = 1;
       gt[i]->hdr_bytes = gemm_header_bytes();
-      gt[i]->pair_ok = i < 4 && !tb[i].jobs.empty() && tb[i].jobs.size() % 2 == 0;
+      gt[i]->pair_ok = !tb[i].jobs.empty() && tb[i].jobs.size() % 2 == 0;
       for (size_t j = 0; gt[i]->pair_ok && j < tb[i].jobs.size(); j += 2) {
         const Job &a = tb[i].jobs[j], &b = tb[i].jobs[j + 1];
         gt[i]->pair_ok = a.n_rows == 64 && b.n_rows == 64 && a.k_total == b.k_total && a.x_koff == b.x_koff;
       }
       if (!tb[i].jobs.empty() &&
-          !gemm_pick_ring(tb[i].w_bytes, tb[i].k_max, gt[i]->hdr_bytes, &gt[i]->n_stages, &gt[i]->bps)) {
-        if (i < 4) return STI_ERR_SHAPE;
-        tb[i] = TableBuilder();          // the LayerNorm form is optional: fall back to partial sums + LayerNorm kernel
-        gt[i]->n_jobs = 0; gt[i]->n_split = 0;
-      }
+          !gemm_pick_ring(tb[i].w_bytes, tb[i].k_max, gt[i]->hdr_bytes, &gt[i]->n_stages, &gt[i]->bps))
+        return STI_ERR_SHAPE;
       gt[i]->smem = gemm_smem_bytes(tb[i].w_bytes, gt[i]->n_stages, gt[i]->bps, gt[i]->hdr_bytes);
       if (gt[i]->smem > kMaxSmem && !tb[i].jobs.empty()) return STI_ERR_SHAPE;
       Fix fx{gt[i], 0, 0};
@@ -1183,9 +1060,6 @@ sti_status sti_plan_finalize(sti_plan* p) {
   CUDA_TRY(cudaMalloc(&p->x_in, Tmax * d.hidden * act_size(c)));
   CUDA_TRY(cudaMalloc(&p->y_out, Tmax * d.hidden * act_size(c)));
   CUDA_TRY(cudaMalloc(&p->lens_dev, static_cast<size_t>(d.max_batch) * 4));
-  CUDA_TRY(cudaMalloc(&p->ln_ctr, static_cast<size_t>(d.n_layers) * 2 * kLnCounters * sizeof(unsigned int)));
-  CUDA_TRY(cudaMemset(p->ln_ctr, 0, static_cast<size_t>(d.n_layers) * 2 * kLnCounters * sizeof(unsigned int)));
-  for (auto& st : p->ln_stats) CUDA_TRY(cudaMalloc(&st, Tmax * kLnMaxTiles * sizeof(float2)));
   CUDA_TRY(cudaMalloc(&p->stamps, static_cast<size_t>(d.n_layers) * kStampKernels * kStampRecord * sizeof(unsigned long long)));
   // 5. events
   const unsigned flags = cudaEventDefault;     // timing-capable; only recorded when profiling
@@ -1300,7 +1174,7 @@ sti_status sti_shard_decode(sti_plan* p, int layer, sti_kind kind, int index, in
 
 sti_status sti_gemm_probe(sti_plan* p, int layer, int gemm, const void* x_bf16_dev, int tokens, void* out_dev,
                           size_t out_capacity_bytes, int variant, int32_t* n_partials) {
-  if (!p || !x_bf16_dev || !out_dev || gemm < 0 || gemm > 3 || variant < 0 || variant > 3) return STI_ERR_ARG;
+  if (!p || !x_bf16_dev || !out_dev || gemm < 0 || gemm > 3 || variant < 0 || variant > 2) return STI_ERR_ARG;
   if (layer < 0 || layer >= static_cast<int>(p->layers.size())) return STI_ERR_ARG;
   if (tokens < 1 || tokens > 65536) return STI_ERR_SHAPE;
   if ((reinterpret_cast<uintptr_t>(x_bf16_dev) & 15) || (reinterpret_cast<uintptr_t>(out_dev) & 15)) return STI_ERR_ARG;
@@ -1312,11 +1186,9 @@ sti_status sti_gemm_probe(sti_plan* p, int layer, int gemm, const void* x_bf16_d
   Layer& L = p->layers[layer];
   const int nh = static_cast<int>(L.kept_heads.size()), ns = static_cast<int>(L.kept_slices.size());
   const int f = d.ffn / d.n_ffn_slices;
-  // variant 3: the O projection / FFN2 tile tables of the LayerNorm-epilogue form (QKV and FFN1 have one form only)
-  const bool ln_tables = variant == 3 && (gemm == 1 || gemm == 3);
-  const GemmTable* tabs[4] = {&L.qkv, ln_tables ? &L.o_ln : &L.o, &L.f1, ln_tables ? &L.f2_ln : &L.f2};
+  const GemmTable* tabs[4] = {&L.qkv, &L.o, &L.f1, &L.f2};
   const GemmTable& tab = *tabs[gemm];
-  if (tab.n_jobs == 0) return STI_ERR_STATE;               // no kept unit feeds this GEMM (or the form is not available)
+  if (tab.n_jobs == 0) return STI_ERR_STATE;               // no kept unit feeds this GEMM
   const int ldx[4] = {d.hidden, nh * 64, d.hidden, ns * f};
   const int ldo[4] = {64, d.hidden, ns * f, d.hidden};
   const int parts[4] = {1, tabs[1]->n_split, 1, tabs[3]->n_split};
@@ -1335,7 +1207,7 @@ sti_status sti_gemm_probe(sti_plan* p, int layer, int gemm, const void* x_bf16_d
   }
   const GemmKind kind = (gemm == 1 || gemm == 3) ? GEMM_BF16_TO_F32 : GEMM_BF16_TO_BF16;
   st = run_gemm(p, kind, tab, x_bf16_dev, ldx[gemm], tokens, out_dev, ldo[gemm], p->zero_bias, -1,
-                variant == 0 ? -1 : (variant == 3 ? 0 : variant - 1));
+                variant == 0 ? -1 : variant - 1);
   if (st != STI_OK) return st;
   if (L.str_bytes > 0) CUDA_TRY(cudaEventRecord(p->slot_free[L.slot], c->compute));
   if (n_partials) *n_partials = parts[gemm];

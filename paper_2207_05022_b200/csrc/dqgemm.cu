@@ -96,164 +96,18 @@ __device__ __forceinline__ void epilogue_tile(uint32_t taddr, uint32_t half, uin
 }
 
 
-// ---------------------------------------------------------------------------------------
-// GEMM_BF16_TO_LN epilogue (Section 2.1: residual connection and layer normalisation after the attention output
-// projection and after the second FFN layer; Section 6: biases and LayerNorm parameters stay in fp32).
-//
-// The CTA holds, in tensor memory, its K split's partial sums for `my_mtiles` token tiles x n_rows features.
-//   1. all warps move the accumulators to shared memory (`red`, row-major, padded rows);
-//   2. cluster barrier; rank r of the cluster owns every c-th slice of the rows and adds up the c partial
-//      sums of its rows out of the c CTAs' shared memories (fixed order), plus bias and residual;
-//   3. per row: mean and sum of squared deviations over this column tile, written to `stats`; the CTAs of the
-//      other column tiles that own the same rows do the same, a counter tells when all of them have;
-//   4. the per-tile statistics are merged (equal counts: mean of means, sum of squares about the common mean),
-//      the rows are normalised and stored.
-// Every CTA passes both cluster barriers and bumps its counter whether or not it has valid data, so that one
-// CTA's bounded wait running out cannot hold up the others for more than their own bound.
-// Returns false when the wait for the other column tiles ran out.
-// ---------------------------------------------------------------------------------------
-__device__ __forceinline__ bool ln_epilogue(const LnEpilogue& ln, const Job& job, float* red, uint32_t tmem_base,
-                                            uint32_t n_rows, uint32_t my_mtiles, int T, uint32_t tid, bool acc_ok,
-                                            volatile uint32_t* abort_flag, unsigned long long* stamps) {
-  const uint32_t lane = tid & 31, warp = tid >> 5;
-  const uint32_t stride = n_rows + 4;                 // floats per row of the exchange buffer
-  const uint32_t R = my_mtiles * kTileM;              // rows this CTA has partial sums for
-  if (acc_ok) {
-    const uint32_t q = warp & 3, cs = warp >> 2, ncol = n_rows / 4;   // TMEM lane quadrant, quarter of the columns
-    for (uint32_t ti = 0; ti < my_mtiles; ++ti) {
-      float* dst = red + static_cast<size_t>(ti * kTileM + q * 32 + lane) * stride + cs * ncol;
-#pragma unroll 1
-      for (uint32_t c0 = 0; c0 < ncol; c0 += 16) {
-        uint32_t v[16];
-        tmem_ld_32x32b_x16(tmem_base + ((q * 32) << 16) + ti * n_rows + cs * ncol + c0, v);
-        tc_wait_ld();
-#pragma unroll
-        for (int i = 0; i < 4; ++i)
-          reinterpret_cast<float4*>(dst + c0)[i] = make_float4(__uint_as_float(v[4 * i]), __uint_as_float(v[4 * i + 1]),
-                                                               __uint_as_float(v[4 * i + 2]), __uint_as_float(v[4 * i + 3]));
-      }
-    }
-  }
-  tc_fence_before_sync();
-  cluster_sync_all();                                 // every CTA's partial sums are in its shared memory
-
-  const uint32_t c = cluster_nctas(), r = cluster_ctarank();
-  const uint32_t rows_per = (R + c - 1) / c;
-  const uint32_t row_lo = r * rows_per;
-  const uint32_t row_hi = row_lo + rows_per < R ? row_lo + rows_per : R;
-  const uint32_t g = n_rows / 4;                      // threads per row (16 or 32), four features each
-  const uint32_t rpp = kThreads / g;                  // rows per pass
-  const uint32_t sub = tid % g, col0 = sub * 4;
-  const uint32_t red_addr = smem_addr(red);
-  const uint32_t nt = job.out_col / n_rows;           // this CTA's column tile
-  const float inv_n = 1.0f / static_cast<float>(n_rows);
-  auto token_of = [&](uint32_t lr) {
-    return static_cast<int>((blockIdx.y + (lr / kTileM) * gridDim.y) * kTileM + lr % kTileM);
-  };
-  auto group_sum = [&](float v) {                     // over the g lanes that share a row
-    for (uint32_t o = g >> 1; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
-    return v;
-  };
-  for (uint32_t base = row_lo; base < row_hi; base += rpp) {
-    const uint32_t lr = base + tid / g;
-    const int t = token_of(lr);
-    const bool valid = acc_ok && lr < row_hi && t < T;
-    float4 z = make_float4(0.f, 0.f, 0.f, 0.f);
-    if (valid) {
-      const uint32_t off = red_addr + (lr * stride + col0) * 4;
-      for (uint32_t peer = 0; peer < c; ++peer) {
-        const float4 v = ld_dsmem_f4(map_to_cta(off, peer));
-        z.x += v.x; z.y += v.y; z.z += v.z; z.w += v.w;
-      }
-      const float4 b = __ldg(reinterpret_cast<const float4*>(ln.bias + job.out_col + col0));
-      const size_t gi = static_cast<size_t>(t) * ln.d + job.out_col + col0;
-      float4 x;
-      if (ln.resid_bf16) {
-        const uint2 rr = *reinterpret_cast<const uint2*>(static_cast<const uint16_t*>(ln.resid) + gi);
-        x = make_float4(__uint_as_float(rr.x << 16), __uint_as_float(rr.x & 0xffff0000u), __uint_as_float(rr.y << 16),
-                        __uint_as_float(rr.y & 0xffff0000u));
-      } else {
-        x = *reinterpret_cast<const float4*>(static_cast<const float*>(ln.resid) + gi);
-      }
-      z.x += b.x + x.x; z.y += b.y + x.y; z.z += b.z + x.z; z.w += b.w + x.w;
-    }
-    const float mean_loc = group_sum((z.x + z.y) + (z.z + z.w)) * inv_n;
-    const float dx = z.x - mean_loc, dy = z.y - mean_loc, dz = z.z - mean_loc, dw = z.w - mean_loc;
-    const float m2_loc = group_sum((dx * dx + dy * dy) + (dz * dz + dw * dw));
-    if (valid) {
-      // the rows this CTA owns are read by nobody else: keep the sums where the partial sums were
-      *reinterpret_cast<float4*>(red + static_cast<size_t>(lr) * stride + col0) = z;
-      if (sub == 0) ln.stats[static_cast<size_t>(t) * ln.n_ntiles + nt] = make_float2(mean_loc, m2_loc);
-    }
-  }
-  cluster_arrive_release();                           // done reading the other CTAs' shared memory
-  __syncthreads();
-  bool ok = true;
-  if (tid == 0) {
-    unsigned int* ctr = ln.counters + blockIdx.y * c + r;   // shared by the column tiles that own the same rows
-    __threadfence();                                  // the CTA's statistics before the count
-    atomicAdd(ctr, 1u);
-    const uint32_t want = static_cast<uint32_t>(ln.n_ntiles);
-    if (ld_acquire_gpu(ctr) < want) {
-      const uint64_t t0 = global_timer_ns();
-      for (;;) {
-        __nanosleep(40);
-        if (ld_acquire_gpu(ctr) >= want) break;
-        if (global_timer_ns() - t0 > 2000000000ull) { *abort_flag = 2; break; }
-      }
-    }
-    __threadfence();
-    stamp_max(stamps, STAMP_EXCHANGED);
-  }
-  __syncthreads();
-  if (*abort_flag == 2) ok = false;
-  const float inv_nt = 1.0f / static_cast<float>(ln.n_ntiles), inv_d = 1.0f / static_cast<float>(ln.d);
-  for (uint32_t base = row_lo; base < row_hi; base += rpp) {
-    const uint32_t lr = base + tid / g;
-    const int t = token_of(lr);
-    const bool valid = acc_ok && ok && lr < row_hi && t < T;
-    // every lane of the row takes the statistics of up to two column tiles (at most 32 tiles: d <= 2048)
-    float2 sa = make_float2(0.f, 0.f), sb = make_float2(0.f, 0.f);
-    const bool has_a = valid && sub < static_cast<uint32_t>(ln.n_ntiles);
-    const bool has_b = valid && sub + g < static_cast<uint32_t>(ln.n_ntiles);
-    if (has_a) sa = __ldcg(ln.stats + static_cast<size_t>(t) * ln.n_ntiles + sub);
-    if (has_b) sb = __ldcg(ln.stats + static_cast<size_t>(t) * ln.n_ntiles + sub + g);
-    const float mean = group_sum(sa.x + sb.x) * inv_nt;
-    const float da = sa.x - mean, db = sb.x - mean;
-    const float dev = (has_a ? sa.y + static_cast<float>(n_rows) * da * da : 0.f) +
-                      (has_b ? sb.y + static_cast<float>(n_rows) * db * db : 0.f);
-    const float var = group_sum(dev) * inv_d;
-    const float rstd = rsqrtf(var + ln.eps);
-    if (valid) {
-      const float4 z = *reinterpret_cast<const float4*>(red + static_cast<size_t>(lr) * stride + col0);
-      const float4 gm = __ldg(reinterpret_cast<const float4*>(ln.gamma + job.out_col + col0));
-      const float4 bt = __ldg(reinterpret_cast<const float4*>(ln.beta + job.out_col + col0));
-      float4 y;
-      y.x = (z.x - mean) * rstd * gm.x + bt.x; y.y = (z.y - mean) * rstd * gm.y + bt.y;
-      y.z = (z.z - mean) * rstd * gm.z + bt.z; y.w = (z.w - mean) * rstd * gm.w + bt.w;
-      const size_t gi = static_cast<size_t>(t) * ln.d + job.out_col + col0;
-      if (ln.out_f32) *reinterpret_cast<float4*>(ln.out_f32 + gi) = y;
-      if (ln.out_bf16) *reinterpret_cast<uint2*>(ln.out_bf16 + gi) = make_uint2(pack_bf16x2(y.x, y.y), pack_bf16x2(y.z, y.w));
-    }
-  }
-  cluster_wait_acquire();                             // nobody leaves while its shared memory may still be read
-  return ok;
-}
-
 template <typename OutT, bool GELU, bool SIMT, bool FEW>
 __global__ void __launch_bounds__(kThreads, 1)
 dqgemm_kernel(const __grid_constant__ CUtensorMap xmap, const Job* __restrict__ jobs, const Seg* __restrict__ segs,
               const __nv_bfloat16* __restrict__ x, int ldx, int T, OutT* __restrict__ out, int ldo,
               const float* __restrict__ bias, int* __restrict__ err, uint32_t n_stages, uint32_t bps,
               uint32_t w_bytes, uint32_t hdr_bytes, uint32_t seg_stride, PrefetchRanges pf, int kind,
-              const __grid_constant__ LnEpilogue ln, unsigned long long* stamps) {
+              unsigned long long* stamps) {
   extern __shared__ __align__(1024) uint8_t smem_raw[];
   uint8_t* smem = smem_raw;
   const uint32_t tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   if (tid == 0) { stamp_min(stamps, STAMP_FIRST_START); stamp_max(stamps, STAMP_LAST_START); }
   const Job job = jobs[blockIdx.x];
-  // LayerNorm epilogue: one accumulator per token tile, all of them kept until the K splits of the cluster meet
-  const bool ln_mode = std::is_void<OutT>::value && !SIMT && kind == GEMM_BF16_TO_LN;
   const Seg* my_segs = segs + static_cast<size_t>(blockIdx.x) * seg_stride;     // independent of the job load
   const uint32_t n_rows = job.n_rows, k_total = job.k_total;
 
@@ -272,7 +126,7 @@ dqgemm_kernel(const __grid_constant__ CUtensorMap xmap, const Job* __restrict__ 
                    (smem_addr(smem_raw) & 1023u) != 0 || job.seg_begin != blockIdx.x * seg_stride || job.n_seg > seg_stride;
   if (bad) {
     if (tid == 0) atomicCAS(err, ERR_NONE, ERR_BAD_JOB);
-    return;               // (a cluster barrier only counts the CTAs that are still running)
+    return;
   }
 
   const int n_mtiles = (T + kTileM - 1) / kTileM;
@@ -281,17 +135,6 @@ dqgemm_kernel(const __grid_constant__ CUtensorMap xmap, const Job* __restrict__ 
   const uint32_t my_mtiles = blockIdx.y < static_cast<uint32_t>(n_mtiles)
                                  ? (n_mtiles - blockIdx.y + gridDim.y - 1) / gridDim.y : 0;
   const uint32_t total = my_mtiles * n_chunks;          // activation chunks this CTA consumes
-  if (ln_mode) {
-    // the whole cluster takes the same decision: these depend on the launch only
-    const bool bad_ln = (n_rows != 64 && n_rows != 128) || my_mtiles * n_rows > 512 || my_mtiles == 0 ||
-                        static_cast<uint32_t>(ln.cluster) != cluster_nctas() || ln.n_ntiles < 1 || ln.n_ntiles > 32 ||
-                        static_cast<uint32_t>(ln.n_ntiles) * n_rows != static_cast<uint32_t>(ln.d) ||
-                        my_mtiles * kTileM * (n_rows + 4) * 4 > n_stages * bps * kBoxBytes + w_bytes;
-    if (bad_ln) {
-      if (tid == 0) atomicCAS(err, ERR_NONE, ERR_BAD_JOB);
-      return;
-    }
-  }
   const uint32_t xsm_addr = smem_addr(xsm);
   // CTAs walk the K range in rotated order so that they do not all ask L2 for the same lines at once
   const uint32_t rot = blockIdx.x % n_chunks;
@@ -316,7 +159,7 @@ dqgemm_kernel(const __grid_constant__ CUtensorMap xmap, const Job* __restrict__ 
   };
 
   uint32_t tmem_cols = 32;
-  while (tmem_cols < (ln_mode ? my_mtiles : 2u) * n_rows) tmem_cols <<= 1;       // two accumulators (LayerNorm: one per token tile)
+  while (tmem_cols < 2 * n_rows) tmem_cols <<= 1;       // two accumulators
   if constexpr (!SIMT) {
     if (tid == 0) {
       for (uint32_t s = 0; s < n_stages; ++s) {
@@ -423,9 +266,9 @@ dqgemm_kernel(const __grid_constant__ CUtensorMap xmap, const Job* __restrict__ 
       // The whole warp runs the loop converged; one elected lane issues.
       uint32_t stage = 0, phase = 0, kc = 0, kcr = rot, ti = 0, issued = 0;
       for (uint32_t c = 0; c < total; ++c) {
-        const uint32_t buf = ln_mode ? ti : (ti & 1);
+        const uint32_t buf = ti & 1;
         bool ok = true;
-        if (!ln_mode && kc == 0 && ti >= 2)        // the epilogue must have drained this accumulator
+        if (kc == 0 && ti >= 2)        // the epilogue must have drained this accumulator
           ok = __all_sync(0xffffffffu, mbar_wait_bounded(smem_addr(&hdr->acc_empty[buf]), ((ti >> 1) - 1) & 1));
         if (ok) ok = __all_sync(0xffffffffu, mbar_wait_bounded(smem_addr(&hdr->full[stage]), phase));
         if (!ok) { failed = true; break; }
@@ -445,10 +288,7 @@ dqgemm_kernel(const __grid_constant__ CUtensorMap xmap, const Job* __restrict__ 
             umma_bf16_ss_x4(d_addr, da, db, 2, b_ks_step, idesc, 1u);
           }
           if (c + n_stages < total) umma_commit(smem_addr(&hdr->empty[stage]));   // only if the stage is refilled
-          if (kc + 1 == n_chunks) {
-            if (!ln_mode) umma_commit(smem_addr(&hdr->acc_full[buf]));
-            else if (c + 1 == total) umma_commit(smem_addr(&hdr->acc_full[0]));    // LayerNorm: everything at once
-          }
+          if (kc + 1 == n_chunks) umma_commit(smem_addr(&hdr->acc_full[buf]));
         }
         __syncwarp();
         issued = c + 1;
@@ -466,7 +306,7 @@ dqgemm_kernel(const __grid_constant__ CUtensorMap xmap, const Job* __restrict__ 
       // ---- otherwise idle: pull the packed shards of a later launch into L2
       const uint32_t n_cta = gridDim.x * gridDim.y, me = (blockIdx.y * gridDim.x + blockIdx.x) * 64 + (tid - 64);
       for (int r = 0; r < 4; ++r) prefetch_range_l2(pf.ptr[r], pf.bytes[r], me, n_cta * 64);
-    } else if (!ln_mode && warp >= kEpilogueWarp0 && warp < kEpilogueWarp0 + kEpilogueWarps) {
+    } else if (warp >= kEpilogueWarp0 && warp < kEpilogueWarp0 + kEpilogueWarps) {
       // ---- epilogue: warp w owns TMEM lanes 32*(w%4).. (token rows) and one half of the columns
       const uint32_t q = warp & 3, half = (warp - kEpilogueWarp0) >> 2, ncol = n_rows / 2;
       for (uint32_t ti = 0; ti < my_mtiles; ++ti) {
@@ -496,22 +336,6 @@ dqgemm_kernel(const __grid_constant__ CUtensorMap xmap, const Job* __restrict__ 
         tc_fence_before_sync();
         __syncwarp();
         if (lane == 0) mbar_arrive(smem_addr(&hdr->acc_empty[buf]));
-      }
-    }
-    if constexpr (std::is_void<OutT>::value) {
-      if (ln_mode) {
-        // all warps: wait for the last accumulator, then the cluster-wide reduction and the LayerNorm
-        uint32_t ok = failed ? 0u : 1u;
-        if (lane == 0 && ok) ok = mbar_wait_bounded_relaxed(smem_addr(&hdr->acc_full[0]), 0) ? 1u : 0u;
-        if (!__all_sync(0xffffffffu, ok != 0)) failed = true;
-        if (failed) hdr->abort = 1;
-        tc_fence_after_sync();
-        __syncthreads();
-        if (tid == 0) stamp_max(stamps, STAMP_ACC);
-        const bool acc_ok = hdr->abort == 0;
-        // the activation stages and the weight tile are dead now: the exchange buffer takes their place
-        if (!ln_epilogue(ln, job, reinterpret_cast<float*>(xsm), tmem_base, n_rows, my_mtiles, T, tid, acc_ok, &hdr->abort, stamps))
-          failed = true;
       }
     }
     if (failed) {
@@ -776,10 +600,9 @@ dqgemm_pair_kernel(const __grid_constant__ CUtensorMap xmap, const Job* __restri
 }
 
 template <typename OutT, bool GELU>
-cudaError_t launch_t(const GemmLaunch& p, cudaStream_t s, bool ln = false) {
+cudaError_t launch_t(const GemmLaunch& p, cudaStream_t s) {
   const __nv_bfloat16* x = static_cast<const __nv_bfloat16*>(p.x);
   if (p.pair && !p.simt_debug) {
-    if (ln) return cudaErrorInvalidValue;
     // clusters of two CTAs along x (consecutive jobs = the two halves of a 128-feature tile)
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(p.n_jobs, p.m_ctas);
@@ -799,29 +622,23 @@ cudaError_t launch_t(const GemmLaunch& p, cudaStream_t s, bool ln = false) {
   dim3 grid(p.n_jobs, p.m_ctas), block(kThreads);
   PrefetchRanges pf;
   for (int r = 0; r < 4; ++r) { pf.ptr[r] = p.pf_ptr[r]; pf.bytes[r] = p.pf_bytes[r]; }
-  const int kind = ln ? GEMM_BF16_TO_LN : (sizeof(OutT) == 4 ? GEMM_BF16_TO_F32 : (GELU ? GEMM_BF16_TO_BF16_GELU : GEMM_BF16_TO_BF16));
+  const int kind = sizeof(OutT) == 4 ? GEMM_BF16_TO_F32 : (GELU ? GEMM_BF16_TO_BF16_GELU : GEMM_BF16_TO_BF16);
   if (p.simt_debug) {
-    if (ln) return cudaErrorInvalidValue;       // the debug path has no LayerNorm epilogue
     return launch_kernel(dqgemm_kernel<OutT, GELU, true, false>, grid, block, p.smem_bytes, s, p.pdl, p.xmap, p.jobs, p.segs, x, p.ldx,
                          p.T, static_cast<OutT*>(p.out), p.ldo, p.bias, p.err, p.n_stages, p.bps, p.w_bytes, p.hdr_bytes,
-                         p.seg_stride, pf, kind, p.ln, p.stamps);
+                         p.seg_stride, pf, kind, p.stamps);
   }
   // every output kind runs the same kernel (the kind is a parameter): one copy of the code for a layer's four GEMMs;
   // two builds of it, for few and for many token tiles per CTA (they differ in the epilogue's shape)
   const int n_mtiles = (p.T + kTileM - 1) / kTileM;
   const bool few = (n_mtiles + p.m_ctas - 1) / p.m_ctas <= 2;
-  unsigned cluster = 1;
-  if (ln) {
-    if (p.ln.cluster < 1 || p.ln.cluster > 8 || p.n_jobs % p.ln.cluster != 0) return cudaErrorInvalidValue;
-    cluster = static_cast<unsigned>(p.ln.cluster);
-  }
   if (few)
-    return launch_kernel_cluster(dqgemm_kernel<void, false, false, true>, grid, block, p.smem_bytes, s, p.pdl, cluster, p.xmap,
+    return launch_kernel(dqgemm_kernel<void, false, false, true>, grid, block, p.smem_bytes, s, p.pdl, p.xmap,
                                  p.jobs, p.segs, x, p.ldx, p.T, p.out, p.ldo, p.bias, p.err, p.n_stages, p.bps, p.w_bytes,
-                                 p.hdr_bytes, p.seg_stride, pf, kind, p.ln, p.stamps);
-  return launch_kernel_cluster(dqgemm_kernel<void, false, false, false>, grid, block, p.smem_bytes, s, p.pdl, cluster, p.xmap,
+                                 p.hdr_bytes, p.seg_stride, pf, kind, p.stamps);
+  return launch_kernel(dqgemm_kernel<void, false, false, false>, grid, block, p.smem_bytes, s, p.pdl, p.xmap,
                                p.jobs, p.segs, x, p.ldx, p.T, p.out, p.ldo, p.bias, p.err, p.n_stages, p.bps, p.w_bytes,
-                               p.hdr_bytes, p.seg_stride, pf, kind, p.ln, p.stamps);
+                               p.hdr_bytes, p.seg_stride, pf, kind, p.stamps);
 }
 
 template <typename K>
@@ -834,10 +651,6 @@ cudaError_t set_smem(K kernel) {
 size_t gemm_weight_bytes(uint32_t n_rows, uint32_t k_total) { return static_cast<size_t>(n_rows) * k_total * 2; }
 
 uint32_t gemm_header_bytes() { return kHeaderBytes; }
-
-size_t gemm_ln_exchange_bytes(uint32_t m_tiles, uint32_t n_rows) {
-  return static_cast<size_t>(m_tiles) * kTileM * (n_rows + 4) * sizeof(float);
-}
 
 size_t gemm_smem_bytes(uint32_t w_bytes, uint32_t n_stages, uint32_t bps, uint32_t hdr_bytes) {
   return hdr_bytes + static_cast<size_t>(w_bytes) + static_cast<size_t>(n_stages) * bps * kBoxBytes;
@@ -870,32 +683,11 @@ cudaError_t gemm_configure() {
   return cudaSuccess;
 }
 
-// How many clusters of `cluster_x` CTAs with `smem_bytes` of shared memory the device can hold at once (0 on error).
-// The LayerNorm epilogue needs the whole launch resident: its CTAs wait for one another.
-int gemm_max_active_clusters(unsigned cluster_x, size_t smem_bytes) {
-  cudaLaunchConfig_t cfg = {};
-  cfg.gridDim = dim3(cluster_x * 64);
-  cfg.blockDim = dim3(kThreads);
-  cfg.dynamicSmemBytes = smem_bytes;
-  cudaLaunchAttribute attr[1];
-  attr[0].id = cudaLaunchAttributeClusterDimension;
-  attr[0].val.clusterDim.x = cluster_x; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
-  cfg.attrs = attr;
-  cfg.numAttrs = 1;
-  int n = 0;
-  if (cudaOccupancyMaxActiveClusters(&n, dqgemm_kernel<void, false, false, true>, &cfg) != cudaSuccess) {
-    (void)cudaGetLastError();
-    return 0;
-  }
-  return n;
-}
-
 cudaError_t launch_gemm(GemmKind kind, const GemmLaunch& p, cudaStream_t s) {
   switch (kind) {
     case GEMM_BF16_TO_BF16: return launch_t<__nv_bfloat16, false>(p, s);
     case GEMM_BF16_TO_BF16_GELU: return launch_t<__nv_bfloat16, true>(p, s);
     case GEMM_BF16_TO_F32: return launch_t<float, false>(p, s);
-    case GEMM_BF16_TO_LN: return launch_t<float, false>(p, s, true);
   }
   return cudaErrorInvalidValue;
 }

@@ -39,29 +39,7 @@ struct Job {
 enum GemmKind : int {
   GEMM_BF16_TO_BF16 = 1,      // bf16 in, bf16 out (+bias)                     : QKV
   GEMM_BF16_TO_BF16_GELU = 2, // bf16 in, bf16 out, +bias, erf-GELU            : FFN1
-  GEMM_BF16_TO_F32 = 3,       // bf16 in, fp32 partial sums out, no bias       : O projection, FFN2 (many tokens, probes)
-  GEMM_BF16_TO_LN = 4         // bf16 in, + bias + residual, LayerNorm, fp32 and/or bf16 out : O projection, FFN2
-};
-
-// Epilogue of GEMM_BF16_TO_LN: out = LayerNorm(x W^T + bias + resid) * gamma + beta with the K range of every
-// 64- or 128-feature column tile split over the CTAs of one thread-block cluster.  The partial sums of a cluster
-// meet in distributed shared memory; the per-row (mean, sum of squared deviations) of every column tile meet in
-// `stats`, counted in `counters` (zero before the launch), so that no partial sum reaches global memory and no
-// separate LayerNorm launch is needed.  Jobs of one column tile are consecutive (cluster rank = K split).
-struct LnEpilogue {
-  const float* bias;        // [d]
-  const void* resid;        // [T][d], fp32 or bf16
-  const float* gamma;
-  const float* beta;
-  float* out_f32;           // optional
-  uint16_t* out_bf16;       // optional
-  float2* stats;            // [T][n_ntiles] scratch
-  unsigned int* counters;   // [m_ctas * cluster] scratch, zero at launch
-  float eps;
-  int resid_bf16;
-  int d;
-  int n_ntiles;             // column tiles = clusters that share a token row
-  int cluster;              // CTAs per cluster = K splits per column tile (1..8)
+  GEMM_BF16_TO_F32 = 3        // bf16 in, fp32 partial sums out, no bias       : O projection, FFN2
 };
 
 struct GemmLaunch {
@@ -88,7 +66,6 @@ struct GemmLaunch {
   bool simt_debug;          // compute the products on the plain ALUs instead of the tensor cores
   bool pdl;                 // launch with programmatic dependent launch
   bool pair;                // two-CTA clusters (cta_group::2): jobs 2i and 2i+1 share one M=256 x N=128 MMA
-  LnEpilogue ln;            // GEMM_BF16_TO_LN only
   unsigned long long* stamps;   // this launch's profiling record (see sti_device.cuh), or null
 };
 
@@ -96,10 +73,7 @@ size_t gemm_weight_bytes(uint32_t n_rows, uint32_t k_total);
 uint32_t gemm_header_bytes();
 bool gemm_pick_ring(uint32_t w_bytes, uint32_t k_total, uint32_t hdr_bytes, uint32_t* n_stages, uint32_t* bps);   // false: does not fit
 size_t gemm_smem_bytes(uint32_t w_bytes, uint32_t n_stages, uint32_t bps, uint32_t hdr_bytes);
-// Shared memory (beyond the header) the LayerNorm epilogue needs for a CTA that owns `m_tiles` token tiles of `n_rows` features.
-size_t gemm_ln_exchange_bytes(uint32_t m_tiles, uint32_t n_rows);
 cudaError_t gemm_configure();   // opt in to large dynamic shared memory (once per device)
-int gemm_max_active_clusters(unsigned cluster_x, size_t smem_bytes);
 cudaError_t launch_gemm(GemmKind kind, const GemmLaunch& p, cudaStream_t s);
 
 // Per-head attention over kept heads.  qkv: [(kept*3 + which)][T][64] bf16; out: [T][n_kept*64] bf16.

@@ -134,7 +134,6 @@ def test_fused_decode_small_shape_all_bitwidths_and_tilings(tune):
     work = _mixed_work(shape, seed=11)
     with _Tune(tune), sti.Session(work) as s:
         _check_all_gemms(work, s)
-        _check_all_gemms(work, s, variant=3)                  # tile tables of the LayerNorm-epilogue form
 
 
 def test_fused_decode_bert_base_elastic_plan():
@@ -143,7 +142,6 @@ def test_fused_decode_bert_base_elastic_plan():
     work = _mixed_work(shape, seed=12, keep_fn=lambda k, i: i not in ((1, 7) if k == ATTN else (0, 5, 10)))
     with sti.Session(work) as s:
         _check_all_gemms(work, s)
-        _check_all_gemms(work, s, variant=3)
 
 
 def test_fused_decode_bert_large_few_and_many_token_tilings():
@@ -151,7 +149,6 @@ def test_fused_decode_bert_large_few_and_many_token_tilings():
     work = _mixed_work(shape, seed=13)
     with sti.Session(work) as s:                              # tiling chosen for few tokens
         _check_all_gemms(work, s)
-        _check_all_gemms(work, s, variant=3)
     with sti.Session(work, max_batch=8, max_seq=512) as s:    # tiling chosen for many tokens
         _check_all_gemms(work, s, variant=1)                  # one-CTA kernel
         _check_all_gemms(work, s, variant=2)                  # two-CTA (cta_group::2) kernel
