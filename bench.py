@@ -41,7 +41,7 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 # dram__bytes_read.sum + dram__bytes_write.sum per dequant-GEMM launch (mean over one layer's QKV, O, FFN1, FFN2
 # launches; BERT-large layer, batch 1, seq 256) from the ncu capture summarised in
 # profiles/dqgemm_bertlarge_seq256_ncu_full.md.  Set to None whenever dqgemm.cu changes after that capture.
-NCU_DRAM_BYTES_PER_GEMM_LAUNCH = 2510720
+NCU_DRAM_BYTES_PER_GEMM_LAUNCH = None
 
 
 def load_peaks():
@@ -160,14 +160,14 @@ def run_reference(args):
     if int(os.environ.get("RANK", "0")) != 0:
         return
     import workloads as W
-    n_sample = 4
-    work = W.make_config(4, n_layers=n_sample, workers=min(4, os.cpu_count() or 1))
+    work = W.make_config(4, workers=min(8, os.cpu_count() or 1))
+    n_sample = work.shape.n_layers                 # the whole model: the same configuration as the GPU arm
     layers = list(range(n_sample))
     for _ in range(args.warmup):
         oracle_forward_timed(work, layers)
     total = sum(oracle_forward_timed(work, layers) for _ in range(args.steps))
     value = work.packed_bytes() * args.steps / total / 1e9
-    sample = f"layers 0-{n_sample - 1} of the 24 (decode + fp64 forward, 1 sequence of 256 tokens) per step"
+    sample = f"all {n_sample} layers (decode + fp64 forward, 1 sequence of 256 tokens) per step"
     print(json.dumps({
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": total / args.steps * 1e3,
@@ -298,7 +298,7 @@ def run_sweep(args):
                       "peak_source": peak_src, "rows": rows}))
 
 
-def planner_profile(args):
+def planner_profile(args, widths=None):
     """Section 5.2's two offline profiles on the device in use: T_io per stored version and T_comp per submodel
     width m (see run_planner).  Returns everything the plan-and-execute modes need."""
     import workloads as W
@@ -308,7 +308,7 @@ def planner_profile(args):
     versions = (2, 3, 4, 5, 6, 32)
     ones = np.ones((1, M), np.uint8)
     shard_bytes = [W.make_planned(ones, ones * k, ones * 0, batch=B, seq=L).packed_bytes() // M for k in versions]
-    widths = list(range(1, M + 1))
+    widths = list(widths) if widths else list(range(1, M + 1))      # submodel widths measured (others interpolated)
     depth = 4
     ring = args.planner_ring
     full = np.ones((depth, M), np.uint8)
@@ -374,7 +374,8 @@ def planner_profile(args):
     t_comp16_6bit = stack_ms(stack6) * 1e3 / depth
     # the 4-shard stack with layers 1.. streamed: its copies are far shorter than its layers, so what it
     # takes longer than the resident stack is the per-layer cost of running inside the pipeline
-    pipe_us = max(0.0, (stack_ms(narrowed(4, streamed_from=1)) * 1e3 - measured[3] * depth) / (depth - 1))
+    pipe_us = max(0.0, (stack_ms(narrowed(4, streamed_from=1)) * 1e3 - float(np.interp(4, widths, measured)) * depth)
+                  / (depth - 1))
     t_comp_us = [0.0] + [float(np.interp(m, widths, measured)) + pipe_us for m in range(1, M + 1)]
     t_comp_us = list(np.maximum.accumulate(t_comp_us))
     return dict(W=W, sti=sti, torch=torch, stream=stream, flush=flush, forward_ms=forward_ms, B=B, L=L, N=N, M=M,
@@ -456,6 +457,96 @@ def run_planner(args):
                       "pipeline_us_per_layer": pipe_us, "t_comp16_us_resident_2bit": measured[-1],
                       "t_comp16_us_resident_6bit": t_comp16_6bit,
                       "ring_slots": ring, "rows": rows, "back_to_back": series}))
+
+
+def planner_point(args, target_ms):
+    """One planner-made plan, end to end, for the default bench line: profile the device on three submodel widths,
+    let sti_plan_auto choose the submodel, the bitwidths and the preload prefix for `target_ms`, execute it streamed
+    and report what the pipeline hid (Section 5)."""
+    pf = planner_profile(args, widths=(4, 8, 16))
+    W, sti, torch, stream, flush, forward_ms = pf["W"], pf["sti"], pf["torch"], pf["stream"], pf["flush"], pf["forward_ms"]
+    B, L, N, M = pf["B"], pf["L"], pf["N"], pf["M"]
+    importance = np.random.default_rng(np.random.SeedSequence([0, 77])).uniform(0, 1, (N, M)).astype(np.float32)
+    preload_bytes = int(args.planner_preload_mb * (1 << 20))
+    plan = sti.sti_plan_auto(target_ms * 1e3, N, M, pf["t_comp_us"], pf["t_io_us"], pf["shard_bytes"], importance,
+                             preload_bytes)
+    streamed_layers = int(((plan["keep"] > 0) & (plan["preload"] == 0)).any(axis=1).sum())
+    work = W.make_planned(plan["keep"], plan["bits"], plan["preload"], batch=B, seq=L, workers=pf["workers"],
+                          ring_slots=max(2, min(pf["ring"], streamed_layers)))
+    kept_bits = plan["bits"][plan["keep"] > 0]
+    with sti.Session(work, compute_stream=stream.cuda_stream) as sess:
+        x = device_act(torch, work)
+        y = torch.empty_like(x)
+        ms = forward_ms(sess, work, x, y, 10)
+        sti.sti_plan_set_profiling(sess.plan, 1)
+        stall, copy = [], []
+        with torch.cuda.stream(stream):
+            for _ in range(5):
+                flush.zero_()
+                sti.sti_model_forward(sess.plan, x.data_ptr(), y.data_ptr(), B, L)
+                st = sti.sti_get_stats(sess.plan)
+                stall.append(sum(st.stall_us[:st.n_layers]))
+                copy.append(sum(st.copy_us[:st.n_layers]))
+        sti.sti_plan_set_profiling(sess.plan, 0)
+    stall_us, copy_us = float(np.median(stall)), float(np.median(copy))
+    return {"workload": "two-stage planner (Section 5) on this device's measured T_comp / T_io, BERT-large 24x16 store, "
+                        f"batch {B}, seq {L}, {args.planner_preload_mb:g} MiB preload buffer, seeded uniform importance",
+            "target_ms": target_ms, "n": plan["n"], "m": plan["m"], "pass1_bits": plan["pass1_bits"],
+            "mean_bits": float(kept_bits.astype(np.float64).mean()), "preloaded_shards": int(plan["preload"].sum()),
+            "predicted_ms": plan["n"] * pf["t_comp_us"][plan["m"]] * 1e-3, "measured_ms": ms,
+            "meets_target": bool(ms <= target_ms), "h2d_copy_ms": copy_us * 1e-3, "stall_ms": stall_us * 1e-3,
+            "hidden_frac": 1.0 - stall_us / copy_us if copy_us > 0 else None, "h2d_GBps": pf["h2d_gbps"]}
+
+
+def model_point(sti, torch, work, stream, flush, peaks, label, steps=12, warm=4):
+    """A model workload resident and streamed: forward ms (median, cold L2), the dequant-GEMMs' stamped time and
+    TFLOP/s under graph replay, and how much of the host-to-device copy time the pipeline hid."""
+    n_layers = work.shape.n_layers
+    B, L = work.batch, work.seq
+    x = device_act(torch, work)
+    y = torch.empty_like(x)
+    out = {"workload": label, "tokens": B * L, "n_layers": n_layers, "packed_bytes": work.packed_bytes()}
+
+    def median_ms(sess):
+        ms = []
+        with torch.cuda.stream(stream):
+            for i in range(warm + steps):
+                flush.zero_()
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                e0.record(stream)
+                sti.sti_model_forward(sess.plan, x.data_ptr(), y.data_ptr(), B, L)
+                e1.record(stream)
+                stream.synchronize()
+                if i >= warm:
+                    ms.append(e0.elapsed_time(e1))
+        sti.sti_sync(sess.ctx)
+        return float(np.median(ms))
+
+    with sti.Session(with_residency(work, n_layers), compute_stream=stream.cuda_stream) as sess:
+        out["ms_resident"] = median_ms(sess)
+        per, count, total = stamped_forwards(sti, torch, sess, stream, flush, x, y, B, L, n_layers, reps=5)
+        gemm_s = float(sum(per[k] for k in GEMM_KERNELS)) * 1e-6
+        out.update({"gemm_ms": gemm_s * 1e3, "gemm_TFLOPs": gemm_flops(work) / gemm_s / 1e12,
+                    "gemm_frac_of_tensor_peak": gemm_flops(work) / gemm_s / 1e12 / peaks["bf16_tflops_sustained"],
+                    "forward_TFLOPs": (gemm_flops(work) + attn_flops(work)) / (out["ms_resident"] * 1e-3) / 1e12,
+                    "packed_GBps_resident": work.packed_bytes() / (out["ms_resident"] * 1e-3) / 1e9,
+                    "kernel_us_per_layer": {KERNEL_NAMES[k]: float(per[k] / n_layers) for k in range(1, 8)}})
+    with sti.Session(work, compute_stream=stream.cuda_stream) as sess:
+        out["ms_streamed"] = median_ms(sess)
+        sti.sti_plan_set_profiling(sess.plan, 1)
+        with torch.cuda.stream(stream):
+            for _ in range(3):
+                flush.zero_()
+                sti.sti_model_forward(sess.plan, x.data_ptr(), y.data_ptr(), B, L)
+                st = sti.sti_get_stats(sess.plan)
+        sti.sti_plan_set_profiling(sess.plan, 0)
+        copy_ms = sum(st.copy_us[:st.n_layers]) * 1e-3
+        out.update({"h2d_copy_ms": copy_ms, "stall_ms": sum(st.stall_us[:st.n_layers]) * 1e-3,
+                    "streamed_bytes": int(sum(st.streamed_bytes[:st.n_layers])),
+                    "hidden_frac": 1.0 - max(0.0, out["ms_streamed"] - out["ms_resident"]) / copy_ms if copy_ms > 0 else None,
+                    "hidden_frac_cap": min(1.0, out["ms_resident"] / copy_ms) if copy_ms > 0 else None,
+                    "streamed_over_resident": out["ms_streamed"] / out["ms_resident"]})
+    return out
 
 
 def run_baselines(args):
@@ -610,6 +701,98 @@ def run_quantize(args):
                                        "kind": "oracle", "sample": "one attention unit and one FFN unit of layer 0"}}))
 
 
+GEMM_KERNELS = (1, 3, 5, 6)          # QKV, O projection, FFN1, FFN2 in the per-layer stamp records
+KERNEL_NAMES = ("cast", "qkv", "attention", "o_proj", "layernorm1", "ffn1", "ffn2", "layernorm2")
+
+
+def stamp_intervals(stamps):
+    """Per-kernel share of one forward from the kernels' own device-timer stamps (profiling level 3, graph replay).
+
+    Kernels overlap (each is launched before its predecessor ends and decodes its weights meanwhile), so a kernel's
+    time is taken as the interval from the previous kernel's last-CTA end to its own: the intervals of a forward add
+    up to the forward.  Returns (us per kernel slot summed over layers [8], launches per slot [8], total us)."""
+    n_layers = stamps.shape[0]
+    per = np.zeros(8)
+    count = np.zeros(8, dtype=np.int64)
+    prev_end = None
+    first = None
+    for l in range(n_layers):
+        for k in range(8):
+            end = int(stamps[l, k, 2])
+            if end == 0:
+                continue                                   # this kernel did not run
+            if prev_end is None:
+                prev_end = first = int(stamps[l, k, 0])    # the forward's first kernel: from its first CTA's start
+            per[k] += (end - prev_end) * 1e-3
+            count[k] += 1
+            prev_end = end
+    total = (prev_end - first) * 1e-3 if prev_end is not None else 0.0
+    return per, count, total
+
+
+def stamped_forwards(sti, torch, sess, stream, flush, x, y, B, L, n_layers, reps, warm=2):
+    """Runs `reps` graph-replayed forwards with kernel stamps on (cold L2 each) and returns the mean per-kernel
+    interval sums, the launches per kernel slot and the mean stamped total, all per forward."""
+    sti.sti_plan_set_profiling(sess.plan, 3)
+    per_acc, total_acc, count = np.zeros(8), 0.0, np.zeros(8, dtype=np.int64)
+    with torch.cuda.stream(stream):
+        for i in range(warm + reps):
+            flush.zero_()
+            sti.sti_model_forward(sess.plan, x.data_ptr(), y.data_ptr(), B, L)
+            stream.synchronize()
+            if i >= warm:
+                per, count, total = stamp_intervals(sti.sti_get_kernel_stamps(sess.plan, n_layers))
+                per_acc += per
+                total_acc += total
+    sti.sti_plan_set_profiling(sess.plan, 0)
+    return per_acc / reps, count, total_acc / reps
+
+
+def plain_h2d_gbps(torch, stream, mb=64, reps=8):
+    """Pinned host -> device cudaMemcpyAsync rate of the box, measured alone (the denominator of the streamed arm)."""
+    src = torch.empty(mb << 20, dtype=torch.uint8).pin_memory()
+    dst = torch.empty(mb << 20, dtype=torch.uint8, device="cuda")
+    rates = []
+    with torch.cuda.stream(stream):
+        for i in range(reps + 2):
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(stream)
+            dst.copy_(src, non_blocking=True)
+            e1.record(stream)
+            stream.synchronize()
+            if i >= 2:
+                rates.append(src.numel() / (e0.elapsed_time(e1) * 1e-3) / 1e9)
+    return float(np.median(rates))
+
+
+def oracle_single_thread(work, layers):
+    """The oracle on one host thread (BLAS pool limited to 1) over `layers`; returns seconds."""
+    try:
+        from threadpoolctl import threadpool_limits
+    except Exception:
+        return None
+    with threadpool_limits(limits=1):
+        return oracle_forward_timed(work, layers)
+
+
+def spawn_ranks(n, argv, extra_env=None, port=None):
+    """Starts `n` copies of the command `argv`, one per GPU of this node, with the rendezvous variables torchrun would
+    set (RANK, LOCAL_RANK, WORLD_SIZE, MASTER_ADDR=127.0.0.1, MASTER_PORT); rank 0 inherits stdout, the others'
+    output goes to stderr.  Returns the largest exit code."""
+    port = port or (29500 + os.getpid() % 2000)
+    procs = []
+    for r in range(n):
+        env = dict(os.environ)
+        env.update({"RANK": str(r), "LOCAL_RANK": str(r), "WORLD_SIZE": str(n), "LOCAL_WORLD_SIZE": str(n),
+                    "MASTER_ADDR": "127.0.0.1", "MASTER_PORT": str(port)})
+        env.setdefault("NCCL_DEBUG", "INFO")               # the communicator's transport choices stay visible
+        if extra_env:
+            env.update(extra_env)
+        procs.append(subprocess.Popen(list(argv), env=env, stdout=None if r == 0 else sys.stderr))
+    codes = [p.wait() for p in procs]
+    return max(codes)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -655,6 +838,10 @@ def main():
         run_baselines(args)
         return
     args.warmup = max(args.warmup, 3)
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
+        # launched plainly with --gpus N: start the N replicas ourselves (the path has no exchange step: one
+        # independent replica per GPU; NCCL only carries the barrier and the max-over-ranks reduction)
+        raise SystemExit(spawn_ranks(args.gpus, [sys.executable, os.path.abspath(__file__)] + sys.argv[1:]))
 
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
@@ -662,7 +849,8 @@ def main():
 
     # inputs first: the quantizer pool is spawned before the first CUDA call
     import workloads as W
-    work_str = W.make_config(4, n_layers=args.layers or None, workers=min(8, os.cpu_count() or 1))
+    workers = min(8, os.cpu_count() or 1)
+    work_str = W.make_config(4, n_layers=args.layers or None, workers=workers)
     work_res = with_residency(work_str, work_str.shape.n_layers)
     packed = work_str.packed_bytes()
 
@@ -677,6 +865,11 @@ def main():
         cpu_baseline = {"value": work_str.packed_bytes(range(n_sample)) * reps / secs / 1e9, "unit": UNIT,
                         "cores": blas_threads(), "kind": "oracle", "seconds": secs,
                         "sample": f"all {n_sample} layers, decode + fp64 forward, {reps} times"}
+        one = list(range(min(2, n_sample)))
+        secs1 = oracle_single_thread(work_str, one)
+        if secs1:
+            cpu_baseline["single_thread"] = {"value": work_str.packed_bytes(one) / secs1 / 1e9, "unit": UNIT, "cores": 1,
+                                             "seconds": secs1, "sample": f"layers 0-{one[-1]}, once"}
 
     import torch
     import torch.distributed as dist
@@ -711,48 +904,48 @@ def main():
     s_str = sti.Session(work_str, device=local_rank, compute_stream=stream.cuda_stream)
     sampler = ClockSampler(local_rank)
 
-    def timed(fn):
+    def timed(fn, cold=True):
+        """W warm-up steps, then exactly K timed ones; returns (job time of the K steps in ms, max over ranks;
+        this rank's per-step times)."""
         with torch.cuda.stream(stream):
             for _ in range(Wm):
-                flush.zero_()
+                if cold:
+                    flush.zero_()
                 fn()
             barrier()
             ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(K)]
             for e0, e1 in ev:
-                flush.zero_()                     # cold L2 for every step (outside the timed interval)
+                if cold:
+                    flush.zero_()                 # cold L2 for every step (outside the timed interval)
                 e0.record(stream)
                 fn()
                 e1.record(stream)
             barrier()
-        return max_over_ranks(sum(e0.elapsed_time(e1) for e0, e1 in ev), world)
+        steps = [e0.elapsed_time(e1) for e0, e1 in ev]
+        return max_over_ranks(sum(steps), world), steps
 
     sampler.start()
     launches0 = sti.sti_ctx_launch_count(s_res.ctx)
-    ms_res = timed(lambda: sti.sti_model_forward(s_res.plan, x_dev.data_ptr(), y_dev.data_ptr(), B, L))
+    ms_res, steps_res = timed(lambda: sti.sti_model_forward(s_res.plan, x_dev.data_ptr(), y_dev.data_ptr(), B, L))
     launches = sti.sti_ctx_launch_count(s_res.ctx) - launches0
     sti.sti_sync(s_res.ctx)
-    ms_e2e = timed(lambda: sti.sti_model_forward_host(s_str.plan, x_host.data_ptr(), y_host.data_ptr(), B, L))
+    ms_e2e, steps_e2e = timed(lambda: sti.sti_model_forward_host(s_str.plan, x_host.data_ptr(), y_host.data_ptr(), B, L))
     sti.sti_sync(s_str.ctx)
-    ms_str_dev = timed(lambda: sti.sti_model_forward(s_str.plan, x_dev.data_ptr(), y_dev.data_ptr(), B, L))
+    ms_str_dev, _ = timed(lambda: sti.sti_model_forward(s_str.plan, x_dev.data_ptr(), y_dev.data_ptr(), B, L))
     sti.sti_sync(s_str.ctx)
     clocks = sampler.stop()
+    # the same forward with whatever the previous step left in L2 (packed weights are 136 MB, L2 126 MB)
+    ms_warm, _ = timed(lambda: sti.sti_model_forward(s_res.plan, x_dev.data_ptr(), y_dev.data_ptr(), B, L), cold=False)
+    sti.sti_sync(s_res.ctx)
 
-    # kernel-level pass for the roofline of the dominant kernel (the fused dequant-GEMM)
-    sti.sti_plan_set_profiling(s_res.plan, 2)
-    gemm_us = attn_us = ln_us = 0.0
-    gemm_launches = 0
-    layer_us = []
-    with torch.cuda.stream(stream):
-        for i in range(Wm + K):
-            flush.zero_()
-            sti.sti_model_forward(s_res.plan, x_dev.data_ptr(), y_dev.data_ptr(), B, L)
-            st = sti.sti_get_stats(s_res.plan)
-            if i >= Wm:
-                n = st.n_layers
-                gemm_us += sum(st.gemm_us[:n]); attn_us += sum(st.attn_us[:n]); ln_us += sum(st.ln_us[:n])
-                gemm_launches += st.gemm_launches
-                layer_us.extend(st.compute_us[:n])
-    sti.sti_plan_set_profiling(s_res.plan, 0)
+    # the dominant kernel's time in the SAME execution mode as the timed value: device-timer stamps written by the
+    # kernels themselves under graph replay
+    n_layers = work_str.shape.n_layers
+    per_kernel_us, kernel_count, stamped_total_us = stamped_forwards(sti, torch, s_res, stream, flush, x_dev, y_dev, B, L,
+                                                                      n_layers, reps=min(K, 10))
+    gemm_us = float(sum(per_kernel_us[k] for k in GEMM_KERNELS))         # per forward
+    gemm_launches = int(sum(kernel_count[k] for k in GEMM_KERNELS))      # per forward
+    attn_us, ln_us = float(per_kernel_us[2]), float(per_kernel_us[4] + per_kernel_us[7])
     # streamed run: copy durations and stalls
     sti.sti_plan_set_profiling(s_str.plan, 1)
     copy_us = stall_us = 0.0
@@ -766,15 +959,30 @@ def main():
             streamed_bytes = sum(st.streamed_bytes[:st.n_layers])
     sti.sti_plan_set_profiling(s_str.plan, 0)
     mem = sti.sti_plan_memory(s_str.plan)
+    h2d_plain = plain_h2d_gbps(torch, stream) if rank == 0 else None
 
+    s_res.close()
+    s_str.close()
     extras = {}
     if rank == 0 and world == 1 and not args.no_extras:
+        # configurations 1 and 2 (single BERT-base layers) and the few-token probes of the same layer
         for num in (1, 2):
             extras[f"config{num}_layer"] = time_layer_config(sti, torch, num, peaks)
         for probe_seq in (8, 32):
             extras[f"config1_layer_probe_seq{probe_seq}"] = time_layer_config(sti, torch, 1, peaks, seq=probe_seq)
-    s_res.close()
-    s_str.close()
+        # configuration 3: 12-layer BERT-base, layers 0-2 preloaded, the rest streamed, two ring slots
+        extras["config3_model"] = model_point(
+            sti, torch, W.make_config(3, workers=workers), stream, flush, peaks,
+            "configs[2]: 12-layer BERT-base, batch 1, seq 128, per-layer random plan (60-100 % kept, 2-6 bits), "
+            "layers 0-2 preloaded, layers 3-11 streamed")
+        # configuration 5: two points of the sweep on a 4-layer BERT-large stack (bf16 activations, uniform 3 bits,
+        # 2-layer preload when streamed); the whole grid is `bench.py --sweep`
+        for b5, s5 in ((8, 512), (32, 512)):
+            w5 = W.make_config(5, n_layers=4, plan="uniform3", resident=False, batch=b5, seq=s5, workers=workers)
+            extras[f"config5_b{b5}_s{s5}_uniform3"] = model_point(
+                sti, torch, w5, stream, flush, peaks,
+                f"configs[4] point: 4-layer BERT-large stack, batch {b5}, seq {s5}, uniform 3-bit plan", steps=6, warm=3)
+        extras["planner_plan"] = planner_point(args, target_ms=0.8)
 
     if rank != 0:
         if world > 1:
@@ -782,7 +990,7 @@ def main():
         return
 
     flops_gemm = gemm_flops(work_str)
-    gemm_s = gemm_us * 1e-6 / K                      # per forward
+    gemm_s = gemm_us * 1e-6                          # per forward (stamped under graph replay)
     ach_tflops = flops_gemm / gemm_s / 1e12 if gemm_s > 0 else 0.0
     peak_tf, peak_hbm = float(peaks["bf16_tflops_sustained"]), float(peaks["hbm_gbs"])
     x_bytes = x_host.numel() * x_host.element_size()
@@ -812,21 +1020,33 @@ def main():
                      "traffic_note": "dram read+write bytes per launch, mean of a layer's four launches, one ncu "
                                      "capture of this kernel build (cold caches); algorithmic: packed shards + bf16 operands",
                      "peak_source": f"bf16_tflops_sustained, {peak_src}",
-                     "flops_per_launch": flops_gemm * K / gemm_launches if gemm_launches else None,
+                     "flops_per_launch": flops_gemm / gemm_launches if gemm_launches else None,
                      "avg_launch_us": gemm_us / gemm_launches if gemm_launches else None,
-                     "launches_timed": gemm_launches,
+                     "launches_per_forward": gemm_launches,
+                     "timing": "device-timer stamps written by the kernels during graph-replayed forwards (the timed "
+                               "mode); kernels overlap, so a launch's time is the interval from the previous "
+                               "kernel's last-CTA end to its own; the intervals of a forward add up to the forward",
                      "hbm_view": {"achieved_GBps": packed / gemm_s / 1e9 if gemm_s > 0 else None, "peak": peak_hbm,
                                   "frac": packed / gemm_s / 1e9 / peak_hbm if gemm_s > 0 else None,
                                   "note": "packed-weight bytes over GEMM time; at 256 tokens the GEMMs are tensor-bound"}},
         "cpu_baseline": cpu_baseline,
-        "latency": {"layer_us_mean": float(np.mean(layer_us)) if layer_us else None,
-                    "model_ms_resident": t_res, "model_ms_streamed": t_str, "model_ms_e2e_host": ms_e2e / K,
+        "latency": {"layer_us_mean": t_res * 1e3 / n_layers,
+                    "model_ms_resident": t_res, "model_ms_resident_p10": float(np.percentile(steps_res, 10)),
+                    "model_ms_resident_p50": float(np.median(steps_res)),
+                    "model_ms_resident_p90": float(np.percentile(steps_res, 90)),
+                    "model_ms_resident_warm_l2": ms_warm / K,
+                    "model_ms_streamed": t_str, "model_ms_e2e_host": ms_e2e / K,
+                    "model_ms_e2e_host_p10": float(np.percentile(steps_e2e, 10)),
+                    "model_ms_e2e_host_p90": float(np.percentile(steps_e2e, 90)),
                     "roofline_floor_ms": t_floor_ms, "x_of_floor": t_res / t_floor_ms,
-                    "gemm_us_per_fwd": gemm_us / K, "attn_us_per_fwd": attn_us / K, "ln_us_per_fwd": ln_us / K},
+                    "stamped_forward_us": stamped_total_us,
+                    "gemm_us_per_fwd": gemm_us, "attn_us_per_fwd": attn_us, "ln_us_per_fwd": ln_us,
+                    "kernel_us_per_layer": {KERNEL_NAMES[k]: float(per_kernel_us[k] / n_layers) for k in range(1, 8)}},
         "pipeline": {"h2d_copy_ms": t_h2d, "h2d_GBps": streamed_bytes / (t_h2d * 1e-3) / 1e9 if t_h2d > 0 else None,
                      "stall_ms": stall_us * 1e-3, "hidden_frac": hidden,
                      "hidden_frac_cap": min(1.0, t_res / t_h2d) if t_h2d > 0 else None,
                      "pipeline_eff": max(t_h2d, t_res) / t_str if t_str > 0 else None,
+                     "h2d_plain_pinned_GBps": h2d_plain,
                      "preload_bytes": mem["preload_bytes"], "pinned_bytes": mem["pinned_bytes"],
                      "ring_bytes": mem["ring_bytes"]},
         "extras": extras,

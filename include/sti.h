@@ -225,6 +225,19 @@ sti_status sti_get_kernel_stamps(sti_plan* plan, uint64_t* out, size_t capacity_
  * only be reused after a layer that has not started).  Takes effect at the next forward. */
 sti_status sti_plan_set_overlap(sti_plan* plan, int overlap);
 
+/* Host-made faults for testing the pipeline's accounting and error paths (no counterpart in the paper, whose
+ * only fault is the operating system reclaiming memory, Section 2.2).  Nothing here touches the device.
+ *   STI_INJECT_SLOW_COPY            : the host sleeps `value` microseconds (<= 1 s) before it enqueues the shard
+ *                                     copy of `layer` in forwards that are launched kernel by kernel (profiling
+ *                                     level 1 or 2); the layer then starts late and its stall_us shows the wait.
+ *                                     Results do not change.
+ *   STI_INJECT_PINNED_ALLOC_FAILURE : with value != 0 the pinned-host allocation of sti_plan_finalize is treated as
+ *                                     failed (STI_ERR_OOM); the plan cannot be used afterwards but can be destroyed.
+ *                                     Only before the plan is finalized (STI_ERR_STATE otherwise); layer is ignored.
+ *   STI_INJECT_NONE                 : clears both. */
+typedef enum { STI_INJECT_NONE = 0, STI_INJECT_SLOW_COPY = 1, STI_INJECT_PINNED_ALLOC_FAILURE = 2 } sti_inject;
+sti_status sti_plan_inject(sti_plan* plan, int what, int layer, unsigned value);
+
 /* Bytes the plan holds: preload buffer in device memory, pinned host arena, ring slots. */
 sti_status sti_plan_memory(sti_plan* plan, uint64_t* preload_bytes, uint64_t* pinned_bytes, uint64_t* ring_bytes);
 
@@ -252,9 +265,12 @@ sti_status sti_host_retile(const uint8_t* src, uint8_t* dst, uint32_t rows, uint
  *   w_dev, codes_dev, wbf16_dev : DEVICE outputs as in sti_shard_decode, caller-owned, any may be NULL
  * Limits: rows*cols*bits/8 <= STI_NOALLOC_MAX_STREAM_BYTES and n_outliers <= STI_NOALLOC_MAX_OUTLIERS
  * (every matrix of BERT-base and BERT-large at up to 6 bits fits); anything larger returns STI_ERR_SIZE
- * and nothing runs.  Host inputs are consumed before the call returns; the kernel runs asynchronously
- * on `stream`.  The first call on a device looks up the array's device address; make that first call
- * before starting any stream capture.  All calls share the one array, which keeps the last call's
+ * and nothing runs.  Host inputs are copied into library-owned staging buffers before the call returns
+ * (pinned or pageable alike: the caller may reuse or free them at once); the kernel runs asynchronously
+ * on `stream`.  The caller's current device is the same after the call as before it.  The first call on a
+ * device looks up the array's device address; make that first call before starting any stream capture.
+ * A call on a stream that is being captured is refused with STI_ERR_STATE, because its copies would read
+ * the shared staging buffers only when the captured work runs.  All calls share the one array, which keeps the last call's
  * contents (each call overwrites everything its kernel reads): calls on the same stream are ordered,
  * calls whose GPU work can overlap (different streams or threads) race on it and must be serialised
  * by the caller. */

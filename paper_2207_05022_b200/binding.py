@@ -87,6 +87,7 @@ def load_library():
         "sti_plan_set_overlap": ([vp, i32], i32),
         "sti_get_stats": ([vp, C.POINTER(StiStats)], i32),
         "sti_plan_memory": ([vp, u64p, u64p, u64p], i32),
+        "sti_plan_inject": ([vp, i32, i32, C.c_uint], i32),
         "sti_ctx_launch_count": ([vp], C.c_uint64),
         "sti_host_retile": ([vp, vp, C.c_uint32, C.c_uint32, C.c_uint32], i32),
         "sti_strerror": ([i32], C.c_char_p),
@@ -103,7 +104,7 @@ def load_library():
 
 EXPORTED = ("sti_ctx_create", "sti_ctx_destroy", "sti_ctx_set_layer_params", "sti_plan_create",
             "sti_plan_destroy", "sti_shard_upload", "sti_plan_finalize", "sti_layer_forward",
-            "sti_model_forward", "sti_model_forward_host", "sti_sync", "sti_shard_decode", "sti_gemm_probe", "sti_get_kernel_stamps",
+            "sti_model_forward", "sti_model_forward_host", "sti_sync", "sti_shard_decode", "sti_gemm_probe", "sti_get_kernel_stamps", "sti_plan_inject",
             "sti_plan_set_profiling", "sti_plan_set_overlap", "sti_get_stats", "sti_plan_memory", "sti_ctx_launch_count",
             "sti_host_retile", "sti_strerror", "sti_matrix_decode_noalloc", "sti_plan_auto",
             "sti_preload_after_run", "sti_quantize_units", "sti_quantize_workspace_bytes")
@@ -248,6 +249,14 @@ def sti_plan_memory(plan: int):
     a, b, c = C.c_uint64(), C.c_uint64(), C.c_uint64()
     _check(load_library().sti_plan_memory(C.c_void_p(plan), C.byref(a), C.byref(b), C.byref(c)), "sti_plan_memory")
     return {"preload_bytes": a.value, "pinned_bytes": b.value, "ring_bytes": c.value}
+
+
+STI_INJECT_NONE, STI_INJECT_SLOW_COPY, STI_INJECT_PINNED_ALLOC_FAILURE = 0, 1, 2
+
+
+def sti_plan_inject(plan: int, what: int, layer: int = 0, value: int = 0):
+    """Host-made faults for tests (see sti.h): a slow shard copy of one layer, a failing pinned allocation."""
+    _check(load_library().sti_plan_inject(C.c_void_p(plan), what, layer, value), "sti_plan_inject")
 
 
 def sti_ctx_launch_count(ctx: int) -> int:

@@ -5,7 +5,9 @@
 #include <cstdlib>
 #include <cstring>
 #include <new>
+#include <chrono>
 #include <string>
+#include <thread>
 #include <vector>
 
 #include <cuda_runtime.h>
@@ -138,6 +140,9 @@ struct sti_plan {
   unsigned long long* stamps = nullptr;   // [layer][kStampKernels][kStampWords] device, profiling level 3
   bool stamping = false;               // the forward being enqueued writes stamps
   bool overlap = true;                 // false: load every streamed layer, then execute (Load&Exec)
+  int slow_copy_layer = -1;            // host-made faults (sti_plan_inject): sleep before enqueueing this layer's copy ...
+  unsigned slow_copy_us = 0;           // ... for this long
+  bool fail_pinned_alloc = false;      // make the pinned-arena allocation of sti_plan_finalize fail
   int n_streamed_layers = 0;
   bool stats_valid = false;
 };
@@ -531,8 +536,10 @@ sti_status enqueue_layer(sti_plan* p, int li, const void* x, void* y, int batch,
   return STI_OK;
 }
 
-sti_status check_forward_args(sti_plan* p, const void* x, void* y, int batch, int seq) {
+sti_status check_forward_args(sti_plan* p, const void* x, void* y, int batch, int seq, bool device_buffers = true) {
   if (!p || !x || !y) return STI_ERR_ARG;
+  // device activations are read through TMA descriptors and vector loads: 16-byte alignment
+  if (device_buffers && ((reinterpret_cast<uintptr_t>(x) | reinterpret_cast<uintptr_t>(y)) & 15)) return STI_ERR_ARG;
   const sti_model_desc& d = p->ctx->desc;
   if (batch < 1 || seq < 1 || seq > d.max_seq) return STI_ERR_SHAPE;
   if (static_cast<long long>(batch) * seq > static_cast<long long>(d.max_batch) * d.max_seq) return STI_ERR_SHAPE;
@@ -543,6 +550,8 @@ sti_status check_forward_args(sti_plan* p, const void* x, void* y, int batch, in
 sti_status enqueue_layer_copy(sti_plan* p, int li, cudaStream_t s) {
   Layer& L = p->layers[li];
   if (L.str_bytes == 0) return STI_OK;
+  if (li == p->slow_copy_layer && p->slow_copy_us)      // injected slow IO: the job reaches the copy engine late
+    std::this_thread::sleep_for(std::chrono::microseconds(p->slow_copy_us));
   CUDA_TRY(cudaMemcpyAsync(p->ring + static_cast<size_t>(L.slot) * p->slot_bytes, L.str_host, L.str_bytes,
                            cudaMemcpyHostToDevice, s));
   return STI_OK;
@@ -675,7 +684,10 @@ sti_status model_forward_impl(sti_plan* p, const ForwardKey& k) {
     if (st != STI_OK || ce != cudaSuccess || !graph) {
       (void)cudaGetLastError();
       if (graph) cudaGraphDestroy(graph);
-      p->graph_off = true;            // fall back to plain stream launches for this plan
+      // an argument or shape error of this call says nothing about later, valid calls: only a failure of the
+      // capture itself switches the plan to plain stream launches
+      if (st == STI_ERR_ARG || st == STI_ERR_SHAPE || st == STI_ERR_STATE) return st;
+      p->graph_off = true;
       return st != STI_OK ? st : enqueue_forward_io(p, k, false);
     }
     cudaGraphExec_t exec = nullptr;
@@ -970,7 +982,10 @@ sti_status sti_plan_finalize(sti_plan* p) {
   p->attempted = true;
   p->preload_bytes = preload_total; p->pinned_bytes = pinned_total; p->slot_bytes = slot_bytes;
   if (preload_total) CUDA_TRY(cudaMalloc(&p->preload, preload_total));
-  if (pinned_total) CUDA_TRY(cudaMallocHost(&p->pinned, pinned_total));
+  if (pinned_total) {
+    if (p->fail_pinned_alloc) return STI_ERR_OOM;          // injected allocation failure
+    CUDA_TRY(cudaMallocHost(&p->pinned, pinned_total));
+  }
   if (slot_bytes) CUDA_TRY(cudaMalloc(&p->ring, slot_bytes * p->ring_slots));
   // 2. fill the preload buffer (device) and the pinned arena (host), one contiguous blob per layer
   size_t pre_cur = 0, pin_cur = 0;
@@ -1119,7 +1134,7 @@ sti_status sti_model_forward(sti_plan* p, const void* x, void* y, int batch, int
 
 sti_status sti_model_forward_host(sti_plan* p, const void* x_host, void* y_host, int batch, int seq,
                                   const int32_t* lens_host) {
-  sti_status st = check_forward_args(p, x_host, y_host, batch, seq);
+  sti_status st = check_forward_args(p, x_host, y_host, batch, seq, false);
   if (st != STI_OK) return st;
   if ((st = sti_plan_finalize(p)) != STI_OK) return st;
   sti_ctx* c = p->ctx;
@@ -1285,6 +1300,25 @@ sti_status sti_get_kernel_stamps(sti_plan* p, uint64_t* out, size_t capacity_wor
   }
   if (n_layers) *n_layers = static_cast<int32_t>(p->layers.size());
   return STI_OK;
+}
+
+sti_status sti_plan_inject(sti_plan* p, int what, int layer, unsigned value) {
+  if (!p) return STI_ERR_ARG;
+  switch (what) {
+    case STI_INJECT_NONE:
+      p->slow_copy_layer = -1; p->slow_copy_us = 0; p->fail_pinned_alloc = false;
+      return STI_OK;
+    case STI_INJECT_SLOW_COPY:
+      if (layer < 0 || layer >= static_cast<int>(p->layers.size()) || value > 1000000u) return STI_ERR_ARG;
+      p->slow_copy_layer = layer; p->slow_copy_us = value;
+      return STI_OK;
+    case STI_INJECT_PINNED_ALLOC_FAILURE:
+      if (p->finalized || p->attempted) return STI_ERR_STATE;
+      p->fail_pinned_alloc = value != 0;
+      return STI_OK;
+    default:
+      return STI_ERR_ARG;
+  }
 }
 
 sti_status sti_plan_memory(sti_plan* p, uint64_t* preload_bytes, uint64_t* pinned_bytes, uint64_t* ring_bytes) {

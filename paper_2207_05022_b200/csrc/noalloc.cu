@@ -36,7 +36,19 @@ constexpr int kMaxDevices = 64;
 std::mutex g_mutex;                           // one call at a time: the host staging buffer is shared too
 unsigned char* g_scratch_dev[kMaxDevices] = {};
 bool g_ready[kMaxDevices] = {};
+// Host side of the staging, shared by all calls (hence the mutex): pageable on purpose, so that cudaMemcpyAsync
+// has read it by the time it returns and the next call may overwrite it.
 unsigned char g_host_stage[kCodesMax];        // re-tiled stream on its way to the device
+float g_host_table[64];
+uint32_t g_host_off[kOutliersMax];
+float g_host_val[kOutliersMax];
+
+// Puts the caller's current device back when the call returns, whatever the outcome.
+struct DeviceGuard {
+  int prev = -1;
+  DeviceGuard() { if (cudaGetDevice(&prev) != cudaSuccess) { (void)cudaGetLastError(); prev = -1; } }
+  ~DeviceGuard() { if (prev >= 0) (void)cudaSetDevice(prev); }
+};
 
 }  // namespace
 
@@ -63,10 +75,20 @@ extern "C" sti_status sti_matrix_decode_noalloc(int device, void* stream, int bi
   }
 
   std::lock_guard<std::mutex> lock(g_mutex);
+  DeviceGuard restore_device;
   if (cudaSetDevice(device) != cudaSuccess) {
     (void)cudaGetLastError();
     return STI_ERR_CUDA;
   }
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  // The copies below read host buffers that the next call reuses and that the caller may free: inside a stream
+  // capture they would only be read when the graph runs.  Such a call is refused.
+  cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
+  if (cudaStreamIsCapturing(s, &cap) != cudaSuccess) {
+    (void)cudaGetLastError();
+    return STI_ERR_CUDA;
+  }
+  if (cap != cudaStreamCaptureStatusNone) return STI_ERR_STATE;
   // ---- first call on this device: find out where the device array lives (not an allocation)
   if (!g_ready[device]) {
     void* p = nullptr;
@@ -79,21 +101,23 @@ extern "C" sti_status sti_matrix_decode_noalloc(int device, void* stream, int bi
     g_ready[device] = true;
   }
   unsigned char* scratch = g_scratch_dev[device];
-  cudaStream_t s = static_cast<cudaStream_t>(stream);
 
   // ---- stage the shard into the scratch: the array still holds the previous call's shard, so every
   // region the kernel will read is overwritten here (stream, table, outlier lists); nothing else is read
   sti::retile_matrix(reinterpret_cast<const unsigned char*>(codes), g_host_stage, rows, cols,
                      static_cast<uint32_t>(bits));
-  float table[64] = {};
-  for (int i = 0; i < (1 << bits); ++i) table[i] = centroids[i];
+  for (int i = 0; i < 64; ++i) g_host_table[i] = i < (1 << bits) ? centroids[i] : 0.f;
+  // the outlier lists go through library-owned pageable buffers too: the caller's arrays may be pinned, and a copy
+  // out of pinned memory would still be reading them after this call has returned
+  for (size_t i = 0; i < n_outliers; ++i) { g_host_off[i] = outlier_off[i]; g_host_val[i] = outlier_val[i]; }
+  auto fail = [] { (void)cudaGetLastError(); return STI_ERR_CUDA; };      // leave no sticky error behind
   if (cudaMemcpyAsync(scratch + kOffCodes, g_host_stage, stream_bytes, cudaMemcpyHostToDevice, s) != cudaSuccess ||
-      cudaMemcpyAsync(scratch + kOffTable, table, kTableBytes, cudaMemcpyHostToDevice, s) != cudaSuccess)
-    return STI_ERR_CUDA;
+      cudaMemcpyAsync(scratch + kOffTable, g_host_table, kTableBytes, cudaMemcpyHostToDevice, s) != cudaSuccess)
+    return fail();
   if (n_outliers) {
-    if (cudaMemcpyAsync(scratch + kOffOutOff, outlier_off, n_outliers * 4, cudaMemcpyHostToDevice, s) != cudaSuccess ||
-        cudaMemcpyAsync(scratch + kOffOutVal, outlier_val, n_outliers * 4, cudaMemcpyHostToDevice, s) != cudaSuccess)
-      return STI_ERR_CUDA;
+    if (cudaMemcpyAsync(scratch + kOffOutOff, g_host_off, n_outliers * 4, cudaMemcpyHostToDevice, s) != cudaSuccess ||
+        cudaMemcpyAsync(scratch + kOffOutVal, g_host_val, n_outliers * 4, cudaMemcpyHostToDevice, s) != cudaSuccess)
+      return fail();
   }
   sti::DecodeLaunch dl{};
   dl.codes = reinterpret_cast<const uint4*>(scratch + kOffCodes);
@@ -108,6 +132,6 @@ extern "C" sti_status sti_matrix_decode_noalloc(int device, void* stream, int bi
   dl.w = w_dev;
   dl.codes_out = codes_dev;
   dl.wbf16 = wbf16_dev;
-  if (sti::launch_decode(dl, s) != cudaSuccess) return STI_ERR_CUDA;
+  if (sti::launch_decode(dl, s) != cudaSuccess) return fail();
   return STI_OK;
 }

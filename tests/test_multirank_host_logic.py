@@ -52,3 +52,42 @@ def test_reference_arm_only_prints_on_rank_zero(monkeypatch, capsys):
     monkeypatch.setenv("RANK", "1")
     bench.run_reference(Args)                              # other ranks leave without work or output
     assert capsys.readouterr().out == ""
+
+
+_RANK_SCRIPT = """
+import json, os, sys
+sys.path.insert(0, {root!r})
+import torch.distributed as dist
+import bench
+rank, world = int(os.environ["RANK"]), int(os.environ["WORLD_SIZE"])
+assert os.environ["MASTER_ADDR"] == "127.0.0.1" and int(os.environ["LOCAL_RANK"]) == rank
+dist.init_process_group("gloo", rank=rank, world_size=world)
+job_ms = bench.max_over_ranks(10.0 + 5.0 * rank, world, device="cpu")
+dist.barrier()
+if rank == 0:
+    print(json.dumps({{"n_gpus": world, "ms": job_ms, "value": bench.aggregate_throughput(1.0e9, world, job_ms)}}))
+else:
+    print("rank", rank, "done")          # must not reach the job's stdout
+dist.destroy_process_group()
+"""
+
+
+def test_plain_launch_with_gpus_n_spawns_n_ranks(tmp_path):
+    """`bench.py --gpus N` started without torchrun starts the N replicas itself (spawn_ranks): every rank gets the
+    rendezvous variables, only rank 0 writes the job's JSON line, the exit code is the worst rank's."""
+    import json
+    import subprocess
+    script = tmp_path / "rank.py"
+    script.write_text(_RANK_SCRIPT.format(root=ROOT))
+    driver = ("import sys; sys.path.insert(0, %r); import bench; "
+              "sys.exit(bench.spawn_ranks(2, [sys.executable, %r], port=%d))" % (ROOT, str(script), 31500 + os.getpid() % 2000))
+    res = subprocess.run([sys.executable, "-c", driver], capture_output=True, text=True, timeout=300)
+    assert res.returncode == 0, res.stderr[-2000:]
+    lines = [ln for ln in res.stdout.splitlines() if ln.strip()]
+    assert len(lines) == 1                                   # one JSON line, from rank 0
+    out = json.loads(lines[0])
+    assert out["n_gpus"] == 2 and out["ms"] == 15.0 and out["value"] == pytest.approx(2 * 1.0e9 / 15.0e-3)
+    assert "rank 1 done" in res.stderr
+    bad = ("import sys; sys.path.insert(0, %r); import bench; "
+           "sys.exit(bench.spawn_ranks(2, [sys.executable, '-c', 'import os, sys; sys.exit(int(os.environ[\"RANK\"]) * 3)']))" % ROOT)
+    assert subprocess.run([sys.executable, "-c", bad], timeout=120).returncode == 3

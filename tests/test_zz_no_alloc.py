@@ -3,8 +3,8 @@
 sti_matrix_decode_noalloc is for callers that cannot allocate device memory (a shard-file check inside a
 serving process whose framework allocator owns the GPU's memory, code under an enforced memory budget):
 it keeps its working copy of the shard in a fixed array inside the library instead of in a plan's arenas.
-Here it must give, bit for bit, what sti_shard_decode gives for the same matrix, on consecutive calls
-that reuse the array (larger matrix first, then smaller ones, so stale contents would show).
+Here it must give, bit for bit, what sti_shard_decode gives for the same matrix and what the CPU oracle decodes,
+on consecutive calls that reuse the array (larger matrix first, then smaller ones, so stale contents would show).
 This file sorts last on purpose: a failure here cannot hide the result of any other test.
 """
 import numpy as np
@@ -13,6 +13,7 @@ import torch
 
 import workloads as W
 from workloads.shards import ATTN, FFN
+from oracle import sti_oracle as O
 
 sti = pytest.importorskip("paper_2207_05022_b200")
 
@@ -48,6 +49,14 @@ def test_noalloc_decode_matches_plan_decode_on_consecutive_calls():
         for kind, idx, m in order:
             blob = work.blobs[(0, kind, idx)]
             r, c, words, off, val = _matrix_inputs(shape, kind, blob, m)
+            # the oracle's decode of the same matrix: indexes, fp32 values with outliers, bf16 operand bits
+            o_w, o_codes = O.decode_unit(blob.bits, blob.codes, blob.centroids, blob.outlier_off, blob.outlier_val,
+                                         shape.hidden, shape.head_dim, shape.slice_width, kind, return_codes=True)
+            name = W.unit_matrix_shapes(shape, kind)[m][0]
+            want_w = torch.from_numpy(o_w[name].reshape(-1).view(np.int32).copy())
+            want_codes = torch.from_numpy(o_codes[name].reshape(-1).astype(np.uint8))
+            want_bf16 = torch.from_numpy((O.bf16_rne(o_w[name]).reshape(-1).view(np.uint32) >> 16).astype(np.uint16)
+                                         .view(np.int16).copy())
             ref = [torch.zeros(r * c, dtype=dt, device="cuda") for dt in (torch.float32, torch.uint8, torch.int16)]
             got = [torch.zeros(r * c, dtype=dt, device="cuda") for dt in (torch.float32, torch.uint8, torch.int16)]
             torch.cuda.synchronize()
@@ -63,6 +72,10 @@ def test_noalloc_decode_matches_plan_decode_on_consecutive_calls():
                 assert torch.equal(got[1], ref[1]), (kind, idx, m, "indexes")
                 assert torch.equal(got[0].view(torch.int32), ref[0].view(torch.int32)), (kind, idx, m, "fp32")
                 assert torch.equal(got[2], ref[2]), (kind, idx, m, "bf16")
+                assert torch.equal(got[1].cpu(), want_codes), (kind, idx, m, "indexes vs oracle")
+                assert torch.equal(got[0].view(torch.int32).cpu(), want_w), (kind, idx, m, "fp32 vs oracle")
+                assert torch.equal(got[2].cpu(), want_bf16), (kind, idx, m, "bf16 vs oracle")
+    assert torch.cuda.current_device() == 0                  # the call leaves the current device as it found it
 
 
 def test_noalloc_rejects_what_the_fixed_array_cannot_hold():
