@@ -225,6 +225,31 @@ sti_status sti_get_kernel_stamps(sti_plan* plan, uint64_t* out, size_t capacity_
  * only be reused after a layer that has not started).  Takes effect at the next forward. */
 sti_status sti_plan_set_overlap(sti_plan* plan, int overlap);
 
+/* Section 3.2 ("back-to-back executions": shards a run loaded stay cached, and the next plan spends the freed IO time
+ * on the others) and Section 5.5 (after a run, loaded shards are evicted from the top layer down until the rest fits
+ * the preload buffer).  Which shards stay is the planner's decision (sti_preload_after_run); these calls keep them in
+ * DEVICE memory across plans, so that the next plan uploads nothing it already holds.
+ *
+ * sti_plan_retain: attn_keep [n_layers*n_heads] and ffn_keep [n_layers*n_ffn_slices] (host, 0/1) mark the kept units
+ * of `plan` that must stay on the device after its next run.  Preloaded units are there already; for the streamed
+ * ones the call allocates a retained arena of their size (*retained_bytes) and the NEXT sti_model_forward on the plan
+ * - launched kernel by kernel once, not as a graph replay - copies each of them device-to-device out of its ring slot
+ * right after the layer that used it.  Marking a unit the plan dropped is STI_ERR_ARG; one retained set per plan
+ * (STI_ERR_STATE on a second call).
+ *
+ * sti_shard_adopt: instead of sti_shard_upload - the unit (layer, kind, index) of the not yet finalized `plan` takes
+ * over the unit that `from` (same context, finalized, still alive until `plan` is finalized) holds in device memory:
+ * preloaded there, or retained and the retaining forward already enqueued.  Same bitwidth in both plans
+ * (STI_ERR_BITS otherwise: a shard is cached at the version it was loaded with), resident in `plan` (STI_ERR_STATE
+ * otherwise, also when `from` does not hold the unit on the device).  sti_plan_finalize then fills that part of the
+ * preload buffer with a device-to-device copy.
+ *
+ * sti_plan_fill_stats: bytes sti_plan_finalize uploaded from the host into the preload buffer, bytes it took over on
+ * the device, bytes of the retained arena (any pointer may be NULL). */
+sti_status sti_plan_retain(sti_plan* plan, const uint8_t* attn_keep, const uint8_t* ffn_keep, uint64_t* retained_bytes);
+sti_status sti_shard_adopt(sti_plan* plan, const sti_plan* from, int layer, sti_kind kind, int index);
+sti_status sti_plan_fill_stats(sti_plan* plan, uint64_t* uploaded_bytes, uint64_t* adopted_bytes, uint64_t* retained_bytes);
+
 /* Host-made faults for testing the pipeline's accounting and error paths (no counterpart in the paper, whose
  * only fault is the operating system reclaiming memory, Section 2.2).  Nothing here touches the device.
  *   STI_INJECT_SLOW_COPY            : the host sleeps `value` microseconds (<= 1 s) before it enqueues the shard

@@ -88,6 +88,9 @@ def load_library():
         "sti_get_stats": ([vp, C.POINTER(StiStats)], i32),
         "sti_plan_memory": ([vp, u64p, u64p, u64p], i32),
         "sti_plan_inject": ([vp, i32, i32, C.c_uint], i32),
+        "sti_plan_retain": ([vp, vp, vp, u64p], i32),
+        "sti_shard_adopt": ([vp, vp, i32, i32, i32], i32),
+        "sti_plan_fill_stats": ([vp, u64p, u64p, u64p], i32),
         "sti_ctx_launch_count": ([vp], C.c_uint64),
         "sti_host_retile": ([vp, vp, C.c_uint32, C.c_uint32, C.c_uint32], i32),
         "sti_strerror": ([i32], C.c_char_p),
@@ -105,6 +108,7 @@ def load_library():
 EXPORTED = ("sti_ctx_create", "sti_ctx_destroy", "sti_ctx_set_layer_params", "sti_plan_create",
             "sti_plan_destroy", "sti_shard_upload", "sti_plan_finalize", "sti_layer_forward",
             "sti_model_forward", "sti_model_forward_host", "sti_sync", "sti_shard_decode", "sti_gemm_probe", "sti_get_kernel_stamps", "sti_plan_inject",
+            "sti_plan_retain", "sti_shard_adopt", "sti_plan_fill_stats",
             "sti_plan_set_profiling", "sti_plan_set_overlap", "sti_get_stats", "sti_plan_memory", "sti_ctx_launch_count",
             "sti_host_retile", "sti_strerror", "sti_matrix_decode_noalloc", "sti_plan_auto",
             "sti_preload_after_run", "sti_quantize_units", "sti_quantize_workspace_bytes")
@@ -257,6 +261,26 @@ STI_INJECT_NONE, STI_INJECT_SLOW_COPY, STI_INJECT_PINNED_ALLOC_FAILURE = 0, 1, 2
 def sti_plan_inject(plan: int, what: int, layer: int = 0, value: int = 0):
     """Host-made faults for tests (see sti.h): a slow shard copy of one layer, a failing pinned allocation."""
     _check(load_library().sti_plan_inject(C.c_void_p(plan), what, layer, value), "sti_plan_inject")
+
+
+def sti_plan_retain(plan: int, attn_keep, ffn_keep) -> int:
+    """Marks kept units (flat, layer-major 0/1 arrays) to stay in device memory after the plan's next run (see sti.h);
+    returns the bytes of the retained arena."""
+    a, f = _host(attn_keep, np.uint8).reshape(-1), _host(ffn_keep, np.uint8).reshape(-1)
+    n = C.c_uint64()
+    _check(load_library().sti_plan_retain(C.c_void_p(plan), _ptr(a), _ptr(f), C.byref(n)), "sti_plan_retain")
+    return int(n.value)
+
+
+def sti_shard_adopt(plan: int, from_plan: int, layer: int, kind: int, index: int):
+    """Takes a unit over from another plan's device memory instead of uploading it (see sti.h)."""
+    _check(load_library().sti_shard_adopt(C.c_void_p(plan), C.c_void_p(from_plan), layer, kind, index), "sti_shard_adopt")
+
+
+def sti_plan_fill_stats(plan: int):
+    a, b, c = C.c_uint64(), C.c_uint64(), C.c_uint64()
+    _check(load_library().sti_plan_fill_stats(C.c_void_p(plan), C.byref(a), C.byref(b), C.byref(c)), "sti_plan_fill_stats")
+    return {"uploaded_bytes": a.value, "adopted_bytes": b.value, "retained_bytes": c.value}
 
 
 def sti_ctx_launch_count(ctx: int) -> int:

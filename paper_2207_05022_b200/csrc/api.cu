@@ -49,6 +49,13 @@ struct Unit {
   std::vector<float> out_val;
   size_t off_codes = 0, off_table = 0, off_ooff = 0, off_oval = 0, bytes = 0;   // inside the layer part
   uint8_t* dev = nullptr;              // where the unit's region starts in device memory
+  size_t codes_bytes = 0;              // size of the index stream (known even when the bytes are not on the host)
+  // Back-to-back executions (Section 3.2): a unit another plan already holds in device memory is taken over with
+  // a device-to-device copy instead of an upload; a streamed unit can be kept after a run for the next plan.
+  const uint8_t* adopt_src = nullptr;  // device address of the whole unit region in the plan it is adopted from
+  bool retain = false;                 // copy this streamed unit out of its ring slot during the next forward
+  uint8_t* retained = nullptr;         // where that copy lives (retained arena), valid once retained_done
+  bool retained_done = false;
 };
 
 struct GemmTable {
@@ -140,6 +147,9 @@ struct sti_plan {
   unsigned long long* stamps = nullptr;   // [layer][kStampKernels][kStampWords] device, profiling level 3
   bool stamping = false;               // the forward being enqueued writes stamps
   bool overlap = true;                 // false: load every streamed layer, then execute (Load&Exec)
+  uint8_t* retain_arena = nullptr; size_t retain_bytes = 0;   // streamed units kept for the next plan
+  bool retain_pending = false;         // the next model forward copies the units marked `retain` out of the ring
+  uint64_t finalize_h2d_bytes = 0, finalize_d2d_bytes = 0;    // how the preload buffer was filled
   int slow_copy_layer = -1;            // host-made faults (sti_plan_inject): sleep before enqueueing this layer's copy ...
   unsigned slow_copy_us = 0;           // ... for this long
   bool fail_pinned_alloc = false;      // make the pinned-arena allocation of sti_plan_finalize fail
@@ -609,6 +619,18 @@ sti_status enqueue_forward(sti_plan* p, const void* x, void* y, int batch, int s
     // the layer's first GEMM also pulls the next layer's packed shards into L2 (if they are on the device yet)
     sti_status st = enqueue_layer(p, li, cur, nxt, batch, seq, lens, li > 0, li + 1 < n, li + 1 < n ? li + 1 : -1);
     if (st != STI_OK) return st;
+    if (p->retain_pending && !capturing && L.str_bytes > 0) {
+      // keep what this run loaded (Section 3.2): the marked units leave their ring slot for the retained arena
+      // before the slot is handed back to the copy stream
+      const uint8_t* slot = p->ring + static_cast<size_t>(L.slot) * p->slot_bytes;
+      auto keep_unit = [&](Unit& u) -> cudaError_t {
+        if (!u.retain || u.retained_done || u.cfg.resident) return cudaSuccess;
+        u.retained_done = true;
+        return cudaMemcpyAsync(u.retained, slot + u.off_codes, u.bytes, cudaMemcpyDeviceToDevice, c->compute);
+      };
+      for (auto& u : L.attn) CUDA_TRY(keep_unit(u));
+      for (auto& u : L.ffn) CUDA_TRY(keep_unit(u));
+    }
     if (prof) CUDA_TRY(cudaEventRecord(L.ev_done, c->compute));
     if (L.str_bytes > 0) {
       CUDA_TRY(cudaEventRecord(capturing ? p->g_slot_free[L.slot] : p->slot_free[L.slot], c->compute));
@@ -667,6 +689,12 @@ sti_status enqueue_forward_io(sti_plan* p, const ForwardKey& k, bool capturing) 
 sti_status model_forward_impl(sti_plan* p, const ForwardKey& k) {
   sti_ctx* c = p->ctx;
   if ((p->profiling && p->profiling < 3) || p->graph_off) return enqueue_forward_io(p, k, false);
+  if (p->retain_pending && k.layer < 0) {
+    // one forward launched kernel by kernel: it also moves the shards to keep out of the ring slots
+    const sti_status st = enqueue_forward_io(p, k, false);
+    if (st == STI_OK) p->retain_pending = false;
+    return st;
+  }
   sti_plan::CachedGraph* hit = nullptr;
   for (auto& g : p->graphs) if (g.exec && g.key == k) hit = &g;
   if (!hit) {
@@ -721,7 +749,7 @@ sti_status model_forward_impl(sti_plan* p, const ForwardKey& k) {
 
 void free_plan_device(sti_plan* p) {
   if (!p) return;
-  cudaFree(p->preload); cudaFree(p->ring); cudaFree(p->tables);
+  cudaFree(p->preload); cudaFree(p->ring); cudaFree(p->tables); cudaFree(p->retain_arena);
   if (p->pinned) cudaFreeHost(p->pinned);
   cudaFree(p->qkv); cudaFree(p->attn_out); cudaFree(p->partial); cudaFree(p->h1_f32); cudaFree(p->h1_bf16);
   cudaFree(p->u); cudaFree(p->x_bf16); cudaFree(p->buf[0]); cudaFree(p->buf[1]); cudaFree(p->x_in); cudaFree(p->y_out);
@@ -926,6 +954,8 @@ sti_status sti_shard_upload(sti_plan* p, int layer, sti_kind kind, int index, co
     if (blob->outlier_off[i] >= n_weights) return STI_ERR_SIZE;
     if (i && blob->outlier_off[i] <= blob->outlier_off[i - 1]) return STI_ERR_ARG;
   }
+  u->adopt_src = nullptr;
+  u->codes_bytes = blob->n_code_words * 4;
   u->codes.assign(blob->n_code_words * 4, 0);
   const uint8_t* src = reinterpret_cast<const uint8_t*>(blob->codes);
   if (bits == 32) {
@@ -962,7 +992,7 @@ sti_status sti_plan_finalize(sti_plan* p) {
       if (!u.uploaded) return false;
       size_t& cursor = u.cfg.resident ? L.res_bytes : L.str_bytes;
       const size_t start = cursor;
-      u.off_codes = cursor; cursor += align16(u.codes.size());
+      u.off_codes = cursor; cursor += align16(u.codes_bytes);
       u.off_table = cursor; cursor += align16(u.table.size() * 4);
       u.off_ooff = cursor; cursor += align16(u.out_off.size() * 4);
       u.off_oval = cursor; cursor += align16(u.out_val.size() * 4);
@@ -995,24 +1025,39 @@ sti_status sti_plan_finalize(sti_plan* p) {
     L.str_host = p->pinned ? p->pinned + pin_cur : nullptr;
     pre_cur += align256(L.res_bytes);
     pin_cur += align256(L.str_bytes);
-    staging.assign(L.res_bytes, 0);
     if (L.str_bytes) memset(L.str_host, 0, L.str_bytes);
+    cudaError_t unit_err = cudaSuccess;
     auto emit = [&](Unit& u) {
-      if (!u.cfg.keep) return;
-      uint8_t* base = u.cfg.resident ? staging.data() : L.str_host;
-      memcpy(base + u.off_codes, u.codes.data(), u.codes.size());
-      if (!u.table.empty()) memcpy(base + u.off_table, u.table.data(), u.table.size() * 4);
+      if (!u.cfg.keep || unit_err != cudaSuccess) return;
+      if (u.adopt_src) {
+        // already in device memory (another plan's preload buffer or retained shards): no host traffic
+        u.dev = L.res_dev;
+        unit_err = cudaMemcpyAsync(L.res_dev + u.off_codes, u.adopt_src, u.bytes, cudaMemcpyDeviceToDevice, c->compute);
+        p->finalize_d2d_bytes += u.bytes;
+        return;
+      }
+      // resident units go up one by one (nothing is uploaded for the units adopted above)
+      staging.assign(u.cfg.resident ? u.bytes : 0, 0);
+      // a resident unit's region is built in `staging` (its first byte = off_codes), a streamed one in the pinned blob
+      auto at = [&](size_t off) { return u.cfg.resident ? staging.data() + (off - u.off_codes) : L.str_host + off; };
+      memcpy(at(u.off_codes), u.codes.data(), u.codes.size());
+      if (!u.table.empty()) memcpy(at(u.off_table), u.table.data(), u.table.size() * 4);
       if (!u.out_off.empty()) {
-        memcpy(base + u.off_ooff, u.out_off.data(), u.out_off.size() * 4);
-        memcpy(base + u.off_oval, u.out_val.data(), u.out_val.size() * 4);
+        memcpy(at(u.off_ooff), u.out_off.data(), u.out_off.size() * 4);
+        memcpy(at(u.off_oval), u.out_val.data(), u.out_val.size() * 4);
       }
       u.dev = u.cfg.resident ? L.res_dev : p->ring + static_cast<size_t>(L.slot) * p->slot_bytes;
+      if (u.cfg.resident) {
+        unit_err = cudaMemcpy(L.res_dev + u.off_codes, staging.data(), u.bytes, cudaMemcpyHostToDevice);
+        p->finalize_h2d_bytes += u.bytes;
+      }
       std::vector<uint8_t>().swap(u.codes);     // the arenas now hold the only copy
     };
     for (auto& u : L.attn) emit(u);
     for (auto& u : L.ffn) emit(u);
-    if (L.res_bytes) CUDA_TRY(cudaMemcpy(L.res_dev, staging.data(), L.res_bytes, cudaMemcpyHostToDevice));
+    CUDA_TRY(unit_err);
   }
+  CUDA_TRY(cudaStreamSynchronize(c->compute));   // adopted units are in place before their source plan may go away
   // 3. tile-job tables
   std::vector<uint8_t> host_tables;
   struct Fix { GemmTable* t; size_t jobs_off, segs_off; };
@@ -1299,6 +1344,78 @@ sti_status sti_get_kernel_stamps(sti_plan* p, uint64_t* out, size_t capacity_wor
     out[i] = v == ~0ull ? 0 : (is_min ? v : ~v);
   }
   if (n_layers) *n_layers = static_cast<int32_t>(p->layers.size());
+  return STI_OK;
+}
+
+sti_status sti_plan_retain(sti_plan* p, const uint8_t* attn_keep, const uint8_t* ffn_keep, uint64_t* retained_bytes) {
+  if (!p || !attn_keep || !ffn_keep) return STI_ERR_ARG;
+  sti_status st = sti_plan_finalize(p);
+  if (st != STI_OK) return st;
+  if (p->retain_arena) return STI_ERR_STATE;               // one retained set per plan
+  sti_ctx* c = p->ctx;
+  const sti_model_desc& d = c->desc;
+  CUDA_TRY(cudaSetDevice(c->device));
+  size_t total = 0;
+  for (int l = 0; l < d.n_layers; ++l) {
+    Layer& L = p->layers[l];
+    for (int h = 0; h < d.n_heads; ++h)
+      if (attn_keep[l * d.n_heads + h] && !L.attn[h].cfg.keep) return STI_ERR_ARG;     // cannot keep what the plan dropped
+    for (int j = 0; j < d.n_ffn_slices; ++j)
+      if (ffn_keep[l * d.n_ffn_slices + j] && !L.ffn[j].cfg.keep) return STI_ERR_ARG;
+  }
+  for (int l = 0; l < d.n_layers; ++l) {
+    Layer& L = p->layers[l];
+    auto mark = [&](Unit& u, bool keep) {
+      u.retain = keep && u.cfg.keep && !u.cfg.resident;    // resident units are on the device anyway
+      if (u.retain) total += align256(u.bytes);
+    };
+    for (int h = 0; h < d.n_heads; ++h) mark(L.attn[h], attn_keep[l * d.n_heads + h] != 0);
+    for (int j = 0; j < d.n_ffn_slices; ++j) mark(L.ffn[j], ffn_keep[l * d.n_ffn_slices + j] != 0);
+  }
+  if (total) {
+    CUDA_TRY(cudaMalloc(&p->retain_arena, total));
+    size_t cur = 0;
+    for (auto& L : p->layers) {
+      auto bind = [&](Unit& u) { if (u.retain) { u.retained = p->retain_arena + cur; cur += align256(u.bytes); } };
+      for (auto& u : L.attn) bind(u);
+      for (auto& u : L.ffn) bind(u);
+    }
+    p->retain_pending = true;
+  }
+  p->retain_bytes = total;
+  if (retained_bytes) *retained_bytes = total;
+  return STI_OK;
+}
+
+sti_status sti_shard_adopt(sti_plan* p, const sti_plan* from, int layer, sti_kind kind, int index) {
+  if (!p || !from || p == from || (kind != STI_ATTN && kind != STI_FFN)) return STI_ERR_ARG;
+  if (p->ctx != from->ctx) return STI_ERR_ARG;             // same device, same streams
+  if (p->finalized || !from->finalized) return STI_ERR_STATE;
+  Unit* u = find_unit(p, layer, kind, index);
+  const Unit* src = find_unit(const_cast<sti_plan*>(from), layer, kind, index);
+  if (!u || !src) return STI_ERR_ARG;
+  if (!u->cfg.keep || !u->cfg.resident || !src->cfg.keep) return STI_ERR_STATE;   // adopted units live in the preload buffer
+  if (u->cfg.bits != src->cfg.bits) return STI_ERR_BITS;                          // a shard is cached at the version it was loaded with
+  const uint8_t* where = nullptr;
+  if (src->cfg.resident) where = src->dev + src->off_codes;
+  else if (src->retained && src->retained_done) where = src->retained;
+  if (!where) return STI_ERR_STATE;                        // not in device memory: it has to be uploaded
+  u->table = src->table;                                   // host-side metadata the tile tables are built from
+  u->out_off = src->out_off;
+  u->out_val = src->out_val;
+  u->codes.clear();
+  u->codes_bytes = src->codes_bytes;
+  u->adopt_src = where;
+  u->uploaded = true;
+  return STI_OK;
+}
+
+sti_status sti_plan_fill_stats(sti_plan* p, uint64_t* uploaded_bytes, uint64_t* adopted_bytes, uint64_t* retained_bytes) {
+  if (!p) return STI_ERR_ARG;
+  if (!p->finalized) return STI_ERR_STATE;
+  if (uploaded_bytes) *uploaded_bytes = p->finalize_h2d_bytes;
+  if (adopted_bytes) *adopted_bytes = p->finalize_d2d_bytes;
+  if (retained_bytes) *retained_bytes = p->retain_bytes;
   return STI_OK;
 }
 
