@@ -37,6 +37,7 @@ struct Tuning {
   int qkv_n = 32, f1_n = 64, o_n = 64, o_group = 4, f2_n = 64, f2_group = 2;
   int cta_budget = 148;                // CTAs a GEMM launch may use when it splits the token tiles over CTAs
   int pair_min_tiles = 8;              // two-CTA GEMM from this many 128-token tiles on (0 = never)
+  int attn_tc_min_items = 96;          // tensor-core attention from this many (sequence, kept head) pairs on, seq >= 256 (0 = never)
   int ln1_ctas = -1, ln2_ctas = -1;    // LayerNorm CTA counts: -1 = chosen per launch (see ln_ctas_hint), 0 = one row per CTA
 };
 
@@ -210,6 +211,7 @@ void parse_tuning(Tuning* t, int tmax, const sti_model_desc& d, int sm_count) {
         else if (k == "f2_n") t->f2_n = v;
         else if (k == "f2_group") t->f2_group = v;
         else if (k == "pair_min_tiles") t->pair_min_tiles = v;
+        else if (k == "attn_tc_min_items") t->attn_tc_min_items = std::max(0, v);
         else if (k == "cta_budget") t->cta_budget = std::max(1, v);
         else if (k == "ln1_ctas") t->ln1_ctas = std::max(-1, v);
         else if (k == "ln2_ctas") t->ln2_ctas = std::max(-1, v);
@@ -489,7 +491,14 @@ sti_status enqueue_layer(sti_plan* p, int li, const void* x, void* y, int batch,
     st = run_gemm(p, GEMM_BF16_TO_BF16, L.qkv, xq, d.hidden, T, p->qkv, 64, dense + c->off_bq, next_layer, -1, stamp(1));
     if (st != STI_OK) return st;
     CUDA_TRY(mark(1));
-    CUDA_TRY(launch_attention(p->qkv, p->attn_out, nh, batch, seq, lens, c->compute, c->pdl, stamp(2)));
+    if (p->tune.attn_tc_min_items > 0 && seq >= 256 && batch * nh >= p->tune.attn_tc_min_items && !c->simt_debug) {
+      // many (sequence, head) pairs: one CTA each on the tensor cores, K and V of the sequence resident in shared memory
+      CUtensorMap qmap;
+      if (!make_xmap(&qmap, p->qkv, 64, 3 * nh * T)) return STI_ERR_CUDA;
+      CUDA_TRY(launch_attention_tc(qmap, p->attn_out, nh, batch, seq, lens, c->err_dev, c->compute, c->pdl, stamp(2)));
+    } else {
+      CUDA_TRY(launch_attention(p->qkv, p->attn_out, nh, batch, seq, lens, c->compute, c->pdl, stamp(2)));
+    }
     c->launches++;
     CUDA_TRY(mark(2));
     st = run_gemm(p, GEMM_BF16_TO_F32, L.o, p->attn_out, nh * 64, T, p->partial, d.hidden, nullptr, -1, -1, stamp(3));
@@ -848,7 +857,7 @@ sti_status sti_ctx_create(const sti_model_desc* desc, int device, void* compute_
   if (cudaMemset(c->dense, 0, c->dense_stride * d.n_layers * sizeof(float)) != cudaSuccess) return fail(STI_ERR_CUDA);
   if (cudaMalloc(&c->err_dev, sizeof(int)) != cudaSuccess) return fail(STI_ERR_OOM);
   if (cudaMemset(c->err_dev, 0, sizeof(int)) != cudaSuccess) return fail(STI_ERR_CUDA);
-  if (gemm_configure() != cudaSuccess || attention_configure() != cudaSuccess)
+  if (gemm_configure() != cudaSuccess || attention_configure() != cudaSuccess || attention_tc_configure() != cudaSuccess)
     return fail(STI_ERR_CUDA);
   if (cudaDeviceGetAttribute(&c->sm_count, cudaDevAttrMultiProcessorCount, device) != cudaSuccess || c->sm_count < 1)
     return fail(STI_ERR_CUDA);
