@@ -498,6 +498,33 @@ def planner_point(args, target_ms):
             "hidden_frac": 1.0 - stall_us / copy_us if copy_us > 0 else None, "h2d_GBps": pf["h2d_gbps"]}
 
 
+def decode_rate_point(sti, torch, sess, work, stream, flush, peaks, token_counts=(8, 32, 128), reps=7):
+    """Steady-state rate of the fused decode: ONE launch over the FFN1 tiles of all layers (sti_decode_rate_probe), timed
+    with events, at few tokens where the decode is all there is to do.  Packed bytes per second against the HBM roof."""
+    d, n_layers, ffn = work.shape.hidden, work.shape.n_layers, work.shape.ffn
+    out = {"what": "one launch of the dequant-GEMM over every layer's FFN1 tiles (weights resident, cold L2)"}
+    for T in token_counts:
+        x = torch.randn(T, d, device="cuda").to(torch.bfloat16)
+        y = torch.empty(T, n_layers * ffn, dtype=torch.bfloat16, device="cuda")
+        ms = []
+        packed = tiles = 0
+        with torch.cuda.stream(stream):
+            for i in range(reps + 2):
+                flush.zero_()
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                e0.record(stream)
+                packed, tiles = sti.sti_decode_rate_probe(sess.plan, x.data_ptr(), T, y.data_ptr(), y.numel() * 2)
+                e1.record(stream)
+                stream.synchronize()
+                if i >= 2:
+                    ms.append(e0.elapsed_time(e1))
+        t = float(np.median(ms)) * 1e-3
+        out[f"tokens_{T}"] = {"ms": t * 1e3, "tiles": tiles, "packed_bytes": packed, "packed_GBps": packed / t / 1e9,
+                              "frac_of_hbm": packed / t / 1e9 / float(peaks["hbm_gbs"]),
+                              "weights_per_s": n_layers * ffn * d / t}
+    return out
+
+
 def model_point(sti, torch, work, stream, flush, peaks, label, steps=12, warm=4):
     """A model workload resident and streamed: forward ms (median, cold L2), the dequant-GEMMs' stamped time and
     TFLOP/s under graph replay, and how much of the host-to-device copy time the pipeline hid."""
@@ -961,6 +988,8 @@ def main():
     mem = sti.sti_plan_memory(s_str.plan)
     h2d_plain = plain_h2d_gbps(torch, stream) if rank == 0 else None
 
+    decode_rate = decode_rate_point(sti, torch, s_res, work_str, stream, flush, peaks) if rank == 0 else None
+
     s_res.close()
     s_str.close()
     extras = {}
@@ -1049,6 +1078,7 @@ def main():
                      "h2d_plain_pinned_GBps": h2d_plain,
                      "preload_bytes": mem["preload_bytes"], "pinned_bytes": mem["pinned_bytes"],
                      "ring_bytes": mem["ring_bytes"]},
+        "decode_rate": decode_rate,
         "extras": extras,
     }
     print(json.dumps(line))

@@ -195,6 +195,18 @@ sti_status sti_shard_decode(sti_plan* plan, int layer, sti_kind kind, int index,
 sti_status sti_gemm_probe(sti_plan* plan, int layer, int gemm, const void* x_bf16_dev, int tokens, void* out_dev,
                           size_t out_capacity_bytes, int variant, int32_t* n_partials);
 
+/* Section 4.2 decompression at its steady-state rate: ONE launch of the fused dequant-GEMM over the FFN1 tiles of
+ * ALL layers (every kept FFN slice's F1 matrix, hundreds of tiles for a 24-layer model), on few tokens, so that the
+ * launch is long enough for the decode's throughput to show instead of one layer's launch and fill latencies.  Used by
+ * the benchmark to report packed-weight GB/s against the HBM roof.  out = x F1^T per layer, no bias, no GELU.
+ *   x_bf16_dev : DEVICE, [tokens, hidden] bf16, 16-byte aligned; tokens <= 128
+ *   out_dev    : DEVICE, bf16 [tokens][n_layers * ffn] (layer l, kept slice number j of that layer at columns
+ *                l * ffn + j * f ...), 16-byte aligned; out_capacity_bytes >= tokens * n_layers * ffn * 2
+ *   packed_bytes, n_tiles : optional outs - index-stream and table bytes the launch reads, weight tiles (CTAs) it runs
+ * Every kept shard must be resident (STI_ERR_STATE otherwise, also when no FFN slice is kept).  Asynchronous. */
+sti_status sti_decode_rate_probe(sti_plan* plan, const void* x_bf16_dev, int tokens, void* out_dev,
+                                 size_t out_capacity_bytes, uint64_t* packed_bytes, int32_t* n_tiles);
+
 /* Section 5.2 (profiling of IO and compute delays): per-layer timings of the last
  * sti_model_forward.  Enable with sti_plan_set_profiling before that forward: level 0 = off,
  * 1 = per-layer events, 2 = additionally events around every kernel (slightly slower; levels 1 and 2 launch

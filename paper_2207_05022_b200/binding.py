@@ -82,6 +82,7 @@ def load_library():
         "sti_sync": ([vp], i32),
         "sti_shard_decode": ([vp, i32, i32, i32, i32, vp, vp, vp], i32),
         "sti_gemm_probe": ([vp, i32, i32, vp, i32, vp, C.c_size_t, i32, C.POINTER(C.c_int32)], i32),
+        "sti_decode_rate_probe": ([vp, vp, i32, vp, C.c_size_t, u64p, C.POINTER(C.c_int32)], i32),
         "sti_plan_set_profiling": ([vp, i32], i32),
         "sti_get_kernel_stamps": ([vp, vp, C.c_size_t, C.POINTER(C.c_int32)], i32),
         "sti_plan_set_overlap": ([vp, i32], i32),
@@ -107,7 +108,7 @@ def load_library():
 
 EXPORTED = ("sti_ctx_create", "sti_ctx_destroy", "sti_ctx_set_layer_params", "sti_plan_create",
             "sti_plan_destroy", "sti_shard_upload", "sti_plan_finalize", "sti_layer_forward",
-            "sti_model_forward", "sti_model_forward_host", "sti_sync", "sti_shard_decode", "sti_gemm_probe", "sti_get_kernel_stamps", "sti_plan_inject",
+            "sti_model_forward", "sti_model_forward_host", "sti_sync", "sti_shard_decode", "sti_gemm_probe", "sti_decode_rate_probe", "sti_get_kernel_stamps", "sti_plan_inject",
             "sti_plan_retain", "sti_shard_adopt", "sti_plan_fill_stats",
             "sti_plan_set_profiling", "sti_plan_set_overlap", "sti_get_stats", "sti_plan_memory", "sti_ctx_launch_count",
             "sti_host_retile", "sti_strerror", "sti_matrix_decode_noalloc", "sti_plan_auto",
@@ -224,6 +225,14 @@ def sti_gemm_probe(plan: int, layer: int, gemm: int, x_bf16_dev: int, tokens: in
 def sti_plan_set_profiling(plan: int, level: int):
     """0 = off, 1 = per-layer events, 2 = events around every kernel."""
     _check(load_library().sti_plan_set_profiling(C.c_void_p(plan), int(level)), "sti_plan_set_profiling")
+
+
+def sti_decode_rate_probe(plan: int, x_bf16_dev: int, tokens: int, out_dev: int, out_capacity_bytes: int):
+    """One launch over every layer's FFN1 tiles on few tokens (see sti.h); returns (packed bytes read, tiles)."""
+    nb, nt = C.c_uint64(0), C.c_int32(0)
+    _check(load_library().sti_decode_rate_probe(C.c_void_p(plan), C.c_void_p(x_bf16_dev), tokens, C.c_void_p(out_dev),
+                                                out_capacity_bytes, C.byref(nb), C.byref(nt)), "sti_decode_rate_probe")
+    return int(nb.value), int(nt.value)
 
 
 STI_STAMP_KERNELS, STI_STAMP_WORDS = 8, 8

@@ -145,6 +145,8 @@ struct sti_plan {
   void* x_in = nullptr; void* y_out = nullptr; int32_t* lens_dev = nullptr;
   int max_partial = 1;
   float* zero_bias = nullptr;          // all-zero bias vector of sti_gemm_probe (allocated by its first call)
+  uint8_t* rate_tables = nullptr;      // every layer's FFN1 tile jobs in one table (sti_decode_rate_probe, built by its first call)
+  int rate_jobs = 0; uint32_t rate_seg_stride = 0; uint64_t rate_packed_bytes = 0;
   unsigned long long* stamps = nullptr;   // [layer][kStampKernels][kStampWords] device, profiling level 3
   bool stamping = false;               // the forward being enqueued writes stamps
   bool overlap = true;                 // false: load every streamed layer, then execute (Load&Exec)
@@ -765,6 +767,7 @@ void free_plan_device(sti_plan* p) {
   cudaFree(p->lens_dev);
   cudaFree(p->stamps);
   cudaFree(p->zero_bias);
+  cudaFree(p->rate_tables);
   for (auto& L : p->layers) {
     if (L.ev_loaded) cudaEventDestroy(L.ev_loaded);
     if (L.g_ev_loaded) cudaEventDestroy(L.g_ev_loaded);
@@ -1280,6 +1283,75 @@ sti_status sti_gemm_probe(sti_plan* p, int layer, int gemm, const void* x_bf16_d
   if (st != STI_OK) return st;
   if (L.str_bytes > 0) CUDA_TRY(cudaEventRecord(p->slot_free[L.slot], c->compute));
   if (n_partials) *n_partials = parts[gemm];
+  return STI_OK;
+}
+
+sti_status sti_decode_rate_probe(sti_plan* p, const void* x_bf16_dev, int tokens, void* out_dev, size_t out_capacity_bytes,
+                                 uint64_t* packed_bytes, int32_t* n_tiles) {
+  if (!p || !x_bf16_dev || !out_dev) return STI_ERR_ARG;
+  if (tokens < 1 || tokens > 128) return STI_ERR_SHAPE;
+  if ((reinterpret_cast<uintptr_t>(x_bf16_dev) & 15) || (reinterpret_cast<uintptr_t>(out_dev) & 15)) return STI_ERR_ARG;
+  sti_status st = sti_plan_finalize(p);
+  if (st != STI_OK) return st;
+  sti_ctx* c = p->ctx;
+  const sti_model_desc& d = c->desc;
+  CUDA_TRY(cudaSetDevice(c->device));
+  const int f = d.ffn / d.n_ffn_slices;
+  for (auto& L : p->layers) if (L.str_bytes) return STI_ERR_STATE;       // every shard must sit in device memory
+  if (!p->rate_tables) {
+    // one table with the FFN1 tile jobs of all layers; layer l's tiles write output columns l * ffn + ...
+    std::vector<Job> jobs;
+    std::vector<Seg> segs;
+    uint32_t stride = 0;
+    for (auto& L : p->layers) stride = std::max(stride, L.f1.seg_stride);
+    if (stride == 0) return STI_ERR_STATE;                               // no FFN slice kept anywhere
+    std::vector<Job> hj;
+    std::vector<Seg> hs;
+    uint64_t bytes = 0;
+    for (size_t l = 0; l < p->layers.size(); ++l) {
+      Layer& L = p->layers[l];
+      if (L.f1.n_jobs == 0) continue;
+      hj.resize(L.f1.n_jobs);
+      hs.resize(static_cast<size_t>(L.f1.n_jobs) * L.f1.seg_stride);
+      CUDA_TRY(cudaMemcpy(hj.data(), L.f1.jobs, hj.size() * sizeof(Job), cudaMemcpyDeviceToHost));
+      CUDA_TRY(cudaMemcpy(hs.data(), L.f1.segs, hs.size() * sizeof(Seg), cudaMemcpyDeviceToHost));
+      for (int j = 0; j < L.f1.n_jobs; ++j) {
+        Job job = hj[j];
+        job.seg_begin = static_cast<uint32_t>(jobs.size()) * stride;
+        job.out_col += static_cast<uint32_t>(l) * d.ffn;
+        job.bias_off = -1;
+        jobs.push_back(job);
+        for (uint32_t k = 0; k < stride; ++k) segs.push_back(k < job.n_seg ? hs[static_cast<size_t>(j) * L.f1.seg_stride + k] : Seg{});
+      }
+      for (int sl : L.kept_slices) {
+        const int bits = L.ffn[sl].cfg.bits;
+        bytes += static_cast<uint64_t>(f) * d.hidden * bits / 8 + (bits == 32 ? 0 : (4ull << bits));
+      }
+    }
+    const size_t jb = align16(jobs.size() * sizeof(Job)), sb = segs.size() * sizeof(Seg);
+    CUDA_TRY(cudaMalloc(&p->rate_tables, jb + sb));
+    CUDA_TRY(cudaMemcpy(p->rate_tables, jobs.data(), jobs.size() * sizeof(Job), cudaMemcpyHostToDevice));
+    CUDA_TRY(cudaMemcpy(p->rate_tables + jb, segs.data(), sb, cudaMemcpyHostToDevice));
+    p->rate_jobs = static_cast<int>(jobs.size());
+    p->rate_seg_stride = stride;
+    p->rate_packed_bytes = bytes;
+  }
+  const int ldo = static_cast<int>(p->layers.size()) * d.ffn;
+  if (out_capacity_bytes < static_cast<size_t>(tokens) * ldo * 2) return STI_ERR_SIZE;
+  const GemmTable& ref = p->layers[0].f1.n_jobs ? p->layers[0].f1 : p->layers.back().f1;
+  GemmTable tab = ref;                                                   // same tile shape, ring and shared memory
+  tab.jobs = reinterpret_cast<Job*>(p->rate_tables);
+  tab.segs = reinterpret_cast<Seg*>(p->rate_tables + align16(static_cast<size_t>(p->rate_jobs) * sizeof(Job)));
+  tab.n_jobs = p->rate_jobs;
+  tab.seg_stride = p->rate_seg_stride;
+  tab.pair_ok = false;
+  for (auto& L : p->layers) {                                            // the widest tile decides the shared-memory shape
+    if (L.f1.n_jobs && L.f1.smem > tab.smem) { tab.smem = L.f1.smem; tab.w_bytes = L.f1.w_bytes; tab.n_stages = L.f1.n_stages; tab.bps = L.f1.bps; }
+  }
+  st = run_gemm(p, GEMM_BF16_TO_BF16, tab, x_bf16_dev, d.hidden, tokens, out_dev, ldo, nullptr, -1, 0);
+  if (st != STI_OK) return st;
+  if (packed_bytes) *packed_bytes = p->rate_packed_bytes;
+  if (n_tiles) *n_tiles = p->rate_jobs;
   return STI_OK;
 }
 
