@@ -4,8 +4,8 @@
  * The library executes a plan that the caller supplies: for every layer, which shard units
  * are kept, at which bitwidth each is stored, and whether it sits in the preload buffer or is
  * streamed while earlier layers compute.  Choosing the plan (the paper's two-stage planner,
- * Section 5) is the caller's business; the paper's engine likewise "simply loads and executes
- * the shards that have been selected in planning" (Section 3.2).
+ * Section 5) is the caller's business; the paper's engine likewise only loads and runs the
+ * shards its planning stage picked (Section 3.2).
  *
  * Vocabulary (Section 4.2, Table 1).  A layer with hidden size d, M heads of width 64 and
  * d_ff FFN neurons is cut into vertical slices.  Here the attention part and the FFN part of a
@@ -118,7 +118,7 @@ typedef struct {
  * `compute_stream` is a cudaStream_t to borrow, or NULL to create one. */
 sti_status sti_ctx_create(const sti_model_desc* desc, int device, void* compute_stream, sti_ctx** out);
 
-/* Section 6 ("layer normalization and biases ... kept in memory in full fidelity").
+/* Section 6: biases and LayerNorm parameters are not quantized; they stay in memory as fp32.
  * Host arrays, copied before return: bq,bk,bv [n_heads*64]; bo [d]; b1 [ffn]; b2 [d];
  * ln1_g, ln1_b, ln2_g, ln2_b [d]. */
 sti_status sti_ctx_set_layer_params(sti_ctx* ctx, int layer,
@@ -133,7 +133,7 @@ sti_status sti_ctx_set_layer_params(sti_ctx* ctx, int layer,
 sti_status sti_plan_create(sti_ctx* ctx, const sti_shard_cfg* attn, const sti_shard_cfg* ffn,
                            int ring_slots, sti_plan** out);
 
-/* Section 4.2 "storing shards per version": hands one unit's blob to the plan.  Host pointers
+/* Section 4.2 (each shard is stored once per fidelity version): hands one unit's blob to the plan.  Host pointers
  * are only read during the call.  The blob's bits must equal the plan's.  Not allowed after
  * the plan has been finalized. */
 sti_status sti_shard_upload(sti_plan* plan, int layer, sti_kind kind, int index, const sti_shard_blob* blob);
@@ -165,8 +165,8 @@ sti_status sti_model_forward_host(sti_plan* plan, const void* x_host, void* y_ho
 /* Waits for everything enqueued on the context; returns the first asynchronous error. */
 sti_status sti_sync(sti_ctx* ctx);
 
-/* Section 4.2 (decompression "substitut[es] dictionary indexes with floating point centroids
- * and outliers"): decodes one matrix of an uploaded unit for inspection.  matrix: 0..3 = Q,K,V,O
+/* Section 4.2 (decompression replaces every index by its centroid and then writes the outliers
+ * over their positions): decodes one matrix of an uploaded unit for inspection.  matrix: 0..3 = Q,K,V,O
  * or 0..1 = F1,F2.  Any of the outputs may be NULL: w_dev fp32 [rows*cols] exact table values
  * with outliers patched, codes_dev one byte per index, wbf16_dev the bf16 (round-to-nearest-
  * even) operand values the GEMMs use.  Device pointers, caller-owned.  Asynchronous. */
@@ -230,14 +230,14 @@ sti_status sti_get_stats(sti_plan* plan, sti_stats* out);
 #define STI_STAMP_WORDS 8
 sti_status sti_get_kernel_stamps(sti_plan* plan, uint64_t* out, size_t capacity_words, int32_t* n_layers);
 
-/* Section 7.1 (the Load&Exec baseline "loads model as a whole and executes it"): with overlap = 0 a model
+/* Section 7.1 (the Load&Exec baseline: the whole model is loaded first, then executed): with overlap = 0 a model
  * forward first copies every streamed layer into its ring slot and only then starts layer 0, so IO and
  * compute delays add up; overlap = 1 (the default) is the layerwise pipeline of Section 3.1.  Results are
  * identical.  overlap = 0 needs one ring slot per streamed layer (STI_ERR_STATE otherwise: a slot could
  * only be reused after a layer that has not started).  Takes effect at the next forward. */
 sti_status sti_plan_set_overlap(sti_plan* plan, int overlap);
 
-/* Section 3.2 ("back-to-back executions": shards a run loaded stay cached, and the next plan spends the freed IO time
+/* Section 3.2 (executions that follow one another: shards a run loaded stay cached, and the next plan spends the freed IO time
  * on the others) and Section 5.5 (after a run, loaded shards are evicted from the top layer down until the rest fits
  * the preload buffer).  Which shards stay is the planner's decision (sti_preload_after_run); these calls keep them in
  * DEVICE memory across plans, so that the next plan uploads nothing it already holds.

@@ -1,8 +1,8 @@
 /*
- * sti_quantize.h - the shard quantizer of STI (arXiv 2207.05022, Section 6 "Gaussian outlier-aware
- * quantization"; Section 4.2 "each shard is stored in K fidelity versions") on the device.
+ * sti_quantize.h - the shard quantizer of STI (arXiv 2207.05022: the outlier-aware quantization of
+ * Section 6, which produces the K fidelity versions Section 4.2 stores per shard) on the device.
  *
- * The paper runs this step offline in the cloud (Python + scikit-learn, "a few minutes per bitwidth");
+ * The paper runs this step offline in the cloud (Python + scikit-learn, minutes per bitwidth);
  * here one call turns fp32 shard units that already sit in device memory into the upload format of
  * sti_shard_upload (sti.h), so that the N x M x K shard versions of a model can be produced where the
  * weights are.  Per unit, on its flat fp32 array of n_weights values:

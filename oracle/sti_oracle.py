@@ -10,16 +10,16 @@ passage states.
 
 What each function follows:
 
-* `unpack_codes`   - Section 4.2 ("k-bit indexes pointing to centroids", the
-  weight matrix "stores K-bit indexes").  The paper does not fix the bit order;
+* `unpack_codes`   - Section 4.2 (a shard's weight matrix holds k-bit indexes
+  into its centroid dictionary).  The paper does not fix the bit order;
   the stream format is the upload format of the library: index i of a matrix
   occupies stream bits [i*k, i*k+k), least-significant bit first, in
   little-endian 32-bit words.
-* `dequantize`     - Section 4.2 (decompression substitutes "dictionary indexes
-  with floating point centroids and outliers") and Section 6 (outliers keep
+* `dequantize`     - Section 4.2 (decompression replaces each index by its
+  centroid, then outliers overwrite their positions) and Section 6 (outliers keep
   their original weights and offsets in the shard).
 * `decode_unit`    - Table 1 (matrix shapes of a vertical slice) and
-  Section 4.2 "storing shards per version".
+  Section 4.2 (one stored copy of a shard per fidelity version).
 * `layer_forward`  - Section 2.1 (MHA over heads backed by Q, K, V, output
   layer O, two FFN layers), Section 4.2 (any subset of shards executes; a
   shard is one head plus 1/M of the FFN neurons), Section 6 (biases and

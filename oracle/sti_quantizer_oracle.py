@@ -1,13 +1,13 @@
 """CPU oracle of the shard quantizer (test infrastructure: only tests, the smoke check and the benchmark's
 CPU baseline may import it; it shares no code with the CUDA path).
 
-Section 6 of the paper ("Gaussian outlier-aware quantization", following GOBO), step by step, in fp64:
+Section 6 of the paper (its outlier-aware quantization with one Gaussian, after GOBO), step by step, in fp64:
   1. fit one Gaussian component to the flat weight array (maximum likelihood: mean and 1/n variance);
   2. a weight whose log-likelihood under that Gaussian is below -4 is an outlier, kept verbatim with its offset;
   3. the other weights are sorted (ties in original order) and cut into 2^k clusters of equal population,
      cluster c = sorted[floor(c n'/2^k) : floor((c+1) n'/2^k));
   4. the arithmetic mean of a cluster is its centroid (fp32); every member gets the cluster's k-bit index;
-  5. an outlier's slot also holds a k-bit index (Section 6: "represent outliers also as k-bit integers"):
+  5. an outlier's slot also holds a k-bit index (Section 6: outliers, too, are represented as k-bit integers in the matrix):
      the nearest centroid, the lower index on a tie (reading: the paper does not say which);
   6. the indexes are written as a bit stream, index i at bits [i k, i k + k), least-significant bit first,
      in little-endian 32-bit words (Section 4.2 gives sizes only; this is the library's upload format).

@@ -1,6 +1,8 @@
-// Stand-alone shard decompression (Section 4.2: "substituting dictionary indexes with floating
-// point centroids and outliers"), used for inspection and for checking the fused path's unpack:
-// it reads the same re-tiled index stream with the same extraction routine as the GEMM.
+// Stand-alone shard decompression (Section 4.2: every k-bit index is replaced by its centroid, and the
+// outlier list then overwrites its positions), used for inspection and parity checks.  It reads the same
+// re-tiled plane layout as the GEMM (one quantum of 128 indexes per lane) but extracts each index by its
+// bit offset (extract_index); the GEMM's own plane-wise unpack is a separate routine (gemm_device.cuh),
+// checked bit for bit through sti_gemm_probe.
 #include <cuda_bf16.h>
 
 #include "sti_device.cuh"
