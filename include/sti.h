@@ -189,7 +189,10 @@ sti_status sti_shard_decode(sti_plan* plan, int layer, sti_kind kind, int index,
  *                         units, each group writes its own partial sum (the caller adds them up)
  *   out_capacity_bytes : size of out_dev; STI_ERR_SIZE when the result would not fit
  *   variant    : 0 = the kernel a forward would choose for this token count, 1 = the one-CTA kernel,
- *                2 = the two-CTA (cta_group::2) kernel, STI_ERR_STATE when the tiling does not allow it
+ *                2 = the two-CTA (cta_group::2) kernel, STI_ERR_STATE when the tiling does not allow it,
+ *                3 = (gemm 3 only) the K-accumulating two-CTA kernel that forwards of many tokens use for FFN2:
+ *                all K groups summed in tensor memory, ONE complete plane written (n_partials = 1);
+ *                STI_ERR_STATE when the plan was not made for that many tokens
  *   n_partials : optional out
  * STI_ERR_STATE when no kept unit feeds the GEMM.  A streamed layer is copied first.  Asynchronous. */
 sti_status sti_gemm_probe(sti_plan* plan, int layer, int gemm, const void* x_bf16_dev, int tokens, void* out_dev,

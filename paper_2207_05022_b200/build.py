@@ -10,7 +10,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB_NAME = "libsti_b200.so"
 LIB_PATH = os.path.join(HERE, LIB_NAME)
-SOURCES = ["api.cu", "dqgemm.cu", "attention.cu", "attention_tc.cu", "layernorm.cu", "decode.cu", "noalloc.cu", "planner.cu", "quantize.cu"]
+SOURCES = ["api.cu", "dqgemm.cu", "dqgemm_kacc.cu", "attention.cu", "attention_tc.cu", "layernorm.cu", "decode.cu", "noalloc.cu", "planner.cu", "quantize.cu"]
 HEADERS = ["sti_kernels.h", "sti_device.cuh", "gemm_device.cuh", "retile.h", os.path.join("..", "..", "include", "sti.h"),
            os.path.join("..", "..", "include", "sti_planner.h"),
            os.path.join("..", "..", "include", "sti_quantize.h")]

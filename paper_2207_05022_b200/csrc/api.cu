@@ -35,8 +35,9 @@ struct MatrixInfo {
 
 struct Tuning {
   int qkv_n = 32, f1_n = 64, o_n = 64, o_group = 4, f2_n = 64, f2_group = 2;
-  int cta_budget = 148;                // CTAs a GEMM launch may use when it splits the token tiles over CTAs
+  int cta_budget = 148;                // (replaced by the device's SM count in parse_tuning) CTAs a GEMM launch may use when it splits the token tiles over CTAs
   int pair_min_tiles = 8;              // two-CTA GEMM from this many 128-token tiles on (0 = never)
+  int f2_kacc_min_tokens = 8192;       // FFN2 through the K-accumulating kernel (one output plane) from this many tokens on (0 = never)
   int attn_tc_min_items = 96;          // tensor-core attention from this many (sequence, kept head) pairs on, seq >= 256 (0 = never)
   int ln1_ctas = -1, ln2_ctas = -1;    // LayerNorm CTA counts: -1 = chosen per launch (see ln_ctas_hint), 0 = one row per CTA
 };
@@ -78,6 +79,7 @@ struct Layer {
   int slot = -1;                       // ring slot of the streamed part
   size_t tables_off = 0, tables_bytes = 0;   // this layer's tile-job descriptors inside the plan's table buffer
   GemmTable qkv, o, f1, f2;
+  GemmTable f2k;                       // FFN2 again, cut for the K-accumulating kernel (plans made for many tokens only)
   cudaEvent_t ev_loaded = nullptr, ev_done = nullptr, ev_copy_start = nullptr, ev_comp_start = nullptr;
   cudaEvent_t g_ev_loaded = nullptr;   // the same role inside graph capture (captured events cannot be reused outside)
   cudaEvent_t ev_k[8] = {};           // boundaries of the seven kernels (kernel-level profiling)
@@ -213,6 +215,7 @@ void parse_tuning(Tuning* t, int tmax, const sti_model_desc& d, int sm_count) {
         else if (k == "f2_n") t->f2_n = v;
         else if (k == "f2_group") t->f2_group = v;
         else if (k == "pair_min_tiles") t->pair_min_tiles = v;
+        else if (k == "f2_kacc_min_tokens") t->f2_kacc_min_tokens = std::max(0, v);
         else if (k == "attn_tc_min_items") t->attn_tc_min_items = std::max(0, v);
         else if (k == "cta_budget") t->cta_budget = std::max(1, v);
         else if (k == "ln1_ctas") t->ln1_ctas = std::max(-1, v);
@@ -297,7 +300,7 @@ struct TableBuilder {
   }
 };
 
-void build_layer_tables(sti_plan* p, Layer& L, TableBuilder tb[4]) {
+void build_layer_tables(sti_plan* p, Layer& L, TableBuilder tb[5]) {
   const sti_ctx* c = p->ctx;
   const sti_model_desc& d = c->desc;
   const Tuning& t = p->tune;
@@ -353,6 +356,25 @@ void build_layer_tables(sti_plan* p, Layer& L, TableBuilder tb[4]) {
       for (int i = 0; i < cnt; ++i)
         ss.push_back(make_seg(c, L.ffn[L.kept_slices[first + i]], STI_FFN, 1, n0, t.f2_n, i * f));
       tb[3].add(j, ss);
+    }
+  }
+  // FFN2 for the K-accumulating kernel: 64-row tiles, K groups of at most 512 columns, group-major order
+  const int kacc_group = f <= 512 && 512 % f == 0 ? static_cast<int>(512 / f) : 0;
+  L.f2k.n_split = 0;
+  if (kacc_group > 0 && ns > 0 && d.hidden % 128 == 0 && t.f2_kacc_min_tokens > 0 &&
+      static_cast<long long>(d.max_batch) * d.max_seq >= t.f2_kacc_min_tokens) {
+    L.f2k.n_split = (ns + kacc_group - 1) / kacc_group;
+    for (int sp = 0; sp < L.f2k.n_split; ++sp) {
+      const int first = sp * kacc_group, cnt = std::min(kacc_group, ns - first);
+      for (uint32_t n0 = 0; n0 < static_cast<uint32_t>(d.hidden); n0 += 64) {
+        Job j{};
+        j.n_rows = 64; j.k_total = cnt * f; j.x_koff = first * f;
+        j.out_mat = 0; j.out_col = n0; j.bias_off = -1;
+        std::vector<Seg> ss;
+        for (int i = 0; i < cnt; ++i)
+          ss.push_back(make_seg(c, L.ffn[L.kept_slices[first + i]], STI_FFN, 1, n0, 64, i * f));
+        tb[4].add(j, ss);
+      }
     }
   }
 }
@@ -446,10 +468,27 @@ sti_status run_gemm(sti_plan* p, GemmKind kind, const GemmTable& tab, const void
   return STI_OK;
 }
 
+// FFN2 through the K-accumulating kernel: one complete fp32 plane [T][ldo] instead of one plane per K group.
+sti_status run_gemm_kacc(sti_plan* p, const GemmTable& tab, const void* x, int ldx, int T, float* out, int ldo,
+                         unsigned long long* stamps) {
+  if (tab.n_jobs == 0 || tab.n_split == 0) return STI_ERR_STATE;
+  KaccLaunch g{};
+  g.jobs = tab.jobs; g.segs = tab.segs; g.n_groups = tab.n_split; g.n_cols64 = tab.n_jobs / tab.n_split;
+  const int n_mpairs = ((T + 127) / 128 + 1) / 2;
+  g.m_ctas = std::max(1, std::min(n_mpairs, p->tune.cta_budget / g.n_cols64));
+  if (!make_xmap(&g.xmap, x, ldx, T)) return STI_ERR_CUDA;
+  g.T = T; g.out = out; g.ldo = ldo; g.err = p->ctx->err_dev;
+  g.n_stages = tab.n_stages; g.hdr_bytes = tab.hdr_bytes; g.seg_stride = tab.seg_stride;
+  g.pdl = p->ctx->pdl; g.stamps = stamps;
+  CUDA_TRY(launch_gemm_kacc(g, p->ctx->compute));
+  p->ctx->launches++;
+  return STI_OK;
+}
+
 // How many CTAs a LayerNorm launch should use, given the GEMM that follows it.  A GEMM CTA needs a whole SM and its
 // CTAs are launched while the LayerNorm runs (they decode their weights meanwhile) - on SMs that hold no LayerNorm
 // CTA.  With one row per CTA the LayerNorm of a few hundred tokens spreads over about 64 SMs; when the next GEMM
-// wants more than the SMs it leaves free (84 of 148), its last CTAs start late and their decode lands on the critical path.  Then the
+// wants more than the SMs it leaves free (84 of a B200's 148), its last CTAs start late and their decode lands on the critical path.  Then the
 // rows are packed into fewer CTAs (measured: 54.6 -> 50.5 us per BERT-large layer at 256 tokens; at 512 tokens
 // packing loses 1-3 us, at BERT-base sizes it changes nothing).  Otherwise one row per CTA.
 int ln_ctas_hint(int tuned, int T, int next_gemm_ctas, int sm_count) {
@@ -499,7 +538,7 @@ sti_status enqueue_layer(sti_plan* p, int li, const void* x, void* y, int batch,
       if (!make_xmap(&qmap, p->qkv, 64, 3 * nh * T)) return STI_ERR_CUDA;
       CUDA_TRY(launch_attention_tc(qmap, p->attn_out, nh, batch, seq, lens, c->err_dev, c->compute, c->pdl, stamp(2)));
     } else {
-      CUDA_TRY(launch_attention(p->qkv, p->attn_out, nh, batch, seq, lens, c->compute, c->pdl, stamp(2)));
+      CUDA_TRY(launch_attention(p->qkv, p->attn_out, nh, batch, seq, lens, c->sm_count, c->compute, c->pdl, stamp(2)));
     }
     c->launches++;
     CUDA_TRY(mark(2));
@@ -524,11 +563,16 @@ sti_status enqueue_layer(sti_plan* p, int li, const void* x, void* y, int batch,
     L.k_ran[3] = true;
   }
   CUDA_TRY(mark(4));
+  bool f2_kacc = false;
   if (ns > 0) {
     st = run_gemm(p, GEMM_BF16_TO_BF16_GELU, L.f1, p->h1_bf16, d.hidden, T, p->u, ns * f, dense + c->off_b1, -1, -1, stamp(5));
     if (st != STI_OK) return st;
     CUDA_TRY(mark(5));
-    st = run_gemm(p, GEMM_BF16_TO_F32, L.f2, p->u, ns * f, T, p->partial, d.hidden, nullptr, -1, -1, stamp(6));
+    f2_kacc = L.f2k.n_jobs > 0 && T >= p->tune.f2_kacc_min_tokens && !c->simt_debug;
+    if (f2_kacc)
+      st = run_gemm_kacc(p, L.f2k, p->u, ns * f, T, p->partial, d.hidden, stamp(6));
+    else
+      st = run_gemm(p, GEMM_BF16_TO_F32, L.f2, p->u, ns * f, T, p->partial, d.hidden, nullptr, -1, -1, stamp(6));
     if (st != STI_OK) return st;
     L.k_ran[4] = L.k_ran[5] = true;
   } else {
@@ -536,7 +580,7 @@ sti_status enqueue_layer(sti_plan* p, int li, const void* x, void* y, int batch,
   }
   CUDA_TRY(mark(6));
   LnLaunch l2{};
-  l2.partial = p->partial; l2.n_partial = ns > 0 ? L.f2.n_split : 0;
+  l2.partial = p->partial; l2.n_partial = ns > 0 ? (f2_kacc ? 1 : L.f2.n_split) : 0;
   l2.bias = dense + c->off_b2; l2.resid = p->h1_f32; l2.resid_bf16 = 0;
   l2.gamma = dense + c->off_ln2g; l2.beta = dense + c->off_ln2b; l2.eps = d.ln_eps; l2.T = T; l2.d = d.hidden;
   l2.out_f32 = bf16_act ? nullptr : static_cast<float*>(y);
@@ -860,7 +904,8 @@ sti_status sti_ctx_create(const sti_model_desc* desc, int device, void* compute_
   if (cudaMemset(c->dense, 0, c->dense_stride * d.n_layers * sizeof(float)) != cudaSuccess) return fail(STI_ERR_CUDA);
   if (cudaMalloc(&c->err_dev, sizeof(int)) != cudaSuccess) return fail(STI_ERR_OOM);
   if (cudaMemset(c->err_dev, 0, sizeof(int)) != cudaSuccess) return fail(STI_ERR_CUDA);
-  if (gemm_configure() != cudaSuccess || attention_configure() != cudaSuccess || attention_tc_configure() != cudaSuccess)
+  if (gemm_configure() != cudaSuccess || gemm_kacc_configure() != cudaSuccess || attention_configure() != cudaSuccess ||
+      attention_tc_configure() != cudaSuccess)
     return fail(STI_ERR_CUDA);
   if (cudaDeviceGetAttribute(&c->sm_count, cudaDevAttrMultiProcessorCount, device) != cudaSuccess || c->sm_count < 1)
     return fail(STI_ERR_CUDA);
@@ -1076,11 +1121,11 @@ sti_status sti_plan_finalize(sti_plan* p) {
   std::vector<Fix> fixes;
   p->max_partial = 1;
   for (auto& L : p->layers) {
-    TableBuilder tb[4];
+    TableBuilder tb[5];
     L.tables_off = align16(host_tables.size());
     build_layer_tables(p, L, tb);
-    GemmTable* gt[4] = {&L.qkv, &L.o, &L.f1, &L.f2};
-    for (int i = 0; i < 4; ++i) {
+    GemmTable* gt[5] = {&L.qkv, &L.o, &L.f1, &L.f2, &L.f2k};
+    for (int i = 0; i < 5; ++i) {
       tb[i].finish();
       gt[i]->seg_stride = tb[i].seg_stride;
       gt[i]->n_jobs = static_cast<int>(tb[i].jobs.size());
@@ -1092,10 +1137,16 @@ sti_status sti_plan_finalize(sti_plan* p) {
         const Job &a = tb[i].jobs[j], &b = tb[i].jobs[j + 1];
         gt[i]->pair_ok = a.n_rows == 64 && b.n_rows == 64 && a.k_total == b.k_total && a.x_koff == b.x_koff;
       }
+      if (i == 4) {                 // two weight buffers, the rest of the shared memory is the ring of single boxes
+        gt[i]->n_stages = 6; gt[i]->bps = 1;
+        gt[i]->smem = gemm_kacc_smem_bytes(gt[i]->hdr_bytes, gt[i]->n_stages);
+        if (gt[i]->smem > kMaxSmem) return STI_ERR_SHAPE;
+      } else {
       if (!tb[i].jobs.empty() &&
           !gemm_pick_ring(tb[i].w_bytes, tb[i].k_max, gt[i]->hdr_bytes, &gt[i]->n_stages, &gt[i]->bps))
         return STI_ERR_SHAPE;
       gt[i]->smem = gemm_smem_bytes(tb[i].w_bytes, gt[i]->n_stages, gt[i]->bps, gt[i]->hdr_bytes);
+      }
       if (gt[i]->smem > kMaxSmem && !tb[i].jobs.empty()) return STI_ERR_SHAPE;
       Fix fx{gt[i], 0, 0};
       fx.jobs_off = align16(host_tables.size());
@@ -1246,7 +1297,8 @@ sti_status sti_shard_decode(sti_plan* p, int layer, sti_kind kind, int index, in
 
 sti_status sti_gemm_probe(sti_plan* p, int layer, int gemm, const void* x_bf16_dev, int tokens, void* out_dev,
                           size_t out_capacity_bytes, int variant, int32_t* n_partials) {
-  if (!p || !x_bf16_dev || !out_dev || gemm < 0 || gemm > 3 || variant < 0 || variant > 2) return STI_ERR_ARG;
+  if (!p || !x_bf16_dev || !out_dev || gemm < 0 || gemm > 3 || variant < 0 || variant > 3) return STI_ERR_ARG;
+  if (variant == 3 && gemm != 3) return STI_ERR_ARG;       // the K-accumulating kernel exists for FFN2 only
   if (layer < 0 || layer >= static_cast<int>(p->layers.size())) return STI_ERR_ARG;
   if (tokens < 1 || tokens > 65536) return STI_ERR_SHAPE;
   if ((reinterpret_cast<uintptr_t>(x_bf16_dev) & 15) || (reinterpret_cast<uintptr_t>(out_dev) & 15)) return STI_ERR_ARG;
@@ -1263,7 +1315,8 @@ sti_status sti_gemm_probe(sti_plan* p, int layer, int gemm, const void* x_bf16_d
   if (tab.n_jobs == 0) return STI_ERR_STATE;               // no kept unit feeds this GEMM
   const int ldx[4] = {d.hidden, nh * 64, d.hidden, ns * f};
   const int ldo[4] = {64, d.hidden, ns * f, d.hidden};
-  const int parts[4] = {1, tabs[1]->n_split, 1, tabs[3]->n_split};
+  const int parts[4] = {1, tabs[1]->n_split, 1, variant == 3 ? 1 : tabs[3]->n_split};
+  if (variant == 3 && L.f2k.n_jobs == 0) return STI_ERR_STATE;   // the plan was not made for many tokens
   const size_t out_elems[4] = {static_cast<size_t>(3) * nh * tokens * 64, static_cast<size_t>(parts[1]) * tokens * d.hidden,
                                static_cast<size_t>(tokens) * ns * f, static_cast<size_t>(parts[3]) * tokens * d.hidden};
   const size_t need = out_elems[gemm] * ((gemm == 1 || gemm == 3) ? 4 : 2);
@@ -1278,6 +1331,9 @@ sti_status sti_gemm_probe(sti_plan* p, int layer, int gemm, const void* x_bf16_d
     if ((st = enqueue_layer_copy(p, layer, c->compute)) != STI_OK) return st;
   }
   const GemmKind kind = (gemm == 1 || gemm == 3) ? GEMM_BF16_TO_F32 : GEMM_BF16_TO_BF16;
+  if (variant == 3)
+    st = run_gemm_kacc(p, L.f2k, x_bf16_dev, ldx[3], tokens, static_cast<float*>(out_dev), ldo[3], nullptr);
+  else
   st = run_gemm(p, kind, tab, x_bf16_dev, ldx[gemm], tokens, out_dev, ldo[gemm], p->zero_bias, -1,
                 variant == 0 ? -1 : variant - 1);
   if (st != STI_OK) return st;

@@ -210,17 +210,18 @@ cudaError_t attention_configure() {
 }
 
 cudaError_t launch_attention(const uint16_t* qkv, uint16_t* out, int n_kept, int batch, int seq,
-                             const int32_t* seq_lens, cudaStream_t s, bool pdl, unsigned long long* stamps) {
+                             const int32_t* seq_lens, int sm_count, cudaStream_t s, bool pdl,
+                             unsigned long long* stamps) {
   if (n_kept <= 0) return cudaSuccess;
   // 128-query CTAs when there are enough of them to fill the GPU (fewer K/V re-reads per head), 64 otherwise
   const long ctas128 = static_cast<long>((seq + 127) / 128) * n_kept * batch;
-  if (seq >= 128 && ctas128 >= 148) {
+  if (seq >= 128 && ctas128 >= sm_count) {
     dim3 grid((seq + 127) / 128, n_kept, batch);
     return launch_kernel(attention_kernel<8>, grid, dim3(256), attn_smem_bytes(seq), s, pdl, qkv, out, n_kept, batch,
                          seq, seq_lens, stamps);
   }
   const long items = static_cast<long>((seq + 63) / 64) * n_kept * batch;
-  if (items <= 2 * 148 && seq > 64) {          // too few CTAs to fill the GPU: shorten each CTA's key loop instead
+  if (items <= 2 * sm_count && seq > 64) {          // too few CTAs to fill the GPU: shorten each CTA's key loop instead
     AttnArgs a{qkv, out, seq_lens, n_kept, batch, seq, batch * seq, stamps};
     return launch_kernel(attention_split_kernel, dim3(static_cast<unsigned>(items)), dim3(kAttnThreads),
                          attn_split_smem_bytes(seq), s, pdl, a);

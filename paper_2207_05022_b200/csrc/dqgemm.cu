@@ -360,47 +360,6 @@ dqgemm_kernel(const __grid_constant__ CUtensorMap xmap, const Job* __restrict__ 
 // CTAs; both CTAs' TMA loads report to CTA 0's `full` barriers; each CTA drains its own accumulator rows
 // (its 128 tokens x all 128 features) and reports to CTA 0's `acc_empty`.
 // ---------------------------------------------------------------------------------------
-__device__ __forceinline__ void tmem_alloc_pair(uint32_t smem_dst, uint32_t n_cols) {     // one warp in each CTA
-  asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_dst), "r"(n_cols)
-               : "memory");
-}
-__device__ __forceinline__ void tmem_relinquish_pair() {
-  asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
-}
-__device__ __forceinline__ void tmem_dealloc_pair(uint32_t taddr, uint32_t n_cols) {
-  asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(n_cols) : "memory");
-}
-// Own tile into own shared memory, completion bytes credited to the barrier at `bar_cluster_addr` (CTA 0's).
-__device__ __forceinline__ void tma_load_2d_pair(uint32_t dst, const CUtensorMap* map, int k0, int m0,
-                                                 uint32_t bar_cluster_addr) {
-  asm volatile(
-      "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
-      ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(k0), "r"(m0), "r"(bar_cluster_addr)
-      : "memory");
-}
-__device__ __forceinline__ void umma_bf16_ss_x4_pair(uint32_t tmem_d, uint64_t desc_a, uint64_t desc_b, uint32_t a_step,
-                                                     uint32_t b_step, uint32_t idesc, uint32_t accumulate_first) {
-  asm volatile(
-      "{\n\t.reg .pred p0, p1;\n\t.reg .b64 a1, a2, a3, b1, b2, b3, as, bs;\n\t"
-      "setp.ne.b32 p0, %6, 0;\n\t"
-      "setp.eq.b32 p1, 0, 0;\n\t"
-      "cvt.u64.u32 as, %3;\n\t"
-      "cvt.u64.u32 bs, %4;\n\t"
-      "add.u64 a1, %1, as;\n\tadd.u64 a2, a1, as;\n\tadd.u64 a3, a2, as;\n\t"
-      "add.u64 b1, %2, bs;\n\tadd.u64 b2, b1, bs;\n\tadd.u64 b3, b2, bs;\n\t"
-      "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %5, p0;\n\t"
-      "tcgen05.mma.cta_group::2.kind::f16 [%0], a1, b1, %5, p1;\n\t"
-      "tcgen05.mma.cta_group::2.kind::f16 [%0], a2, b2, %5, p1;\n\t"
-      "tcgen05.mma.cta_group::2.kind::f16 [%0], a3, b3, %5, p1;\n\t}"
-      ::"r"(tmem_d), "l"(desc_a), "l"(desc_b), "r"(a_step), "r"(b_step), "r"(idesc), "r"(accumulate_first)
-      : "memory");
-}
-// Completion of all MMAs issued so far -> the barrier at this offset in both CTAs.
-__device__ __forceinline__ void umma_commit_pair(uint32_t bar) {
-  asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
-               ::"r"(bar), "h"(static_cast<uint16_t>(3)) : "memory");
-}
-
 template <typename OutT, bool GELU>
 __global__ void __launch_bounds__(kThreads, 1)
 dqgemm_pair_kernel(const __grid_constant__ CUtensorMap xmap, const Job* __restrict__ jobs, const Seg* __restrict__ segs,

@@ -1,0 +1,313 @@
+// K-accumulating form of the fused dequant-GEMM for many tokens (FFN2: out = u F2^T, K = all kept FFN neurons).
+//
+// The ordinary kernels keep one decoded weight tile per CTA, so a GEMM whose K does not fit one tile is cut into
+// K groups that each write their own fp32 plane of partial sums, which the LayerNorm kernel then adds up.  With
+// thousands of tokens those planes are most of the traffic of the layer's second half.  Here a pair of CTAs
+// (cta_group::2, M = 256 tokens, N = 128 features) keeps the accumulators of up to four token-tile pairs in tensor
+// memory (4 x 128 columns = all of it) and walks ALL K groups over them, so the result is written once, complete.
+// The price is that the pair's weight tile changes with every K group: the tiles are small (64 rows x <= 512
+// columns, 64 KB), two of them sit in shared memory, and eight warps decode K group g + 1 (Section 4.2
+// decompression, the same routine as everywhere) while the tensor core works on K group g.  The same eight
+// warps drain the accumulators at the end of a block of token tiles.
+//
+//   warp 0     TMA producer: activation boxes [128 tokens x 64] of (block, K group, tile, box) into a ring
+//   warp 1     MMA issuer (CTA 0 of the pair): tcgen05.mma.cta_group::2, commits free ring stages / weight buffers
+//   warps 4-11 decode weight tiles into the two buffers; epilogue (tcgen05.ld -> fp32 rows in global memory)
+//
+// Every wait is bounded; a role that gives up raises the CTA's abort flag, the others stop waiting but keep
+// walking their loops (the decode group meets at named barriers), and the status word reports the timeout.
+#include "gemm_device.cuh"
+
+namespace sti {
+namespace {
+
+constexpr uint32_t kKaccTiles = 4;                    // token-tile pairs whose accumulators are live at once
+constexpr uint32_t kKaccAccCols = 128;                // columns of one accumulator (N of the pair's MMA)
+constexpr uint32_t kKaccTmemCols = kKaccTiles * kKaccAccCols;
+constexpr uint32_t kKaccWBytes = 64 * 512 * 2;        // one weight buffer: 64 rows x 512 columns of bf16
+constexpr uint32_t kKaccKMax = 512;
+constexpr int kKaccGroupWarp0 = 4, kKaccGroupWarps = 8;
+constexpr uint32_t kKaccGroupBarrier = 1;
+
+struct KaccHeader {
+  uint64_t full[kMaxStages];     // CTA 0: both CTAs' activation boxes of the stage have landed
+  uint64_t empty[kMaxStages];    // both CTAs: the MMAs that read the stage have completed
+  uint64_t w_full[2];            // CTA 0: both CTAs' halves of the weight tile in this buffer are decoded (2 arrivals)
+  uint64_t w_empty[2];           // both CTAs: the MMAs that read the buffer have completed
+  uint64_t acc_full;             // both CTAs: the block's accumulators are complete
+  uint64_t acc_empty;            // CTA 0: both CTAs' epilogue warps have read them (2 x 8 arrivals)
+  uint64_t drain;                // failure path only
+  uint32_t tmem_base;
+  volatile uint32_t abort;
+};
+static_assert(sizeof(KaccHeader) <= 256, "barriers must fit the first 256 bytes of the header");
+
+__device__ __forceinline__ void fence_acq_rel_cluster() { asm volatile("fence.acq_rel.cluster;" ::: "memory"); }
+
+__global__ void __launch_bounds__(kThreads, 1)
+dqgemm_kacc_kernel(const __grid_constant__ CUtensorMap xmap, const Job* __restrict__ jobs, const Seg* __restrict__ segs,
+                   int n_groups, int T, float* __restrict__ out, int ldo, int* __restrict__ err, uint32_t n_stages,
+                   uint32_t hdr_bytes, uint32_t seg_stride, unsigned long long* stamps) {
+  extern __shared__ __align__(1024) uint8_t smem_raw[];
+  uint8_t* smem = smem_raw;
+  const uint32_t tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  if (tid == 0) { stamp_min(stamps, STAMP_FIRST_START); stamp_max(stamps, STAMP_LAST_START); }
+  const uint32_t rank = cluster_ctarank();
+  const uint32_t pair_base = blockIdx.x & ~1u;
+  const uint32_t n_cols64 = gridDim.x;                 // 64-feature tiles: job (g, c) = jobs[g * n_cols64 + c]
+
+  KaccHeader* hdr = reinterpret_cast<KaccHeader*>(smem);
+  uint16_t* tables = reinterpret_cast<uint16_t*>(smem + 768);
+  uint8_t* xsm = smem + hdr_bytes;
+  uint8_t* wsm = xsm + n_stages * kBoxBytes;            // two buffers of kKaccWBytes
+
+  // both CTAs look at both halves of every K group, so a refused pair leaves together
+  bool bad = n_groups < 1 || n_stages < 2 || n_stages > kMaxStages || (gridDim.x & 1) != 0 || (hdr_bytes & 1023) != 0 ||
+             768 + kWarps * kTableStride * 2 > hdr_bytes || (smem_addr(smem_raw) & 1023u) != 0;
+  for (int g = 0; !bad && g < n_groups; ++g) {
+    const uint32_t i0 = g * n_cols64 + pair_base;
+    const Job a = jobs[i0], b = jobs[i0 + 1];
+    bad = a.n_rows != 64 || b.n_rows != 64 || a.k_total != b.k_total || a.x_koff != b.x_koff || a.k_total == 0 ||
+          a.k_total > kKaccKMax || (a.k_total % kChunkK) != 0 || a.n_seg == 0 || b.n_seg == 0 || a.n_seg > seg_stride ||
+          b.n_seg > seg_stride || a.n_seg > kMaxSegs || b.n_seg > kMaxSegs || a.seg_begin != i0 * seg_stride ||
+          b.seg_begin != (i0 + 1) * seg_stride || a.out_col != pair_base * 64 || b.out_col != (pair_base + 1) * 64;
+  }
+  if (bad) {
+    if (tid == 0) atomicCAS(err, ERR_NONE, ERR_BAD_JOB);
+    return;
+  }
+
+  const int n_mtiles = (T + kTileM - 1) / kTileM;
+  const uint32_t n_mpairs = (n_mtiles + 1) / 2;
+  const uint32_t my_pairs = blockIdx.y < n_mpairs ? (n_mpairs - blockIdx.y + gridDim.y - 1) / gridDim.y : 0;
+  const uint32_t n_blocks = (my_pairs + kKaccTiles - 1) / kKaccTiles;
+  const uint32_t n_steps = n_blocks * static_cast<uint32_t>(n_groups);       // (block, K group) steps of this pair
+  const uint32_t xsm_addr = smem_addr(xsm);
+  auto tile_row0 = [&](uint32_t ti) { return static_cast<int>((2 * (blockIdx.y + ti * gridDim.y) + rank) * kTileM); };
+  auto tiles_in = [&](uint32_t blk) { return my_pairs - blk * kKaccTiles < kKaccTiles ? my_pairs - blk * kKaccTiles : kKaccTiles; };
+  // activation boxes the pair brings in over the whole launch (for the "does anybody still wait" rule of the commits)
+  uint32_t boxes_per_tile = 0;
+  for (int g = 0; g < n_groups; ++g) boxes_per_tile += jobs[g * n_cols64 + pair_base].k_total / kChunkK;
+  const uint32_t total_boxes = my_pairs * boxes_per_tile;
+
+  if (tid == 0) {
+    for (uint32_t s = 0; s < n_stages; ++s) {
+      mbar_init(smem_addr(&hdr->full[s]), 1);
+      mbar_init(smem_addr(&hdr->empty[s]), 1);
+    }
+    for (int b = 0; b < 2; ++b) {
+      mbar_init(smem_addr(&hdr->w_full[b]), 2);
+      mbar_init(smem_addr(&hdr->w_empty[b]), 1);
+    }
+    mbar_init(smem_addr(&hdr->acc_full), 1);
+    mbar_init(smem_addr(&hdr->acc_empty), 2 * kKaccGroupWarps);
+    mbar_init(smem_addr(&hdr->drain), 1);
+    hdr->abort = 0;
+    mbar_fence_init();
+    fence_proxy_async_smem();
+  }
+  if (warp == 1) {
+    tmem_alloc_pair(smem_addr(&hdr->tmem_base), kKaccTmemCols);
+    tmem_relinquish_pair();
+  }
+  tc_fence_before_sync();
+  __syncthreads();
+  tc_fence_after_sync();
+  const uint32_t tmem_base = hdr->tmem_base;
+  cluster_sync_all();               // the partner's barriers are initialised before anything arrives on them
+  pdl_launch_dependents();
+
+  bool failed = false;
+  if (warp == 0) {
+    // ---- producer (one in each CTA): own token tile into own ring, bytes credited to CTA 0's barrier
+    if (lane == 0) {
+      pdl_wait();                   // the activations are the previous kernel's output
+      stamp_min(stamps, STAMP_RELEASE);
+      uint32_t c = 0, stage = 0, round = 0;
+      for (uint32_t blk = 0; blk < n_blocks && !failed; ++blk) {
+        const uint32_t nt = tiles_in(blk);
+        for (int g = 0; g < n_groups && !failed; ++g) {
+          const Job jb = jobs[g * n_cols64 + pair_base];
+          const uint32_t nb = jb.k_total / kChunkK, rot = (blockIdx.x >> 1) % nb;
+          for (uint32_t t = 0; t < nt && !failed; ++t) {
+            const int row0 = tile_row0(blk * kKaccTiles + t);
+            for (uint32_t bi = 0; bi < nb; ++bi, ++c) {
+              if (round > 0 && !mbar_wait_bounded_relaxed(smem_addr(&hdr->empty[stage]), (round - 1) & 1)) {
+                failed = true;
+                break;
+              }
+              const uint32_t b = bi + rot < nb ? bi + rot : bi + rot - nb;
+              if (rank == 0) mbar_expect_tx(smem_addr(&hdr->full[stage]), 2 * kBoxBytes);
+              tma_load_2d_pair(xsm_addr + stage * kBoxBytes, &xmap, static_cast<int>(jb.x_koff + b * kChunkK), row0,
+                               map_to_cta(smem_addr(&hdr->full[stage]), 0));
+              if (++stage == n_stages) { stage = 0; ++round; }
+            }
+          }
+        }
+      }
+    }
+    __syncwarp();
+  } else if (warp == 1) {
+    if (rank == 0) {
+      // ---- MMA issuer of the pair
+      const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((128u >> 3) << 17) | ((256u >> 4) << 24);
+      const uint32_t w_lbo = 64 * 16;
+      const uint64_t a_desc0 = umma_smem_desc_sw128(xsm_addr);
+      const uint64_t b_desc_buf[2] = {umma_smem_desc(smem_addr(wsm), w_lbo, 128),
+                                      umma_smem_desc(smem_addr(wsm + kKaccWBytes), w_lbo, 128)};
+      const uint32_t a_stage_step = kBoxBytes >> 4;
+      const uint32_t b_ks_step = (2 * w_lbo) >> 4, b_chunk_step = 4 * b_ks_step;
+      uint32_t c = 0, stage = 0, round = 0, step = 0, issued = 0;
+      for (uint32_t blk = 0; blk < n_blocks && !failed; ++blk) {
+        const uint32_t nt = tiles_in(blk);
+        if (blk > 0 && !__all_sync(0xffffffffu, mbar_wait_bounded(smem_addr(&hdr->acc_empty), (blk - 1) & 1))) {
+          failed = true;
+          break;
+        }
+        for (int g = 0; g < n_groups && !failed; ++g, ++step) {
+          const uint32_t wb = step & 1;
+          const Job jb = jobs[g * n_cols64 + pair_base];
+          const uint32_t nb = jb.k_total / kChunkK, rot = (blockIdx.x >> 1) % nb;
+          if (!__all_sync(0xffffffffu, mbar_wait_bounded(smem_addr(&hdr->w_full[wb]), (step >> 1) & 1))) {
+            failed = true;
+            break;
+          }
+          fence_acq_rel_cluster();      // the other CTA's half of the tile was written by the other CTA's threads
+          tc_fence_after_sync();
+          for (uint32_t t = 0; t < nt && !failed; ++t) {
+            const uint32_t d_addr = tmem_base + t * kKaccAccCols;
+            for (uint32_t bi = 0; bi < nb; ++bi, ++c) {
+              if (!__all_sync(0xffffffffu, mbar_wait_bounded(smem_addr(&hdr->full[stage]), round & 1))) {
+                failed = true;
+                break;
+              }
+              tc_fence_after_sync();
+              const uint32_t b = bi + rot < nb ? bi + rot : bi + rot - nb;
+              if (elect_one()) {
+                umma_bf16_ss_x4_pair(d_addr, a_desc0 + stage * a_stage_step, b_desc_buf[wb] + b * b_chunk_step, 2,
+                                     b_ks_step, idesc, (g != 0 || bi != 0) ? 1u : 0u);
+                if (c + n_stages < total_boxes) umma_commit_pair(smem_addr(&hdr->empty[stage]));
+              }
+              __syncwarp();
+              issued = c + 1;
+              if (++stage == n_stages) { stage = 0; ++round; }
+            }
+          }
+          if (!failed) {
+            if (elect_one()) {
+              if (step + 2 < n_steps) umma_commit_pair(smem_addr(&hdr->w_empty[wb]));
+              if (g + 1 == n_groups) umma_commit_pair(smem_addr(&hdr->acc_full));
+            }
+            __syncwarp();
+          }
+        }
+      }
+      if (failed && issued > 0) {
+        if (elect_one()) umma_commit_pair(smem_addr(&hdr->drain));
+        __syncwarp();
+        (void)mbar_wait_bounded(smem_addr(&hdr->drain), 0);
+      }
+    }
+  } else if (warp >= kKaccGroupWarp0 && warp < kKaccGroupWarp0 + kKaccGroupWarps) {
+    // ---- decode group / epilogue.  No early exit: the group meets at named barriers inside the decode.
+    const uint32_t gtid = tid - kKaccGroupWarp0 * 32;
+    const uint32_t q = warp & 3, half = (warp - kKaccGroupWarp0) >> 2;
+    bool released = false;
+    // lane 0 polls and the warp takes its verdict; once the CTA has given up nobody waits any more
+    auto wait_uniform = [&](uint32_t bar, uint32_t parity) {
+      uint32_t ok = 1;
+      if (lane == 0) ok = (failed || hdr->abort) ? 0u : (mbar_wait_bounded(bar, parity) ? 1u : 0u);
+      ok = __shfl_sync(0xffffffffu, ok, 0);
+      if (!ok) {
+        failed = true;
+        if (lane == 0) hdr->abort = 1;
+      }
+    };
+    auto epilogue = [&](uint32_t blk) {
+      if (!released) { pdl_wait(); released = true; }               // `out` may still be read by an earlier kernel
+      wait_uniform(smem_addr(&hdr->acc_full), blk & 1);
+      tc_fence_after_sync();
+      const uint32_t nt = tiles_in(blk);
+      for (uint32_t t = 0; t < nt; ++t) {
+        const int row = tile_row0(blk * kKaccTiles + t) + static_cast<int>(q * 32 + lane);
+        float* drow = out + static_cast<size_t>(row < T ? row : 0) * ldo + pair_base * 64 + half * 64;
+        const uint32_t taddr = tmem_base + ((q * 32) << 16) + t * kKaccAccCols + half * 64;
+#pragma unroll
+        for (uint32_t col = 0; col < 64; col += 32) {
+          uint32_t r[32];
+          tmem_ld_32x32b_x32(taddr + col, r);
+          tc_wait_ld();
+          if (row < T) {
+#pragma unroll
+            for (int h = 0; h < 2; ++h) {
+              float v[16];
+#pragma unroll
+              for (int i = 0; i < 16; ++i) v[i] = __uint_as_float(r[h * 16 + i]);
+              store_row16<float>(drow + col + h * 16, v);
+            }
+          }
+        }
+      }
+      tc_fence_before_sync();
+      __syncwarp();
+      if (lane == 0) mbar_arrive_cluster(map_to_cta(smem_addr(&hdr->acc_empty), 0));
+    };
+    uint32_t step = 0;
+    for (uint32_t blk = 0; blk < n_blocks; ++blk) {
+      for (int g = 0; g < n_groups; ++g, ++step) {
+        const uint32_t wb = step & 1;
+        if (step >= 2) wait_uniform(smem_addr(&hdr->w_empty[wb]), ((step >> 1) - 1) & 1);
+        const uint32_t ji = g * n_cols64 + blockIdx.x;
+        const Job job = jobs[ji];
+        decode_weight_tile_group<kKaccGroupWarps>(job, segs + static_cast<size_t>(ji) * seg_stride, tables,
+                                                  wsm + wb * kKaccWBytes, gtid, kKaccGroupBarrier);
+        if (gtid == 0) {
+          if (step == 0) stamp_max(stamps, STAMP_DECODED);
+          mbar_arrive_cluster(map_to_cta(smem_addr(&hdr->w_full[wb]), 0));
+        }
+        // the previous block is drained after this block's first tile is decoded: that decode ran under the
+        // previous block's last MMAs
+        if (g == 0 && blk > 0) epilogue(blk - 1);
+      }
+    }
+    if (n_blocks > 0) epilogue(n_blocks - 1);
+  }
+  if (failed) {
+    hdr->abort = 1;
+    if (lane == 0) atomicCAS(err, ERR_NONE, ERR_WAIT_TIMEOUT);
+  }
+  tc_fence_before_sync();
+  __syncthreads();
+  cluster_sync_all();      // neither CTA frees tensor memory or exits while the pair's MMAs may still use it
+  if (warp == 1) tmem_dealloc_pair(tmem_base, kKaccTmemCols);
+  if (tid == 0) stamp_max(stamps, STAMP_LAST_END);
+}
+
+}  // namespace
+
+size_t gemm_kacc_smem_bytes(uint32_t hdr_bytes, uint32_t n_stages) {
+  return static_cast<size_t>(hdr_bytes) + static_cast<size_t>(n_stages) * kBoxBytes + 2 * kKaccWBytes;
+}
+
+cudaError_t gemm_kacc_configure() {
+  return cudaFuncSetAttribute(dqgemm_kacc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 232448);
+}
+
+cudaError_t launch_gemm_kacc(const KaccLaunch& p, cudaStream_t s) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(p.n_cols64, p.m_ctas);
+  cfg.blockDim = dim3(kThreads);
+  cfg.dynamicSmemBytes = gemm_kacc_smem_bytes(p.hdr_bytes, p.n_stages);
+  cfg.stream = s;
+  cudaLaunchAttribute attr[2];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+  attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[1].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = p.pdl ? 2 : 1;
+  return cudaLaunchKernelEx(&cfg, dqgemm_kacc_kernel, p.xmap, p.jobs, p.segs, p.n_groups, p.T, p.out, p.ldo, p.err,
+                            p.n_stages, p.hdr_bytes, p.seg_stride, p.stamps);
+}
+
+}  // namespace sti

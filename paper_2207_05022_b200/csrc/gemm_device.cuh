@@ -309,5 +309,139 @@ __device__ __forceinline__ void decode_weight_tile(const Job& job, const Seg* __
   __syncthreads();
 }
 
+// ---------------------------------------------------------------------------------------
+// Two-CTA (cta_group::2) forms of the tensor-memory, TMA and MMA helpers
+// ---------------------------------------------------------------------------------------
+__device__ __forceinline__ void tmem_alloc_pair(uint32_t smem_dst, uint32_t n_cols) {     // one warp in each CTA
+  asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_dst), "r"(n_cols)
+               : "memory");
+}
+__device__ __forceinline__ void tmem_relinquish_pair() {
+  asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc_pair(uint32_t taddr, uint32_t n_cols) {
+  asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(n_cols) : "memory");
+}
+// Own tile into own shared memory, completion bytes credited to the barrier at `bar_cluster_addr` (CTA 0's).
+__device__ __forceinline__ void tma_load_2d_pair(uint32_t dst, const CUtensorMap* map, int k0, int m0,
+                                                 uint32_t bar_cluster_addr) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+      ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(k0), "r"(m0), "r"(bar_cluster_addr)
+      : "memory");
+}
+__device__ __forceinline__ void umma_bf16_ss_x4_pair(uint32_t tmem_d, uint64_t desc_a, uint64_t desc_b, uint32_t a_step,
+                                                     uint32_t b_step, uint32_t idesc, uint32_t accumulate_first) {
+  asm volatile(
+      "{\n\t.reg .pred p0, p1;\n\t.reg .b64 a1, a2, a3, b1, b2, b3, as, bs;\n\t"
+      "setp.ne.b32 p0, %6, 0;\n\t"
+      "setp.eq.b32 p1, 0, 0;\n\t"
+      "cvt.u64.u32 as, %3;\n\t"
+      "cvt.u64.u32 bs, %4;\n\t"
+      "add.u64 a1, %1, as;\n\tadd.u64 a2, a1, as;\n\tadd.u64 a3, a2, as;\n\t"
+      "add.u64 b1, %2, bs;\n\tadd.u64 b2, b1, bs;\n\tadd.u64 b3, b2, bs;\n\t"
+      "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %5, p0;\n\t"
+      "tcgen05.mma.cta_group::2.kind::f16 [%0], a1, b1, %5, p1;\n\t"
+      "tcgen05.mma.cta_group::2.kind::f16 [%0], a2, b2, %5, p1;\n\t"
+      "tcgen05.mma.cta_group::2.kind::f16 [%0], a3, b3, %5, p1;\n\t}"
+      ::"r"(tmem_d), "l"(desc_a), "l"(desc_b), "r"(a_step), "r"(b_step), "r"(idesc), "r"(accumulate_first)
+      : "memory");
+}
+// Completion of all MMAs issued so far -> the barrier at this offset in both CTAs.
+__device__ __forceinline__ void umma_commit_pair(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+               ::"r"(bar), "h"(static_cast<uint16_t>(3)) : "memory");
+}
+
+
+// ---------------------------------------------------------------------------------------
+// The same decode run by a group of NWARPS warps of the CTA (the others do something else meanwhile):
+// `gtid` is the thread's index inside the group, `warp_tables` the group's first centroid table, `bar_id`
+// a named barrier reserved for the group.  Ends with the tile visible to the tensor core (proxy fence +
+// group barrier).  Every thread of the group must call it the same number of times.
+// ---------------------------------------------------------------------------------------
+template <int NWARPS>
+__device__ __forceinline__ void group_barrier(uint32_t bar_id) {
+  asm volatile("bar.sync %0, %1;" ::"r"(bar_id), "n"(NWARPS * 32) : "memory");
+}
+
+template <int NWARPS>
+__device__ __forceinline__ void decode_weight_tile_group(const Job& job, const Seg* __restrict__ segs,
+                                                         uint16_t* warp_tables, uint8_t* wsm, uint32_t gtid,
+                                                         uint32_t bar_id) {
+  constexpr uint32_t kGroupThreads = NWARPS * 32;
+  const uint32_t lane = gtid & 31, warp = gtid >> 5;
+  const uint32_t n_rows = job.n_rows, k_total = job.k_total;
+  const Seg& s0 = segs[0];
+  const uint32_t rows_per_group = s0.kc >= 128 ? 32 : 64;
+  const uint32_t chunks = s0.kc >= 128 ? s0.kc / 128 : 1;
+  const uint32_t tasks_per_seg = (n_rows / rows_per_group) * chunks;
+  const uint32_t n_tasks = tasks_per_seg * job.n_seg;
+  uint32_t o_seg = 0xffffffffu, o_off = 0, n_out_total = 0;
+  float o_val = 0.f;
+  for (uint32_t si = 0; si < job.n_seg; ++si) {
+    const uint32_t n = segs[si].n_out;
+    if (o_seg == 0xffffffffu && gtid >= n_out_total && gtid - n_out_total < n) {
+      o_seg = si;
+      o_off = __ldg(segs[si].out_off + (gtid - n_out_total));
+      o_val = __ldg(segs[si].out_val + (gtid - n_out_total));
+    }
+    n_out_total += n;
+  }
+  uint16_t* tab = warp_tables + warp * kTableStride;
+  for (uint32_t t = warp; t < n_tasks; t += NWARPS) {
+    const uint32_t si = t / tasks_per_seg, task = t % tasks_per_seg;
+    const Seg& sg = segs[si];
+    const uint32_t bits = sg.bits;
+    if (bits > 6) continue;
+    const uint32_t n_entries = 1u << bits;
+    const float c0 = lane < n_entries ? __ldg(sg.table + lane) : 0.f;
+    const float c1 = lane + 32 < n_entries ? __ldg(sg.table + lane + 32) : 0.f;
+    uint32_t planes[24];
+    load_planes(sg, task, lane, planes);
+    tab[lane] = bf16_bits(c0);
+    tab[lane + 32] = bf16_bits(c1);
+    __syncwarp();
+    switch (bits) {
+      case 2: unpack_task<2>(planes, sg, tab, wsm, n_rows, task, lane); break;
+      case 3: unpack_task<3>(planes, sg, tab, wsm, n_rows, task, lane); break;
+      case 4: unpack_task<4>(planes, sg, tab, wsm, n_rows, task, lane); break;
+      case 5: unpack_task<5>(planes, sg, tab, wsm, n_rows, task, lane); break;
+      case 6: unpack_task<6>(planes, sg, tab, wsm, n_rows, task, lane); break;
+      default: break;
+    }
+    __syncwarp();
+  }
+  for (uint32_t si = 0; si < job.n_seg; ++si) {
+    const Seg& sg = segs[si];
+    if (sg.bits == 32) {             // uncompressed version: fp32 rows, rounded to bf16 on the way in
+      const float* src = reinterpret_cast<const float*>(sg.codes);
+      const uint32_t pieces_per_row = sg.kc / 8;
+      const uint32_t total = n_rows * pieces_per_row;
+      for (uint32_t idx = gtid; idx < total; idx += kGroupThreads) {
+        const uint32_t row = idx % n_rows, piece = idx / n_rows;
+        const float4 a = __ldg(reinterpret_cast<const float4*>(src + static_cast<size_t>(row) * sg.kc + piece * 8));
+        const float4 b = __ldg(reinterpret_cast<const float4*>(src + static_cast<size_t>(row) * sg.kc + piece * 8 + 4));
+        const uint32_t kcore = (sg.koff >> 3) + piece;
+        *reinterpret_cast<uint4*>(wsm + (static_cast<size_t>(kcore) * n_rows + row) * 16) =
+            make_uint4(pack_bf16x2(a.x, a.y), pack_bf16x2(a.z, a.w), pack_bf16x2(b.x, b.y), pack_bf16x2(b.z, b.w));
+      }
+    }
+  }
+  group_barrier<NWARPS>(bar_id);
+  if (o_seg != 0xffffffffu) patch_outlier(segs[o_seg], o_off, o_val, wsm, n_rows, k_total);
+  if (n_out_total > kGroupThreads) {
+    uint32_t base = 0;
+    for (uint32_t si = 0; si < job.n_seg; ++si) {
+      const Seg& sg = segs[si];
+      for (uint32_t o = gtid; o < sg.n_out; o += kGroupThreads)
+        if (base + o >= kGroupThreads) patch_outlier(sg, __ldg(sg.out_off + o), __ldg(sg.out_val + o), wsm, n_rows, k_total);
+      base += sg.n_out;
+    }
+  }
+  fence_proxy_async_smem();
+  group_barrier<NWARPS>(bar_id);
+}
+
 }  // namespace
 }  // namespace sti

@@ -76,10 +76,32 @@ size_t gemm_smem_bytes(uint32_t w_bytes, uint32_t n_stages, uint32_t bps, uint32
 cudaError_t gemm_configure();   // opt in to large dynamic shared memory (once per device)
 cudaError_t launch_gemm(GemmKind kind, const GemmLaunch& p, cudaStream_t s);
 
+// K-accumulating two-CTA dequant-GEMM (fp32 output written once, all K groups summed in tensor memory).
+// jobs: n_groups x n_cols64 tile jobs of 64 rows and at most 512 columns, job (g, c) at index g * n_cols64 + c,
+// segments at the fixed stride; out: [T][ldo] fp32, tile c writes columns [64 c, 64 c + 64).
+struct KaccLaunch {
+  const Job* jobs;
+  const Seg* segs;
+  int n_groups, n_cols64, m_ctas;
+  CUtensorMap xmap;         // x: [T rows, ldx columns] bf16, box 64 x 128, 128-byte swizzle
+  int T;
+  float* out;
+  int ldo;
+  int* err;
+  uint32_t n_stages, hdr_bytes, seg_stride;
+  bool pdl;
+  unsigned long long* stamps;
+};
+cudaError_t gemm_kacc_configure();
+size_t gemm_kacc_smem_bytes(uint32_t hdr_bytes, uint32_t n_stages);
+cudaError_t launch_gemm_kacc(const KaccLaunch& p, cudaStream_t s);
+
 // Per-head attention over kept heads.  qkv: [(kept*3 + which)][T][64] bf16; out: [T][n_kept*64] bf16.
+// sm_count (the device's multiprocessor count) picks the CTA shape: large query tiles once they fill the GPU.
 cudaError_t attention_configure();
 cudaError_t launch_attention(const uint16_t* qkv, uint16_t* out, int n_kept, int batch, int seq,
-                             const int32_t* seq_lens, cudaStream_t s, bool pdl, unsigned long long* stamps);
+                             const int32_t* seq_lens, int sm_count, cudaStream_t s, bool pdl,
+                             unsigned long long* stamps);
 
 // The same attention on the tcgen05 tensor cores, one CTA per (sequence, kept head), for many tokens (attention_tc.cu).
 // `qkv_map`: TMA view of qkv as [3 * n_kept * T rows, 64 columns] bf16, boxes of 128 rows x 64 columns, 128-byte swizzle.

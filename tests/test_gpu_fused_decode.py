@@ -167,6 +167,47 @@ def test_fused_decode_more_outliers_than_threads_in_a_tile():
         _check_all_gemms(work, s, variant=2)
 
 
+def _check_ffn2_kacc(work, sess):
+    """FFN2 through the K-accumulating kernel: one complete plane, every weight exactly once."""
+    sh = work.shape
+    f = sh.slice_width
+    slices = work.kept(0, FFN)
+    ns = len(slices)
+    out, n_part = _probe(sess, 3, ns * f, (1, ns * f, sh.hidden), torch.float32, 3)
+    assert n_part == 1
+    got = out[0].cpu().numpy()
+    assert np.isfinite(got).all()
+    for ji, j in enumerate(slices):
+        want = O.bf16_rne(_oracle_unit(work, FFN, j)["F2"]).T               # [f][d]
+        assert np.array_equal(got[ji * f:(ji + 1) * f].view(np.uint32), want.view(np.uint32)), ("FFN2 kacc", j)
+
+
+@pytest.mark.parametrize("tune,keep_ffn", [
+    ("f2_kacc_min_tokens=1024", lambda i: True),                       # 3 K groups of 512, one tile pair per CTA pair
+    ("f2_kacc_min_tokens=1024,cta_budget=4", lambda i: True),          # one CTA pair per column pair: 2 blocks (4 + 2 tiles)
+    ("f2_kacc_min_tokens=1024,cta_budget=8", lambda i: i != 2),        # 5 slices kept: the last K group is 256 wide
+])
+def test_fused_decode_k_accumulating_ffn2_small_shape(tune, keep_ffn):
+    shape = W.ModelShape(n_layers=1, hidden=256, n_heads=4, head_dim=64, ffn=1536, n_ffn_slices=6)
+    work = _mixed_work(shape, seed=16, keep_fn=lambda k, i: True if k == ATTN else keep_ffn(i))
+    with _Tune(tune), sti.Session(work, max_batch=8, max_seq=256) as s:
+        _check_ffn2_kacc(work, s)
+
+
+def test_fused_decode_k_accumulating_ffn2_bert_large():
+    shape = W.BERT_LARGE.with_layers(1)
+    work = _mixed_work(shape, seed=17)
+    with sti.Session(work, max_batch=32, max_seq=512) as s:                # made for 16,384 tokens: the default rule applies
+        _check_ffn2_kacc(work, s)
+        _check_all_gemms(work, s, variant=2)
+    with sti.Session(work, max_batch=8, max_seq=512) as s:                 # 4,096 tokens: no K-accumulating table
+        x = _identity_bf16(64)
+        out = torch.zeros(64 * 1024, dtype=torch.float32, device="cuda")
+        with pytest.raises(sti.StiError) as e:
+            sti.sti_gemm_probe(s.plan, 0, 3, x.data_ptr(), 64, out.data_ptr(), out.numel() * 4, 3)
+        assert e.value.status == 5
+
+
 def test_probe_argument_checks():
     shape = W.ModelShape(n_layers=1, hidden=256, n_heads=4, head_dim=64, ffn=1024, n_ffn_slices=4)
     attn, ffn = _plan(shape, lambda k, i: 4, lambda k, i: k == ATTN)      # no FFN slice kept
