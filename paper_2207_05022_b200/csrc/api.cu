@@ -37,7 +37,9 @@ struct Tuning {
   int qkv_n = 32, f1_n = 64, o_n = 64, o_group = 4, f2_n = 64, f2_group = 2;
   int cta_budget = 148;                // (replaced by the device's SM count in parse_tuning) CTAs a GEMM launch may use when it splits the token tiles over CTAs
   int pair_min_tiles = 8;              // two-CTA GEMM from this many 128-token tiles on (0 = never)
-  int f2_kacc_min_tokens = 8192;       // FFN2 through the K-accumulating kernel (one output plane) from this many tokens on (0 = never)
+  int f2_kacc_min_tokens = 4096;       // FFN2 through the K-accumulating kernel (one output plane) from this many tokens on (0 = never)
+  int f2_kacc_k = 512;                 // columns per K group there
+  int f2_kacc_bps = 2;                 // boxes of 64 columns per ring stage there (1 or 2)
   int attn_tc_min_items = 96;          // tensor-core attention from this many (sequence, kept head) pairs on, seq >= 256 (0 = never)
   int ln1_ctas = -1, ln2_ctas = -1;    // LayerNorm CTA counts: -1 = chosen per launch (see ln_ctas_hint), 0 = one row per CTA
 };
@@ -216,6 +218,8 @@ void parse_tuning(Tuning* t, int tmax, const sti_model_desc& d, int sm_count) {
         else if (k == "f2_group") t->f2_group = v;
         else if (k == "pair_min_tiles") t->pair_min_tiles = v;
         else if (k == "f2_kacc_min_tokens") t->f2_kacc_min_tokens = std::max(0, v);
+        else if (k == "f2_kacc_k") t->f2_kacc_k = std::max(64, std::min(v, 1024));
+        else if (k == "f2_kacc_bps") t->f2_kacc_bps = v == 1 ? 1 : 2;
         else if (k == "attn_tc_min_items") t->attn_tc_min_items = std::max(0, v);
         else if (k == "cta_budget") t->cta_budget = std::max(1, v);
         else if (k == "ln1_ctas") t->ln1_ctas = std::max(-1, v);
@@ -359,7 +363,7 @@ void build_layer_tables(sti_plan* p, Layer& L, TableBuilder tb[5]) {
     }
   }
   // FFN2 for the K-accumulating kernel: 64-row tiles, K groups of at most 512 columns, group-major order
-  const int kacc_group = f <= 512 && 512 % f == 0 ? static_cast<int>(512 / f) : 0;
+  const int kacc_group = static_cast<int>(t.f2_kacc_k / f);      // whole slices per K group (0: a slice does not fit)
   L.f2k.n_split = 0;
   if (kacc_group > 0 && ns > 0 && d.hidden % 128 == 0 && t.f2_kacc_min_tokens > 0 &&
       static_cast<long long>(d.max_batch) * d.max_seq >= t.f2_kacc_min_tokens) {
@@ -478,7 +482,7 @@ sti_status run_gemm_kacc(sti_plan* p, const GemmTable& tab, const void* x, int l
   g.m_ctas = std::max(1, std::min(n_mpairs, p->tune.cta_budget / g.n_cols64));
   if (!make_xmap(&g.xmap, x, ldx, T)) return STI_ERR_CUDA;
   g.T = T; g.out = out; g.ldo = ldo; g.err = p->ctx->err_dev;
-  g.n_stages = tab.n_stages; g.hdr_bytes = tab.hdr_bytes; g.seg_stride = tab.seg_stride;
+  g.n_stages = tab.n_stages; g.bps = tab.bps; g.hdr_bytes = tab.hdr_bytes; g.seg_stride = tab.seg_stride; g.k_group = tab.k_max;
   g.pdl = p->ctx->pdl; g.stamps = stamps;
   CUDA_TRY(launch_gemm_kacc(g, p->ctx->compute));
   p->ctx->launches++;
@@ -1138,9 +1142,13 @@ sti_status sti_plan_finalize(sti_plan* p) {
         gt[i]->pair_ok = a.n_rows == 64 && b.n_rows == 64 && a.k_total == b.k_total && a.x_koff == b.x_koff;
       }
       if (i == 4) {                 // two weight buffers, the rest of the shared memory is the ring of single boxes
-        gt[i]->n_stages = 6; gt[i]->bps = 1;
-        gt[i]->smem = gemm_kacc_smem_bytes(gt[i]->hdr_bytes, gt[i]->n_stages);
-        if (gt[i]->smem > kMaxSmem) return STI_ERR_SHAPE;
+        gt[i]->k_max = tb[i].k_max;
+        gt[i]->bps = p->tune.f2_kacc_bps;
+        for (const Job& j : tb[i].jobs)
+          if (j.k_total % (128 * gt[i]->bps / 2) != 0) gt[i]->bps = 1;      // an odd number of boxes somewhere
+        gt[i]->n_stages = gemm_kacc_stages(gt[i]->hdr_bytes, tb[i].k_max, gt[i]->bps, kMaxSmem);
+        gt[i]->smem = gemm_kacc_smem_bytes(gt[i]->hdr_bytes, gt[i]->n_stages, gt[i]->bps, tb[i].k_max);
+        if (!tb[i].jobs.empty() && (gt[i]->n_stages < 2 || gt[i]->smem > kMaxSmem)) return STI_ERR_SHAPE;
       } else {
       if (!tb[i].jobs.empty() &&
           !gemm_pick_ring(tb[i].w_bytes, tb[i].k_max, gt[i]->hdr_bytes, &gt[i]->n_stages, &gt[i]->bps))

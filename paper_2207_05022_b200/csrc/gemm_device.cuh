@@ -365,7 +365,51 @@ __device__ __forceinline__ void group_barrier(uint32_t bar_id) {
   asm volatile("bar.sync %0, %1;" ::"r"(bar_id), "n"(NWARPS * 32) : "memory");
 }
 
-template <int NWARPS>
+// Half of unpack_task: index groups [2 * half, 2 * half + 2) of the quantum, so that two warps share a task (both
+// hold the task's planes) and the decode of a small tile has the latency of half a task.
+template <int BITS>
+__device__ __forceinline__ void unpack_task_half(const uint32_t (&planes)[24], const Seg& sg, const uint16_t* __restrict__ tab,
+                                                 uint8_t* wsm, uint32_t n_rows, uint32_t task, uint32_t lane, uint32_t half) {
+  uint32_t w[2 * BITS];
+  if (half == 0) {
+#pragma unroll
+    for (int i = 0; i < 2 * BITS; ++i) w[i] = planes[i];
+  } else {
+#pragma unroll
+    for (int i = 0; i < 2 * BITS; ++i) w[i] = planes[i + 2 * BITS];
+  }
+  const uint32_t chunks = sg.kc >= 128 ? sg.kc / 128 : 1;
+  const uint32_t g = task / chunks, j = task % chunks;
+  const bool narrow = sg.kc < 128;
+  const uint32_t row0 = narrow ? g * 64 + lane : g * 32 + lane;
+  const uint32_t kcore0 = (sg.koff + (narrow ? 0 : j * 128)) >> 3;
+#pragma unroll 1
+  for (int grp = 0; grp < 2; ++grp) {
+    uint32_t lo[BITS];
+#pragma unroll
+    for (int i = 0; i < BITS; ++i) lo[i] = w[i];
+#pragma unroll
+    for (int ss = 0; ss < 4; ++ss) {
+      uint32_t pk[4];
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        const uint32_t c0 = extract_index_words<BITS>(lo, 8 * ss + 2 * e);
+        const uint32_t c1 = extract_index_words<BITS>(lo, 8 * ss + 2 * e + 1);
+        pk[e] = static_cast<uint32_t>(tab[c0]) | (static_cast<uint32_t>(tab[c1]) << 16);
+      }
+      const uint32_t sidx = 8 * half + 4 * grp + ss;
+      const uint32_t row = narrow ? row0 + 32 * (sidx >> 3) : row0;
+      const uint32_t kcore = narrow ? kcore0 + (sidx & 7) : kcore0 + sidx;
+      *reinterpret_cast<uint4*>(wsm + (static_cast<size_t>(kcore) * n_rows + row) * 16) =
+          make_uint4(pk[0], pk[1], pk[2], pk[3]);
+    }
+#pragma unroll
+    for (int i = 0; i < BITS; ++i) w[i] = w[i + BITS];
+  }
+}
+
+// SPLIT: every task is shared by two warps (unit u = 2 * task + half), for tiles with fewer tasks than warps.
+template <int NWARPS, bool SPLIT = false>
 __device__ __forceinline__ void decode_weight_tile_group(const Job& job, const Seg* __restrict__ segs,
                                                          uint16_t* warp_tables, uint8_t* wsm, uint32_t gtid,
                                                          uint32_t bar_id) {
@@ -389,7 +433,8 @@ __device__ __forceinline__ void decode_weight_tile_group(const Job& job, const S
     n_out_total += n;
   }
   uint16_t* tab = warp_tables + warp * kTableStride;
-  for (uint32_t t = warp; t < n_tasks; t += NWARPS) {
+  for (uint32_t u = warp; u < (SPLIT ? 2 * n_tasks : n_tasks); u += NWARPS) {
+    const uint32_t t = SPLIT ? u >> 1 : u;
     const uint32_t si = t / tasks_per_seg, task = t % tasks_per_seg;
     const Seg& sg = segs[si];
     const uint32_t bits = sg.bits;
@@ -402,6 +447,16 @@ __device__ __forceinline__ void decode_weight_tile_group(const Job& job, const S
     tab[lane] = bf16_bits(c0);
     tab[lane + 32] = bf16_bits(c1);
     __syncwarp();
+    if (SPLIT) {
+      switch (bits) {
+        case 2: unpack_task_half<2>(planes, sg, tab, wsm, n_rows, task, lane, u & 1); break;
+        case 3: unpack_task_half<3>(planes, sg, tab, wsm, n_rows, task, lane, u & 1); break;
+        case 4: unpack_task_half<4>(planes, sg, tab, wsm, n_rows, task, lane, u & 1); break;
+        case 5: unpack_task_half<5>(planes, sg, tab, wsm, n_rows, task, lane, u & 1); break;
+        case 6: unpack_task_half<6>(planes, sg, tab, wsm, n_rows, task, lane, u & 1); break;
+        default: break;
+      }
+    } else {
     switch (bits) {
       case 2: unpack_task<2>(planes, sg, tab, wsm, n_rows, task, lane); break;
       case 3: unpack_task<3>(planes, sg, tab, wsm, n_rows, task, lane); break;
@@ -409,6 +464,7 @@ __device__ __forceinline__ void decode_weight_tile_group(const Job& job, const S
       case 5: unpack_task<5>(planes, sg, tab, wsm, n_rows, task, lane); break;
       case 6: unpack_task<6>(planes, sg, tab, wsm, n_rows, task, lane); break;
       default: break;
+    }
     }
     __syncwarp();
   }

@@ -77,7 +77,7 @@ cudaError_t gemm_configure();   // opt in to large dynamic shared memory (once p
 cudaError_t launch_gemm(GemmKind kind, const GemmLaunch& p, cudaStream_t s);
 
 // K-accumulating two-CTA dequant-GEMM (fp32 output written once, all K groups summed in tensor memory).
-// jobs: n_groups x n_cols64 tile jobs of 64 rows and at most 512 columns, job (g, c) at index g * n_cols64 + c,
+// jobs: n_groups x n_cols64 tile jobs of 64 rows and at most k_group columns, job (g, c) at index g * n_cols64 + c,
 // segments at the fixed stride; out: [T][ldo] fp32, tile c writes columns [64 c, 64 c + 64).
 struct KaccLaunch {
   const Job* jobs;
@@ -88,12 +88,14 @@ struct KaccLaunch {
   float* out;
   int ldo;
   int* err;
-  uint32_t n_stages, hdr_bytes, seg_stride;
+  uint32_t n_stages, bps, hdr_bytes, seg_stride;   // ring: n_stages stages of bps boxes (1 or 2; K groups are multiples of 64 * bps)
+  uint32_t k_group;         // columns of the widest K group (a multiple of 64): the size of the two weight buffers
   bool pdl;
   unsigned long long* stamps;
 };
 cudaError_t gemm_kacc_configure();
-size_t gemm_kacc_smem_bytes(uint32_t hdr_bytes, uint32_t n_stages);
+uint32_t gemm_kacc_stages(uint32_t hdr_bytes, uint32_t k_group, uint32_t bps, size_t smem_limit);
+size_t gemm_kacc_smem_bytes(uint32_t hdr_bytes, uint32_t n_stages, uint32_t bps, uint32_t k_group);
 cudaError_t launch_gemm_kacc(const KaccLaunch& p, cudaStream_t s);
 
 // Per-head attention over kept heads.  qkv: [(kept*3 + which)][T][64] bf16; out: [T][n_kept*64] bf16.

@@ -46,18 +46,19 @@ def _run(work, tune):
             os.environ["STI_TUNE"] = old
 
 
-@pytest.mark.parametrize("batch,seq,act,budget,keep", [
-    (16, 128, "bf16", 148, lambda i: True),        # 2,048 tokens: 8 tile pairs over 8 CTA pairs per column pair
-    (16, 128, "f32", 4, lambda i: True),           # one CTA pair per column pair: two full blocks of four
-    (11, 100, "bf16", 4, lambda i: i != 4),        # 1,100 tokens: 9 tiles (odd), ragged rows, 5 slices (a 256-wide group)
-    (24, 128, "bf16", 8, lambda i: i % 2 == 0),    # 3,072 tokens: 12 tile pairs over two CTA pairs: blocks of 4 + 2
+@pytest.mark.parametrize("batch,seq,act,budget,kgroup,keep", [
+    (16, 128, "bf16", 148, 256, lambda i: True),   # 2,048 tokens: 8 tile pairs over 8 CTA pairs per column pair
+    (16, 128, "f32", 4, 256, lambda i: True),      # one CTA pair per column pair: two full blocks of four
+    (11, 100, "bf16", 4, 512, lambda i: i != 4),   # 1,100 tokens: 9 tiles (odd), ragged rows, 5 slices (a 256-wide group)
+    (24, 128, "bf16", 8, 256, lambda i: i % 2 == 0),    # 3,072 tokens: 12 tile pairs over two CTA pairs: blocks of 4 + 2
+    (24, 128, "f32", 8, 512, lambda i: True),
 ])
-def test_layer_with_k_accumulating_ffn2(batch, seq, act, budget, keep):
+def test_layer_with_k_accumulating_ffn2(batch, seq, act, budget, kgroup, keep):
     from gpu_util import rel_err, REL_TOL
     work = _work(batch, seq, act, seed=batch * 100 + seq, keep=keep)
     a, f = O.decode_layer(work, 0)
     ref = O.layer_forward(work.x, work.dense[0], a, f, eps=work.ln_eps)
-    y_k, _ = _run(work, f"f2_kacc_min_tokens=1024,cta_budget={budget}")
+    y_k, _ = _run(work, f"f2_kacc_min_tokens=1024,f2_kacc_k={kgroup},cta_budget={budget}")
     y_p, _ = _run(work, f"f2_kacc_min_tokens=0,cta_budget={budget}")
     assert rel_err(y_k, ref) <= REL_TOL
     assert rel_err(y_p, ref) <= REL_TOL

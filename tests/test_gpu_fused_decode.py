@@ -183,9 +183,11 @@ def _check_ffn2_kacc(work, sess):
 
 
 @pytest.mark.parametrize("tune,keep_ffn", [
-    ("f2_kacc_min_tokens=1024", lambda i: True),                       # 3 K groups of 512, one tile pair per CTA pair
+    ("f2_kacc_min_tokens=1024", lambda i: True),                       # 6 K groups of 256, one tile pair per CTA pair
     ("f2_kacc_min_tokens=1024,cta_budget=4", lambda i: True),          # one CTA pair per column pair: 2 blocks (4 + 2 tiles)
-    ("f2_kacc_min_tokens=1024,cta_budget=8", lambda i: i != 2),        # 5 slices kept: the last K group is 256 wide
+    ("f2_kacc_min_tokens=1024,cta_budget=8", lambda i: i != 2),        # 5 slices kept
+    ("f2_kacc_min_tokens=1024,f2_kacc_k=512", lambda i: True),         # K groups of two slices, whole decode tasks per warp
+    ("f2_kacc_min_tokens=1024,f2_kacc_k=512,cta_budget=4", lambda i: i != 2),   # ... the last K group is 256 wide
 ])
 def test_fused_decode_k_accumulating_ffn2_small_shape(tune, keep_ffn):
     shape = W.ModelShape(n_layers=1, hidden=256, n_heads=4, head_dim=64, ffn=1536, n_ffn_slices=6)
@@ -200,7 +202,7 @@ def test_fused_decode_k_accumulating_ffn2_bert_large():
     with sti.Session(work, max_batch=32, max_seq=512) as s:                # made for 16,384 tokens: the default rule applies
         _check_ffn2_kacc(work, s)
         _check_all_gemms(work, s, variant=2)
-    with sti.Session(work, max_batch=8, max_seq=512) as s:                 # 4,096 tokens: no K-accumulating table
+    with sti.Session(work, max_batch=4, max_seq=512) as s:                 # 2,048 tokens: no K-accumulating table
         x = _identity_bf16(64)
         out = torch.zeros(64 * 1024, dtype=torch.float32, device="cuda")
         with pytest.raises(sti.StiError) as e:
