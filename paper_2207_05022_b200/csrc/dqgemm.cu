@@ -415,7 +415,7 @@ dqgemm_pair_kernel(const __grid_constant__ CUtensorMap xmap, const Job* __restri
     }
     for (int b = 0; b < 2; ++b) {
       mbar_init(smem_addr(&hdr->acc_full[b]), 1);
-      mbar_init(smem_addr(&hdr->acc_empty[b]), 2 * kEpilogueWarps);   // CTA 0 only: both CTAs' epilogue warps
+      mbar_init(smem_addr(&hdr->acc_empty[b]), 2 * kPairEpilogueWarps);   // CTA 0 only: both CTAs' epilogue warps
     }
     mbar_init(smem_addr(&hdr->drain), 1);
     hdr->abort = 0;
@@ -510,10 +510,11 @@ dqgemm_pair_kernel(const __grid_constant__ CUtensorMap xmap, const Job* __restri
         (void)mbar_wait_bounded(smem_addr(&hdr->drain), 0);
       }
     }
-  } else if (warp >= kEpilogueWarp0 && warp < kEpilogueWarp0 + kEpilogueWarps) {
-    // ---- epilogue: this CTA's 128 token rows; warp = (lane quadrant, which job's 64 columns)
-    const uint32_t q = warp & 3, half = (warp - kEpilogueWarp0) >> 2;
-    const Job& jb = half ? job1 : job0;
+  } else if (warp >= kEpilogueWarp0 && warp < kEpilogueWarp0 + kPairEpilogueWarps) {
+    // ---- epilogue: this CTA's 128 token rows x 128 features.  Twelve warps, three per tensor-memory lane quadrant
+    // (a warp reads only the 32 lanes of quadrant warp % 4); the three share the eight 16-column chunks 3 + 3 + 2.
+    const uint32_t q = warp & 3, part = (warp - kEpilogueWarp0) >> 2;
+    const uint32_t chunk0 = part * 3, chunk1 = part == 2 ? 8 : chunk0 + 3;
     for (uint32_t ti = 0; ti < my_pairs; ++ti) {
       const uint32_t buf = ti & 1;
       uint32_t ok = 1;
@@ -522,23 +523,27 @@ dqgemm_pair_kernel(const __grid_constant__ CUtensorMap xmap, const Job* __restri
       if (!ok) { failed = true; break; }
       tc_fence_after_sync();
       const int t = tile_row0(ti) + static_cast<int>(q * 32 + lane);
-      OutT* drow = out + (static_cast<size_t>(jb.out_mat) * T + (t < T ? t : 0)) * ldo + jb.out_col;
-      const uint32_t taddr = tmem_base + ((q * 32) << 16) + buf * kAccCols + half * 64;
+      const size_t trow = static_cast<size_t>(t < T ? t : 0);
+      OutT* drow0 = out + (static_cast<size_t>(job0.out_mat) * T + trow) * ldo + job0.out_col;
+      OutT* drow1 = out + (static_cast<size_t>(job1.out_mat) * T + trow) * ldo + job1.out_col;
+      const uint32_t taddr = tmem_base + ((q * 32) << 16) + buf * kAccCols;
+      uint32_t r[3][16];
 #pragma unroll
-      for (uint32_t col = 0; col < 64; col += 32) {
-        uint32_t r[32];
-        tmem_ld_32x32b_x32(taddr + col, r);
-        tc_wait_ld();
-        if (t < T) {
+      for (uint32_t c = 0; c < 3; ++c)
+        if (chunk0 + c < chunk1) tmem_ld_32x32b_x16(taddr + (chunk0 + c) * 16, r[c]);
+      tc_wait_ld();
+      if (t < T) {
 #pragma unroll
-          for (int h = 0; h < 2; ++h) {
+        for (uint32_t c = 0; c < 3; ++c) {
+          if (chunk0 + c < chunk1) {
+            const uint32_t col = (chunk0 + c) * 16;            // 0..127: the first 64 are job 0's features
             float v[16];
 #pragma unroll
             for (int i = 0; i < 16; ++i) {
-              const float a = __uint_as_float(r[h * 16 + i]) + bias_sm[half * 64 + col + h * 16 + i];
+              const float a = __uint_as_float(r[c][i]) + bias_sm[col + i];
               v[i] = GELU ? gelu_erf(a) : a;
             }
-            store_row16<OutT>(drow + col + h * 16, v);
+            store_row16<OutT>((col < 64 ? drow0 : drow1) + (col & 63), v);
           }
         }
       }

@@ -23,6 +23,7 @@ constexpr int kMaxSegs = 16;
 constexpr int kTableStride = 64;            // bf16 entries per segment table
 constexpr int kEpilogueWarp0 = 4;             // epilogue warps 4..11: two per TMEM lane quadrant
 constexpr int kEpilogueWarps = 8;
+constexpr int kPairEpilogueWarps = 12;        // the two-CTA kernel drains with warps 4..15: three per lane quadrant
 
 struct SmemHeader {
   uint64_t full[kMaxStages];     // activation chunk landed (TMA transaction bytes)
