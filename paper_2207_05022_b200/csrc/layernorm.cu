@@ -179,6 +179,87 @@ layernorm_rows_kernel(LnLaunch p, int tpr, int rows_per_cta) {
   }
 }
 
+// Many tokens: a warp per row, lane l holding float4 number l, l + 32, ... of it (V = d / 128 of them).  Every load of
+// a row - residual and one partial-sum plane at a time - is issued before the first use, 8 rows per CTA, and the two
+// reductions are warp shuffles: no barrier, and enough bytes in flight per SM to keep the memory system busy.
+constexpr int kLnWarpRows = 8;
+constexpr int kLnWarpMinRows = 2048;
+template <int V>
+__global__ void __launch_bounds__(kLnWarpRows * 32)
+layernorm_warp_kernel(LnLaunch p) {
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int r = blockIdx.x * kLnWarpRows + warp;
+  pdl_launch_dependents();
+  if (threadIdx.x == 0) { stamp_min(p.stamps, STAMP_FIRST_START); stamp_max(p.stamps, STAMP_LAST_START); }
+  float4 a[V];
+#pragma unroll
+  for (int v = 0; v < V; ++v) a[v] = __ldg(reinterpret_cast<const float4*>(p.bias + (lane + v * 32) * 4));
+  pdl_wait();
+  if (threadIdx.x == 0) stamp_min(p.stamps, STAMP_RELEASE);
+  if (r < p.T) {
+    const size_t row = static_cast<size_t>(r) * p.d;
+    if (p.resid_bf16) {
+      uint2 rr[V];
+#pragma unroll
+      for (int v = 0; v < V; ++v)
+        rr[v] = __ldg(reinterpret_cast<const uint2*>(static_cast<const uint16_t*>(p.resid) + row + (lane + v * 32) * 4));
+#pragma unroll
+      for (int v = 0; v < V; ++v) {
+        a[v].x += __uint_as_float(rr[v].x << 16); a[v].y += __uint_as_float(rr[v].x & 0xffff0000u);
+        a[v].z += __uint_as_float(rr[v].y << 16); a[v].w += __uint_as_float(rr[v].y & 0xffff0000u);
+      }
+    } else {
+      float4 rr[V];
+#pragma unroll
+      for (int v = 0; v < V; ++v)
+        rr[v] = __ldg(reinterpret_cast<const float4*>(static_cast<const float*>(p.resid) + row + (lane + v * 32) * 4));
+#pragma unroll
+      for (int v = 0; v < V; ++v) { a[v].x += rr[v].x; a[v].y += rr[v].y; a[v].z += rr[v].z; a[v].w += rr[v].w; }
+    }
+    const size_t pstride = static_cast<size_t>(p.T) * p.d;
+#pragma unroll 1
+    for (int q = 0; q < p.n_partial; ++q) {
+      float4 s[V];
+#pragma unroll
+      for (int v = 0; v < V; ++v)
+        s[v] = __ldg(reinterpret_cast<const float4*>(p.partial + q * pstride + row + (lane + v * 32) * 4));
+#pragma unroll
+      for (int v = 0; v < V; ++v) { a[v].x += s[v].x; a[v].y += s[v].y; a[v].z += s[v].z; a[v].w += s[v].w; }
+    }
+    float part = 0.f;
+#pragma unroll
+    for (int v = 0; v < V; ++v) part += (a[v].x + a[v].y) + (a[v].z + a[v].w);
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) part += __shfl_xor_sync(0xffffffffu, part, o);
+    const float mean = part / static_cast<float>(p.d);
+    part = 0.f;
+#pragma unroll
+    for (int v = 0; v < V; ++v) {
+      a[v].x -= mean; a[v].y -= mean; a[v].z -= mean; a[v].w -= mean;
+      part += (a[v].x * a[v].x + a[v].y * a[v].y) + (a[v].z * a[v].z + a[v].w * a[v].w);
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) part += __shfl_xor_sync(0xffffffffu, part, o);
+    const float rstd = rsqrtf(part / static_cast<float>(p.d) + p.eps);
+#pragma unroll
+    for (int v = 0; v < V; ++v) {
+      const int c = (lane + v * 32) * 4;
+      const float4 g = __ldg(reinterpret_cast<const float4*>(p.gamma + c));
+      const float4 b = __ldg(reinterpret_cast<const float4*>(p.beta + c));
+      float4 y;
+      y.x = a[v].x * rstd * g.x + b.x; y.y = a[v].y * rstd * g.y + b.y;
+      y.z = a[v].z * rstd * g.z + b.z; y.w = a[v].w * rstd * g.w + b.w;
+      if (p.out_f32) *reinterpret_cast<float4*>(p.out_f32 + row + c) = y;
+      if (p.out_bf16)
+        *reinterpret_cast<uint2*>(p.out_bf16 + row + c) = make_uint2(pack_bf16x2(y.x, y.y), pack_bf16x2(y.z, y.w));
+    }
+  }
+  if (p.stamps != nullptr) {
+    __syncthreads();
+    if (threadIdx.x == 0) stamp_max(p.stamps, STAMP_LAST_END);
+  }
+}
+
 __global__ void cast_bf16_kernel(const float* __restrict__ in, uint16_t* __restrict__ out, size_t n4,
                                  unsigned long long* stamps) {
   const size_t i = static_cast<size_t>(blockIdx.x) * blockDim.x + threadIdx.x;
@@ -220,6 +301,20 @@ cudaError_t launch_layernorm(const LnLaunch& p, cudaStream_t s, bool pdl) {
         case 4: return launch_kernel(layernorm_rows_kernel<4>, grid, block, 0, s, pdl, p, tpr, rows);
         default: break;
       }
+    }
+  }
+  if (p.T >= kLnWarpMinRows && p.d <= 1024) {      // thousands of rows: a warp per row
+    const dim3 grid((p.T + kLnWarpRows - 1) / kLnWarpRows), block(kLnWarpRows * 32);
+    switch (p.d / 128) {
+      case 1: return launch_kernel(layernorm_warp_kernel<1>, grid, block, 0, s, pdl, p);
+      case 2: return launch_kernel(layernorm_warp_kernel<2>, grid, block, 0, s, pdl, p);
+      case 3: return launch_kernel(layernorm_warp_kernel<3>, grid, block, 0, s, pdl, p);
+      case 4: return launch_kernel(layernorm_warp_kernel<4>, grid, block, 0, s, pdl, p);
+      case 5: return launch_kernel(layernorm_warp_kernel<5>, grid, block, 0, s, pdl, p);
+      case 6: return launch_kernel(layernorm_warp_kernel<6>, grid, block, 0, s, pdl, p);
+      case 7: return launch_kernel(layernorm_warp_kernel<7>, grid, block, 0, s, pdl, p);
+      case 8: return launch_kernel(layernorm_warp_kernel<8>, grid, block, 0, s, pdl, p);
+      default: break;
     }
   }
   return launch_kernel(layernorm_kernel, dim3(p.T), dim3(p.d / 4), 0, s, pdl, p);
