@@ -185,14 +185,19 @@ __device__ __forceinline__ uint32_t ld_acquire_gpu(const unsigned int* p) {
 // below 1.5e-7, three orders of magnitude under the bf16 rounding of the result) with the hardware
 // exponential; the epilogue runs it for every element of the FFN1 output.
 __device__ __forceinline__ float gelu_erf(float v) {
+  // gelu(v) = v/2 + |v|/2 * erf(|v| / sqrt 2), erf(x) = 1 - poly(t) t exp(-x^2), t = 1 / (1 + p x)
   const float x = fabsf(v) * 0.70710678118654752440f;
-  const float t = __fdividef(1.0f, fmaf(0.3275911f, x, 1.0f));
+  float t;
+  asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(t) : "f"(fmaf(0.3275911f, x, 1.0f)));
   float poly = fmaf(1.061405429f, t, -1.453152027f);
   poly = fmaf(poly, t, 1.421413741f);
   poly = fmaf(poly, t, -0.284496736f);
   poly = fmaf(poly, t, 0.254829592f);
-  const float erf_abs = 1.0f - poly * t * __expf(-x * x);
-  return 0.5f * v * (1.0f + copysignf(erf_abs, v));
+  float e;                                                   // exp(-x^2) = 2^(v^2 * (-log2(e) / 2))
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(e) : "f"((v * v) * -0.72134752044448170368f));
+  const float erf_abs = fmaf(-(poly * t), e, 1.0f);
+  const float h = 0.5f * v;
+  return fmaf(fabsf(h), erf_abs, h);
 }
 
 template <typename OutT>
