@@ -549,7 +549,7 @@ dqgemm_pair_kernel(const __grid_constant__ CUtensorMap xmap, const Job* __restri
       }
       tc_fence_before_sync();
       __syncwarp();
-      if (lane == 0) mbar_arrive_cluster(map_to_cta(smem_addr(&hdr->acc_empty[buf]), 0));
+      if (lane == 0) mbar_arrive_cluster_cta_scope(map_to_cta(smem_addr(&hdr->acc_empty[buf]), 0));
     }
   }
   if (failed) {

@@ -158,6 +158,12 @@ __device__ __forceinline__ uint32_t map_to_cta(uint32_t saddr, uint32_t rank) { 
 __device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr) {
   asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
 }
+// The same arrival with release semantics at CTA scope only: enough where the arrival hands over tensor memory
+// (ordered by the tcgen05 fences), and it does not wait for the thread's earlier global stores to reach the
+// cluster's point of coherence, which the cluster-scope form does.
+__device__ __forceinline__ void mbar_arrive_cluster_cta_scope(uint32_t cluster_addr) {
+  asm volatile("mbarrier.arrive.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+}
 __device__ __forceinline__ uint32_t cluster_nctas() {      // CTAs in this cluster (1 without a cluster launch)
   uint32_t r;
   asm volatile("mov.u32 %0, %%cluster_nctarank;" : "=r"(r));
