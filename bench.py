@@ -823,8 +823,8 @@ def spawn_ranks(n, argv, extra_env=None, port=None):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=30)
-    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--steps", type=int, default=100)
+    ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--layers", type=int, default=0, help="shorten the stack (profiler captures only)")
     ap.add_argument("--no-extras", action="store_true", help="skip the cpu baseline and single-layer extras")

@@ -57,12 +57,19 @@ __device__ __forceinline__ void load_planes(const Seg& sg, uint32_t task, uint32
 
 // Index unpack in registers -> bf16 table lookup in shared memory -> 16-byte stores into the K-major
 // core-matrix layout.  Each lane holds 128 consecutive indexes of its own row.
+// `half`: 0 = the whole quantum (four index groups), 1 / 2 = its first / second two groups only (two warps share a
+// task when a tile has fewer tasks than the CTA has warps; both hold the task's planes).
 template <int BITS>
 __device__ __forceinline__ void unpack_task(const uint32_t (&planes)[24], const Seg& sg, const uint16_t* __restrict__ tab,
-                                            uint8_t* wsm, uint32_t n_rows, uint32_t task, uint32_t lane) {
+                                            uint8_t* wsm, uint32_t n_rows, uint32_t task, uint32_t lane, uint32_t half = 0) {
   uint32_t w[4 * BITS];
 #pragma unroll
   for (int i = 0; i < 4 * BITS; ++i) w[i] = planes[i];
+  if (half == 2) {
+#pragma unroll
+    for (int i = 0; i < 2 * BITS; ++i) w[i] = planes[i + 2 * BITS];
+  }
+  const int grp0 = half == 2 ? 2 : 0, grp1 = half == 1 ? 2 : 4;
   const uint32_t chunks = sg.kc >= 128 ? sg.kc / 128 : 1;
   const uint32_t g = task / chunks, j = task % chunks;
   const bool narrow = sg.kc < 128;     // 64 in-features: the quantum is rows (l, l + 32) of a 64-row group
@@ -73,7 +80,7 @@ __device__ __forceinline__ void unpack_task(const uint32_t (&planes)[24], const 
   // quarter of the instructions of the fully unrolled form: the decode runs once per CTA, so its code is
   // fetched cold and its size is what it costs.
 #pragma unroll 1
-  for (int grp = 0; grp < 4; ++grp) {
+  for (int grp = grp0; grp < grp1; ++grp) {
     uint32_t lo[BITS];
 #pragma unroll
     for (int i = 0; i < BITS; ++i) lo[i] = w[i];
@@ -279,7 +286,11 @@ __device__ __forceinline__ void decode_weight_tile(const Job& job, const Seg* __
     n_out_total += n;
   }
   uint16_t* tab = warp_tables + warp * kTableStride;
-  for (uint32_t t = warp; t < n_tasks; t += kWarps) {
+  // a tile with at most half as many tasks as the CTA has warps: two warps share a task (half the decode latency)
+  const bool split = 2 * n_tasks <= kWarps;
+  const uint32_t n_units = split ? 2 * n_tasks : n_tasks;
+  for (uint32_t u = warp; u < n_units; u += kWarps) {
+    const uint32_t t = split ? u >> 1 : u, half = split ? 1 + (u & 1) : 0;
     const uint32_t si = t / tasks_per_seg, task = t % tasks_per_seg;
     const Seg& sg = segs[si];
     const uint32_t bits = sg.bits;
@@ -293,11 +304,11 @@ __device__ __forceinline__ void decode_weight_tile(const Job& job, const Seg* __
     tab[lane + 32] = bf16_bits(c1);
     __syncwarp();
     switch (bits) {
-      case 2: unpack_task<2>(planes, sg, tab, wsm, n_rows, task, lane); break;
-      case 3: unpack_task<3>(planes, sg, tab, wsm, n_rows, task, lane); break;
-      case 4: unpack_task<4>(planes, sg, tab, wsm, n_rows, task, lane); break;
-      case 5: unpack_task<5>(planes, sg, tab, wsm, n_rows, task, lane); break;
-      case 6: unpack_task<6>(planes, sg, tab, wsm, n_rows, task, lane); break;
+      case 2: unpack_task<2>(planes, sg, tab, wsm, n_rows, task, lane, half); break;
+      case 3: unpack_task<3>(planes, sg, tab, wsm, n_rows, task, lane, half); break;
+      case 4: unpack_task<4>(planes, sg, tab, wsm, n_rows, task, lane, half); break;
+      case 5: unpack_task<5>(planes, sg, tab, wsm, n_rows, task, lane, half); break;
+      case 6: unpack_task<6>(planes, sg, tab, wsm, n_rows, task, lane, half); break;
       default: break;
     }
     __syncwarp();                      // the table is overwritten by the warp's next task
@@ -377,49 +388,6 @@ __device__ __forceinline__ void group_barrier(uint32_t bar_id) {
   asm volatile("bar.sync %0, %1;" ::"r"(bar_id), "n"(NWARPS * 32) : "memory");
 }
 
-// Half of unpack_task: index groups [2 * half, 2 * half + 2) of the quantum, so that two warps share a task (both
-// hold the task's planes) and the decode of a small tile has the latency of half a task.
-template <int BITS>
-__device__ __forceinline__ void unpack_task_half(const uint32_t (&planes)[24], const Seg& sg, const uint16_t* __restrict__ tab,
-                                                 uint8_t* wsm, uint32_t n_rows, uint32_t task, uint32_t lane, uint32_t half) {
-  uint32_t w[2 * BITS];
-  if (half == 0) {
-#pragma unroll
-    for (int i = 0; i < 2 * BITS; ++i) w[i] = planes[i];
-  } else {
-#pragma unroll
-    for (int i = 0; i < 2 * BITS; ++i) w[i] = planes[i + 2 * BITS];
-  }
-  const uint32_t chunks = sg.kc >= 128 ? sg.kc / 128 : 1;
-  const uint32_t g = task / chunks, j = task % chunks;
-  const bool narrow = sg.kc < 128;
-  const uint32_t row0 = narrow ? g * 64 + lane : g * 32 + lane;
-  const uint32_t kcore0 = (sg.koff + (narrow ? 0 : j * 128)) >> 3;
-#pragma unroll 1
-  for (int grp = 0; grp < 2; ++grp) {
-    uint32_t lo[BITS];
-#pragma unroll
-    for (int i = 0; i < BITS; ++i) lo[i] = w[i];
-#pragma unroll
-    for (int ss = 0; ss < 4; ++ss) {
-      uint32_t pk[4];
-#pragma unroll
-      for (int e = 0; e < 4; ++e) {
-        const uint32_t c0 = extract_index_words<BITS>(lo, 8 * ss + 2 * e);
-        const uint32_t c1 = extract_index_words<BITS>(lo, 8 * ss + 2 * e + 1);
-        pk[e] = static_cast<uint32_t>(tab[c0]) | (static_cast<uint32_t>(tab[c1]) << 16);
-      }
-      const uint32_t sidx = 8 * half + 4 * grp + ss;
-      const uint32_t row = narrow ? row0 + 32 * (sidx >> 3) : row0;
-      const uint32_t kcore = narrow ? kcore0 + (sidx & 7) : kcore0 + sidx;
-      *reinterpret_cast<uint4*>(wsm + (static_cast<size_t>(kcore) * n_rows + row) * 16) =
-          make_uint4(pk[0], pk[1], pk[2], pk[3]);
-    }
-#pragma unroll
-    for (int i = 0; i < BITS; ++i) w[i] = w[i + BITS];
-  }
-}
-
 // SPLIT: every task is shared by two warps (unit u = 2 * task + half), for tiles with fewer tasks than warps.
 template <int NWARPS, bool SPLIT = false>
 __device__ __forceinline__ void decode_weight_tile_group(const Job& job, const Seg* __restrict__ segs,
@@ -461,11 +429,11 @@ __device__ __forceinline__ void decode_weight_tile_group(const Job& job, const S
     __syncwarp();
     if (SPLIT) {
       switch (bits) {
-        case 2: unpack_task_half<2>(planes, sg, tab, wsm, n_rows, task, lane, u & 1); break;
-        case 3: unpack_task_half<3>(planes, sg, tab, wsm, n_rows, task, lane, u & 1); break;
-        case 4: unpack_task_half<4>(planes, sg, tab, wsm, n_rows, task, lane, u & 1); break;
-        case 5: unpack_task_half<5>(planes, sg, tab, wsm, n_rows, task, lane, u & 1); break;
-        case 6: unpack_task_half<6>(planes, sg, tab, wsm, n_rows, task, lane, u & 1); break;
+        case 2: unpack_task<2>(planes, sg, tab, wsm, n_rows, task, lane, 1 + (u & 1)); break;
+        case 3: unpack_task<3>(planes, sg, tab, wsm, n_rows, task, lane, 1 + (u & 1)); break;
+        case 4: unpack_task<4>(planes, sg, tab, wsm, n_rows, task, lane, 1 + (u & 1)); break;
+        case 5: unpack_task<5>(planes, sg, tab, wsm, n_rows, task, lane, 1 + (u & 1)); break;
+        case 6: unpack_task<6>(planes, sg, tab, wsm, n_rows, task, lane, 1 + (u & 1)); break;
         default: break;
       }
     } else {
