@@ -75,3 +75,32 @@ def test_config5_point_sampled_sequences(plan):
         ref = O.run_workload(dataclasses.replace(work, seq_lens=[lens[b]]), x=xv[b:b + 1])
         e = rel_err(got[b:b + 1, :lens[b]], ref[:, :lens[b]])    # padded query rows carry no meaning
         assert e <= REL_TOL, (b, e)
+
+
+def test_config5_largest_bench_point_sampled_sequences():
+    # 32 x 512 = 16,384 tokens: the launch shapes bench.py times (two-CTA GEMMs, K-accumulating FFN2 with two
+    # blocks of tile pairs per CTA pair, tensor-core attention, warp-per-row LayerNorm), two layers, streamed
+    from gpu_util import rel_err, REL_TOL
+    B, L, n_layers = 32, 512, 2
+    work = W.make_config(5, n_layers=n_layers, plan="mixed", resident=False, resident_layers=1, batch=1, seq=L, workers=3)
+    rng = np.random.default_rng(6)
+    bits16, xv = round_to_bf16(rng.standard_normal((B, L, work.shape.hidden), dtype=np.float32))
+    lens = [L] * B
+    lens[5], lens[30] = 131, 400
+    x = torch.from_numpy(bits16.view(np.int16)).cuda().view(torch.bfloat16)
+    y = torch.empty_like(x)
+    lens_dev = torch.tensor(lens, dtype=torch.int32).cuda()
+    torch.cuda.synchronize()
+    with sti.Session(work, max_batch=B, max_seq=L) as s:
+        sti.sti_model_forward(s.plan, x.data_ptr(), y.data_ptr(), B, L, lens_dev.data_ptr())
+        sti.sti_sync(s.ctx)
+        y2 = torch.empty_like(x)
+        sti.sti_model_forward(s.plan, x.data_ptr(), y2.data_ptr(), B, L, lens_dev.data_ptr())   # graph replay
+        sti.sti_sync(s.ctx)
+    assert torch.equal(y.view(torch.int16), y2.view(torch.int16))
+    got = y.float().cpu().numpy().astype(np.float64)
+    assert np.isfinite(got).all()
+    for b in (0, 5, 17, 30, 31):                         # first, last, middle and the padded sequences
+        ref = O.run_workload(dataclasses.replace(work, seq_lens=[lens[b]]), x=xv[b:b + 1])
+        e = rel_err(got[b:b + 1, :lens[b]], ref[:, :lens[b]])
+        assert e <= REL_TOL, (b, e)
