@@ -281,6 +281,14 @@ sti_status sti_plan_inject(sti_plan* plan, int what, int layer, unsigned value);
 /* Bytes the plan holds: preload buffer in device memory, pinned host arena, ring slots. */
 sti_status sti_plan_memory(sti_plan* plan, uint64_t* preload_bytes, uint64_t* pinned_bytes, uint64_t* ring_bytes);
 
+/* Debugging aid (no counterpart in the paper): the preload buffer and every ring slot of the working buffer are
+ * followed (and the buffers preceded) by 256 guard bytes of a fixed pattern that nothing may write - only the upload
+ * and the per-layer copies write those buffers, each with the size the plan computed.  Waits for the plan's work on
+ * both streams, reads the guards back and returns in *damaged how many of them no longer hold the pattern (0 = intact).
+ * Together with sti_plan_inject's delayed copies this is the stream-order check of the pipeline: results and guards
+ * must not depend on when a copy reaches the copy engine.  ring_bytes of sti_plan_memory includes the guards. */
+sti_status sti_plan_check_guards(sti_plan* plan, int32_t* damaged);
+
 /* Host-only utility: re-tiles one matrix's canonical index stream (rows x cols indexes of `bits`
  * bits) into the order the device holds it (see the upload format above; the size is unchanged).
  * For every group of 32 rows (64 rows when cols == 64) and every 128-column chunk, the `bits`

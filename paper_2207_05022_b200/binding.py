@@ -88,6 +88,7 @@ def load_library():
         "sti_plan_set_overlap": ([vp, i32], i32),
         "sti_get_stats": ([vp, C.POINTER(StiStats)], i32),
         "sti_plan_memory": ([vp, u64p, u64p, u64p], i32),
+        "sti_plan_check_guards": ([vp, C.POINTER(C.c_int32)], i32),
         "sti_plan_inject": ([vp, i32, i32, C.c_uint], i32),
         "sti_plan_retain": ([vp, vp, vp, u64p], i32),
         "sti_shard_adopt": ([vp, vp, i32, i32, i32], i32),
@@ -110,7 +111,7 @@ EXPORTED = ("sti_ctx_create", "sti_ctx_destroy", "sti_ctx_set_layer_params", "st
             "sti_plan_destroy", "sti_shard_upload", "sti_plan_finalize", "sti_layer_forward",
             "sti_model_forward", "sti_model_forward_host", "sti_sync", "sti_shard_decode", "sti_gemm_probe", "sti_decode_rate_probe", "sti_get_kernel_stamps", "sti_plan_inject",
             "sti_plan_retain", "sti_shard_adopt", "sti_plan_fill_stats",
-            "sti_plan_set_profiling", "sti_plan_set_overlap", "sti_get_stats", "sti_plan_memory", "sti_ctx_launch_count",
+            "sti_plan_set_profiling", "sti_plan_set_overlap", "sti_get_stats", "sti_plan_memory", "sti_plan_check_guards", "sti_ctx_launch_count",
             "sti_host_retile", "sti_strerror", "sti_matrix_decode_noalloc", "sti_plan_auto",
             "sti_preload_after_run", "sti_quantize_units", "sti_quantize_workspace_bytes")
 
@@ -256,6 +257,13 @@ def sti_get_stats(plan: int) -> StiStats:
     st = StiStats()
     _check(load_library().sti_get_stats(C.c_void_p(plan), C.byref(st)), "sti_get_stats")
     return st
+
+
+def sti_plan_check_guards(plan: int) -> int:
+    """Number of damaged guard regions around the preload buffer and the ring slots (0 = intact; see sti.h)."""
+    n = C.c_int32(-1)
+    _check(load_library().sti_plan_check_guards(C.c_void_p(plan), C.byref(n)), "sti_plan_check_guards")
+    return int(n.value)
 
 
 def sti_plan_memory(plan: int):

@@ -22,6 +22,10 @@ namespace {
 
 constexpr int kMaxLayersStats = 64;
 constexpr size_t kMaxSmem = 227 * 1024;
+// Guard words around the preload buffer and around every ring slot: nothing may ever write them (only the layer
+// copies and the upload write those buffers), sti_plan_check_guards reads them back.
+constexpr size_t kGuardBytes = 256;
+constexpr int kGuardPattern = 0xA5;
 constexpr int kStampKernels = 8;       // per layer: cast, QKV, attention, O projection, LayerNorm 1, FFN1, FFN2, LayerNorm 2
 constexpr int kStampRecord = 8;        // 64-bit words per kernel launch (kStampWords of the device code)
 
@@ -132,7 +136,8 @@ struct sti_plan {
   Tuning tune;
   uint8_t* preload = nullptr;  size_t preload_bytes = 0;
   uint8_t* pinned = nullptr;   size_t pinned_bytes = 0;
-  uint8_t* ring = nullptr;     size_t slot_bytes = 0;
+  uint8_t* ring = nullptr;     size_t slot_bytes = 0;      // a slot = its data followed by kGuardBytes of guard pattern
+  uint8_t* ring_alloc = nullptr; uint8_t* preload_alloc = nullptr;   // the allocations: a leading guard, then `ring` / `preload`
   uint8_t* tables = nullptr;   size_t tables_bytes = 0;       // job/segment descriptors
   std::vector<cudaEvent_t> slot_free, g_slot_free;   // direct launches / graph capture
   cudaEvent_t ev_copy_tail = nullptr, ev_begin = nullptr, ev_end = nullptr, ev_fork = nullptr, g_ev_join = nullptr;
@@ -808,7 +813,7 @@ sti_status model_forward_impl(sti_plan* p, const ForwardKey& k) {
 
 void free_plan_device(sti_plan* p) {
   if (!p) return;
-  cudaFree(p->preload); cudaFree(p->ring); cudaFree(p->tables); cudaFree(p->retain_arena);
+  cudaFree(p->preload_alloc); cudaFree(p->ring_alloc); cudaFree(p->tables); cudaFree(p->retain_arena);
   if (p->pinned) cudaFreeHost(p->pinned);
   cudaFree(p->qkv); cudaFree(p->attn_out); cudaFree(p->partial); cudaFree(p->h1_f32); cudaFree(p->h1_bf16);
   cudaFree(p->u); cudaFree(p->x_bf16); cudaFree(p->buf[0]); cudaFree(p->buf[1]); cudaFree(p->x_in); cudaFree(p->y_out);
@@ -1064,7 +1069,7 @@ sti_status sti_plan_finalize(sti_plan* p) {
     for (auto& u : L.ffn) if (!place(u)) return STI_ERR_SHARD_MISSING;
     preload_total += align256(L.res_bytes);
     pinned_total += align256(L.str_bytes);
-    slot_bytes = std::max(slot_bytes, align256(L.str_bytes));
+    if (L.str_bytes) slot_bytes = std::max(slot_bytes, align256(L.str_bytes) + kGuardBytes);
     if (L.str_bytes) L.slot = (n_streamed++) % p->ring_slots;
     p->n_streamed_layers = n_streamed;
     max_heads = std::max<int>(max_heads, L.kept_heads.size());
@@ -1072,12 +1077,20 @@ sti_status sti_plan_finalize(sti_plan* p) {
   }
   p->attempted = true;
   p->preload_bytes = preload_total; p->pinned_bytes = pinned_total; p->slot_bytes = slot_bytes;
-  if (preload_total) CUDA_TRY(cudaMalloc(&p->preload, preload_total));
+  if (preload_total) {
+    CUDA_TRY(cudaMalloc(&p->preload_alloc, preload_total + 2 * kGuardBytes));
+    CUDA_TRY(cudaMemset(p->preload_alloc, kGuardPattern, preload_total + 2 * kGuardBytes));
+    p->preload = p->preload_alloc + kGuardBytes;
+  }
   if (pinned_total) {
     if (p->fail_pinned_alloc) return STI_ERR_OOM;          // injected allocation failure
     CUDA_TRY(cudaMallocHost(&p->pinned, pinned_total));
   }
-  if (slot_bytes) CUDA_TRY(cudaMalloc(&p->ring, slot_bytes * p->ring_slots));
+  if (slot_bytes) {
+    CUDA_TRY(cudaMalloc(&p->ring_alloc, kGuardBytes + slot_bytes * p->ring_slots));
+    CUDA_TRY(cudaMemset(p->ring_alloc, kGuardPattern, kGuardBytes + slot_bytes * p->ring_slots));
+    p->ring = p->ring_alloc + kGuardBytes;
+  }
   // 2. fill the preload buffer (device) and the pinned arena (host), one contiguous blob per layer
   size_t pre_cur = 0, pin_cur = 0;
   std::vector<uint8_t> staging;
@@ -1589,6 +1602,34 @@ sti_status sti_plan_memory(sti_plan* p, uint64_t* preload_bytes, uint64_t* pinne
   if (preload_bytes) *preload_bytes = p->preload_bytes;
   if (pinned_bytes) *pinned_bytes = p->pinned_bytes;
   if (ring_bytes) *ring_bytes = p->slot_bytes * p->ring_slots;
+  return STI_OK;
+}
+
+sti_status sti_plan_check_guards(sti_plan* p, int32_t* damaged) {
+  if (!p || !damaged) return STI_ERR_ARG;
+  if (!p->finalized) return STI_ERR_STATE;
+  sti_ctx* c = p->ctx;
+  CUDA_TRY(cudaSetDevice(c->device));
+  CUDA_TRY(cudaStreamSynchronize(c->copy));
+  CUDA_TRY(cudaStreamSynchronize(c->compute));
+  std::vector<const uint8_t*> guards;
+  if (p->preload_alloc) {
+    guards.push_back(p->preload_alloc);
+    guards.push_back(p->preload + p->preload_bytes);
+  }
+  if (p->ring_alloc) {
+    guards.push_back(p->ring_alloc);
+    for (int i = 1; i <= p->ring_slots; ++i) guards.push_back(p->ring + static_cast<size_t>(i) * p->slot_bytes - kGuardBytes);
+  }
+  uint8_t host[kGuardBytes];
+  int bad = 0;
+  for (const uint8_t* g : guards) {
+    CUDA_TRY(cudaMemcpy(host, g, kGuardBytes, cudaMemcpyDeviceToHost));
+    bool ok = true;
+    for (size_t i = 0; i < kGuardBytes; ++i) ok = ok && host[i] == static_cast<uint8_t>(kGuardPattern);
+    if (!ok) ++bad;
+  }
+  *damaged = bad;
   return STI_OK;
 }
 

@@ -91,3 +91,39 @@ def test_bad_argument_does_not_change_later_forwards():
         assert e.value.status == 1
         assert sti.sti_ctx_launch_count(s.ctx) == launches   # nothing was launched for the refused call
         assert torch.equal(_forward(s, work, x), y0)
+
+
+def test_randomised_copy_delays_change_neither_results_nor_guard_words():
+    # stream-order check of the pipeline: whenever a layer's copy reaches the copy engine, the layer computes on
+    # its own bytes (two ring slots for seven streamed layers, so every slot is reused three times per forward),
+    # and nothing writes past a slot or past the preload buffer
+    work = _work(n_layers=8, resident_layers=1)
+    x = torch.from_numpy(work.x_dev).cuda()
+    rng = np.random.default_rng(8)
+    with sti.Session(work) as s:
+        assert sti.sti_plan_check_guards(s.plan) == 0          # right after the upload
+        y_ref = _forward(s, work, x)
+        assert sti.sti_plan_check_guards(s.plan) == 0
+        sti.sti_plan_set_profiling(s.plan, 1)                  # forwards launched kernel by kernel: delays apply
+        for _ in range(12):
+            layer = int(rng.integers(1, 8))
+            sti.sti_plan_inject(s.plan, sti.STI_INJECT_SLOW_COPY, layer, int(rng.integers(50, 1500)))
+            y = _forward(s, work, x)
+            assert torch.equal(y, y_ref), layer
+            st = sti.sti_get_stats(s.plan)
+            assert all(st.streamed_bytes[l] > 0 for l in range(1, 8)) and st.streamed_bytes[0] == 0
+        sti.sti_plan_inject(s.plan, sti.STI_INJECT_NONE)
+        sti.sti_plan_set_profiling(s.plan, 0)
+        assert torch.equal(_forward(s, work, x), y_ref)
+        assert sti.sti_plan_check_guards(s.plan) == 0
+        mem = sti.sti_plan_memory(s.plan)
+        assert mem["ring_bytes"] > 0 and mem["preload_bytes"] > 0
+
+
+def test_guard_words_of_a_fully_resident_plan():
+    work = _work(n_layers=2, resident_layers=2)
+    x = torch.from_numpy(work.x_dev).cuda()
+    with sti.Session(work) as s:
+        _forward(s, work, x)
+        assert sti.sti_plan_check_guards(s.plan) == 0
+        assert sti.sti_plan_memory(s.plan)["ring_bytes"] == 0
