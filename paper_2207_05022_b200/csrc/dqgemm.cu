@@ -35,21 +35,17 @@ namespace {
 // unrolled (each thread writes 128 or 64 contiguous bytes of its row).
 template <typename OutT, bool GELU, bool FEW>
 __device__ __forceinline__ void epilogue_tile(uint32_t taddr, uint32_t half, uint32_t ncol, const float* bias_sm, OutT* drow,
-                                              bool row_ok, uint32_t acc2_off = 0) {
+                                              bool row_ok) {
   if constexpr (FEW) {
-    // acc2_off != 0: the tile was accumulated by two MMA issuers into two accumulators, acc2_off columns apart
 #pragma unroll 1
     for (uint32_t col = half * ncol; col < (half + 1) * ncol; col += 8) {
-      uint32_t r[8], r2[8];
+      uint32_t r[8];
       tmem_ld_32x32b_x8(taddr + col, r);
-      if (acc2_off) tmem_ld_32x32b_x8(taddr + acc2_off + col, r2);
       tc_wait_ld();
       float v[8];
 #pragma unroll
       for (int i = 0; i < 8; ++i) {
-        float a = __uint_as_float(r[i]);
-        if (acc2_off) a += __uint_as_float(r2[i]);
-        a += bias_sm[col + i];
+        const float a = __uint_as_float(r[i]) + bias_sm[col + i];
         v[i] = GELU ? gelu_erf(a) : a;
       }
       if constexpr (sizeof(OutT) == 2) {
@@ -162,13 +158,8 @@ dqgemm_kernel(const __grid_constant__ CUtensorMap xmap, const Job* __restrict__ 
     if (++p_kc == n_chunks) { p_kc = 0; ++p_ti; }
   };
 
-  // Few token tiles per CTA: the MMA phase is bound by the rate at which ONE warp can issue tcgen05.mma (about 80
-  // cycles per instruction here, against 34 cycles of tensor time at N = 64), so two warps issue, each the chunks of
-  // its own parity into its own accumulator; the epilogue adds the two.
-  const bool dual = FEW && n_chunks >= 2;
-  const uint32_t n_iss = dual ? 2 : 1;
   uint32_t tmem_cols = 32;
-  while (tmem_cols < 2 * n_iss * n_rows) tmem_cols <<= 1;       // two accumulator buffers (per issuer)
+  while (tmem_cols < 2 * n_rows) tmem_cols <<= 1;       // two accumulators
   if constexpr (!SIMT) {
     if (tid == 0) {
       for (uint32_t s = 0; s < n_stages; ++s) {
@@ -176,11 +167,10 @@ dqgemm_kernel(const __grid_constant__ CUtensorMap xmap, const Job* __restrict__ 
         mbar_init(smem_addr(&hdr->empty[s]), 1);
       }
       for (int b = 0; b < 2; ++b) {
-        mbar_init(smem_addr(&hdr->acc_full[b]), n_iss);               // one commit per issuer
+        mbar_init(smem_addr(&hdr->acc_full[b]), 1);
         mbar_init(smem_addr(&hdr->acc_empty[b]), kEpilogueWarps);     // one arrival per epilogue warp
       }
       mbar_init(smem_addr(&hdr->drain), 1);
-      mbar_init(smem_addr(&hdr->drain2), 1);
       hdr->abort = 0;
       mbar_fence_init();
       fence_proxy_async_smem();
@@ -263,9 +253,8 @@ dqgemm_kernel(const __grid_constant__ CUtensorMap xmap, const Job* __restrict__ 
         }
       }
       __syncwarp();
-    } else if (warp == 1 || (dual && warp == kSecondIssuerWarp)) {
-      // ---- MMA issuer(s).  Descriptors are built once; per instruction only their start address moves.
-      const uint32_t iss = warp == 1 ? 0u : 1u;
+    } else if (warp == 1) {
+      // ---- MMA issuer.  Descriptors are built once; per instruction only their start address moves.
       const uint32_t idesc = umma_idesc_bf16_m128(n_rows);
       const uint32_t w_lbo = n_rows * 16;
       const uint64_t a_desc0 = umma_smem_desc_sw128(xsm_addr);
@@ -276,13 +265,10 @@ dqgemm_kernel(const __grid_constant__ CUtensorMap xmap, const Job* __restrict__ 
       const uint32_t b_chunk_step = 4 * b_ks_step;             // next 64 columns
       // The whole warp runs the loop converged; one elected lane issues.
       uint32_t stage = 0, phase = 0, kc = 0, kcr = rot, ti = 0, issued = 0;
-      // this issuer's last chunk of a tile: the largest kc < n_chunks of its parity
-      const uint32_t last_kc = ((n_chunks - 1 - iss) / n_iss) * n_iss + iss;
       for (uint32_t c = 0; c < total; ++c) {
         const uint32_t buf = ti & 1;
-        if (kc % n_iss == iss) {
         bool ok = true;
-        if (kc == iss && ti >= 2)      // the epilogue must have drained this accumulator
+        if (kc == 0 && ti >= 2)        // the epilogue must have drained this accumulator
           ok = __all_sync(0xffffffffu, mbar_wait_bounded(smem_addr(&hdr->acc_empty[buf]), ((ti >> 1) - 1) & 1));
         if (ok) ok = __all_sync(0xffffffffu, mbar_wait_bounded(smem_addr(&hdr->full[stage]), phase));
         if (!ok) { failed = true; break; }
@@ -291,32 +277,30 @@ dqgemm_kernel(const __grid_constant__ CUtensorMap xmap, const Job* __restrict__ 
         const uint32_t nb = n_boxes - box0 < bps ? n_boxes - box0 : bps;
         const uint64_t da0 = a_desc0 + stage * a_stage_step;
         const uint64_t db0 = b_desc0 + box0 * b_chunk_step;
-        const uint32_t d_addr = tmem_base + (buf * n_iss + iss) * n_rows;
+        const uint32_t d_addr = tmem_base + buf * n_rows;
         if (elect_one()) {
           uint64_t da = da0, db = db0;
           // per box: four K = 16 steps, +32 bytes inside the swizzled activation row, +2 core-matrix columns of W
-          umma_bf16_ss_x4(d_addr, da, db, 2, b_ks_step, idesc, kc >= n_iss ? 1u : 0u);
+          umma_bf16_ss_x4(d_addr, da, db, 2, b_ks_step, idesc, kc != 0 ? 1u : 0u);
           for (uint32_t b = 1; b < nb; ++b) {
             da += a_box_step;
             db += b_chunk_step;
             umma_bf16_ss_x4(d_addr, da, db, 2, b_ks_step, idesc, 1u);
           }
           if (c + n_stages < total) umma_commit(smem_addr(&hdr->empty[stage]));   // only if the stage is refilled
-          if (kc == last_kc) umma_commit(smem_addr(&hdr->acc_full[buf]));
+          if (kc + 1 == n_chunks) umma_commit(smem_addr(&hdr->acc_full[buf]));
         }
         __syncwarp();
         issued = c + 1;
-        }
         if (++stage == n_stages) { stage = 0; phase ^= 1; }
         if (++kcr == n_chunks) kcr = 0;
         if (++kc == n_chunks) { kc = 0; ++ti; }
       }
       if (failed && issued > 0) {
         // outstanding MMAs: a commit of its own and one more bounded chance before TMEM is freed
-        const uint32_t drain_bar = smem_addr(iss == 0 ? &hdr->drain : &hdr->drain2);
-        if (elect_one()) umma_commit(drain_bar);
+        if (elect_one()) umma_commit(smem_addr(&hdr->drain));
         __syncwarp();
-        (void)mbar_wait_bounded(drain_bar, 0);
+        (void)mbar_wait_bounded(smem_addr(&hdr->drain), 0);
       }
     } else if (warp == 2 || warp == 3) {
       // ---- otherwise idle: pull the packed shards of a later launch into L2
@@ -336,19 +320,18 @@ dqgemm_kernel(const __grid_constant__ CUtensorMap xmap, const Job* __restrict__ 
         tc_fence_after_sync();
         const int t = static_cast<int>((blockIdx.y + ti * gridDim.y) * kTileM + q * 32 + lane);
         const size_t row_off = (static_cast<size_t>(job.out_mat) * T + (t < T ? t : 0)) * ldo + job.out_col;
-        const uint32_t taddr = tmem_base + ((q * 32) << 16) + buf * n_iss * n_rows;
-        const uint32_t acc2 = dual ? n_rows : 0u;
+        const uint32_t taddr = tmem_base + ((q * 32) << 16) + buf * n_rows;
         if constexpr (std::is_void<OutT>::value) {
           // one kernel for every GEMM of a layer: the output kind is a launch parameter, the code stays in the
           // instruction caches from launch to launch
           if (kind == GEMM_BF16_TO_F32)
-            epilogue_tile<float, false, FEW>(taddr, half, ncol, bias_sm, static_cast<float*>(out) + row_off, t < T, acc2);
+            epilogue_tile<float, false, FEW>(taddr, half, ncol, bias_sm, static_cast<float*>(out) + row_off, t < T);
           else if (kind == GEMM_BF16_TO_BF16_GELU)
-            epilogue_tile<__nv_bfloat16, true, FEW>(taddr, half, ncol, bias_sm, static_cast<__nv_bfloat16*>(out) + row_off, t < T, acc2);
+            epilogue_tile<__nv_bfloat16, true, FEW>(taddr, half, ncol, bias_sm, static_cast<__nv_bfloat16*>(out) + row_off, t < T);
           else
-            epilogue_tile<__nv_bfloat16, false, FEW>(taddr, half, ncol, bias_sm, static_cast<__nv_bfloat16*>(out) + row_off, t < T, acc2);
+            epilogue_tile<__nv_bfloat16, false, FEW>(taddr, half, ncol, bias_sm, static_cast<__nv_bfloat16*>(out) + row_off, t < T);
         } else {
-          epilogue_tile<OutT, GELU, FEW>(taddr, half, ncol, bias_sm, out + row_off, t < T, acc2);
+          epilogue_tile<OutT, GELU, FEW>(taddr, half, ncol, bias_sm, out + row_off, t < T);
         }
         tc_fence_before_sync();
         __syncwarp();

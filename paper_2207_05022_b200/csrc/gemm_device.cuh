@@ -23,7 +23,6 @@ constexpr int kMaxSegs = 16;
 constexpr int kTableStride = 64;            // bf16 entries per segment table
 constexpr int kEpilogueWarp0 = 4;             // epilogue warps 4..11: two per TMEM lane quadrant
 constexpr int kEpilogueWarps = 8;
-constexpr int kSecondIssuerWarp = 12;         // one-CTA kernel, few token tiles: a second MMA-issuing warp
 constexpr int kPairEpilogueWarps = 12;        // the two-CTA kernel drains with warps 4..15: three per lane quadrant
 
 struct SmemHeader {
@@ -32,7 +31,6 @@ struct SmemHeader {
   uint64_t acc_full[2];          // accumulator buffer complete
   uint64_t acc_empty[2];         // accumulator buffer drained by the epilogue warps
   uint64_t drain;                // failure path only: all issued MMAs have completed
-  uint64_t drain2;               // ... of the second issuer
   uint32_t tmem_base;
   volatile uint32_t abort;       // a bounded wait ran out somewhere in the CTA
 };
