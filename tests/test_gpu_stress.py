@@ -47,3 +47,20 @@ def test_queued_forwards_meet_every_wait_and_repeat_bit_for_bit(batch, seq, resi
         sti.sti_sync(s.ctx)                                   # raises if a device-side wait ran out
         for y in ys:
             assert torch.equal(y.view(torch.int16), y0.view(torch.int16))
+
+
+@pytest.mark.parametrize("seq", [128, 256, 512])
+def test_queued_forwards_bert_base_layers(seq):
+    # hidden 768: rings of four stages, so both MMA-issuing warps are at work in every GEMM of the layer
+    work = W.make_config(3, n_layers=4, seq=seq, workers=3)          # fp32 activations, layers 0-2 preloaded
+    x = torch.from_numpy(work.x_dev).cuda()
+    with sti.Session(work) as s:
+        y0 = torch.empty_like(x)
+        sti.sti_model_forward(s.plan, x.data_ptr(), y0.data_ptr(), work.batch, seq)
+        sti.sti_sync(s.ctx)
+        ys = [torch.empty_like(x) for _ in range(3)]
+        for i in range(400):
+            sti.sti_model_forward(s.plan, x.data_ptr(), ys[i % 3].data_ptr(), work.batch, seq)
+        sti.sti_sync(s.ctx)
+        for y in ys:
+            assert torch.equal(y.view(torch.int32), y0.view(torch.int32))
