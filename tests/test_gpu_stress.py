@@ -51,7 +51,7 @@ def test_queued_forwards_meet_every_wait_and_repeat_bit_for_bit(batch, seq, resi
 
 @pytest.mark.parametrize("seq", [128, 256, 512])
 def test_queued_forwards_bert_base_layers(seq):
-    # hidden 768: rings of four stages, so both MMA-issuing warps are at work in every GEMM of the layer
+    # hidden 768: 96 KB weight tiles, rings of four two-box stages, 12 K boxes per tile (a ragged last ring round)
     work = W.make_config(3, n_layers=4, seq=seq, workers=3)          # fp32 activations, layers 0-2 preloaded
     x = torch.from_numpy(work.x_dev).cuda()
     with sti.Session(work) as s:
