@@ -435,21 +435,91 @@ def run_planner(args):
         rows.append(execute(plan, target_ms))
 
     # back-to-back executions (Section 3.2): the buffer grows between runs, the shards already loaded stay
-    # cached bottom-up, and the next plan spends the freed IO time on higher versions of the rest
+    # cached bottom-up ON THE DEVICE (sti_plan_retain / sti_shard_adopt: one context, the next plan takes over what
+    # the previous one holds and uploads only the rest), and the next plan spends the freed IO time on higher
+    # versions of the other shards
     series = []
     target_ms = targets[-1]
-    plan = None
-    for mb in [float(v) for v in args.planner_series_mb.split(",")]:
-        if plan is None:
-            plan = sti.sti_plan_auto(target_ms * 1e3, N, M, t_comp_us, t_io_us, shard_bytes, importance,
-                                     int(mb * (1 << 20)))
-        else:
-            cached, used = sti.sti_preload_after_run(plan["keep"], plan["bits"], shard_bytes, int(mb * (1 << 20)))
-            plan = sti.sti_plan_auto(target_ms * 1e3, N, M, t_comp_us, t_io_us, shard_bytes, importance,
-                                     int(mb * (1 << 20)), cached)
-        row = execute(plan, target_ms)
-        row["buffer_mb"] = mb
-        series.append(row)
+    buffers = [int(float(v) * (1 << 20)) for v in args.planner_series_mb.split(",")]
+    plan, prev, ctx = None, None, 0
+    plans_alive = []
+    try:
+        for step, buf in enumerate(buffers):
+            cached = None
+            if plan is not None:
+                cached, _ = sti.sti_preload_after_run(plan["keep"], plan["bits"], shard_bytes, buf)
+            plan = sti.sti_plan_auto(target_ms * 1e3, N, M, t_comp_us, t_io_us, shard_bytes, importance, buf, cached)
+            streamed_layers = int(((plan["keep"] > 0) & (plan["preload"] == 0)).any(axis=1).sum())
+            work = W.make_planned(plan["keep"], plan["bits"], plan["preload"], batch=B, seq=L, workers=workers,
+                                  ring_slots=max(2, min(ring, streamed_layers)))
+            sh = work.shape
+            desc = sti.StiModelDesc(n_layers=sh.n_layers, hidden=sh.hidden, n_heads=sh.n_heads, head_dim=sh.head_dim,
+                                    ffn=sh.ffn, n_ffn_slices=sh.n_ffn_slices, max_batch=B, max_seq=L,
+                                    act_dtype=sti.STI_BF16 if work.act_dtype == "bf16" else sti.STI_F32,
+                                    ln_eps=work.ln_eps)
+            if not ctx:
+                ctx = sti.sti_ctx_create(desc, 0, stream.cuda_stream)
+                for l, p in enumerate(work.dense):
+                    sti.sti_ctx_set_layer_params(ctx, l, p["bq"], p["bk"], p["bv"], p["bo"], p["b1"], p["b2"],
+                                                 p["ln1_g"], p["ln1_b"], p["ln2_g"], p["ln2_b"])
+            attn = [(u.keep, u.bits, u.resident) for layer in work.attn_plan for u in layer]
+            ffn = [(u.keep, u.bits, u.resident) for layer in work.ffn_plan for u in layer]
+            handle = sti.sti_plan_create(ctx, attn, ffn, work.ring_slots)
+            plans_alive.append(handle)
+            for (l, kind, idx), b in work.blobs.items():
+                if cached is not None and cached[l][idx] != 0:
+                    sti.sti_shard_adopt(handle, prev, l, kind, idx)
+                else:
+                    sti.sti_shard_upload(handle, l, kind, idx, b.bits, b.codes, b.centroids, b.outlier_off, b.outlier_val)
+            sti.sti_plan_finalize(handle)
+            fill = sti.sti_plan_fill_stats(handle)
+            if prev:                                            # the previous plan has handed its shards over
+                sti.sti_plan_destroy(prev)
+                plans_alive.remove(prev)
+            x = device_act(torch, work)
+            y = torch.empty_like(x)
+            retained = 0
+            if step + 1 < len(buffers):                         # what the next execution will find cached stays on the device
+                keep_next, _ = sti.sti_preload_after_run(plan["keep"], plan["bits"], shard_bytes, buffers[step + 1])
+                mask = (keep_next != 0).astype(np.uint8)
+                retained = sti.sti_plan_retain(handle, mask, mask)
+            ms = []
+            with torch.cuda.stream(stream):
+                for i in range(3 + args.steps):
+                    flush.zero_()
+                    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                    e0.record(stream)
+                    sti.sti_model_forward(handle, x.data_ptr(), y.data_ptr(), B, L)
+                    e1.record(stream)
+                    stream.synchronize()
+                    if i >= 3:
+                        ms.append(e0.elapsed_time(e1))
+            sti.sti_plan_set_profiling(handle, 1)
+            stall = []
+            with torch.cuda.stream(stream):
+                for _ in range(5):
+                    flush.zero_()
+                    sti.sti_model_forward(handle, x.data_ptr(), y.data_ptr(), B, L)
+                    st = sti.sti_get_stats(handle)
+                    stall.append(sum(st.stall_us[:st.n_layers]))
+            sti.sti_plan_set_profiling(handle, 0)
+            sti.sti_sync(ctx)
+            kept_bits = plan["bits"][plan["keep"] > 0]
+            series.append({"buffer_mb": buf / (1 << 20), "n": plan["n"], "m": plan["m"], "pass1_bits": plan["pass1_bits"],
+                           "bits_hist": {int(b): int((kept_bits == b).sum()) for b in np.unique(kept_bits)},
+                           "mean_bits": float(kept_bits.astype(np.float64).mean()),
+                           "preloaded_shards": int(plan["preload"].sum()),
+                           "cached_shards_taken_over": 0 if cached is None else int((cached != 0).sum()),
+                           "uploaded_bytes": fill["uploaded_bytes"], "adopted_bytes": fill["adopted_bytes"],
+                           "retained_bytes_for_next": int(retained),
+                           "measured_ms": float(np.median(ms)), "meets_target": bool(np.median(ms) <= target_ms),
+                           "stall_ms": float(np.median(stall)) * 1e-3})
+            prev = handle
+    finally:
+        for h in plans_alive:
+            sti.sti_plan_destroy(h)
+        if ctx:
+            sti.sti_ctx_destroy(ctx)
 
     print(json.dumps({"planner": "two-stage planner on profiled device tables, BERT-large 24x16 store",
                       "batch": B, "seq": L, "preload_budget_bytes": preload_bytes, "h2d_GBps": h2d_gbps,
