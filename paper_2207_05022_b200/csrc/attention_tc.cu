@@ -78,7 +78,7 @@ __device__ __forceinline__ float fast_exp2(float x) {
   return y;
 }
 
-// One lane polls, the warp takes its verdict (keeps the barrier word free of a warp's worth of pollers).  The poll
+// One lane polls, the warp takes its result (keeps the barrier word free of a warp's worth of pollers).  The poll
 // does not sleep: these waits sit on the per-chunk critical path and are short.
 __device__ __forceinline__ bool warp_wait(uint32_t bar, uint32_t parity, uint32_t lane) {
   uint32_t ok = 1;

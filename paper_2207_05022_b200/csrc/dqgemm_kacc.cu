@@ -272,7 +272,7 @@ dqgemm_kacc_kernel(const __grid_constant__ CUtensorMap xmap, const Job* __restri
     const uint32_t gtid = tid - kKaccGroupWarp0 * 32;
     const uint32_t q = warp & 3, half = (warp - kKaccGroupWarp0) >> 2;
     bool released = false;
-    // lane 0 polls and the warp takes its verdict; once the CTA has given up nobody waits any more
+    // lane 0 polls and the warp takes its result; once the CTA has given up nobody waits any more
     auto wait_uniform = [&](uint32_t bar, uint32_t parity) {
       uint32_t ok = 1;
       if (lane == 0) ok = (failed || hdr->abort) ? 0u : (mbar_wait_bounded(bar, parity) ? 1u : 0u);
