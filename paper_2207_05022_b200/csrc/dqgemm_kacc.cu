@@ -28,6 +28,7 @@ constexpr uint32_t kKaccAccCols = 128;                // columns of one accumula
 constexpr uint32_t kKaccTmemCols = kKaccTiles * kKaccAccCols;
 constexpr int kKaccMaxStages = 12;
 constexpr int kKaccGroupWarp0 = 4, kKaccGroupWarps = 8;
+constexpr int kKaccPrefetchWarp0 = 12;               // warps 12-15: L2 prefetch of the activation stream
 constexpr uint32_t kKaccGroupBarrier = 1;
 
 struct KaccHeader {
@@ -60,7 +61,8 @@ __device__ __forceinline__ void fence_acq_rel_cluster() { asm volatile("fence.ac
 template <bool SPLIT>
 __global__ void __launch_bounds__(kThreads, 1)
 dqgemm_kacc_kernel(const __grid_constant__ CUtensorMap xmap, const Job* __restrict__ jobs, const Seg* __restrict__ segs,
-                   int n_groups, int T, float* __restrict__ out, int ldo, int* __restrict__ err, uint32_t n_stages,
+                   const __nv_bfloat16* __restrict__ x, int ldx, int n_groups, int T, float* __restrict__ out, int ldo,
+                   int* __restrict__ err, uint32_t n_stages,
                    uint32_t bps, uint32_t w_buf_bytes, uint32_t hdr_bytes, uint32_t seg_stride,
                    unsigned long long* stamps) {
   extern __shared__ __align__(1024) uint8_t smem_raw[];
@@ -267,6 +269,37 @@ dqgemm_kacc_kernel(const __grid_constant__ CUtensorMap xmap, const Job* __restri
         (void)mbar_wait_bounded(smem_addr(&hdr->drain), 0);
       }
     }
+  } else if (warp >= kKaccPrefetchWarp0 && x != nullptr) {
+    // ---- otherwise idle: pull the activations of the step after next into L2 (the host passes x only when the
+    // operand is larger than L2: 16,384 tokens x 4096 columns of bf16 are 134 MB).  Without this every box's first
+    // reader - and the seven other column pairs
+    // that ask for the same lines at the same moment - waits for DRAM.  The column pairs share the work: pair p
+    // takes the boxes p, p + n_pairs, ... of a K group, each thread one 128-byte line of one token row.  Paced by the
+    // same barrier as the decode (a weight buffer is free = the step two back has been computed).
+    pdl_wait();
+    const uint32_t n_pairs = gridDim.x >> 1, pair = blockIdx.x >> 1;
+    const uint32_t r_in_tile = (warp - kKaccPrefetchWarp0) * 32 + lane;        // 0..127: the CTA's rows of a tile
+    uint32_t step = 0;
+    for (uint32_t blk = 0; blk < n_blocks && !failed; ++blk) {
+      const uint32_t nt = tiles_in(blk);
+      for (int g = 0; g < n_groups; ++g, ++step) {
+        if (step >= 2) {
+          uint32_t ok = 1;
+          if (lane == 0) ok = hdr->abort ? 0u : (mbar_wait_bounded_relaxed(smem_addr(&hdr->w_empty[step & 1]), ((step >> 1) - 1) & 1) ? 1u : 0u);
+          ok = __shfl_sync(0xffffffffu, ok, 0);
+          if (!ok) { failed = true; break; }
+        }
+        const uint32_t nb = ginfo[g].n_boxes, x_koff = ginfo[g].x_koff;
+        for (uint32_t t = 0; t < nt; ++t) {
+          const int row = tile_row0(blk * kKaccTiles + t) + static_cast<int>(r_in_tile);
+          if (row < T) {
+            const __nv_bfloat16* line = x + static_cast<size_t>(row) * ldx + x_koff;
+            for (uint32_t b = pair; b < nb; b += n_pairs)
+              asm volatile("prefetch.global.L2 [%0];" ::"l"(line + b * kChunkK));
+          }
+        }
+      }
+    }
   } else if (warp >= kKaccGroupWarp0 && warp < kKaccGroupWarp0 + kKaccGroupWarps) {
     // ---- decode group / epilogue.  No early exit: the group meets at named barriers inside the decode.
     const uint32_t gtid = tid - kKaccGroupWarp0 * 32;
@@ -379,9 +412,9 @@ cudaError_t launch_gemm_kacc(const KaccLaunch& p, cudaStream_t s) {
   cfg.numAttrs = p.pdl ? 2 : 1;
   const uint32_t w_buf_bytes = 64u * p.k_group * 2u;
   if (p.k_group <= 256)      // at most four decode tasks per weight tile: two warps share each
-    return cudaLaunchKernelEx(&cfg, dqgemm_kacc_kernel<true>, p.xmap, p.jobs, p.segs, p.n_groups, p.T, p.out, p.ldo, p.err,
+    return cudaLaunchKernelEx(&cfg, dqgemm_kacc_kernel<true>, p.xmap, p.jobs, p.segs, static_cast<const __nv_bfloat16*>(p.x), p.ldx, p.n_groups, p.T, p.out, p.ldo, p.err,
                               p.n_stages, p.bps, w_buf_bytes, p.hdr_bytes, p.seg_stride, p.stamps);
-  return cudaLaunchKernelEx(&cfg, dqgemm_kacc_kernel<false>, p.xmap, p.jobs, p.segs, p.n_groups, p.T, p.out, p.ldo, p.err,
+  return cudaLaunchKernelEx(&cfg, dqgemm_kacc_kernel<false>, p.xmap, p.jobs, p.segs, static_cast<const __nv_bfloat16*>(p.x), p.ldx, p.n_groups, p.T, p.out, p.ldo, p.err,
                             p.n_stages, p.bps, w_buf_bytes, p.hdr_bytes, p.seg_stride, p.stamps);
 }
 

@@ -84,6 +84,8 @@ struct KaccLaunch {
   const Seg* segs;
   int n_groups, n_cols64, m_ctas;
   CUtensorMap xmap;         // x: [T rows, ldx columns] bf16, box 64 x 128, 128-byte swizzle
+  const void* x;            // the same operand as a plain pointer: idle warps prefetch it into L2; null = no prefetch
+  int ldx;
   int T;
   float* out;
   int ldo;
