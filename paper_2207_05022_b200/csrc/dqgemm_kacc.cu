@@ -8,11 +8,15 @@
 // The price is that the pair's weight tile changes with every K group: the tiles are small (64 rows x <= 512
 // columns, 64 KB), two of them sit in shared memory, and eight warps decode K group g + 1 (Section 4.2
 // decompression, the same routine as everywhere) while the tensor core works on K group g.  The same eight
-// warps drain the accumulators at the end of a block of token tiles.
+// warps drain the accumulators, tile pair by tile pair, when a block's last K group is through.
 //
-//   warp 0     TMA producer: activation boxes [128 tokens x 64] of (block, K group, tile, box) into a ring
-//   warp 1     MMA issuer (CTA 0 of the pair): tcgen05.mma.cta_group::2, commits free ring stages / weight buffers
-//   warps 4-11 decode weight tiles into the two buffers; epilogue (tcgen05.ld -> fp32 rows in global memory)
+//   warp 0      TMA producer: activation boxes [128 tokens x 64] of (block, K group, tile, box) into a ring
+//   warp 1      MMA issuer (CTA 0 of the pair): tcgen05.mma.cta_group::2, commits free ring stages / weight buffers
+//   warps 4-11  decode weight tiles into the two buffers; epilogue (tcgen05.ld -> fp32 rows in global memory)
+//   warps 12-15 L2 prefetch of the activations of the step after next, when the operand does not fit L2
+//
+// An mbarrier parity wait only tells "the phase of this parity has completed": every waiter here meets every phase
+// of the barriers it waits on, in order (a waiter that skipped a phase would take the one two back for its own).
 //
 // Every wait is bounded; a role that gives up raises the CTA's abort flag, the others stop waiting but keep
 // walking their loops (the decode group meets at named barriers), and the status word reports the timeout.
