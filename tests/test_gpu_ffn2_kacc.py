@@ -52,6 +52,8 @@ def _run(work, tune):
     (11, 100, "bf16", 4, 512, lambda i: i != 4),   # 1,100 tokens: 9 tiles (odd), ragged rows, 5 slices (a 256-wide group)
     (24, 128, "bf16", 8, 256, lambda i: i % 2 == 0),    # 3,072 tokens: 12 tile pairs over two CTA pairs: blocks of 4 + 2
     (24, 128, "f32", 8, 512, lambda i: True),
+    (16, 128, "bf16", 148, 512, lambda i: i == 3),      # one FFN slice kept: a single 256-wide K group
+    (16, 128, "f32", 4, 256, lambda i: i in (0, 5)),    # two slices, one group each, two blocks per CTA pair
 ])
 def test_layer_with_k_accumulating_ffn2(batch, seq, act, budget, kgroup, keep):
     from gpu_util import rel_err, REL_TOL
