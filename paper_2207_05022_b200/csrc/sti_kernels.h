@@ -107,11 +107,13 @@ cudaError_t launch_attention(const uint16_t* qkv, uint16_t* out, int n_kept, int
                              const int32_t* seq_lens, int sm_count, cudaStream_t s, bool pdl,
                              unsigned long long* stamps);
 
-// The same attention on the tcgen05 tensor cores, one CTA per (sequence, kept head), for many tokens (attention_tc.cu).
+// The same attention on the tcgen05 tensor cores, one CTA per (sequence, kept head) with two query tiles in flight, for
+// many tokens (attention_tc.cu).
 // `qkv_map`: TMA view of qkv as [3 * n_kept * T rows, 64 columns] bf16, boxes of 128 rows x 64 columns, 128-byte swizzle.
 cudaError_t attention_tc_configure();
 cudaError_t launch_attention_tc(const CUtensorMap& qkv_map, uint16_t* out, int n_kept, int batch, int seq,
                                 const int32_t* seq_lens, int* err, cudaStream_t s, bool pdl, unsigned long long* stamps);
+
 
 // out = LayerNorm(sum_p partial[p] + bias + resid) * gamma + beta, one warp per token row.
 struct LnLaunch {
