@@ -46,7 +46,8 @@ struct TcBarriers {
   uint64_t q_full[2];      // a query tile has landed in the group's slot
   uint64_t q_empty[2];     // the score MMAs of the slot's tile have completed
   uint64_t s_full[2];      // the group's score chunk is complete in tensor memory
-  uint64_t p_full[2];      // the group's probabilities are in shared memory (and its scores have been read)
+  uint64_t s_empty[2];     // the group has read its score chunk for the last time (the chunk's last tcgen05.ld is complete)
+  uint64_t p_full[2];      // the group's probabilities are in shared memory
   uint64_t o_full[2];      // the group's O_c is complete in tensor memory (and its probabilities have been read)
   uint32_t tmem_base;
   volatile uint32_t abort;
@@ -108,6 +109,7 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap qkv_map, uint16_t* __res
       mbar_init(smem_addr(&bar->q_full[g]), 1);
       mbar_init(smem_addr(&bar->q_empty[g]), 1);
       mbar_init(smem_addr(&bar->s_full[g]), 1);
+      mbar_init(smem_addr(&bar->s_empty[g]), kTcGroupWarps);
       mbar_init(smem_addr(&bar->p_full[g]), kTcGroupWarps);
       mbar_init(smem_addr(&bar->o_full[g]), 1);
     }
@@ -179,26 +181,50 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap qkv_map, uint16_t* __res
       bool ok = warp_wait(smem_addr(&bar->kv_full), 0, lane, &bar->abort);
       for (int g = 0; ok && g < 2; ++g)
         if (steps[g] > 0) ok = issue_scores(g, 0);
-      const int n_max = steps[0] > steps[1] ? steps[0] : steps[1];
-      for (int n = 0; ok && n < n_max; ++n) {
+      // Serve whichever group has something ready: its scores read for the last time -> the next chunk's S; its
+      // probabilities in shared memory -> O_c = P V.  Neither group waits for the other's softmax.
+      int next_s[2] = {1, 1}, next_pv[2] = {0, 0};               // S of step 0 is issued above
+      uint64_t t_idle = global_timer_ns();
+      while (ok && (next_pv[0] < steps[0] || next_pv[1] < steps[1])) {
+        bool progressed = false;
         for (int g = 0; ok && g < 2; ++g) {
-          if (n >= steps[g]) continue;
-          const int c = n % nc;
-          // the group's probabilities of step n are in shared memory, and its scores have been read
-          ok = warp_wait(smem_addr(&bar->p_full[g]), n & 1, lane, &bar->abort);
-          if (!ok) break;
-          if (n + 1 < steps[g]) ok = issue_scores(g, n + 1);     // the group's next scores first: it needs them first
-          if (!ok) break;
-          tc_fence_after_sync();
-          if (elect_one()) {
-            // O_c = P V_c: two boxes of 64 keys; per K = 16 step P moves 32 bytes in its swizzled row, V 16 rows
-            const uint64_t vd = v_desc0 + c * (kTcBox >> 4), pd = p_desc0 + g * (2 * kTcBox >> 4);
-            const uint32_t od = tmem + kTcColO + g * kTcHead;
-            umma_bf16_ss_x4(od, pd, vd, 2, 2048 >> 4, idesc_o, 0u);
-            umma_bf16_ss_x4(od, pd + (kTcBox >> 4), vd + (8192 >> 4), 2, 2048 >> 4, idesc_o, 1u);
-            umma_commit(smem_addr(&bar->o_full[g]));
+          if (next_s[g] < steps[g]) {                            // S(next_s) needs the reads of step next_s - 1 done
+            uint32_t ready = 0;
+            if (lane == 0) ready = mbar_try_wait(smem_addr(&bar->s_empty[g]), (next_s[g] - 1) & 1);
+            if (__shfl_sync(0xffffffffu, ready, 0)) {
+              ok = issue_scores(g, next_s[g]);
+              if (!ok) break;
+              ++next_s[g];
+              progressed = true;
+            }
           }
-          __syncwarp();
+          const int n = next_pv[g];
+          if (n < steps[g]) {
+            uint32_t ready = 0;
+            if (lane == 0) ready = mbar_try_wait(smem_addr(&bar->p_full[g]), n & 1);
+            if (__shfl_sync(0xffffffffu, ready, 0)) {
+              const int c = n % nc;
+              tc_fence_after_sync();
+              if (elect_one()) {
+                // O_c = P V_c: two boxes of 64 keys; per K = 16 step P moves 32 bytes in its swizzled row, V 16 rows
+                const uint64_t vd = v_desc0 + c * (kTcBox >> 4), pd = p_desc0 + g * (2 * kTcBox >> 4);
+                const uint32_t od = tmem + kTcColO + g * kTcHead;
+                umma_bf16_ss_x4(od, pd, vd, 2, 2048 >> 4, idesc_o, 0u);
+                umma_bf16_ss_x4(od, pd + (kTcBox >> 4), vd + (8192 >> 4), 2, 2048 >> 4, idesc_o, 1u);
+                umma_commit(smem_addr(&bar->o_full[g]));
+              }
+              __syncwarp();
+              next_pv[g] = n + 1;
+              progressed = true;
+            }
+          }
+        }
+        if (progressed) {
+          t_idle = global_timer_ns();
+        } else {
+          uint32_t give_up = 0;
+          if (lane == 0) give_up = (bar->abort || global_timer_ns() - t_idle > 2000000000ull) ? 1u : 0u;
+          if (__shfl_sync(0xffffffffu, give_up, 0)) ok = false;
         }
       }
       if (!ok) failed = true;
@@ -271,7 +297,13 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap qkv_map, uint16_t* __res
         for (int pc = 0; pc < 4; ++pc) {
           uint32_t (&r)[32] = rr[pc & 1];
           tmem_wait_ld_x32(r);
-          if (pc + 1 < 4) tmem_ld_32x32b_x32(s_addr + (pc + 1) * 32, rr[(pc + 1) & 1]);
+          if (pc + 1 < 4) {
+            tmem_ld_32x32b_x32(s_addr + (pc + 1) * 32, rr[(pc + 1) & 1]);
+          } else {                                               // the scores are in registers: their buffer may be refilled
+            tc_fence_before_sync();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(smem_addr(&bar->s_empty[g]));
+          }
           if (n_valid < (pc + 1) * 32) {
 #pragma unroll
             for (int k = 0; k < 32; ++k)
