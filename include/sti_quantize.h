@@ -34,12 +34,25 @@ extern "C" {
 #endif
 
 /* Bytes of device workspace sti_quantize_units needs for n_units units of n_weights weights each
- * (two ping-pong (key, offset) buffers for the sort and one byte per index: 17 bytes per weight). */
+ * (per unit 17 bytes per weight - two ping-pong (key, offset) buffers and one byte per index for the
+ * sorting method, the gathered bin members for the selecting one - plus one byte per unit that says
+ * which method did it). */
 size_t sti_quantize_workspace_bytes(uint32_t n_units, uint32_t n_weights);
 
-/* Quantizes n_units units in one launch (one CTA per unit), asynchronously on `stream` (a cudaStream_t,
- * NULL = default stream) of `device`.  All pointers are device pointers owned by the caller:
- *   w_dev            [n_units][n_weights] fp32, read only
+/* How step 3 is carried out.  Both give the same output (index streams, outlier lists and counts bit for
+ * bit; centroids up to the order of their fp64 sums).
+ *   STI_QUANTIZE_SELECT  no sort: clusters are equal-population slices of the sorted order, so only the
+ *                        2^bits - 1 weights at the slice boundaries are looked for (a histogram over value
+ *                        bins, then rank selection inside the few bins that hold a boundary); a unit this
+ *                        cannot take (zero variance, very many equal values) is sorted instead
+ *   STI_QUANTIZE_SORT    every unit: a stable radix sort of the (value, offset) pairs */
+#define STI_QUANTIZE_SELECT 0
+#define STI_QUANTIZE_SORT 1
+
+/* Quantizes n_units units (one CTA per unit), asynchronously on `stream` (a cudaStream_t,
+ * NULL = default stream) of `device`; the caller's current device is left as it was.  All pointers are
+ * device pointers owned by the caller:
+ *   w_dev            [n_units][n_weights] fp32, read only, 16-byte aligned
  *   codes_dev        [n_units][n_weights*bits/32] 32-bit words of the index stream
  *   centroids_dev    [n_units][2^bits] fp32, ascending where clusters are non-empty
  *   outlier_off_dev  [n_units][max_outliers] offsets within the unit, ascending; outlier_val_dev the values
@@ -51,11 +64,19 @@ size_t sti_quantize_workspace_bytes(uint32_t n_units, uint32_t n_weights);
  * Errors: STI_ERR_ARG (NULL or misaligned pointer), STI_ERR_BITS (bits outside 2..6), STI_ERR_SHAPE
  * (n_weights not a positive multiple of 32 or above 2^26, n_units 0 or above 65535, max_outliers 0),
  * STI_ERR_SIZE (workspace too small), STI_ERR_CUDA (no such device, launch failure).  Nothing is launched
- * on error. */
+ * on error.  Uses STI_QUANTIZE_SELECT. */
 sti_status sti_quantize_units(int device, void* stream, const float* w_dev, uint32_t n_units, uint32_t n_weights,
                               int bits, uint32_t* codes_dev, float* centroids_dev, uint32_t* outlier_off_dev,
                               float* outlier_val_dev, uint32_t max_outliers, uint32_t* n_outliers_dev,
                               void* workspace_dev, size_t workspace_bytes);
+
+/* The same with the method chosen by the caller (STI_ERR_ARG for an unknown one).  sorted_units_dev, when
+ * not NULL, is a device array of n_units bytes that receives 1 for every unit the sort did and 0 for the
+ * others. */
+sti_status sti_quantize_units_by(int device, void* stream, const float* w_dev, uint32_t n_units, uint32_t n_weights,
+                                 int bits, uint32_t* codes_dev, float* centroids_dev, uint32_t* outlier_off_dev,
+                                 float* outlier_val_dev, uint32_t max_outliers, uint32_t* n_outliers_dev,
+                                 void* workspace_dev, size_t workspace_bytes, int method, uint8_t* sorted_units_dev);
 
 #if defined(__GNUC__)
 #pragma GCC visibility pop

@@ -12,6 +12,6 @@ from .binding import (  # noqa: F401
     sti_sync, sti_shard_decode, sti_gemm_probe, sti_decode_rate_probe, sti_get_kernel_stamps, sti_plan_inject, sti_plan_retain, sti_shard_adopt, sti_plan_fill_stats, STI_INJECT_NONE, STI_INJECT_SLOW_COPY,
     STI_INJECT_PINNED_ALLOC_FAILURE, STAMP_KERNEL_NAMES, sti_plan_set_profiling, sti_plan_set_overlap, sti_get_stats, sti_plan_memory, sti_plan_check_guards,
     sti_ctx_launch_count, sti_host_retile, sti_strerror, sti_matrix_decode_noalloc, sti_plan_auto, sti_preload_after_run,
-    sti_quantize_units, sti_quantize_workspace_bytes,
+    sti_quantize_units, sti_quantize_units_by, sti_quantize_workspace_bytes, STI_QUANTIZE_SELECT, STI_QUANTIZE_SORT,
     Session,
 )

@@ -113,7 +113,7 @@ EXPORTED = ("sti_ctx_create", "sti_ctx_destroy", "sti_ctx_set_layer_params", "st
             "sti_plan_retain", "sti_shard_adopt", "sti_plan_fill_stats",
             "sti_plan_set_profiling", "sti_plan_set_overlap", "sti_get_stats", "sti_plan_memory", "sti_plan_check_guards", "sti_ctx_launch_count",
             "sti_host_retile", "sti_strerror", "sti_matrix_decode_noalloc", "sti_plan_auto",
-            "sti_preload_after_run", "sti_quantize_units", "sti_quantize_workspace_bytes")
+            "sti_preload_after_run", "sti_quantize_units", "sti_quantize_units_by", "sti_quantize_workspace_bytes")
 
 
 def _check(status: int, where: str):
@@ -415,6 +415,27 @@ def sti_quantize_units(w_dev: int, n_units: int, n_weights: int, bits: int, code
                                   C.c_void_p(codes_dev), C.c_void_p(centroids_dev), C.c_void_p(outlier_off_dev),
                                   C.c_void_p(outlier_val_dev), max_outliers, C.c_void_p(n_outliers_dev),
                                   C.c_void_p(workspace_dev), workspace_bytes), "sti_quantize_units")
+
+
+STI_QUANTIZE_SELECT, STI_QUANTIZE_SORT = 0, 1
+
+
+def sti_quantize_units_by(w_dev: int, n_units: int, n_weights: int, bits: int, codes_dev: int, centroids_dev: int,
+                          outlier_off_dev: int, outlier_val_dev: int, max_outliers: int, n_outliers_dev: int,
+                          workspace_dev: int, workspace_bytes: int, method: int, sorted_units_dev: int = 0,
+                          device: int = 0, stream: int = 0):
+    """sti_quantize_units with the method named (STI_QUANTIZE_SELECT / STI_QUANTIZE_SORT); sorted_units_dev, when
+    not 0, is a device array of n_units bytes that says which units the sort did (see sti_quantize.h)."""
+    lib = load_library()
+    lib.sti_quantize_units_by.restype = C.c_int
+    lib.sti_quantize_units_by.argtypes = [C.c_int, C.c_void_p, C.c_void_p, C.c_uint32, C.c_uint32, C.c_int, C.c_void_p,
+                                          C.c_void_p, C.c_void_p, C.c_void_p, C.c_uint32, C.c_void_p, C.c_void_p,
+                                          C.c_size_t, C.c_int, C.c_void_p]
+    _check(lib.sti_quantize_units_by(device, C.c_void_p(stream or None), C.c_void_p(w_dev), n_units, n_weights, int(bits),
+                                     C.c_void_p(codes_dev), C.c_void_p(centroids_dev), C.c_void_p(outlier_off_dev),
+                                     C.c_void_p(outlier_val_dev), max_outliers, C.c_void_p(n_outliers_dev),
+                                     C.c_void_p(workspace_dev), workspace_bytes, int(method),
+                                     C.c_void_p(sorted_units_dev or None)), "sti_quantize_units_by")
 
 
 class Session:

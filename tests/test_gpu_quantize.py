@@ -1,6 +1,7 @@
 """GPU parity of the device quantizer (Section 6) against the CPU oracle on the same seeded weights: index
 streams, outlier offsets, values and counts bit-exact; centroids equal up to one fp32 unit in the last place
-(both sides round an fp64 mean once, the summation orders differ)."""
+(both sides round an fp64 mean once, the summation orders differ).  Every case runs through both methods of the
+library (rank selection, the default, and the stable sort it falls back to)."""
 import numpy as np
 import pytest
 import torch
@@ -21,7 +22,7 @@ def _built():
     sti.load_library()
 
 
-def _run(units, bits, max_out=4096):
+def _run(units, bits, max_out=4096, method=None, want_sorted=False):
     """units: [n_units][n] fp32 on the host -> (words, centroids, offsets, values, counts) from the device."""
     n_units, n = units.shape
     w = torch.from_numpy(units).cuda()
@@ -34,11 +35,18 @@ def _run(units, bits, max_out=4096):
     ws_bytes = sti.sti_quantize_workspace_bytes(n_units, n)
     ws = torch.empty(ws_bytes, dtype=torch.uint8, device="cuda")
     torch.cuda.synchronize()
-    sti.sti_quantize_units(w.data_ptr(), n_units, n, bits, codes.data_ptr(), cents.data_ptr(), off.data_ptr(),
-                           val.data_ptr(), max_out, cnt.data_ptr(), ws.data_ptr(), ws_bytes)
+    by_sort = torch.full((n_units,), 7, dtype=torch.uint8, device="cuda")
+    if method is None:
+        sti.sti_quantize_units(w.data_ptr(), n_units, n, bits, codes.data_ptr(), cents.data_ptr(), off.data_ptr(),
+                               val.data_ptr(), max_out, cnt.data_ptr(), ws.data_ptr(), ws_bytes)
+    else:
+        sti.sti_quantize_units_by(w.data_ptr(), n_units, n, bits, codes.data_ptr(), cents.data_ptr(), off.data_ptr(),
+                                  val.data_ptr(), max_out, cnt.data_ptr(), ws.data_ptr(), ws_bytes, method,
+                                  by_sort.data_ptr())
     torch.cuda.synchronize()
-    return (codes.cpu().numpy().view(np.uint32), cents.cpu().numpy(), off.cpu().numpy().view(np.uint32),
-            val.cpu().numpy(), cnt.cpu().numpy())
+    res = (codes.cpu().numpy().view(np.uint32), cents.cpu().numpy(), off.cpu().numpy().view(np.uint32),
+           val.cpu().numpy(), cnt.cpu().numpy())
+    return res + (by_sort.cpu().numpy(),) if want_sorted else res
 
 
 def _ulp_diff(a, b):
@@ -49,9 +57,24 @@ def _ulp_diff(a, b):
 
 
 def _check(units, bits, max_out=4096):
-    words, cents, off, val, cnt = _run(units, bits, max_out)
+    """Both methods against the oracle; returns which units the default method handed to the sort."""
+    refs = [Q.quantize_unit(units[u], bits) for u in range(units.shape[0])]
+    _check_one(units, bits, max_out, refs, sti.STI_QUANTIZE_SORT)
+    return _check_one(units, bits, max_out, refs, sti.STI_QUANTIZE_SELECT)
+
+
+def _check_one(units, bits, max_out, refs, method):
+    words, cents, off, val, cnt, by_sort = _run(units, bits, max_out, method, want_sorted=True)
+    assert set(np.unique(by_sort)) <= {0, 1}
+    if method == sti.STI_QUANTIZE_SORT:
+        assert by_sort.all()
+    _compare(units, bits, max_out, refs, words, cents, off, val, cnt)
+    return by_sort
+
+
+def _compare(units, bits, max_out, refs, words, cents, off, val, cnt):
     for u in range(units.shape[0]):
-        rw, rc, ro, rv = Q.quantize_unit(units[u], bits)
+        rw, rc, ro, rv = refs[u]
         assert cnt[u] == ro.size, (u, bits)
         m = min(ro.size, max_out)
         assert np.array_equal(off[u, :m], ro[:m]) and np.array_equal(val[u, :m].view(np.uint32), rv[:m].view(np.uint32))
@@ -71,15 +94,15 @@ def test_bert_base_units_every_bitwidth(bits):
     shape = W.BERT_BASE
     units = np.stack([np.concatenate([m.reshape(-1) for m in make_unit_weights(shape, 11, l, ATTN, i)])
                       for l, i in ((0, 0), (1, 5), (2, 11))])
-    _check(units, bits)
+    assert not _check(units, bits).any()                  # Gaussian-like weights never need the sort
 
 
 def test_bert_large_ffn_unit_with_heavy_tails():
     shape = W.BERT_LARGE
     mats = make_unit_weights(shape, 12, 3, FFN, 7, outlier_stress=0.0015)       # 524,288 weights, ~0.15 % outliers
     units = np.concatenate([m.reshape(-1) for m in mats])[None, :]
-    _check(units, 3)
-    _check(units, 6)
+    assert not _check(units, 3).any()
+    assert not _check(units, 6).any()
 
 
 def test_ties_constant_and_tiny_units():
@@ -92,9 +115,34 @@ def test_ties_constant_and_tiny_units():
     ramp = np.arange(8192, dtype=np.float32) * np.float32(1e-5) - np.float32(0.04)
     units = np.stack([few_values, signed_zero, const, ramp])
     for bits in (2, 4, 6):
-        _check(units, bits)
+        by_sort = _check(units, bits)
+        assert by_sort[2] == 1                             # zero variance: no value bins to select in
     _check(rng.standard_normal((2, 32)).astype(np.float32) * np.float32(0.02), 5)            # fewer weights than 2 clusters' worth
     _check(rng.standard_normal((1, 1056)).astype(np.float32) * np.float32(0.02), 3)          # ragged last chunk
+
+
+def test_units_the_selection_hands_to_the_sort():
+    """Many equal values: one value bin holds more members than the counting selection accepts.  Mixed in one launch
+    with units that the selection does itself."""
+    rng = np.random.default_rng(6)
+    n = 65536
+    ties = rng.choice(np.linspace(-0.05, 0.05, 9).astype(np.float32), size=n)
+    normal = (rng.standard_normal(n) * 0.03).astype(np.float32)
+    half = normal.copy()
+    half[: n // 2] = np.float32(0.01)                     # half the unit is one value
+    units = np.stack([normal, ties, half, normal[::-1].copy()])
+    for bits in (2, 5):
+        by_sort = _check(units, bits)
+        assert list(by_sort) == [0, 1, 1, 0]
+
+
+def test_selection_is_deterministic():
+    shape = W.BERT_LARGE
+    units = np.stack([np.concatenate([m.reshape(-1) for m in make_unit_weights(shape, 14, 0, ATTN, i)]) for i in range(3)])
+    a = _run(units, 6)
+    b = _run(units, 6)
+    for x, y in zip(a, b):
+        assert np.array_equal(x.view(np.uint32) if x.dtype == np.float32 else x, y.view(np.uint32) if y.dtype == np.float32 else y)
 
 
 def test_outlier_lists_shorter_than_the_outliers_found():
