@@ -731,14 +731,20 @@ def run_baselines(args):
                       "t_io_us": t_io_us, "t_comp_us": t_comp_us[1:], "rows": rows}))
 
 
+def shape_layers_default():
+    """The quantizer's default workload is the whole model: every launch then holds more units than the GPU has SMs."""
+    import workloads as W
+    return W.BERT_LARGE.n_layers
+
+
 def run_quantize(args):
-    """Section 6 on the device: every shard unit of `--layers` BERT-large layers (16 attention units of 262,144
+    """Section 6 on the device: every shard unit of `--layers` BERT-large layers (default: all 24; 16 attention units of 262,144
     weights and 16 FFN units of 524,288 weights per layer) quantized at `--baseline-bits` bits by
     sti_quantize_units, timed with CUDA events, next to the CPU oracle on a sample of the same units."""
     import workloads as W
     from workloads.shards import ATTN, FFN, make_unit_weights
     from oracle import sti_quantizer_oracle as Q
-    n_layers = args.layers or 4
+    n_layers = args.layers or shape_layers_default()
     bits = args.baseline_bits
     shape = W.BERT_LARGE
     groups = {}
