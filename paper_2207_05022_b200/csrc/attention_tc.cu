@@ -12,7 +12,8 @@
 //                   register accumulator (which also says that the probability buffer is free); pass 2 reads the
 //                   scores again, exponentiates, sums, and writes the bf16 probabilities into shared memory in the
 //                   swizzled K-major layout the second MMA reads
-//   warp 8          TMA: K and V once, then query tiles into the two slots
+//   warp 8          TMA: K and V once (a barrier per 128-key chunk, so the first scores start after 16 KB of K have
+//                   landed, not after the sequence's 128 KB), query tiles into the two slots
 //   warp 9          MMA issuer: for each group in turn  S(next chunk)  and  O_c = P V(this chunk)
 //
 // Tensor memory: S of group g at columns 128 g, O_c of group g at 256 + 64 g.  Every barrier has one class of
@@ -42,7 +43,8 @@ constexpr uint32_t kTcTmemCols = 512;
 constexpr uint32_t kTcColS = 0, kTcColO = 256;
 
 struct TcBarriers {
-  uint64_t kv_full;        // K and V of the sequence have landed
+  uint64_t k_full[4];      // key chunk c has landed (one phase each: K and V are loaded once per CTA)
+  uint64_t v_full[4];      // value chunk c has landed
   uint64_t q_full[2];      // a query tile has landed in the group's slot
   uint64_t q_empty[2];     // the score MMAs of the slot's tile have completed
   uint64_t s_full[2];      // the group's score chunk is complete in tensor memory
@@ -104,7 +106,7 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap qkv_map, uint16_t* __res
     return;
   }
   if (tid == 0) {
-    mbar_init(smem_addr(&bar->kv_full), 1);
+    for (int c = 0; c < 4; ++c) { mbar_init(smem_addr(&bar->k_full[c]), 1); mbar_init(smem_addr(&bar->v_full[c]), 1); }
     for (int g = 0; g < 2; ++g) {
       mbar_init(smem_addr(&bar->q_full[g]), 1);
       mbar_init(smem_addr(&bar->q_empty[g]), 1);
@@ -144,16 +146,28 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap qkv_map, uint16_t* __res
 
   if (warp == kTcProducerWarp) {
     if (lane == 0 && nc > 0) {
-      mbar_expect_tx(smem_addr(&bar->kv_full), 2u * nc * kTcBox);
-      for (int c = 0; c < nc; ++c) {
-        tma_load_2d(k_sm + c * kTcBox, &qkv_map, 0, k_row + c * kTcChunk, smem_addr(&bar->kv_full));
-        tma_load_2d(v_sm + c * kTcBox, &qkv_map, 0, v_row + c * kTcChunk, smem_addr(&bar->kv_full));
-      }
-      for (int qt = 0; qt < n_qt; ++qt) {
-        const uint32_t g = qt & 1, i = qt >> 1;                  // the group's i-th tile
-        if (i >= 1 && !mbar_wait_bounded_relaxed(smem_addr(&bar->q_empty[g]), (i - 1) & 1)) { failed = true; break; }
+      // in the order the MMA warp needs them: the first key chunk, the first two query tiles, then V and K chunk by chunk
+      auto load_k = [&](int c) {
+        mbar_expect_tx(smem_addr(&bar->k_full[c]), kTcBox);
+        tma_load_2d(k_sm + c * kTcBox, &qkv_map, 0, k_row + c * kTcChunk, smem_addr(&bar->k_full[c]));
+      };
+      auto load_v = [&](int c) {
+        mbar_expect_tx(smem_addr(&bar->v_full[c]), kTcBox);
+        tma_load_2d(v_sm + c * kTcBox, &qkv_map, 0, v_row + c * kTcChunk, smem_addr(&bar->v_full[c]));
+      };
+      auto load_q = [&](int qt) {
+        const uint32_t g = qt & 1;
         mbar_expect_tx(smem_addr(&bar->q_full[g]), kTcBox);
         tma_load_2d(q_sm + g * kTcBox, &qkv_map, 0, q_row + qt * kTcQTile, smem_addr(&bar->q_full[g]));
+      };
+      load_k(0);
+      for (int qt = 0; qt < n_qt && qt < 2; ++qt) load_q(qt);
+      load_v(0);
+      for (int c = 1; c < nc; ++c) { load_k(c); load_v(c); }
+      for (int qt = 2; qt < n_qt; ++qt) {
+        const uint32_t g = qt & 1, i = qt >> 1;                  // the group's i-th tile
+        if (!mbar_wait_bounded_relaxed(smem_addr(&bar->q_empty[g]), (i - 1) & 1)) { failed = true; break; }
+        load_q(qt);
       }
     }
     __syncwarp();
@@ -168,6 +182,7 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap qkv_map, uint16_t* __res
       auto issue_scores = [&](int g, int n) -> bool {
         const int i = n / nc, c = n - i * nc;
         if (c == 0 && !warp_wait(smem_addr(&bar->q_full[g]), i & 1, lane, &bar->abort)) return false;
+        if (i == 0 && !warp_wait(smem_addr(&bar->k_full[c]), 0, lane, &bar->abort)) return false;   // later tiles: long landed
         tc_fence_after_sync();
         if (elect_one()) {
           umma_bf16_ss_x4(tmem + kTcColS + g * kTcChunk, q_desc0 + g * (kTcBox >> 4), k_desc0 + c * (kTcBox >> 4), 2, 2,
@@ -178,7 +193,7 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap qkv_map, uint16_t* __res
         __syncwarp();
         return true;
       };
-      bool ok = warp_wait(smem_addr(&bar->kv_full), 0, lane, &bar->abort);
+      bool ok = true;
       for (int g = 0; ok && g < 2; ++g)
         if (steps[g] > 0) ok = issue_scores(g, 0);
       // Serve whichever group has something ready: its scores read for the last time -> the next chunk's S; its
@@ -204,6 +219,7 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap qkv_map, uint16_t* __res
             if (lane == 0) ready = mbar_try_wait(smem_addr(&bar->p_full[g]), n & 1);
             if (__shfl_sync(0xffffffffu, ready, 0)) {
               const int c = n % nc;
+              if (n < nc && !warp_wait(smem_addr(&bar->v_full[c]), 0, lane, &bar->abort)) { ok = false; break; }
               tc_fence_after_sync();
               if (elect_one()) {
                 // O_c = P V_c: two boxes of 64 keys; per K = 16 step P moves 32 bytes in its swizzled row, V 16 rows
