@@ -165,6 +165,14 @@ def test_argument_checks():
     with pytest.raises(sti.StiError) as e:
         sti.sti_quantize_units(w.data_ptr(), 1, 64, 4, p, p, p, p, 4, p, p, 100)
     assert e.value.status == 4
+    big = torch.zeros(1 << 16, dtype=torch.uint8, device="cuda")
+    q = big.data_ptr()
+    with pytest.raises(sti.StiError) as e:                               # no such method
+        sti.sti_quantize_units_by(w.data_ptr(), 1, 64, 4, q, q, q, q, 4, q, q, 1 << 16, 2)
+    assert e.value.status == 1
+    with pytest.raises(sti.StiError) as e:                               # weights not 16-byte aligned
+        sti.sti_quantize_units(w.data_ptr() + 4, 1, 32, 4, q, q, q, q, 4, q, q, 1 << 16)
+    assert e.value.status == 1
 
 
 def test_device_quantized_units_run_through_the_layer():
