@@ -133,3 +133,25 @@ def test_agrees_with_the_input_generator_written_separately():
         words, cents, off, val = Q.quantize_unit(np.concatenate([m.reshape(-1) for m in mats]), bits)
         assert np.array_equal(words, blob.codes) and np.array_equal(off, blob.outlier_off)
         assert np.array_equal(val, blob.outlier_val) and np.array_equal(cents, blob.centroids)
+
+
+@pytest.mark.parametrize("bits", [2, 4, 6])
+def test_index_is_the_count_of_boundary_elements_not_above(bits):
+    """The property the device's selecting method rests on: in the stable sorted order (= the order of (value,
+    offset) pairs) cluster c starts at rank floor(c n'/2^k), so an inlier's index is the number of those boundary
+    elements, c = 1 .. 2^k - 1, whose pair is not above its own.  Checked on arrays with many ties, where the
+    offset decides, and with fewer inliers than clusters, where boundaries coincide."""
+    rng = np.random.default_rng(40 + bits)
+    cases = [(rng.standard_normal(4096) * 0.03).astype(np.float32),
+             rng.choice(np.linspace(-0.05, 0.05, 7).astype(np.float32), size=2048),
+             (rng.standard_normal(24) * 0.02).astype(np.float32)]
+    for w in cases:
+        codes, _, out_off, _ = Q.quantize(w, bits)
+        inl = np.setdiff1d(np.arange(w.size), out_off)
+        # -0 and +0 compare equal; the pair order is (value, offset)
+        order = sorted(inl, key=lambda i: (float(w[i]), int(i)))
+        n_in, K = len(order), 1 << bits
+        bounds = [order[(c * n_in) // K] for c in range(1, K)] if n_in else []
+        for i in inl:
+            count = sum(1 for b in bounds if (float(w[b]), int(b)) <= (float(w[i]), int(i)))
+            assert codes[i] == count
