@@ -567,7 +567,9 @@ sti_status enqueue_layer(sti_plan* p, int li, const void* x, void* y, int batch,
     ln.partial = p->partial; ln.n_partial = nh > 0 ? L.o.n_split : 0;
     ln.bias = dense + c->off_bo; ln.resid = x; ln.resid_bf16 = bf16_act ? 1 : 0;
     ln.gamma = dense + c->off_ln1g; ln.beta = dense + c->off_ln1b; ln.eps = d.ln_eps; ln.T = T; ln.d = d.hidden;
-    ln.out_f32 = p->h1_f32; ln.out_bf16 = p->h1_bf16;
+    // With bf16 activations every activation that crosses a kernel boundary is bf16 (the layer's input and output are):
+    // the second LayerNorm then takes its residual from the bf16 copy the FFN reads, and no fp32 copy is written.
+    ln.out_f32 = bf16_act ? nullptr : p->h1_f32; ln.out_bf16 = p->h1_bf16;
     ln.ctas_hint = ln_ctas_hint(p->tune.ln1_ctas, T, ns > 0 ? L.f1.n_jobs * m_ctas_for(L.f1.n_jobs, T, p->tune.cta_budget) : 0, c->sm_count);
     ln.stamps = stamp(4);
     CUDA_TRY(launch_layernorm(ln, c->compute, c->pdl));
@@ -593,7 +595,9 @@ sti_status enqueue_layer(sti_plan* p, int li, const void* x, void* y, int batch,
   CUDA_TRY(mark(6));
   LnLaunch l2{};
   l2.partial = p->partial; l2.n_partial = ns > 0 ? (f2_kacc ? 1 : L.f2.n_split) : 0;
-  l2.bias = dense + c->off_b2; l2.resid = p->h1_f32; l2.resid_bf16 = 0;
+  l2.bias = dense + c->off_b2;
+  l2.resid = bf16_act ? static_cast<const void*>(p->h1_bf16) : static_cast<const void*>(p->h1_f32);
+  l2.resid_bf16 = bf16_act ? 1 : 0;
   l2.gamma = dense + c->off_ln2g; l2.beta = dense + c->off_ln2b; l2.eps = d.ln_eps; l2.T = T; l2.d = d.hidden;
   l2.out_f32 = bf16_act ? nullptr : static_cast<float*>(y);
   l2.out_bf16 = bf16_act ? static_cast<uint16_t*>(y) : (want_next_bf16 ? p->x_bf16 : nullptr);

@@ -62,7 +62,9 @@ def test_tensor_core_attention_layer_matches_oracle_and_the_other_kernel(batch, 
     assert np.isfinite(y_tc).all()
     assert rel_err(y_tc, ref) <= REL_TOL, rel_err(y_tc, ref)
     assert rel_err(y_old, ref) <= REL_TOL
-    assert rel_err(y_tc, y_old) <= 5e-3                      # same arithmetic, different order
+    # same arithmetic, different order; with bf16 activations the LayerNorm output that feeds the FFN and the second
+    # residual is bf16, so a one-step difference there can move an output by two bf16 steps (2 x 2^-8 of the maximum)
+    assert rel_err(y_tc, y_old) <= (1e-2 if act == "bf16" else 5e-3)
 
 
 def test_tensor_core_attention_is_the_default_for_many_sequences():
