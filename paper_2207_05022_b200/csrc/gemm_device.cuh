@@ -40,19 +40,37 @@ struct SmemHeader {
 // ---------------------------------------------------------------------------------------
 // The k index planes of one task = (row group, 128-column chunk), one coalesced 128-bit load per plane.
 // `bits` is only known at run time here, so that the loads can be issued before anything else of the
-// task is ready; planes beyond `bits` are not touched.
+// task is ready.  All six loads are issued back to back and unconditionally - a plane number beyond `bits`
+// re-reads the last plane (a cache hit) - so that the task pays one memory round trip: with a load under
+// `if (p < bits)` each plane's load waited for the one before it.
 __device__ __forceinline__ void load_planes(const Seg& sg, uint32_t task, uint32_t lane, uint32_t (&w)[24]) {
   const uint32_t bits = sg.bits;
   const uint32_t chunks = sg.kc >= 128 ? sg.kc / 128 : 1;
   const uint32_t g = task / chunks, j = task % chunks;
   const uint4* src = sg.codes + (static_cast<size_t>(g) * chunks + j) * (bits * 32) + lane;
+  uint4 v[6];
 #pragma unroll
-  for (int p = 0; p < 6; ++p) {
-    if (static_cast<uint32_t>(p) < bits) {
-      const uint4 v = __ldg(src + p * 32);
-      w[4 * p + 0] = v.x; w[4 * p + 1] = v.y; w[4 * p + 2] = v.z; w[4 * p + 3] = v.w;
-    }
+  for (int p = 0; p < 6; ++p) v[p] = __ldg(src + (static_cast<uint32_t>(p) < bits ? p : (bits ? bits - 1 : 0)) * 32);
+#pragma unroll
+  for (int p = 0; p < 6; ++p) { w[4 * p + 0] = v[p].x; w[4 * p + 1] = v[p].y; w[4 * p + 2] = v[p].z; w[4 * p + 3] = v[p].w; }
+}
+
+// Which outlier of the tile a thread patches: outlier number `t` in the order of the tile's segments.  The segments'
+// counts are read in one go (lane s reads segment s: one memory round trip for up to kMaxSegs descriptors instead of
+// one per segment) and handed round by shuffles.  Returns the total; `seg` stays 0xffffffff when t is beyond it.
+__device__ __forceinline__ uint32_t find_outlier_slot(const Seg* __restrict__ segs, uint32_t n_seg, uint32_t t, uint32_t lane,
+                                                      uint32_t& seg, uint32_t& index) {
+  const uint32_t mine = lane < n_seg ? segs[lane].n_out : 0u;
+  uint32_t before = 0;
+  seg = 0xffffffffu;
+  index = 0;
+#pragma unroll 1
+  for (uint32_t si = 0; si < n_seg; ++si) {
+    const uint32_t n = __shfl_sync(0xffffffffu, mine, static_cast<int>(si));
+    if (seg == 0xffffffffu && t >= before && t - before < n) { seg = si; index = t - before; }
+    before += n;
   }
+  return before;
 }
 
 // Index unpack in registers -> bf16 table lookup in shared memory -> 16-byte stores into the K-major
@@ -274,16 +292,12 @@ __device__ __forceinline__ void decode_weight_tile(const Job& job, const Seg* __
   const uint32_t tasks_per_seg = (n_rows / rows_per_group) * chunks;
   const uint32_t n_tasks = tasks_per_seg * job.n_seg;
   // outlier number `tid` of the tile (segments in order): fetched now, applied once the tile is written
-  uint32_t o_seg = 0xffffffffu, o_off = 0, n_out_total = 0;
+  uint32_t o_seg, o_idx, o_off = 0;
   float o_val = 0.f;
-  for (uint32_t si = 0; si < job.n_seg; ++si) {
-    const uint32_t n = segs[si].n_out;
-    if (o_seg == 0xffffffffu && tid >= n_out_total && tid - n_out_total < n) {
-      o_seg = si;
-      o_off = __ldg(segs[si].out_off + (tid - n_out_total));
-      o_val = __ldg(segs[si].out_val + (tid - n_out_total));
-    }
-    n_out_total += n;
+  const uint32_t n_out_total = find_outlier_slot(segs, job.n_seg, tid, lane, o_seg, o_idx);
+  if (o_seg != 0xffffffffu) {
+    o_off = __ldg(segs[o_seg].out_off + o_idx);
+    o_val = __ldg(segs[o_seg].out_val + o_idx);
   }
   uint16_t* tab = warp_tables + warp * kTableStride;
   // a tile with at most half as many tasks as the CTA has warps: two warps share a task (half the decode latency)
@@ -401,16 +415,12 @@ __device__ __forceinline__ void decode_weight_tile_group(const Job& job, const S
   const uint32_t chunks = s0.kc >= 128 ? s0.kc / 128 : 1;
   const uint32_t tasks_per_seg = (n_rows / rows_per_group) * chunks;
   const uint32_t n_tasks = tasks_per_seg * job.n_seg;
-  uint32_t o_seg = 0xffffffffu, o_off = 0, n_out_total = 0;
+  uint32_t o_seg, o_idx, o_off = 0;
   float o_val = 0.f;
-  for (uint32_t si = 0; si < job.n_seg; ++si) {
-    const uint32_t n = segs[si].n_out;
-    if (o_seg == 0xffffffffu && gtid >= n_out_total && gtid - n_out_total < n) {
-      o_seg = si;
-      o_off = __ldg(segs[si].out_off + (gtid - n_out_total));
-      o_val = __ldg(segs[si].out_val + (gtid - n_out_total));
-    }
-    n_out_total += n;
+  const uint32_t n_out_total = find_outlier_slot(segs, job.n_seg, gtid, lane, o_seg, o_idx);
+  if (o_seg != 0xffffffffu) {
+    o_off = __ldg(segs[o_seg].out_off + o_idx);
+    o_val = __ldg(segs[o_seg].out_val + o_idx);
   }
   uint16_t* tab = warp_tables + warp * kTableStride;
   for (uint32_t u = warp; u < (SPLIT ? 2 * n_tasks : n_tasks); u += NWARPS) {
