@@ -41,7 +41,7 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 # dram__bytes_read.sum + dram__bytes_write.sum per dequant-GEMM launch (mean over one layer's QKV, O, FFN1, FFN2
 # launches; BERT-large layer, batch 1, seq 256) from the ncu capture summarised in
 # profiles/dqgemm_bertlarge_seq256_ncu_full.md.  Set to None whenever dqgemm.cu changes after that capture.
-NCU_DRAM_BYTES_PER_GEMM_LAUNCH = 2512256
+NCU_DRAM_BYTES_PER_GEMM_LAUNCH = 2510720
 
 
 def load_peaks():
